@@ -1,0 +1,146 @@
+/*
+ * vatp.h - C ABI of the Value-Aware Token Pruning (VATP) hot path for NVIDIA B200 (sm_100a).
+ *
+ * Method (arXiv 2406.12335, Section 3.2): every cached token k of an attention head has an
+ * importance I_k = S_k * ||v_k||_1 (Eq. 4), where S_k is an attention indicator: the attention
+ * probability accumulated over all queries so far (Eq. 2, H2O) or over a history window of the
+ * last w queries (Eq. 3, Scissorhands).  The lowest-importance tokens are dropped down to a KV
+ * budget B; the first F tokens ("Attention Sink Tokens" paragraph) and a local window of the R
+ * most recent tokens (Appendix A) are always kept.  Budgets are uniform over heads (Appendix A),
+ * so every (batch, head) pair - a "unit" - is an independent problem of identical shape.
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers owned by the caller; the library never allocates,
+ *     frees or synchronises.  `params`, `cache` structs are HOST structs read during the call.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and the call returns at once; outputs are valid after the caller synchronises the stream.
+ *   - q/k/v are [batch, heads, seq_len, head_dim] with innermost stride 1 and element strides
+ *     stride_b / stride_h / stride_t (0 = the contiguous default).  head_dim is 64 or 128.
+ *     dtype VATP_BF16 or VATP_F32; all arithmetic accumulates in fp32.
+ *   - Data pointers must be 16-byte aligned and row strides multiples of 16 bytes.
+ *   - Errors that the host can see (null pointer, bad shape, F + R > B, workspace too small,
+ *     misalignment) return a status before anything is launched.  A failed launch returns
+ *     VATP_ERR_CUDA.  Device-side conditions (a bounded wait that ran out) are written to
+ *     *dev_status (device int32, 0 = fine; caller zeroes it and reads it after sync); the
+ *     kernels never trap.
+ *   - Inputs are assumed finite.
+ */
+#ifndef VATP_H_
+#define VATP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  VATP_OK = 0,
+  VATP_ERR_INVALID_ARG = 1,
+  VATP_ERR_UNSUPPORTED = 2,
+  VATP_ERR_WORKSPACE = 3,
+  VATP_ERR_CUDA = 4,
+  VATP_ERR_TIMEOUT = 5
+} vatp_status;
+
+typedef enum { VATP_BF16 = 0, VATP_F32 = 1 } vatp_dtype;
+typedef enum { VATP_IND_H2O = 0, VATP_IND_WINDOW = 1 } vatp_indicator;
+
+/* Problem description shared by the four calls (host struct). */
+typedef struct {
+  int32_t batch, heads;      /* units = batch * heads                                          */
+  int32_t seq_len;           /* T: prompt length (prefill / select / compact)                  */
+  int32_t head_dim;          /* d: 64 or 128                                                   */
+  int32_t dtype;             /* vatp_dtype of q, k, v, the caches and `out`                    */
+  int32_t indicator;         /* vatp_indicator: Eq. 2 or Eq. 3                                 */
+  int32_t window_w;          /* w of Eq. 3 (last w queries); ignored for VATP_IND_H2O          */
+  float   scale;             /* softmax scale, normally 1/sqrt(d)                              */
+  int32_t budget;            /* B: tokens kept per unit                                        */
+  int32_t n_sink;            /* F: leading tokens always kept                                  */
+  int32_t n_recent;          /* R: most recent tokens always kept; F + R <= B                  */
+  int64_t stride_b, stride_h, stride_t; /* element strides of q, k, v; 0 = contiguous          */
+} vatp_params;
+
+/*
+ * Decode-time state of all units (host struct of caller-owned DEVICE arrays).
+ * cap = budget + 1 slots per unit.  Slot order is not positional after evictions; pos[] gives
+ * each slot's original token position (-1 = empty slot).
+ */
+typedef struct {
+  void    *k_cache, *v_cache; /* [batch, heads, cap, head_dim], params dtype                   */
+  float   *acc;               /* [batch, heads, cap] indicator S per slot (Eq. 2 / Eq. 3)      */
+  float   *vnorm;             /* [batch, heads, cap] ||v||_1 per slot (Eq. 4)                  */
+  int32_t *pos;               /* [batch, heads, cap] original position per slot, -1 = empty    */
+  int32_t *len;               /* [batch, heads] live tokens                                    */
+  int32_t *free_slot;         /* [batch, heads] slot the next token is written to              */
+  int32_t *next_pos;          /* [batch, heads] position t of the next token                   */
+  float   *ring;              /* windowed only: [batch, heads, w, cap] last w probability rows,
+                                 row (j mod w) holds query position j; else NULL                */
+  int64_t *acc_fixed;         /* windowed only: [batch, heads, cap] exact fixed-point window sum */
+} vatp_cache;
+
+/* Bytes of device scratch that vatp_prefill_scores / vatp_select need for `params`. */
+size_t vatp_workspace_bytes(const vatp_params* params);
+
+/*
+ * Prefill scoring (Eq. 1-4 at t = T-1), without materialising the T x T matrix.
+ *   pass 1: lse[j] = log sum_{i<=j} exp(scale * <q_j, k_i>)           (row normaliser of Eq. 1)
+ *   pass 2: attn_acc[k] = sum_j exp(scale * <q_j, k_k> - lse[j]) over j >= k (Eq. 2), or over
+ *           j >= max(T - w, k) (Eq. 3, last w queries); QK^T is recomputed, never stored
+ *   vnorm[k] = sum_c |v[k][c]|,  score[k] = attn_acc[k] * vnorm[k]     (Eq. 4)
+ * q, k, v: inputs as described above (read only).
+ * lse_out:  [batch, heads, T] fp32, nullable (then the row normalisers live in the workspace).
+ * attn_acc, vnorm, score: [batch, heads, T] fp32 outputs.
+ * win_rows: VATP_IND_WINDOW only: [batch, heads, w, T] fp32 output, row r = probabilities of
+ *           query T - w + r (zero where masked or where T - w + r < 0); NULL for H2O.
+ * workspace: >= vatp_workspace_bytes(params) bytes of device scratch, 256-byte aligned.
+ * bf16 with head_dim 128 runs on the tensor cores; other combinations use an fp32 FMA kernel.
+ */
+vatp_status vatp_prefill_scores(const vatp_params* params, const void* q, const void* k, const void* v,
+                                float* lse_out, float* attn_acc, float* vnorm, float* score,
+                                float* win_rows, void* workspace, size_t workspace_bytes,
+                                int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Budgeted selection (Section 3.2 with Appendix A's budget split): per unit keep the first F
+ * tokens, the last R tokens and the B - F - R highest-`score` tokens of the range [F, T - R);
+ * among equal scores the lower index is kept.  T <= B keeps every token.
+ * score: [batch, heads, T] fp32 (non-negative).
+ * kept_idx: [batch, heads, B] int32 output, ascending; when T < B entries T..B-1 are -1.
+ */
+vatp_status vatp_select(const vatp_params* params, const float* score, int32_t* kept_idx,
+                        void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Compaction: gather the surviving K/V rows (bit-exact copies, ascending original index) into
+ * the budgeted cache and initialise the decode state: acc <- attn_acc[kept], vnorm <- vnorm[kept],
+ * pos <- kept index, len <- min(T, B), free_slot <- len, next_pos <- T; unused slots get pos -1.
+ * VATP_IND_WINDOW also gathers win_rows columns into `ring` (row (T - w + r) mod w) and sets
+ * acc_fixed to the fixed-point window sums.
+ */
+vatp_status vatp_compact(const vatp_params* params, const void* k, const void* v, const float* attn_acc,
+                         const float* vnorm, const float* win_rows, const int32_t* kept_idx,
+                         const vatp_cache* cache, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * One generation step on the budgeted cache (Eq. 1-4 at step t = next_pos):
+ *   write (k_new, v_new) into free_slot with pos = t; p = softmax(scale * <q_new, k_i>) over all
+ *   live slots (the new token included); out = sum_i p_i v_i (Eq. 1); acc_i += p_i (Eq. 2; the
+ *   new token starts at its own probability) or the window update of Eq. 3; then, if more than
+ *   B tokens are live, the slot with the smallest acc_i * vnorm_i among tokens with
+ *   F <= pos <= t - R is released (ties: the highest position goes).
+ * q_new, k_new, v_new: [batch, heads, head_dim]; out: same shape and dtype.
+ * evicted_pos: [batch, heads] int32, nullable; position released this step or -1.
+ * State arrays are updated in place.  seq_len in params is ignored.
+ */
+vatp_status vatp_decode_step(const vatp_params* params, const vatp_cache* cache, const void* q_new,
+                             const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
+                             int32_t* dev_status, void* cuda_stream);
+
+const char* vatp_status_string(vatp_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* VATP_H_ */

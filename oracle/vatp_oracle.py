@@ -217,7 +217,7 @@ def decode_step(state: DecodeState, q, k, v, scale: float, B: int, F: int, R: in
     oracle's own minimum, otherwise ValueError.
 
     Returns dict(out, p, evicted (position or -1), runner_up, I_evicted,
-    I_runner_up, I (importances before eviction), pos (positions before
+    I_runner_up, adopted (a forced near-tie was taken), I (importances before eviction), pos (positions before
     eviction)).
     """
     t = state.t
@@ -244,7 +244,7 @@ def decode_step(state: DecodeState, q, k, v, scale: float, B: int, F: int, R: in
     I = state.importance()
     pos_before = list(state.pos)
     res = {"out": out, "p": p, "evicted": -1, "runner_up": -1,
-           "I_evicted": None, "I_runner_up": None, "I": I, "pos": pos_before}
+           "I_evicted": None, "I_runner_up": None, "I": I, "pos": pos_before, "adopted": False}
 
     if len(state.pos) > B:
         elig = [i for i, pp in enumerate(state.pos) if pp >= F and pp <= t - R]
@@ -260,6 +260,7 @@ def decode_step(state: DecodeState, q, k, v, scale: float, B: int, F: int, R: in
             if gap > tie_tol * max(abs(I[victim]), abs(I[cand])) + tie_abs:
                 raise ValueError("forced eviction is not a near-tie")
             victim = cand
+            res["adopted"] = True
         res["evicted"] = state.pos[victim]
         res["I_evicted"] = float(I[victim])
         if runner >= 0:

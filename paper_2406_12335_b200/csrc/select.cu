@@ -1,0 +1,142 @@
+// Budgeted selection: per unit, the top (B - F - R) scores of the middle range [F, T - R) by a
+// block-wide radix select on the fp32 bit pattern, ties resolved towards the lower index, and
+// the kept indices written in ascending order (first F, selected middle, last R).
+// One CTA per unit; the unit's scores are staged in shared memory once when they fit and read
+// from global memory (L2-resident) otherwise.  Pure integer work after the key transform.
+#include "vatp_internal.cuh"
+
+namespace vatp {
+namespace {
+
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_WARPS = SEL_THREADS / 32;
+
+// order-preserving map float -> uint32 (larger float = larger key), valid for any sign
+__device__ __forceinline__ uint32_t order_key(float x) {
+  uint32_t b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+
+template <bool STAGED>
+__global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F, int R, const float* __restrict__ score,
+                                                             int32_t* __restrict__ kept) {
+  extern __shared__ uint32_t keys_s[];  // STAGED: keys of the middle range
+  __shared__ uint32_t hist[256];
+  __shared__ uint32_t sh_prefix, sh_need;
+  __shared__ uint32_t warp_keep[SEL_WARPS], warp_eq[SEL_WARPS];
+  __shared__ uint32_t run_keep, run_eq;
+
+  const int u = blockIdx.x;
+  const float* sc = score + (int64_t)u * T;
+  int32_t* out = kept + (int64_t)u * B;
+  const int tid = threadIdx.x;
+
+  if (T <= B) {  // everything survives
+    for (int i = tid; i < B; i += SEL_THREADS) out[i] = i < T ? i : -1;
+    return;
+  }
+  const int n = T - R - F;   // middle range length (> 0 here because T > B >= F + R)
+  const int ksel = B - F - R;  // how many of the middle range survive
+  for (int i = tid; i < F; i += SEL_THREADS) out[i] = i;
+  for (int i = tid; i < R; i += SEL_THREADS) out[B - R + i] = T - R + i;
+  if (ksel == 0) return;
+
+  if (STAGED) {
+    for (int i = tid; i < n; i += SEL_THREADS) keys_s[i] = order_key(sc[F + i]);
+    __syncthreads();
+  }
+  auto key_at = [&](int i) -> uint32_t { return STAGED ? keys_s[i] : order_key(sc[F + i]); };
+
+  // radix select, most significant byte first: find the key value tau of rank ksel (descending)
+  uint32_t prefix = 0, mask = 0, need = (uint32_t)ksel;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    for (int i = tid; i < n; i += SEL_THREADS) {
+      const uint32_t key = key_at(i);
+      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (tid < 32) {
+      // walk the 256 bins from the top: 8 bins per lane, suffix sums by shuffles
+      uint32_t c[8], tot = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { c[j] = hist[255 - (tid * 8 + j)]; tot += c[j]; }
+      uint32_t incl = tot;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const uint32_t y = __shfl_up_sync(0xffffffffu, incl, off);
+        if (tid >= off) incl += y;
+      }
+      uint32_t before = incl - tot;  // keys in strictly higher bins than this lane's first bin
+      if (before < need && need <= incl) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (need <= before + c[j]) {
+            sh_prefix = prefix | ((uint32_t)(255 - (tid * 8 + j)) << shift);
+            sh_need = need - before;
+            break;
+          }
+          before += c[j];
+        }
+      }
+    }
+    __syncthreads();
+    prefix = sh_prefix;
+    need = sh_need;
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+  const uint32_t tau = prefix;     // the ksel-th largest key; `need` of the keys equal to tau survive
+  const uint32_t need_eq = need;
+
+  // ordered compaction: keep key > tau, and the first need_eq (lowest index) keys equal to tau
+  if (tid == 0) { run_keep = 0; run_eq = 0; }
+  __syncthreads();
+  const int lane = tid & 31, wid = tid >> 5;
+  for (int base = 0; base < n; base += SEL_THREADS) {
+    const int i = base + tid;
+    uint32_t key = 0;
+    bool gt = false, eq = false;
+    if (i < n) { key = key_at(i); gt = key > tau; eq = key == tau; }
+    const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
+    if (lane == 0) warp_eq[wid] = __popc(eq_ballot);
+    __syncthreads();
+    uint32_t eq_before = run_eq;
+    for (int w = 0; w < wid; ++w) eq_before += warp_eq[w];
+    eq_before += __popc(eq_ballot & ((1u << lane) - 1u));
+    const bool keep = gt || (eq && eq_before < need_eq);
+    const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
+    if (lane == 0) warp_keep[wid] = __popc(keep_ballot);
+    __syncthreads();
+    uint32_t keep_before = run_keep;
+    for (int w = 0; w < wid; ++w) keep_before += warp_keep[w];
+    keep_before += __popc(keep_ballot & ((1u << lane) - 1u));
+    if (keep) out[F + keep_before] = F + i;
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t a = 0, b = 0;
+      for (int w = 0; w < SEL_WARPS; ++w) { a += warp_keep[w]; b += warp_eq[w]; }
+      run_keep += a;
+      run_eq += b;
+    }
+    __syncthreads();
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st) {
+  const int n = T > B ? T - R - F : 0;
+  const size_t bytes = (size_t)n * sizeof(uint32_t);
+  if (bytes <= 200 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+    if (e != cudaSuccess) return e;
+    select_kernel<true><<<units, SEL_THREADS, bytes, st>>>(T, B, F, R, score, kept);
+  } else {
+    select_kernel<false><<<units, SEL_THREADS, 0, st>>>(T, B, F, R, score, kept);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace vatp

@@ -1,0 +1,154 @@
+// Host side of the C ABI: argument checks, workspace carving, dispatch to the kernels.
+#include <cstring>
+
+#include "vatp_internal.cuh"
+
+using namespace vatp;
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+vatp_status check_params(const vatp_params* p, bool need_T) {
+  if (!p) return VATP_ERR_INVALID_ARG;
+  if (p->batch <= 0 || p->heads <= 0) return VATP_ERR_INVALID_ARG;
+  if (need_T && p->seq_len <= 0) return VATP_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return VATP_ERR_UNSUPPORTED;
+  if (p->dtype != VATP_BF16 && p->dtype != VATP_F32) return VATP_ERR_UNSUPPORTED;
+  if (p->indicator != VATP_IND_H2O && p->indicator != VATP_IND_WINDOW) return VATP_ERR_UNSUPPORTED;
+  if (p->indicator == VATP_IND_WINDOW && p->window_w <= 0) return VATP_ERR_INVALID_ARG;
+  if (p->budget <= 0 || p->n_sink < 0 || p->n_recent < 0) return VATP_ERR_INVALID_ARG;
+  if ((int64_t)p->n_sink + p->n_recent > p->budget) return VATP_ERR_INVALID_ARG;
+  if (!(p->scale > 0.f)) return VATP_ERR_INVALID_ARG;
+  if (p->stride_b < 0 || p->stride_h < 0 || p->stride_t < 0) return VATP_ERR_INVALID_ARG;
+  return VATP_OK;
+}
+
+vatp_status make_shape(const vatp_params* p, Shape* s) {
+  s->units = p->batch * p->heads;
+  s->heads = p->heads;
+  s->T = p->seq_len;
+  s->d = p->head_dim;
+  s->st = p->stride_t ? p->stride_t : p->head_dim;
+  s->sh = p->stride_h ? p->stride_h : (int64_t)p->seq_len * s->st;
+  s->sb = p->stride_b ? p->stride_b : (int64_t)p->heads * s->sh;
+  s->scale = p->scale;
+  s->window = p->indicator == VATP_IND_WINDOW ? p->window_w : 0;
+  const int eb = p->dtype == VATP_F32 ? 4 : 2;
+  if (s->st < s->d) return VATP_ERR_INVALID_ARG;
+  if ((s->st * eb) % 16 || (s->sh * eb) % 16 || (s->sb * eb) % 16) return VATP_ERR_INVALID_ARG;
+  return VATP_OK;
+}
+
+inline size_t lse_bytes(const vatp_params* p) {
+  size_t n = (size_t)p->batch * p->heads * (size_t)p->seq_len * sizeof(float);
+  return (n + 255) / 256 * 256;
+}
+
+bool cache_ok(const vatp_cache* c, bool windowed) {
+  if (!c || !c->k_cache || !c->v_cache || !c->acc || !c->vnorm || !c->pos || !c->len || !c->free_slot || !c->next_pos)
+    return false;
+  if (!aligned16(c->k_cache) || !aligned16(c->v_cache)) return false;
+  if (windowed && (!c->ring || !c->acc_fixed)) return false;
+  return true;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* vatp_status_string(vatp_status s) {
+  switch (s) {
+    case VATP_OK: return "ok";
+    case VATP_ERR_INVALID_ARG: return "invalid argument";
+    case VATP_ERR_UNSUPPORTED: return "unsupported configuration";
+    case VATP_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case VATP_ERR_CUDA: return "CUDA error";
+    case VATP_ERR_TIMEOUT: return "device-side wait ran out";
+  }
+  return "unknown status";
+}
+
+size_t vatp_workspace_bytes(const vatp_params* p) {
+  if (check_params(p, true) != VATP_OK) return 0;
+  return lse_bytes(p);
+}
+
+vatp_status vatp_prefill_scores(const vatp_params* p, const void* q, const void* k, const void* v, float* lse_out,
+                                float* attn_acc, float* vnorm, float* score, float* win_rows, void* workspace,
+                                size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  vatp_status s = check_params(p, true);
+  if (s != VATP_OK) return s;
+  if (!q || !k || !v || !attn_acc || !vnorm || !score) return VATP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
+  const bool windowed = p->indicator == VATP_IND_WINDOW;
+  if (windowed && !win_rows) return VATP_ERR_INVALID_ARG;
+  Shape sh;
+  s = make_shape(p, &sh);
+  if (s != VATP_OK) return s;
+  float* lse = lse_out;
+  if (!lse) {
+    if (!workspace || workspace_bytes < lse_bytes(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+      return VATP_ERR_WORKSPACE;
+    lse = static_cast<float*>(workspace);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (p->dtype == VATP_BF16 && p->head_dim == 128 && !windowed && vatp_tc_available())
+    e = launch_prefill_tc(sh, q, k, v, lse, attn_acc, vnorm, score, win_rows, dev_status, st);
+  else
+    e = launch_prefill_simt(sh, p->dtype, q, k, v, lse, attn_acc, vnorm, score, win_rows, st);
+  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+}
+
+vatp_status vatp_select(const vatp_params* p, const float* score, int32_t* kept_idx, void* workspace,
+                        size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  (void)workspace; (void)workspace_bytes; (void)dev_status;
+  vatp_status s = check_params(p, true);
+  if (s != VATP_OK) return s;
+  if (!score || !kept_idx) return VATP_ERR_INVALID_ARG;
+  cudaError_t e = launch_select(p->batch * p->heads, p->seq_len, p->budget, p->n_sink, p->n_recent, score, kept_idx,
+                                static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+}
+
+vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, const float* attn_acc,
+                         const float* vnorm, const float* win_rows, const int32_t* kept_idx, const vatp_cache* cache,
+                         int32_t* dev_status, void* cuda_stream) {
+  (void)dev_status;
+  vatp_status s = check_params(p, true);
+  if (s != VATP_OK) return s;
+  const bool windowed = p->indicator == VATP_IND_WINDOW;
+  if (!k || !v || !attn_acc || !vnorm || !kept_idx || !cache_ok(cache, windowed)) return VATP_ERR_INVALID_ARG;
+  if (windowed && !win_rows) return VATP_ERR_INVALID_ARG;
+  if (!aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
+  Shape sh;
+  s = make_shape(p, &sh);
+  if (s != VATP_OK) return s;
+  cudaError_t e = launch_compact(sh, p->dtype, p->budget, k, v, attn_acc, vnorm, win_rows, kept_idx, *cache,
+                                 static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+}
+
+vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, const void* q_new, const void* k_new,
+                             const void* v_new, void* out, int32_t* evicted_pos, int32_t* dev_status,
+                             void* cuda_stream) {
+  (void)dev_status;
+  vatp_status s = check_params(p, false);
+  if (s != VATP_OK) return s;
+  const bool windowed = p->indicator == VATP_IND_WINDOW;
+  if (!q_new || !k_new || !v_new || !out || !cache_ok(cache, windowed)) return VATP_ERR_INVALID_ARG;
+  if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return VATP_ERR_INVALID_ARG;
+  Shape sh;
+  std::memset(&sh, 0, sizeof(sh));
+  sh.units = p->batch * p->heads;
+  sh.heads = p->heads;
+  sh.d = p->head_dim;
+  sh.scale = p->scale;
+  sh.window = windowed ? p->window_w : 0;
+  cudaError_t e = launch_decode(sh, p->dtype, p->budget, p->n_sink, p->n_recent, *cache, q_new, k_new, v_new, out,
+                                evicted_pos, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+}
+
+}  // extern "C"

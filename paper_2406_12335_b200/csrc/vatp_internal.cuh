@@ -1,0 +1,48 @@
+// Internal declarations shared by the kernels of libvatp (not part of the public C ABI).
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vatp.h"
+
+namespace vatp {
+
+struct Shape {
+  int units;           // batch * heads
+  int heads;
+  int T, d;
+  int64_t sb, sh, st;  // element strides of q/k/v
+  float scale;
+  int window;          // 0 = accumulate over all queries (Eq. 2); >0 = last `window` queries (Eq. 3)
+};
+
+// offset (in elements) of unit u's first row
+__host__ __device__ inline int64_t unit_offset(const Shape& s, int u) {
+  return (int64_t)(u / s.heads) * s.sb + (int64_t)(u % s.heads) * s.sh;
+}
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// true once the tensor-core prefill kernel is usable on the current device (sm_100, driver entry points found)
+bool vatp_tc_available();
+
+// ---- launchers (each returns cudaGetLastError()) ----
+cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const void* k, const void* v, float* lse,
+                                float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st);
+cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse,
+                              float* attn_acc, float* vnorm, float* score, float* win_rows, int32_t* dev_status,
+                              cudaStream_t st);
+cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st);
+cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, const void* v, const float* attn_acc,
+                           const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
+                           cudaStream_t st);
+cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
+                          const void* k, const void* v, void* out, int32_t* evicted, cudaStream_t st);
+
+// fixed-point image of a probability for the exact window sums (Eq. 3): p in [0, 1] -> p * 2^52
+__host__ __device__ inline long long prob_to_fixed(float p) { return (long long)((double)p * 4503599627370496.0); }
+__host__ __device__ inline float fixed_to_prob(long long x) { return (float)((double)x * (1.0 / 4503599627370496.0)); }
+
+}  // namespace vatp

@@ -1,0 +1,142 @@
+"""ctypes binding to libvatp.so: the same four calls as include/vatp.h, taking torch tensors.
+
+Argument marshalling only - every step of the path runs in the CUDA kernels of the library.
+There is no fallback: if the library is missing the import raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libvatp.so")
+if not os.path.exists(_LIB_PATH):
+    raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2406_12335_b200.build`")
+lib = C.CDLL(_LIB_PATH)
+
+OK = 0
+BF16, F32 = 0, 1
+IND_H2O, IND_WINDOW = 0, 1
+EXPORTS = ["vatp_workspace_bytes", "vatp_prefill_scores", "vatp_select", "vatp_compact", "vatp_decode_step",
+           "vatp_status_string"]
+
+
+class Params(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("heads", C.c_int32), ("seq_len", C.c_int32), ("head_dim", C.c_int32),
+                ("dtype", C.c_int32), ("indicator", C.c_int32), ("window_w", C.c_int32), ("scale", C.c_float),
+                ("budget", C.c_int32), ("n_sink", C.c_int32), ("n_recent", C.c_int32),
+                ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
+
+
+class CacheStruct(C.Structure):
+    _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("acc", C.c_void_p), ("vnorm", C.c_void_p),
+                ("pos", C.c_void_p), ("len", C.c_void_p), ("free_slot", C.c_void_p), ("next_pos", C.c_void_p),
+                ("ring", C.c_void_p), ("acc_fixed", C.c_void_p)]
+
+
+_vp = C.c_void_p
+lib.vatp_workspace_bytes.restype = C.c_size_t
+lib.vatp_workspace_bytes.argtypes = [C.POINTER(Params)]
+lib.vatp_prefill_scores.restype = C.c_int
+lib.vatp_prefill_scores.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.vatp_select.restype = C.c_int
+lib.vatp_select.argtypes = [C.POINTER(Params), _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.vatp_compact.restype = C.c_int
+lib.vatp_compact.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(CacheStruct), _vp, _vp]
+lib.vatp_decode_step.restype = C.c_int
+lib.vatp_decode_step.argtypes = [C.POINTER(Params), C.POINTER(CacheStruct), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.vatp_status_string.restype = C.c_char_p
+lib.vatp_status_string.argtypes = [C.c_int]
+
+
+class VatpError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {lib.vatp_status_string(code).decode()} ({code})")
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise VatpError(code, where)
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def make_params(*, batch, heads, seq_len, head_dim, dtype, budget, n_sink=0, n_recent=0, scale=None,
+                indicator="h2o", window=0, strides=(0, 0, 0)) -> Params:
+    dt = {torch.bfloat16: BF16, torch.float32: F32, "bf16": BF16, "f32": F32}[dtype]
+    return Params(batch, heads, seq_len, head_dim, dt, IND_WINDOW if indicator == "window" else IND_H2O, window,
+                  float(scale if scale is not None else head_dim ** -0.5), budget, n_sink, n_recent, *strides)
+
+
+def params_for(x: torch.Tensor, **kw) -> Params:
+    """Params for a [batch, heads, T, d] tensor, taking shape, dtype and strides from it."""
+    b, h, T, d = x.shape
+    assert x.stride(3) == 1
+    return make_params(batch=b, heads=h, seq_len=T, head_dim=d, dtype=x.dtype,
+                       strides=(x.stride(0), x.stride(1), x.stride(2)), **kw)
+
+
+def vatp_workspace_bytes(p: Params) -> int:
+    return int(lib.vatp_workspace_bytes(C.byref(p)))
+
+
+class Cache:
+    """Device arrays of the decode state (allocated with torch, owned by this object)."""
+
+    def __init__(self, p: Params, device="cuda"):
+        b, h, d, cap = p.batch, p.heads, p.head_dim, p.budget + 1
+        dt = torch.float32 if p.dtype == F32 else torch.bfloat16
+        self.cap = cap
+        self.k_cache = torch.zeros(b, h, cap, d, dtype=dt, device=device)
+        self.v_cache = torch.zeros(b, h, cap, d, dtype=dt, device=device)
+        self.acc = torch.zeros(b, h, cap, dtype=torch.float32, device=device)
+        self.vnorm = torch.zeros(b, h, cap, dtype=torch.float32, device=device)
+        self.pos = torch.full((b, h, cap), -1, dtype=torch.int32, device=device)
+        self.len = torch.zeros(b, h, dtype=torch.int32, device=device)
+        self.free_slot = torch.zeros(b, h, dtype=torch.int32, device=device)
+        self.next_pos = torch.zeros(b, h, dtype=torch.int32, device=device)
+        self.ring = self.acc_fixed = None
+        if p.indicator == IND_WINDOW:
+            self.ring = torch.zeros(b, h, p.window_w, cap, dtype=torch.float32, device=device)
+            self.acc_fixed = torch.zeros(b, h, cap, dtype=torch.int64, device=device)
+        self.struct = CacheStruct(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.acc, self.vnorm, self.pos,
+                                                       self.len, self.free_slot, self.next_pos, self.ring,
+                                                       self.acc_fixed)])
+
+    def nbytes(self) -> int:
+        return sum(t.numel() * t.element_size() for t in (self.k_cache, self.v_cache, self.acc, self.vnorm, self.pos))
+
+
+def vatp_prefill_scores(p: Params, q, k, v, *, lse_out=None, attn_acc, vnorm, score, win_rows=None,
+                        workspace=None, dev_status=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vatp_prefill_scores(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse_out), _ptr(attn_acc), _ptr(vnorm),
+                                   _ptr(score), _ptr(win_rows), _ptr(workspace), ws_bytes, _ptr(dev_status),
+                                   _stream(stream)), "vatp_prefill_scores")
+
+
+def vatp_select(p: Params, score, kept_idx, *, workspace=None, dev_status=None, stream=None):
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vatp_select(C.byref(p), _ptr(score), _ptr(kept_idx), _ptr(workspace), ws_bytes, _ptr(dev_status),
+                           _stream(stream)), "vatp_select")
+
+
+def vatp_compact(p: Params, k, v, attn_acc, vnorm, kept_idx, cache: Cache, *, win_rows=None, dev_status=None,
+                 stream=None):
+    _check(lib.vatp_compact(C.byref(p), _ptr(k), _ptr(v), _ptr(attn_acc), _ptr(vnorm), _ptr(win_rows), _ptr(kept_idx),
+                            C.byref(cache.struct), _ptr(dev_status), _stream(stream)), "vatp_compact")
+
+
+def vatp_decode_step(p: Params, cache: Cache, q_new, k_new, v_new, out, *, evicted_pos=None, dev_status=None,
+                     stream=None):
+    _check(lib.vatp_decode_step(C.byref(p), C.byref(cache.struct), _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(out),
+                                _ptr(evicted_pos), _ptr(dev_status), _stream(stream)), "vatp_decode_step")

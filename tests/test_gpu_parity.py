@@ -1,0 +1,139 @@
+"""GPU parity: the CUDA path through the C ABI against the float64 oracle, element by element,
+on the same seeded inputs.  Tolerances: scores 1e-5 relative for fp32 inputs, 1e-3 for bf16;
+kept sets exact except for scores within that tolerance of the boundary score; compacted K/V
+bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2406_12335_b200 import synth
+from tests import parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+def _small(dtype, d, T, B, F, R, b=1, h=2, indicator="h2o", window=0, steps=0, cid=90):
+    return synth.Workload(cid, f"case_T{T}", dtype, b, h, 1, d, T, B, F, R, indicator, window, steps)
+
+
+def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4):
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink).run()
+    P.gpu_invariants(g)
+    tol = P.TOL[wl.dtype]
+    units = units or [(b, h) for b in range(wl.batch) for h in range(wl.heads)]
+    refs, nb = {}, 0
+    for (b, h) in units:
+        ref, kept, n_boundary = P.check_prefill_unit(g, b, h, tol)
+        refs[(b, h)] = (ref, kept)
+        nb += n_boundary
+    adopted = 0
+    if decode and wl.decode_steps:
+        dq, dk, dv = synth.decode_inputs(wl, 0, device="cuda")
+        adopted = P.run_decode_and_check(g, refs, dq, dk, dv, wl.decode_steps, tol, check_state_every)
+    return g, nb, adopted
+
+
+def test_config0_fp32_tiny():
+    """Config 0: fp32, 2 heads, d 64, T 512, budget 256, recent 32, 16 decode steps."""
+    _run_case(synth.CONFIGS[0])
+
+
+@pytest.mark.parametrize("F", [2, 20])
+def test_config0_with_sink_retention(F):
+    g, _, _ = _run_case(synth.CONFIGS[0], n_sink=F)
+    assert torch.all(g.kept[..., :F].cpu() == torch.arange(F))
+
+
+@pytest.mark.parametrize("dtype,d,T,B,F,R", [
+    ("f32", 64, 333, 100, 3, 17),      # ragged tail, several 64-tiles
+    ("f32", 128, 200, 64, 0, 8),
+    ("bf16", 64, 257, 128, 2, 16),
+    ("bf16", 128, 1000, 300, 4, 50),   # ragged against 64- and 128-tiles
+    ("bf16", 128, 130, 65, 1, 1),
+    ("f32", 64, 40, 20, 2, 3),         # shorter than one tile
+])
+def test_ragged_shapes(dtype, d, T, B, F, R):
+    _run_case(_small(dtype, d, T, B, F, R, steps=6))
+
+
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("bf16", 128)])
+def test_degenerate_budgets(dtype, d):
+    # budget = F + R: sinks and window only, whatever the scores
+    wl = _small(dtype, d, 300, 24, 8, 16, steps=5)
+    g, _, _ = _run_case(wl)
+    assert g.kept[0, 0].cpu().tolist() == list(range(8)) + list(range(284, 300))
+    # budget >= T: every token kept, cache grows before evictions start
+    wl = _small(dtype, d, 100, 103, 2, 5, steps=8)
+    g, _, _ = _run_case(wl)
+    assert int(g.cache.len[0, 0]) == 103
+    # T == B exactly
+    _run_case(_small(dtype, d, 96, 96, 0, 0, steps=3))
+    # no recent window and no sinks
+    _run_case(_small(dtype, d, 150, 50, 0, 0, steps=4))
+
+
+def test_exact_ties_prefer_lower_index():
+    """select on hand-made scores with many exact ties (integer work: bit-exact)."""
+    V = P.vatp()
+    T, B, F, R = 5000, 1200, 3, 100
+    rng = np.random.default_rng(0)
+    score = torch.from_numpy(rng.integers(0, 7, size=(2, 3, T)).astype(np.float32)).cuda()
+    p = V.make_params(batch=2, heads=3, seq_len=T, head_dim=64, dtype="f32", budget=B, n_sink=F, n_recent=R)
+    kept = torch.empty(2, 3, B, dtype=torch.int32, device="cuda")
+    V.vatp_select(p, score, kept)
+    torch.cuda.synchronize()
+    from oracle import vatp_oracle as O
+    for b in range(2):
+        for h in range(3):
+            want = O.select_keep(score[b, h].cpu().numpy(), B, F, R)
+            assert kept[b, h].cpu().numpy().tolist() == want.tolist()
+
+
+def test_select_large_T_unstaged_path():
+    """T beyond what one CTA can stage in shared memory."""
+    V = P.vatp()
+    T, B, F, R = 70000, 7000, 20, 512
+    g = torch.Generator(device="cuda").manual_seed(5)
+    score = torch.rand(1, 2, T, generator=g, device="cuda")
+    score[0, 0, 1000:1100] = 0.5          # a run of ties
+    p = V.make_params(batch=1, heads=2, seq_len=T, head_dim=128, dtype="bf16", budget=B, n_sink=F, n_recent=R)
+    kept = torch.empty(1, 2, B, dtype=torch.int32, device="cuda")
+    V.vatp_select(p, score, kept)
+    torch.cuda.synchronize()
+    from oracle import vatp_oracle as O
+    for h in range(2):
+        want = O.select_keep(score[0, h].cpu().numpy(), B, F, R)
+        assert kept[0, h].cpu().numpy().tolist() == want.tolist()
+
+
+def test_strided_inputs():
+    """q/k/v as [b, T, h, d] storage viewed as [b, h, T, d] (non-contiguous token stride)."""
+    wl = _small("bf16", 128, 300, 100, 2, 10, b=2, h=3)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    qs, ks, vs = (x.transpose(1, 2).contiguous().transpose(1, 2) for x in (q, k, v))
+    assert not qs.is_contiguous()
+    g1 = P.GpuPrefill(wl, q, k, v).run()
+    g2 = P.GpuPrefill(wl, qs, ks, vs).run()
+    assert torch.equal(g1.score, g2.score) and torch.equal(g1.kept, g2.kept)
+    assert torch.equal(g1.cache.k_cache, g2.cache.k_cache) and torch.equal(g1.cache.v_cache, g2.cache.v_cache)
+
+
+def test_run_to_run_determinism():
+    wl = _small("bf16", 128, 700, 200, 2, 20, b=1, h=4)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    a = P.GpuPrefill(wl, q, k, v).run()
+    b = P.GpuPrefill(wl, q, k, v).run()
+    assert torch.equal(a.score, b.score) and torch.equal(a.kept, b.kept)
+
+
+def test_config1_llama_layer():
+    """Config 1: bf16, 32 heads, d 128, T 4096, budget 2048, recent 128; 256 decode steps on a
+    sample of heads (the oracle's python loop is the limit), invariants on all heads."""
+    wl = synth.CONFIGS[1]
+    _run_case(wl, units=[(0, 0), (0, 13), (0, 31)], check_state_every=64)
+
+
+def test_config1_prefill_all_heads():
+    wl = synth.CONFIGS[1].with_(decode_steps=0)
+    _run_case(wl, decode=False)
