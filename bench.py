@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the VATP hot path on B200: prefill score+prune tokens/s and decode us/layer-step.
+
+One "step" = one pass of the whole path over one batch of synthetic input:
+  for each layer: vatp_prefill_scores -> vatp_select -> vatp_compact      (score + prune)
+  then `decode_steps` generation steps, each visiting every layer with vatp_decode_step.
+The workload is config 1 (LLaMA2-7B layer shape: bf16, 32 heads, d 128, prompt 4096, budget 2048,
+recent 128, 256 decode steps) held as LAYERS independently seeded layers, so that the decode
+working set (LAYERS x 34.6 MB) does not sit in the 126 MB L2 between visits - as in a real model,
+where the layers are visited in turn.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the float64 CPU oracle on a bounded
+sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "prefill_score_prune_tokens_per_s"
+UNIT = "tokens/s"
+LAYERS = 8
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[1])); mx.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for name, col in (("hw_slowdown", 5), ("hw_thermal_slowdown", 6), ("sw_thermal_slowdown", 7),
+                              ("sw_power_cap", 8)):
+                if len(r) > col and r[col].lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ reference arm
+def oracle_sample(wl, units: int, decode_steps: int):
+    """Times the oracle, as it stands, on `units` heads of layer 0 of the workload (prefill, select,
+    compact and `decode_steps` generation steps).  Returns (seconds prefill+prune, seconds decode)."""
+    import numpy as np
+    from oracle import vatp_oracle as O
+    from paper_2406_12335_b200 import synth
+    sub = wl.with_(heads=units)
+    q, k, v = (x.double().numpy() for x in synth.prefill_inputs(sub, 0, "cpu"))
+    dq, dk, dv = (x.double().numpy() for x in synth.decode_inputs(sub, 0, decode_steps, "cpu"))
+    t_pre = t_dec = 0.0
+    for h in range(units):
+        t0 = time.perf_counter()
+        r = O.prefill(q[0, h], k[0, h], v[0, h], wl.scale)
+        kept = O.select_keep(r["I"], wl.budget, wl.n_sink, wl.n_recent)
+        O.compact_rows(k[0, h], kept); O.compact_rows(v[0, h], kept)
+        st = O.DecodeState(k[0, h], v[0, h], r["S"], r["n1"], kept, wl.seq_len)
+        t1 = time.perf_counter()
+        for s in range(decode_steps):
+            O.decode_step(st, dq[s, 0, h], dk[s, 0, h], dv[s, 0, h], wl.scale, wl.budget, wl.n_sink, wl.n_recent)
+        t2 = time.perf_counter()
+        t_pre += t1 - t0
+        t_dec += t2 - t1
+        del r
+    return t_pre, t_dec
+
+
+def cpu_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [i.get("num_threads", 1) for i in threadpool_info() if i.get("user_api") == "blas"]
+        if n:
+            return max(n)
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    units, dsteps = 2, 16
+    for _ in range(args.warmup and 1):
+        oracle_sample(wl, 1, 2)
+    pre, dec = [], []
+    for _ in range(args.steps):
+        a, b = oracle_sample(wl, units, dsteps)
+        pre.append(a); dec.append(b)
+    t_unit = statistics.mean(pre) / units                       # seconds per (layer, head) unit
+    all_units = wl.batch * wl.heads
+    value = wl.batch * wl.seq_len / (t_unit * all_units)        # tokens/s of one layer, extrapolated from the sample
+    dec_us = statistics.mean(dec) / (units * dsteps) * all_units * 1e6
+    sample = (f"{units} of {all_units} heads of one layer, full prompt {wl.seq_len}, {dsteps} decode steps each; "
+              f"per-layer figure extrapolated x{all_units // units}")
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": (statistics.mean(pre) + statistics.mean(dec)) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config1 {wl.name} (oracle on a sample)", "sample": sample},
+            "decode_us_per_layer_step": dec_us,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------ CUDA arm
+class LayerState:
+    def __init__(self, V, wl, layer, dev):
+        from paper_2406_12335_b200 import synth
+        self.q, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
+        self.p = V.params_for(self.q, budget=wl.budget, n_sink=wl.n_sink, n_recent=wl.n_recent, scale=wl.scale,
+                              indicator=wl.indicator, window=wl.window)
+        b, h, T = wl.batch, wl.heads, wl.seq_len
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.attn_acc = torch.empty(b, h, T, **f32)
+        self.vnorm = torch.empty(b, h, T, **f32)
+        self.score = torch.empty(b, h, T, **f32)
+        self.kept = torch.empty(b, h, wl.budget, dtype=torch.int32, device=dev)
+        self.ws = torch.empty(max(V.vatp_workspace_bytes(self.p), 256), dtype=torch.uint8, device=dev)
+        self.cache = V.Cache(self.p, device=dev)
+        self.dq, self.dk, self.dv = synth.decode_inputs(wl, layer, device=dev)
+        self.out = torch.empty(wl.decode_steps, b, h, wl.head_dim, dtype=self.q.dtype, device=dev)
+        self.evicted = torch.empty(wl.decode_steps, b, h, dtype=torch.int32, device=dev)
+
+
+def run_cuda(args, wl):
+    from paper_2406_12335_b200 import build as _b
+    _b.build()
+    from paper_2406_12335_b200 import vatp as V      # raises if libvatp.so is missing: no fallback
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    L, steps_dec = LAYERS, wl.decode_steps
+    layers = [LayerState(V, wl, l, dev) for l in range(L)]
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def prefill_all(ev=None):
+        for i, ls in enumerate(layers):
+            if ev: ev[i][0].record()
+            V.vatp_prefill_scores(ls.p, ls.q, ls.k, ls.v, attn_acc=ls.attn_acc, vnorm=ls.vnorm, score=ls.score,
+                                  workspace=ls.ws, dev_status=status)
+            if ev: ev[i][1].record()
+            V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
+            if ev: ev[i][2].record()
+            V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, dev_status=status)
+            if ev: ev[i][3].record()
+
+    def decode_all():
+        for s in range(steps_dec):
+            for ls in layers:
+                V.vatp_decode_step(ls.p, ls.cache, ls.dq[s], ls.dk[s], ls.dv[s], ls.out[s], evicted_pos=ls.evicted[s],
+                                   dev_status=status)
+
+    # warm up once outside any capture (first calls set kernel attributes), then capture the
+    # launch-bound decode loop in a CUDA graph
+    prefill_all(); decode_all(); torch.cuda.synchronize()
+    graph = None
+    if not args.no_graph:
+        prefill_all(); torch.cuda.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            decode_all()
+        torch.cuda.synchronize()
+
+    def run_decode():
+        if graph is not None:
+            graph.replay()
+        else:
+            decode_all()
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    E = lambda: torch.cuda.Event(enable_timing=True)
+
+    def one_step(timed):
+        flush.fill_(rank + 1)                       # evict L2 between iterations
+        ev = [[E() for _ in range(4)] for _ in range(L)]
+        e0, e1, e2 = E(), E(), E()
+        e0.record()
+        prefill_all(ev)
+        e1.record()
+        run_decode()
+        e2.record()
+        return e0, e1, e2, ev
+
+    for _ in range(args.warmup):
+        one_step(False)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    recs = [one_step(True) for _ in range(args.steps)]
+    barrier()
+    clocks = sampler.stop()
+    assert int(status.item()) == 0, "device status word set"
+
+    t_pre = [a.elapsed_time(b) for a, b, _, _ in recs]               # ms, all layers
+    t_dec = [b.elapsed_time(c) for _, b, c, _ in recs]
+    t_all = [a.elapsed_time(c) for a, _, c, _ in recs]
+    t_score = [sum(e[0].elapsed_time(e[1]) for e in r[3]) / L for r in recs]    # ms per layer
+    t_select = [sum(e[1].elapsed_time(e[2]) for e in r[3]) / L for r in recs]
+    t_compact = [sum(e[2].elapsed_time(e[3]) for e in r[3]) / L for r in recs]
+    stats = torch.tensor([sum(t_pre), sum(t_dec), sum(t_all)], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(stats, op=torch.distributed.ReduceOp.MAX)
+    pre_ms, dec_ms, all_ms = (stats / args.steps).tolist()
+
+    # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
+    host = [[x.cpu().pin_memory() for x in (ls.q, ls.k, ls.v, ls.dq, ls.dk, ls.dv)] for ls in layers]
+    host_kept = [torch.empty_like(ls.kept, device="cpu").pin_memory() for ls in layers]
+    host_out = [torch.empty_like(ls.out, device="cpu").pin_memory() for ls in layers]
+    h2d = sum(x.numel() * x.element_size() for hl in host for x in hl)
+    d2h = sum(x.numel() * x.element_size() for x in host_kept + host_out)
+
+    def e2e_step():
+        flush.fill_(3)
+        e0, e1, e2 = E(), E(), E()
+        e0.record()
+        for ls, hl in zip(layers, host):
+            for dst, src in zip((ls.q, ls.k, ls.v, ls.dq, ls.dk, ls.dv), hl):
+                dst.copy_(src, non_blocking=True)
+        prefill_all()
+        for ls, hk in zip(layers, host_kept):
+            hk.copy_(ls.kept, non_blocking=True)
+        e1.record()
+        run_decode()
+        for ls, ho in zip(layers, host_out):
+            ho.copy_(ls.out, non_blocking=True)
+        e2.record()
+        return e0, e1, e2
+
+    e2e_step(); barrier()
+    e2e_recs = [e2e_step() for _ in range(max(2, min(args.steps, 5)))]
+    barrier()
+    e2e_pre = torch.tensor([statistics.mean(a.elapsed_time(b) for a, b, _ in e2e_recs)], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(e2e_pre, op=torch.distributed.ReduceOp.MAX)
+    e2e_dec_ms = statistics.mean(b.elapsed_time(c) for _, b, c in e2e_recs)
+
+    if rank != 0:
+        return
+    units = wl.batch * wl.heads
+    T, d, B = wl.seq_len, wl.head_dim, wl.budget
+    tokens = wl.batch * T * L                                  # layer-tokens scored and pruned per step
+    value = world * tokens / (pre_ms * 1e-3)
+    dec_us = dec_ms * 1e3 / (steps_dec * L)
+
+    # ---- rooflines (algorithmic work only) ----
+    flops_score = 2 * (2.0 * d) * T * (T + 1) / 2 * units      # two passes of the causal half of QK^T
+    bytes_compact = units * (2 * 2 * B * d * 2 + 12 * B)       # K,V rows read + written, 12 B of state per slot
+    bytes_decode = units * (B + 1) * (2 * d * 2 + 16)          # K,V rows once, acc r+w, vnorm, pos
+    bytes_select = units * (4 * T + 4 * B)
+    ms = statistics.mean
+    kernels = {
+        "prefill_scores": {"bound": "tensor", "achieved": flops_score / (ms(t_score) * 1e-3) / 1e12,
+                           "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "ms_per_launch_pair": ms(t_score)},
+        "select": {"bound": "hbm", "achieved": bytes_select / (ms(t_select) * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                   "unit": "GB/s", "us_per_launch": ms(t_select) * 1e3},
+        "compact": {"bound": "hbm", "achieved": bytes_compact / (ms(t_compact) * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "us_per_launch": ms(t_compact) * 1e3},
+        "decode_step": {"bound": "hbm", "achieved": bytes_decode / (dec_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"],
+                        "unit": "GB/s", "us_per_launch": dec_us},
+    }
+    for kd in kernels.values():
+        kd["frac"] = kd["achieved"] / kd["peak"]
+        kd["peak_source"] = peaks["source"]
+    share = {"prefill_scores": ms(t_score) * L, "select": ms(t_select) * L, "compact": ms(t_compact) * L,
+             "decode_step": dec_ms}
+    dominant = max(share, key=share.get)
+    roof = dict(kernels[dominant])
+    roof["kernel"] = dominant
+    roof["traffic"] = None
+    roof["time_share"] = share[dominant] / sum(share.values())
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": all_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
+        "config": {"workload": f"config1 {wl.name}: b{wl.batch} h{wl.heads} d{d} T{T} budget{B} recent{wl.n_recent} "
+                               f"sinkF{wl.n_sink} h2o, {steps_dec} decode steps, x{L} independently seeded layers",
+                   "l2": "256 MB flush write between steps; layer rotation keeps the decode state (277 MB) out of L2",
+                   "replicas": "each GPU runs the whole workload (path does not shard within a call)",
+                   "decode_graph": graph is not None},
+        "prefill_ms_per_layer": pre_ms / L, "decode_us_per_layer_step": dec_us,
+        "roofline": roof, "roofline_all": kernels,
+        "e2e": {"value": world * tokens / (float(e2e_pre.item()) * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "decode_us_per_layer_step": e2e_dec_ms * 1e3 / (steps_dec * L)},
+        "gpu_launches": args.steps * (L * 4 + steps_dec * L),
+        "clocks": clocks,
+    }
+    if not args.no_cpu_baseline and world == 1:
+        cu, cs = 2, 16
+        a, b = oracle_sample(wl, cu, cs)
+        v = wl.batch * T / (a / cu * units)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+                                "sample": f"{cu} of {units} heads of one layer (full prompt {T}, {cs} decode steps), "
+                                          f"{a + b:.1f} s of CPU work, per-layer figure extrapolated x{units // cu}",
+                                "decode_us_per_layer_step": b / (cu * cs) * units * 1e6}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-graph", action="store_true", help="launch decode steps directly instead of replaying a CUDA graph")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    from paper_2406_12335_b200 import synth
+    wl = synth.CONFIGS[1]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_cuda(args, wl)
+
+
+if __name__ == "__main__":
+    main()
