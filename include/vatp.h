@@ -64,8 +64,10 @@ typedef struct {
 
 /*
  * Decode-time state of all units (host struct of caller-owned DEVICE arrays).
- * cap = budget + 1 slots per unit.  Slot order is not positional after evictions; pos[] gives
- * each slot's original token position (-1 = empty slot).
+ * cap = vatp_cache_capacity(budget) slots per unit: budget + 1 rounded up to a multiple of 8 (one
+ * slot beyond the budget receives the incoming token before the eviction; the padding keeps every
+ * unit's arrays 32-byte aligned).  Slot order is not positional after evictions; pos[] gives each
+ * slot's original token position (-1 = empty slot).  acc, vnorm and pos must be 16-byte aligned.
  */
 typedef struct {
   void    *k_cache, *v_cache; /* [batch, heads, cap, head_dim], params dtype                   */
@@ -79,6 +81,9 @@ typedef struct {
                                  row (j mod w) holds query position j; else NULL                */
   int64_t *acc_fixed;         /* windowed only: [batch, heads, cap] exact fixed-point window sum */
 } vatp_cache;
+
+/* Slots per unit of the decode state for a budget of B tokens (see vatp_cache). */
+int32_t vatp_cache_capacity(int32_t budget);
 
 /* Bytes of device scratch that vatp_prefill_scores / vatp_select need for `params`. */
 size_t vatp_workspace_bytes(const vatp_params* params);

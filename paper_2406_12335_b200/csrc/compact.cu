@@ -88,7 +88,7 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
                            cudaStream_t st) {
   const int eb = dtype == VATP_F32 ? 4 : 2;
-  const int cap = B + 1;
+  const int cap = cache_capacity(B);
   const int cpr = s.d * eb / 16;
   const int64_t total = (int64_t)s.units * cap * 2 * cpr;
   const int64_t per_block = (int64_t)CP_THREADS * CP_UNROLL;

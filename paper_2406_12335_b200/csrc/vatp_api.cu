@@ -48,7 +48,8 @@ inline size_t lse_bytes(const vatp_params* p) {
 bool cache_ok(const vatp_cache* c, bool windowed) {
   if (!c || !c->k_cache || !c->v_cache || !c->acc || !c->vnorm || !c->pos || !c->len || !c->free_slot || !c->next_pos)
     return false;
-  if (!aligned16(c->k_cache) || !aligned16(c->v_cache)) return false;
+  if (!aligned16(c->k_cache) || !aligned16(c->v_cache) || !aligned16(c->acc) || !aligned16(c->vnorm) || !aligned16(c->pos))
+    return false;
   if (windowed && (!c->ring || !c->acc_fixed)) return false;
   return true;
 }
@@ -68,6 +69,8 @@ const char* vatp_status_string(vatp_status s) {
   }
   return "unknown status";
 }
+
+int32_t vatp_cache_capacity(int32_t budget) { return budget > 0 ? cache_capacity(budget) : 0; }
 
 size_t vatp_workspace_bytes(const vatp_params* p) {
   if (check_params(p, true) != VATP_OK) return 0;
@@ -133,7 +136,6 @@ vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, con
 vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, const void* q_new, const void* k_new,
                              const void* v_new, void* out, int32_t* evicted_pos, int32_t* dev_status,
                              void* cuda_stream) {
-  (void)dev_status;
   vatp_status s = check_params(p, false);
   if (s != VATP_OK) return s;
   const bool windowed = p->indicator == VATP_IND_WINDOW;
@@ -147,7 +149,7 @@ vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, cons
   sh.scale = p->scale;
   sh.window = windowed ? p->window_w : 0;
   cudaError_t e = launch_decode(sh, p->dtype, p->budget, p->n_sink, p->n_recent, *cache, q_new, k_new, v_new, out,
-                                evicted_pos, static_cast<cudaStream_t>(cuda_stream));
+                                evicted_pos, dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
 

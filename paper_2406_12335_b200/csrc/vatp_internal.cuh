@@ -17,6 +17,10 @@ struct Shape {
   int window;          // 0 = accumulate over all queries (Eq. 2); >0 = last `window` queries (Eq. 3)
 };
 
+// slots per unit in the decode state: budget + 1, rounded up to a multiple of 8 so that every
+// per-slot array of a unit starts on a 32-byte boundary (bulk copies need 16)
+__host__ __device__ inline int cache_capacity(int budget) { return (budget + 1 + 7) & ~7; }
+
 // offset (in elements) of unit u's first row
 __host__ __device__ inline int64_t unit_offset(const Shape& s, int u) {
   return (int64_t)(u / s.heads) * s.sb + (int64_t)(u % s.heads) * s.sh;
@@ -39,7 +43,7 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
                            cudaStream_t st);
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
-                          const void* k, const void* v, void* out, int32_t* evicted, cudaStream_t st);
+                          const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st);
 
 // fixed-point image of a probability for the exact window sums (Eq. 3): p in [0, 1] -> p * 2^52
 __host__ __device__ inline long long prob_to_fixed(float p) { return (long long)((double)p * 4503599627370496.0); }

@@ -18,7 +18,7 @@ lib = C.CDLL(_LIB_PATH)
 OK = 0
 BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
-EXPORTS = ["vatp_workspace_bytes", "vatp_prefill_scores", "vatp_select", "vatp_compact", "vatp_decode_step",
+EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_select", "vatp_compact", "vatp_decode_step",
            "vatp_status_string"]
 
 
@@ -36,6 +36,8 @@ class CacheStruct(C.Structure):
 
 
 _vp = C.c_void_p
+lib.vatp_cache_capacity.restype = C.c_int32
+lib.vatp_cache_capacity.argtypes = [C.c_int32]
 lib.vatp_workspace_bytes.restype = C.c_size_t
 lib.vatp_workspace_bytes.argtypes = [C.POINTER(Params)]
 lib.vatp_prefill_scores.restype = C.c_int
@@ -93,7 +95,7 @@ class Cache:
     """Device arrays of the decode state (allocated with torch, owned by this object)."""
 
     def __init__(self, p: Params, device="cuda"):
-        b, h, d, cap = p.batch, p.heads, p.head_dim, p.budget + 1
+        b, h, d, cap = p.batch, p.heads, p.head_dim, int(lib.vatp_cache_capacity(p.budget))
         dt = torch.float32 if p.dtype == F32 else torch.bfloat16
         self.cap = cap
         self.k_cache = torch.zeros(b, h, cap, d, dtype=dt, device=device)
