@@ -95,11 +95,12 @@ size_t vatp_workspace_bytes(const vatp_params* params);
  *           j >= max(T - w, k) (Eq. 3, last w queries); QK^T is recomputed, never stored
  *   vnorm[k] = sum_c |v[k][c]|,  score[k] = attn_acc[k] * vnorm[k]     (Eq. 4)
  * q, k, v: inputs as described above (read only).
- * lse_out:  [batch, heads, T] fp32, nullable (then the row normalisers live in the workspace).
+ * lse_out:  [batch, heads, T] fp32 output (natural log), nullable.
  * attn_acc, vnorm, score: [batch, heads, T] fp32 outputs.
  * win_rows: VATP_IND_WINDOW only: [batch, heads, w, T] fp32 output, row r = probabilities of
  *           query T - w + r (zero where masked or where T - w + r < 0); NULL for H2O.
- * workspace: >= vatp_workspace_bytes(params) bytes of device scratch, 256-byte aligned.
+ * workspace: >= vatp_workspace_bytes(params) bytes of device scratch, 256-byte aligned; holds the
+ *           row normalisers between the two passes.
  * bf16 with head_dim 128 runs on the tensor cores; other combinations use an fp32 FMA kernel.
  */
 vatp_status vatp_prefill_scores(const vatp_params* params, const void* q, const void* k, const void* v,

@@ -1,7 +1,495 @@
-// placeholder until the tcgen05 kernel lands
+// Tensor-core prefill scoring for bf16, head_dim 128 (sm_100a: tcgen05 MMA, TMEM accumulators, TMA).
+//
+// Two launches of one persistent kernel, never materialising the T x T matrix:
+//   pass 1  rows = 128 queries (fixed tile), streamed tiles = keys 0..diagonal:
+//           per query the running max and sum of exp2 give lse (the normaliser of Eq. 1);
+//   pass 2  rows = 128 keys (fixed tile), streamed tiles = queries diagonal..end: S^T = K Q^T is
+//           recomputed, every thread owns one key and adds exp2(s - lse_j) over the query columns
+//           of its TMEM lane (Eq. 2) - a per-thread running sum, no shuffles, no atomics - then
+//           multiplies by the value l1 norm computed by a side warp (Eq. 4).
+// Both operands are [token, d] row-major, i.e. K-major for A and B alike.
+//
+// Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two
+// softmax warpgroups that take alternate accumulators, warp 10 value-norm reduction.
+// Every wait is bounded; on expiry the CTA raises a flag, writes VATP_ERR_TIMEOUT to the status
+// word, drains, frees its TMEM and returns.
+#include <cuda.h>
+
 #include "vatp_internal.cuh"
+
 namespace vatp {
-bool vatp_tc_available() { return false; }
-cudaError_t launch_prefill_tc(const Shape&, const void*, const void*, const void*, float*, float*, float*, float*,
-                              float*, int32_t*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int TC_THREADS = 352;
+constexpr int TILE = 128;          // rows of the fixed tile = columns of a streamed tile
+constexpr int HD = 128;            // head_dim
+constexpr int NS = 4;              // streamed-tile stages in shared memory
+constexpr int NACC = 4;            // TMEM accumulators (128 columns each)
+constexpr int SLAB_BYTES = TILE * 128;        // 128 rows x 64 bf16, 128-byte swizzled
+constexpr int TILE_BYTES = 2 * SLAB_BYTES;    // two K halves
+constexpr uint64_t WAIT_NS = 1000000000ull;
+
+struct Smem {
+  alignas(1024) unsigned char fixed[2][TILE_BYTES];
+  alignas(1024) unsigned char stream[NS][TILE_BYTES];
+  float vn[2][TILE];
+  float part_a[2][TILE];   // pass 1: running max of warpgroup 1; pass 2: its column sums
+  float part_b[2][TILE];   // pass 1: running sum of warpgroup 1
+  alignas(8) uint64_t full[NS], empty[NS];
+  uint64_t fixed_full[2], fixed_empty[2];
+  uint64_t acc_full[NACC], acc_empty[NACC];
+  uint64_t comb_full[2], comb_empty[2];
+  uint64_t vn_full[2], vn_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(bar)), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(s32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t now_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this or another waiter ran out of time).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
+  if (mbar_try(bar, parity)) return true;
+  const uint64_t t0 = now_ns();
+  for (;;) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (now_ns() - t0 > WAIT_NS) {
+      *abort_flag = 1;
+      if (dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(s32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(s32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M 128, N 128.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t addr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(addr)
+      : "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+struct TcArgs {
+  int units, heads, T, nt, Tpad;
+  float scale_log2;
+  const __nv_bfloat16* v;
+  int64_t sb, sh, st;       // element strides of v
+  float* lse2;              // [units][Tpad] log2-domain row normalisers (+inf beyond T)
+  float* lse_out;           // [units][T] natural-log copy, nullable
+  float* attn_acc;
+  float* vnorm;
+  float* score;
+  int32_t* dev_status;
+};
+
+// Work items are (unit, fixed tile), longest first and dealt round-robin to the persistent CTAs.
+// PASS 1: fixed = query tile, streamed key tiles 0..tile.  PASS 2: fixed = key tile, streamed
+// query tiles tile..nt-1.
+template <int PASS>
+__device__ __forceinline__ void item_of(int id, const TcArgs& a, int& u, int& tile, int& s_first, int& s_count) {
+  const int r = id / a.units;
+  u = id - r * a.units;
+  if (PASS == 1) { tile = a.nt - 1 - r; s_first = 0; s_count = tile + 1; }
+  else           { tile = r;            s_first = tile; s_count = a.nt - tile; }
+}
+
+template <int PASS>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, TcArgs a) {
+  extern __shared__ unsigned char smem_raw[];
+  Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  volatile int* abort_flag = &sm.abort_flag;
+  const int items = a.units * a.nt;
+
+  if (tid == 0) {
+    for (int i = 0; i < NS; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sm.fixed_full[i], 1); mbar_init(&sm.fixed_empty[i], 1);
+      mbar_init(&sm.comb_full[i], 128); mbar_init(&sm.comb_empty[i], 128);
+      mbar_init(&sm.vn_full[i], 1); mbar_init(&sm.vn_empty[i], 128);
+    }
+    for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 4); }
+    sm.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (wid == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+
+  // the operand that stays fixed per item and the one that streams
+  const CUtensorMap* tm_fixed = PASS == 1 ? &tm_q : &tm_k;
+  const CUtensorMap* tm_stream = PASS == 1 ? &tm_k : &tm_q;
+
+  if (wid == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t n = 0, itl = 0;
+      for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+        int u, tile, s_first, s_count;
+        item_of<PASS>(id, a, u, tile, s_first, s_count);
+        const int b = u / a.heads, h = u - b * a.heads;
+        const int fb = itl & 1;
+        ok = mbar_wait(&sm.fixed_empty[fb], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        mbar_expect_tx(&sm.fixed_full[fb], TILE_BYTES);
+        tma_load_4d(sm.fixed[fb], tm_fixed, &sm.fixed_full[fb], 0, tile * TILE, h, b);
+        tma_load_4d(sm.fixed[fb] + SLAB_BYTES, tm_fixed, &sm.fixed_full[fb], 64, tile * TILE, h, b);
+        for (int s = 0; s < s_count; ++s, ++n) {
+          const int stg = n % NS;
+          ok = mbar_wait(&sm.empty[stg], ((n / NS) & 1) ^ 1, abort_flag, a.dev_status);
+          if (!ok) break;
+          mbar_expect_tx(&sm.full[stg], TILE_BYTES);
+          tma_load_4d(sm.stream[stg], tm_stream, &sm.full[stg], 0, (s_first + s) * TILE, h, b);
+          tma_load_4d(sm.stream[stg] + SLAB_BYTES, tm_stream, &sm.full[stg], 64, (s_first + s) * TILE, h, b);
+        }
+      }
+    }
+  } else if (wid == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t n = 0, itl = 0;
+      for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+        int u, tile, s_first, s_count;
+        item_of<PASS>(id, a, u, tile, s_first, s_count);
+        const int fb = itl & 1;
+        ok = mbar_wait(&sm.fixed_full[fb], (itl >> 1) & 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        const uint32_t fixed_addr = s32(sm.fixed[fb]);
+        for (int s = 0; s < s_count; ++s, ++n) {
+          const int stg = n % NS, ab = n % NACC;
+          ok = mbar_wait(&sm.full[stg], (n / NS) & 1, abort_flag, a.dev_status) &&
+               mbar_wait(&sm.acc_empty[ab], ((n / NACC) & 1) ^ 1, abort_flag, a.dev_status);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t stream_addr = s32(sm.stream[stg]);
+          const uint32_t d_addr = tmem + ab * TILE;
+#pragma unroll
+          for (int kk = 0; kk < HD / 16; ++kk) {
+            const uint32_t off = (kk / 4) * SLAB_BYTES + (kk % 4) * 32;
+            umma_bf16(d_addr, umma_desc(fixed_addr + off), umma_desc(stream_addr + off), kk > 0 ? 1u : 0u);
+          }
+          umma_commit(&sm.empty[stg]);      // the streamed tile may be overwritten once these MMAs have read it
+          umma_commit(&sm.acc_full[ab]);    // accumulator ready for the softmax warps
+        }
+        if (ok) umma_commit(&sm.fixed_empty[fb]);
+      }
+    }
+  } else if (wid < 10) {
+    // ------------------------------------------------------------------ softmax warpgroups
+    const int g = (wid - 2) >> 2;                 // warpgroup 0 or 1: alternate accumulators
+    const int quarter = wid & 3;                  // TMEM lanes this warp may touch
+    const int row = quarter * 32 + lane;          // row of the fixed tile = TMEM lane
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    bool ok = true;
+    uint32_t n = 0, itl = 0;
+    for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+      int u, tile, s_first, s_count;
+      item_of<PASS>(id, a, u, tile, s_first, s_count);
+      const int pi = itl & 1;
+      const uint32_t ipar = (itl >> 1) & 1;
+      const float* lse2_u = a.lse2 + (int64_t)u * a.Tpad;
+      float m_run = -INFINITY, l_run = 0.f;       // pass 1
+      float cs0 = 0.f, cs1 = 0.f, cs2 = 0.f, cs3 = 0.f;   // pass 2
+      for (int s = 0; s < s_count; ++s, ++n) {
+        if ((int)(n & 1) != g) continue;
+        const int ab = n % NACC;
+        ok = mbar_wait(&sm.acc_full[ab], (n / NACC) & 1, abort_flag, a.dev_status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const int st_tile = s_first + s;
+        const bool diag = st_tile == tile;
+#pragma unroll 1
+        for (int c0 = 0; c0 < TILE; c0 += 64) {
+          float x[64];
+          tmem_ld32(lane_addr + ab * TILE + c0, *reinterpret_cast<float(*)[32]>(&x[0]));
+          tmem_ld32(lane_addr + ab * TILE + c0 + 32, *reinterpret_cast<float(*)[32]>(&x[32]));
+          tmem_ld_wait();
+          if (c0 + 64 == TILE) {                  // accumulator fully read: hand it back to the MMA warp
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
+          }
+          if (PASS == 1) {
+            // x_i = scale_log2 * s_i over keys; causal: key <= query on the diagonal tile
+            float cmax = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 64; ++i) {
+              if (diag && c0 + i > row) x[i] = -INFINITY;
+              cmax = fmaxf(cmax, x[i]);
+            }
+            cmax *= a.scale_log2;                 // scale > 0 keeps the order
+            if (cmax > m_run) { l_run *= ex2(m_run - cmax); m_run = cmax; }
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 64; i += 4) {
+              a0 += ex2(fmaf(x[i], a.scale_log2, -m_run));
+              a1 += ex2(fmaf(x[i + 1], a.scale_log2, -m_run));
+              a2 += ex2(fmaf(x[i + 2], a.scale_log2, -m_run));
+              a3 += ex2(fmaf(x[i + 3], a.scale_log2, -m_run));
+            }
+            l_run += (a0 + a1) + (a2 + a3);
+          } else {
+            // p = exp2(scale_log2 * s - lse2[query]); causal: query >= key on the diagonal tile
+            const float4* lp = reinterpret_cast<const float4*>(lse2_u + st_tile * TILE + c0);
+#pragma unroll
+            for (int i = 0; i < 64; i += 4) {
+              const float4 L = __ldg(lp + (i >> 2));
+              float p0 = ex2(fmaf(x[i], a.scale_log2, -L.x));
+              float p1 = ex2(fmaf(x[i + 1], a.scale_log2, -L.y));
+              float p2 = ex2(fmaf(x[i + 2], a.scale_log2, -L.z));
+              float p3 = ex2(fmaf(x[i + 3], a.scale_log2, -L.w));
+              if (diag) {
+                if (c0 + i < row) p0 = 0.f;
+                if (c0 + i + 1 < row) p1 = 0.f;
+                if (c0 + i + 2 < row) p2 = 0.f;
+                if (c0 + i + 3 < row) p3 = 0.f;
+              }
+              cs0 += p0; cs1 += p1; cs2 += p2; cs3 += p3;
+            }
+          }
+        }
+      }
+      if (!ok) break;
+      // ---- end of item: warpgroup 1 hands its partial to warpgroup 0, which finishes the rows
+      const int tok = tile * TILE + row;           // query (pass 1) or key (pass 2) index of this thread
+      if (g == 1) {
+        ok = mbar_wait(&sm.comb_empty[pi], ipar ^ 1, abort_flag, a.dev_status);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        if (PASS == 1) { sm.part_a[pi][row] = m_run; sm.part_b[pi][row] = l_run; }
+        else           { sm.part_a[pi][row] = (cs0 + cs1) + (cs2 + cs3); }
+        mbar_arrive(&sm.comb_full[pi]);
+      } else {
+        ok = mbar_wait(&sm.comb_full[pi], ipar, abort_flag, a.dev_status);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        if (PASS == 1) {
+          const float m1 = sm.part_a[pi][row], l1 = sm.part_b[pi][row];
+          mbar_arrive(&sm.comb_empty[pi]);
+          const float m = fmaxf(m_run, m1);
+          float l = 0.f;
+          if (l_run > 0.f) l += l_run * ex2(m_run - m);
+          if (l1 > 0.f) l += l1 * ex2(m1 - m);
+          const float lse2 = m + log2f(l);
+          a.lse2[(int64_t)u * a.Tpad + tok] = tok < a.T ? lse2 : INFINITY;
+          if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
+        } else {
+          const float tot = ((cs0 + cs1) + (cs2 + cs3)) + sm.part_a[pi][row];
+          mbar_arrive(&sm.comb_empty[pi]);
+          ok = mbar_wait(&sm.vn_full[pi], ipar, abort_flag, a.dev_status);
+          if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+          const float n1 = sm.vn[pi][row];
+          mbar_arrive(&sm.vn_empty[pi]);
+          if (tok < a.T) {
+            const int64_t o = (int64_t)u * a.T + tok;
+            a.attn_acc[o] = tot;
+            a.vnorm[o] = n1;
+            a.score[o] = tot * n1;
+          }
+        }
+      }
+    }
+  } else if (PASS == 2) {
+    // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
+    bool ok = true;
+    uint32_t itl = 0;
+    for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+      int u, tile, s_first, s_count;
+      item_of<PASS>(id, a, u, tile, s_first, s_count);
+      const int pi = itl & 1;
+      ok = mbar_wait(&sm.vn_empty[pi], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
+      if (!__all_sync(0xffffffffu, ok)) break;
+      const int b = u / a.heads, h = u - b * a.heads;
+      const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
+      // 16 lanes per row, two rows per pass: coalesced 16-byte loads
+      const int sub = lane >> 4, part = lane & 15;
+      for (int r0 = 0; r0 < TILE; r0 += 8) {
+        float acc[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int tok = tile * TILE + r0 + 2 * j + sub;
+          acc[j] = 0.f;
+          if (tok < a.T) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              acc[j] += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+          for (int o = 8; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
+          if (part == 0) sm.vn[pi][r0 + 2 * j + sub] = acc[j];
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.vn_full[pi]);
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (sm.abort_flag) {
+    // give copies that may still be in flight time to land before the shared memory is released
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (wid == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+// ---- host side -------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+// [batch, heads, T, 128] bf16 with element strides (sb, sh, st, 1); box = 64 x 128 rows, 128-byte swizzle
+bool make_map(CUtensorMap* m, const void* base, const Shape& s) {
+  const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)s.T, (cuuint64_t)s.heads, (cuuint64_t)(s.units / s.heads)};
+  const cuuint64_t strides[3] = {(cuuint64_t)s.st * 2, (cuuint64_t)s.sh * 2, (cuuint64_t)s.sb * 2};
+  const cuuint32_t box[4] = {64, TILE, 1, 1};
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  return encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool vatp_tc_available() {
+  static int cached = -1;
+  if (cached < 0) {
+    int dev = 0, major = 0;
+    cached = cudaGetDevice(&dev) == cudaSuccess &&
+             cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10 &&
+             encode_fn() != nullptr;
+  }
+  return cached == 1;
+}
+
+size_t prefill_tc_workspace_bytes(int units, int T) {
+  const size_t Tpad = (size_t)(T + TILE - 1) / TILE * TILE;
+  return (size_t)units * Tpad * sizeof(float);
+}
+
+cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
+                              float* lse_out, float* attn_acc, float* vnorm, float* score, int32_t* dev_status,
+                              cudaStream_t st) {
+  CUtensorMap tm_q, tm_k;
+  if (!make_map(&tm_q, q, s) || !make_map(&tm_k, k, s)) return cudaErrorInvalidValue;
+  TcArgs a;
+  a.units = s.units; a.heads = s.heads; a.T = s.T;
+  a.nt = (s.T + TILE - 1) / TILE;
+  a.Tpad = a.nt * TILE;
+  a.scale_log2 = s.scale * 1.4426950408889634f;
+  a.v = static_cast<const __nv_bfloat16*>(v);
+  a.sb = s.sb; a.sh = s.sh; a.st = s.st;
+  a.lse2 = lse_ws; a.lse_out = lse_out; a.attn_acc = attn_acc; a.vnorm = vnorm; a.score = score;
+  a.dev_status = dev_status;
+  const size_t smem = sizeof(Smem) + 1024;
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int items = a.units * a.nt;
+  const int grid = items < sms ? items : sms;
+  prefill_tc_kernel<1><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  prefill_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  return cudaGetLastError();
+}
+
+}  // namespace vatp

@@ -40,8 +40,9 @@ vatp_status make_shape(const vatp_params* p, Shape* s) {
   return VATP_OK;
 }
 
+// row normalisers of pass 1, padded to whole 128-row tiles per unit
 inline size_t lse_bytes(const vatp_params* p) {
-  size_t n = (size_t)p->batch * p->heads * (size_t)p->seq_len * sizeof(float);
+  size_t n = prefill_tc_workspace_bytes(p->batch * p->heads, p->seq_len);
   return (n + 255) / 256 * 256;
 }
 
@@ -89,18 +90,15 @@ vatp_status vatp_prefill_scores(const vatp_params* p, const void* q, const void*
   Shape sh;
   s = make_shape(p, &sh);
   if (s != VATP_OK) return s;
-  float* lse = lse_out;
-  if (!lse) {
-    if (!workspace || workspace_bytes < lse_bytes(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
-      return VATP_ERR_WORKSPACE;
-    lse = static_cast<float*>(workspace);
-  }
+  if (!workspace || workspace_bytes < lse_bytes(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return VATP_ERR_WORKSPACE;
+  float* ws = static_cast<float*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e;
   if (p->dtype == VATP_BF16 && p->head_dim == 128 && !windowed && vatp_tc_available())
-    e = launch_prefill_tc(sh, q, k, v, lse, attn_acc, vnorm, score, win_rows, dev_status, st);
+    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, dev_status, st);
   else
-    e = launch_prefill_simt(sh, p->dtype, q, k, v, lse, attn_acc, vnorm, score, win_rows, st);
+    e = launch_prefill_simt(sh, p->dtype, q, k, v, lse_out ? lse_out : ws, attn_acc, vnorm, score, win_rows, st);
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
 
