@@ -191,7 +191,7 @@ def run_cuda(args, wl):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
-    L, steps_dec = LAYERS, wl.decode_steps
+    L, steps_dec = args.layers, wl.decode_steps
     layers = [LayerState(V, wl, l, dev) for l in range(L)]
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -270,10 +270,10 @@ def run_cuda(args, wl):
     pre_ms, dec_ms, all_ms = (stats / args.steps).tolist()
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
-    host = [[x.cpu().pin_memory() for x in (ls.q, ls.k, ls.v, ls.dq, ls.dk, ls.dv)] for ls in layers]
+    host = None if args.no_e2e else [[x.cpu().pin_memory() for x in (ls.q, ls.k, ls.v, ls.dq, ls.dk, ls.dv)] for ls in layers]
     host_kept = [torch.empty_like(ls.kept, device="cpu").pin_memory() for ls in layers]
     host_out = [torch.empty_like(ls.out, device="cpu").pin_memory() for ls in layers]
-    h2d = sum(x.numel() * x.element_size() for hl in host for x in hl)
+    h2d = sum(x.numel() * x.element_size() for hl in (host or []) for x in hl)
     d2h = sum(x.numel() * x.element_size() for x in host_kept + host_out)
 
     def e2e_step():
@@ -293,13 +293,15 @@ def run_cuda(args, wl):
         e2.record()
         return e0, e1, e2
 
-    e2e_step(); barrier()
-    e2e_recs = [e2e_step() for _ in range(max(2, min(args.steps, 5)))]
-    barrier()
-    e2e_pre = torch.tensor([statistics.mean(a.elapsed_time(b) for a, b, _ in e2e_recs)], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(e2e_pre, op=torch.distributed.ReduceOp.MAX)
-    e2e_dec_ms = statistics.mean(b.elapsed_time(c) for _, b, c in e2e_recs)
+    if host is not None:
+        e2e_step(); barrier()
+        e2e_recs = [e2e_step() for _ in range(max(2, min(args.steps, 5)))]
+        barrier()
+        e2e_pre = torch.tensor([statistics.mean(a.elapsed_time(b) for a, b, _ in e2e_recs)], dtype=torch.float64,
+                               device=dev)
+        if world > 1:
+            torch.distributed.all_reduce(e2e_pre, op=torch.distributed.ReduceOp.MAX)
+        e2e_dec_ms = statistics.mean(b.elapsed_time(c) for _, b, c in e2e_recs)
 
     if rank != 0:
         return
@@ -342,12 +344,14 @@ def run_cuda(args, wl):
         "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
         "config": {"workload": f"config1 {wl.name}: b{wl.batch} h{wl.heads} d{d} T{T} budget{B} recent{wl.n_recent} "
                                f"sinkF{wl.n_sink} h2o, {steps_dec} decode steps, x{L} independently seeded layers",
+                   "layers": L,
                    "l2": "256 MB flush write between steps; layer rotation keeps the decode state (277 MB) out of L2",
                    "replicas": "each GPU runs the whole workload (path does not shard within a call)",
                    "decode_graph": graph is not None},
         "prefill_ms_per_layer": pre_ms / L, "decode_us_per_layer_step": dec_us,
         "roofline": roof, "roofline_all": kernels,
-        "e2e": {"value": world * tokens / (float(e2e_pre.item()) * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": None if host is None else
+               {"value": world * tokens / (float(e2e_pre.item()) * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "decode_us_per_layer_step": e2e_dec_ms * 1e3 / (steps_dec * L)},
         "gpu_launches": args.steps * (L * 4 + steps_dec * L),
         "clocks": clocks,
@@ -373,9 +377,14 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch decode steps directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--layers", type=int, default=LAYERS, help="independently seeded layers held on the device")
+    ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps (profiling runs)")
     args = ap.parse_args()
     from paper_2406_12335_b200 import synth
     wl = synth.CONFIGS[1]
+    if args.decode_steps is not None:
+        wl = wl.with_(decode_steps=args.decode_steps)
     if args.impl == "reference":
         run_reference(args, wl)
     else:

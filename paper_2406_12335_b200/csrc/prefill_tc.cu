@@ -6,7 +6,7 @@
 //   pass 2  rows = 128 keys (fixed tile), streamed tiles = queries diagonal..end: S^T = K Q^T is
 //           recomputed, every thread owns one key and adds exp2(s - lse_j) over the query columns
 //           of its TMEM lane (Eq. 2) - a per-thread running sum, no shuffles, no atomics - then
-//           multiplies by the value l1 norm computed by a side warp (Eq. 4).
+//           multiplies by the value l1 norm (Eq. 4), which a side warp of pass 1 has reduced.
 // Both operands are [token, d] row-major, i.e. K-major for A and B alike.
 //
 // Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two
@@ -32,14 +32,13 @@ constexpr uint64_t WAIT_NS = 1000000000ull;
 struct Smem {
   alignas(1024) unsigned char fixed[2][TILE_BYTES];
   alignas(1024) unsigned char stream[NS][TILE_BYTES];
-  float vn[2][TILE];
   float part_a[2][TILE];   // pass 1: running max of warpgroup 1; pass 2: its column sums
   float part_b[2][TILE];   // pass 1: running sum of warpgroup 1
+  alignas(16) float lse_s[8][2][TILE];   // pass 2: per softmax warp, double-buffered normalisers of a query tile
   alignas(8) uint64_t full[NS], empty[NS];
   uint64_t fixed_full[2], fixed_empty[2];
   uint64_t acc_full[NACC], acc_empty[NACC];
   uint64_t comb_full[2], comb_empty[2];
-  uint64_t vn_full[2], vn_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -135,6 +134,61 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
+// One 32-column slice of an accumulator row.  x holds raw dot products; c0 is the slice's first
+// column inside the tile, row the thread's row.
+//   PASS 1 (row = query, columns = keys): online max / sum of exp2(scale_log2 * s); on the diagonal
+//           tile keys beyond the query are masked.
+//   PASS 2 (row = key, columns = queries): cs += exp2(scale_log2 * s - lse2[query]); on the diagonal
+//           tile queries before the key are masked.  lse_t: the tile's 128 normalisers in shared memory.
+template <int PASS, bool DIAG>
+__device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float scale_log2, float& m_run, float& l_run,
+                                          float (&cs)[4], const float* lse_t) {
+  if (PASS == 1) {
+    if (DIAG) {
+#pragma unroll
+      for (int i = 0; i < 32; ++i)
+        if (c0 + i > row) x[i] = -INFINITY;
+    }
+    float cmax = max3(x[0], x[1], x[2]);
+#pragma unroll
+    for (int i = 3; i + 1 < 32; i += 2) cmax = max3(cmax, x[i], x[i + 1]);
+    cmax = fmaxf(cmax, x[31]) * scale_log2;            // scale > 0 keeps the order
+    if (cmax > m_run) { l_run *= ex2(m_run - cmax); m_run = cmax; }
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+      a0 += ex2(fmaf(x[i], scale_log2, -m_run));
+      a1 += ex2(fmaf(x[i + 1], scale_log2, -m_run));
+      a2 += ex2(fmaf(x[i + 2], scale_log2, -m_run));
+      a3 += ex2(fmaf(x[i + 3], scale_log2, -m_run));
+    }
+    l_run += (a0 + a1) + (a2 + a3);
+  } else {
+    const float4* lp = reinterpret_cast<const float4*>(lse_t + c0);
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+      const float4 L = lp[i >> 2];
+      float p0 = ex2(fmaf(x[i], scale_log2, -L.x));
+      float p1 = ex2(fmaf(x[i + 1], scale_log2, -L.y));
+      float p2 = ex2(fmaf(x[i + 2], scale_log2, -L.z));
+      float p3 = ex2(fmaf(x[i + 3], scale_log2, -L.w));
+      if (DIAG) {
+        if (c0 + i < row) p0 = 0.f;
+        if (c0 + i + 1 < row) p1 = 0.f;
+        if (c0 + i + 2 < row) p2 = 0.f;
+        if (c0 + i + 3 < row) p3 = 0.f;
+      }
+      cs[0] += p0; cs[1] += p1; cs[2] += p2; cs[3] += p3;
+    }
+  }
+}
+
 struct TcArgs {
   int units, heads, T, nt, Tpad;
   float scale_log2;
@@ -151,6 +205,10 @@ struct TcArgs {
 // Work items are (unit, fixed tile), longest first and dealt round-robin to the persistent CTAs.
 // PASS 1: fixed = query tile, streamed key tiles 0..tile.  PASS 2: fixed = key tile, streamed
 // query tiles tile..nt-1.
+// id of the n-th item of CTA c: rounds alternate direction so that the longest-first order is dealt
+// like a snake draft (load spread within ~2% instead of ~14% for plain round-robin)
+__device__ __forceinline__ int item_id(int n, int c, int G) { return n * G + ((n & 1) ? G - 1 - c : c); }
+
 template <int PASS>
 __device__ __forceinline__ void item_of(int id, const TcArgs& a, int& u, int& tile, int& s_first, int& s_count) {
   const int r = id / a.units;
@@ -173,7 +231,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sm.fixed_full[i], 1); mbar_init(&sm.fixed_empty[i], 1);
       mbar_init(&sm.comb_full[i], 128); mbar_init(&sm.comb_empty[i], 128);
-      mbar_init(&sm.vn_full[i], 1); mbar_init(&sm.vn_empty[i], 128);
     }
     for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 4); }
     sm.abort_flag = 0;
@@ -198,7 +255,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (lane == 0) {
       bool ok = true;
       uint32_t n = 0, itl = 0;
-      for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+      for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
         int u, tile, s_first, s_count;
         item_of<PASS>(id, a, u, tile, s_first, s_count);
         const int b = u / a.heads, h = u - b * a.heads;
@@ -223,7 +280,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (lane == 0) {
       bool ok = true;
       uint32_t n = 0, itl = 0;
-      for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+      for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
         int u, tile, s_first, s_count;
         item_of<PASS>(id, a, u, tile, s_first, s_count);
         const int fb = itl & 1;
@@ -257,75 +314,83 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
     bool ok = true;
     uint32_t n = 0, itl = 0;
-    for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+    for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
       int u, tile, s_first, s_count;
       item_of<PASS>(id, a, u, tile, s_first, s_count);
       const int pi = itl & 1;
       const uint32_t ipar = (itl >> 1) & 1;
       const float* lse2_u = a.lse2 + (int64_t)u * a.Tpad;
+      // pass 2: this key's value norm, written by pass 1; fetched now, used in the item's epilogue
+      float n1 = 0.f;
+      if (PASS == 2 && g == 0 && tile * TILE + row < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tile * TILE + row);
       float m_run = -INFINITY, l_run = 0.f;       // pass 1
-      float cs0 = 0.f, cs1 = 0.f, cs2 = 0.f, cs3 = 0.f;   // pass 2
-      for (int s = 0; s < s_count; ++s, ++n) {
-        if ((int)(n & 1) != g) continue;
-        const int ab = n % NACC;
-        ok = mbar_wait(&sm.acc_full[ab], (n / NACC) & 1, abort_flag, a.dev_status);
-        ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+      float cs[4] = {0.f, 0.f, 0.f, 0.f};         // pass 2
+      // this warpgroup's tiles of the item: s = s0, s0 + 2, ... (running tile index n0 + s)
+      const uint32_t n0 = n;
+      n += s_count;
+      int s = ((n0 & 1u) == (uint32_t)g) ? 0 : 1;
+      float* lse_w = &sm.lse_s[wid - 2][0][0];
+      int buf = 0;
+      float xa[32], xb[32];
+      auto acc_of = [&](int ss) { return (int)((n0 + ss) % NACC); };
+      auto tile_wait = [&](int ss) -> bool {
+        bool w = mbar_wait(&sm.acc_full[acc_of(ss)], ((n0 + ss) / NACC) & 1, abort_flag, a.dev_status);
+        w = __all_sync(0xffffffffu, w);
         tc_fence_after();
-        const int st_tile = s_first + s;
-        const bool diag = st_tile == tile;
-#pragma unroll 1
-        for (int c0 = 0; c0 < TILE; c0 += 64) {
-          float x[64];
-          tmem_ld32(lane_addr + ab * TILE + c0, *reinterpret_cast<float(*)[32]>(&x[0]));
-          tmem_ld32(lane_addr + ab * TILE + c0 + 32, *reinterpret_cast<float(*)[32]>(&x[32]));
-          tmem_ld_wait();
-          if (c0 + 64 == TILE) {                  // accumulator fully read: hand it back to the MMA warp
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
-          }
-          if (PASS == 1) {
-            // x_i = scale_log2 * s_i over keys; causal: key <= query on the diagonal tile
-            float cmax = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < 64; ++i) {
-              if (diag && c0 + i > row) x[i] = -INFINITY;
-              cmax = fmaxf(cmax, x[i]);
-            }
-            cmax *= a.scale_log2;                 // scale > 0 keeps the order
-            if (cmax > m_run) { l_run *= ex2(m_run - cmax); m_run = cmax; }
-            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-            for (int i = 0; i < 64; i += 4) {
-              a0 += ex2(fmaf(x[i], a.scale_log2, -m_run));
-              a1 += ex2(fmaf(x[i + 1], a.scale_log2, -m_run));
-              a2 += ex2(fmaf(x[i + 2], a.scale_log2, -m_run));
-              a3 += ex2(fmaf(x[i + 3], a.scale_log2, -m_run));
-            }
-            l_run += (a0 + a1) + (a2 + a3);
-          } else {
-            // p = exp2(scale_log2 * s - lse2[query]); causal: query >= key on the diagonal tile
-            const float4* lp = reinterpret_cast<const float4*>(lse2_u + st_tile * TILE + c0);
-#pragma unroll
-            for (int i = 0; i < 64; i += 4) {
-              const float4 L = __ldg(lp + (i >> 2));
-              float p0 = ex2(fmaf(x[i], a.scale_log2, -L.x));
-              float p1 = ex2(fmaf(x[i + 1], a.scale_log2, -L.y));
-              float p2 = ex2(fmaf(x[i + 2], a.scale_log2, -L.z));
-              float p3 = ex2(fmaf(x[i + 3], a.scale_log2, -L.w));
-              if (diag) {
-                if (c0 + i < row) p0 = 0.f;
-                if (c0 + i + 1 < row) p1 = 0.f;
-                if (c0 + i + 2 < row) p2 = 0.f;
-                if (c0 + i + 3 < row) p3 = 0.f;
-              }
-              cs0 += p0; cs1 += p1; cs2 += p2; cs3 += p3;
-            }
-          }
+        return w;
+      };
+      if (s < s_count) {
+        ok = tile_wait(s);
+        if (!ok) break;
+        tmem_ld32(lane_addr + acc_of(s) * TILE, xa);
+        if (PASS == 2) {
+          reinterpret_cast<float4*>(lse_w)[lane] = __ldg(reinterpret_cast<const float4*>(lse2_u + (s_first + s) * TILE) + lane);
+          __syncwarp();
         }
+        tmem_ld_wait();
+      }
+      while (s < s_count) {
+        const bool diag = (s_first + s) == tile;
+        const bool has_next = s + 2 < s_count;
+        const uint32_t t_addr = lane_addr + acc_of(s) * TILE;
+        const float* lse_t = lse_w + buf * TILE;
+        float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (PASS == 2 && has_next)
+          lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + (s_first + s + 2) * TILE) + lane);
+        // software pipeline: the TMEM load of the next 32 columns is in flight while these are consumed
+        tmem_ld32(t_addr + 32, xb);
+        if (diag) consume32<PASS, true>(xa, 0, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        else      consume32<PASS, false>(xa, 0, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        tmem_ld_wait();
+        tmem_ld32(t_addr + 64, xa);
+        if (diag) consume32<PASS, true>(xb, 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        else      consume32<PASS, false>(xb, 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        tmem_ld_wait();
+        tmem_ld32(t_addr + 96, xb);
+        if (diag) consume32<PASS, true>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        else      consume32<PASS, false>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        tmem_ld_wait();
+        // accumulator fully read: hand it back to the MMA warp
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.acc_empty[acc_of(s)]);
+        if (has_next) {
+          ok = tile_wait(s + 2);
+          if (!ok) break;
+          tmem_ld32(lane_addr + acc_of(s + 2) * TILE, xa);
+        }
+        if (diag) consume32<PASS, true>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        else      consume32<PASS, false>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        if (PASS == 2 && has_next) {
+          reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
+          __syncwarp();
+        }
+        tmem_ld_wait();
+        s += 2;
+        buf ^= 1;
       }
       if (!ok) break;
+      const float cs0 = cs[0], cs1 = cs[1], cs2 = cs[2], cs3 = cs[3];
       // ---- end of item: warpgroup 1 hands its partial to warpgroup 0, which finishes the rows
       const int tok = tile * TILE + row;           // query (pass 1) or key (pass 2) index of this thread
       if (g == 1) {
@@ -350,56 +415,47 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         } else {
           const float tot = ((cs0 + cs1) + (cs2 + cs3)) + sm.part_a[pi][row];
           mbar_arrive(&sm.comb_empty[pi]);
-          ok = mbar_wait(&sm.vn_full[pi], ipar, abort_flag, a.dev_status);
-          if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-          const float n1 = sm.vn[pi][row];
-          mbar_arrive(&sm.vn_empty[pi]);
           if (tok < a.T) {
             const int64_t o = (int64_t)u * a.T + tok;
             a.attn_acc[o] = tot;
-            a.vnorm[o] = n1;
             a.score[o] = tot * n1;
           }
         }
       }
     }
-  } else if (PASS == 2) {
+  } else if (PASS == 1) {
     // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
-    bool ok = true;
+    // Independent of the attention work of this pass: every (unit, token tile) is an item exactly
+    // once, so this warp covers all tokens.  Pass 2 reads the norms back in its epilogue.
     uint32_t itl = 0;
-    for (int id = blockIdx.x; ok && id < items; id += gridDim.x, ++itl) {
+    for (int id = item_id(0, blockIdx.x, gridDim.x); id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
       int u, tile, s_first, s_count;
       item_of<PASS>(id, a, u, tile, s_first, s_count);
-      const int pi = itl & 1;
-      ok = mbar_wait(&sm.vn_empty[pi], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
-      if (!__all_sync(0xffffffffu, ok)) break;
       const int b = u / a.heads, h = u - b * a.heads;
       const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
-      // 16 lanes per row, two rows per pass: coalesced 16-byte loads
+      // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
       const int sub = lane >> 4, part = lane & 15;
-      for (int r0 = 0; r0 < TILE; r0 += 8) {
-        float acc[4];
+      for (int r0 = 0; r0 < TILE; r0 += 32) {
+        uint4 raw[16];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 16; ++j) {
           const int tok = tile * TILE + r0 + 2 * j + sub;
-          acc[j] = 0.f;
-          if (tok < a.T) {
-            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
-            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              acc[j] += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
-          }
+          raw[j] = make_uint4(0u, 0u, 0u, 0u);
+          if (tok < a.T) raw[j] = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
         }
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < 16; ++j) {
+          const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+          float acc = 0.f;
 #pragma unroll
-          for (int o = 8; o; o >>= 1) acc[j] += __shfl_xor_sync(0xffffffffu, acc[j], o);
-          if (part == 0) sm.vn[pi][r0 + 2 * j + sub] = acc[j];
+          for (int i = 0; i < 4; ++i)
+            acc += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
+#pragma unroll
+          for (int o = 8; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+          const int tok = tile * TILE + r0 + 2 * j + sub;
+          if (part == 0 && tok < a.T) a.vnorm[(int64_t)u * a.T + tok] = acc;
         }
       }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sm.vn_full[pi]);
     }
   }
 
