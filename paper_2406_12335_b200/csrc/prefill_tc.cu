@@ -10,7 +10,8 @@
 // Both operands are [token, d] row-major, i.e. K-major for A and B alike.
 //
 // Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two
-// softmax warpgroups that take alternate accumulators, warp 10 value-norm reduction.
+// softmax warpgroups (one per fixed tile of the item, two TMEM accumulators each), warp 10 the
+// value-norm reduction (pass 1 only).
 // Every wait is bounded; on expiry the CTA raises a flag, writes VATP_ERR_TIMEOUT to the status
 // word, drains, frees its TMEM and returns.
 #include <cuda.h>
@@ -28,17 +29,17 @@ constexpr int NACC = 4;            // TMEM accumulators (128 columns each)
 constexpr int SLAB_BYTES = TILE * 128;        // 128 rows x 64 bf16, 128-byte swizzled
 constexpr int TILE_BYTES = 2 * SLAB_BYTES;    // two K halves
 constexpr uint64_t WAIT_NS = 1000000000ull;
+#ifndef VATP_POLY_EVERY
+#define VATP_POLY_EVERY 4   // one exponential in this many goes to the FMA pipe (0 = none)
+#endif
 
 struct Smem {
-  alignas(1024) unsigned char fixed[2][TILE_BYTES];
+  alignas(1024) unsigned char fixed[2][TILE_BYTES];      // the item's two fixed tiles
   alignas(1024) unsigned char stream[NS][TILE_BYTES];
-  float part_a[2][TILE];   // pass 1: running max of warpgroup 1; pass 2: its column sums
-  float part_b[2][TILE];   // pass 1: running sum of warpgroup 1
   alignas(16) float lse_s[8][2][TILE];   // pass 2: per softmax warp, double-buffered normalisers of a query tile
   alignas(8) uint64_t full[NS], empty[NS];
-  uint64_t fixed_full[2], fixed_empty[2];
-  uint64_t acc_full[NACC], acc_empty[NACC];
-  uint64_t comb_full[2], comb_empty[2];
+  uint64_t fixed_full, fixed_empty;
+  uint64_t acc_full[NACC], acc_empty[NACC];  // accumulators 2f, 2f+1 belong to warpgroup f
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -68,16 +69,24 @@ __device__ __forceinline__ uint64_t now_ns() {
   return t;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this or another waiter ran out of time).
+// SLEEP_NS > 0 backs off between polls: used by the single-lane producer / MMA roles so that their
+// polling does not take issue slots from the softmax warps.
+template <int SLEEP_NS = 0>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int32_t* dev_status) {
   if (mbar_try(bar, parity)) return true;
-  const uint64_t t0 = now_ns();
-  for (;;) {
+  uint64_t t0 = 0;
+  for (uint32_t spins = 1;; ++spins) {
+    if (SLEEP_NS > 0) __nanosleep(SLEEP_NS);
     if (mbar_try(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (now_ns() - t0 > WAIT_NS) {
-      *abort_flag = 1;
-      if (dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
-      return false;
+    if ((spins & 255u) == 0) {
+      if (*abort_flag) return false;
+      const uint64_t now = now_ns();
+      if (t0 == 0) t0 = now;
+      if (now - t0 > WAIT_NS) {
+        *abort_flag = 1;
+        if (dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+        return false;
+      }
     }
   }
 }
@@ -96,13 +105,26 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
 // Instruction descriptor: D fp32, A and B bf16, both K-major, M 128, N 128.
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
 
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t accumulate) {
+// One 128 x 128 x 16 MMA.  ACC = false overwrites the accumulator, true adds to it.  Issued by a
+// single thread, so every instruction between two MMAs costs tensor-pipe time: the descriptors are
+// built once per tile and advanced by adding compile-time constants.
+template <bool ACC>
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "r"(accumulate)
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "n"(ACC ? 1 : 0)
       : "memory");
+}
+// descriptor offset (16-byte units) of the kk-th 16-element K step inside a two-slab tile
+__host__ __device__ constexpr uint64_t k_step_offset(int kk) { return (uint64_t)(((kk / 4) * SLAB_BYTES + (kk % 4) * 32) >> 4); }
+template <int KK>
+__device__ __forceinline__ void umma_tile(uint32_t d_addr, uint64_t da, uint64_t db) {
+  if constexpr (KK < HD / 16) {
+    umma_bf16<(KK > 0)>(d_addr, da + k_step_offset(KK), db + k_step_offset(KK));
+    umma_tile<KK + 1>(d_addr, da, db);
+  }
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s32(bar)) : "memory");
@@ -132,6 +154,26 @@ __device__ __forceinline__ float ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
+}
+
+// exp2 on the FMA pipe for x <= 0: round-to-nearest split x = n + f with f in [-0.5, 0.5] (adding
+// 1.5 * 2^23 leaves n in the low mantissa bits), a degree-3 minimax polynomial for 2^f (relative
+// error 7.5e-5) and an exponent-field add for 2^n.  The special-function unit issues 16 exp2 per
+// clock per SM, which bounds this kernel before the tensor pipe does; sending one element in four
+// here moves that share of the exponentials onto otherwise idle FMA issue slots.
+__device__ __forceinline__ float ex2_fma(float x) {
+  x = fmaxf(x, -126.f);
+  const float t = x + 12582912.f;
+  const float f = x - (t - 12582912.f);
+  const float p = fmaf(fmaf(fmaf(0.05517164617776871f, f, 0.2426111251115799f), f, 0.6932609677314758f), f,
+                       0.9999280571937561f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
+// i is the unrolled element index (a multiple of 4): compile-time choice of the pipe
+__device__ __forceinline__ float exp2_mixed(int i, float x) {
+  if (VATP_POLY_EVERY > 0 && ((i + 4) % VATP_POLY_EVERY) == 0) return ex2_fma(x);
+  return ex2(x);
 }
 
 __device__ __forceinline__ float max3(float a, float b, float c) {
@@ -166,7 +208,7 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
       a0 += ex2(fmaf(x[i], scale_log2, -m_run));
       a1 += ex2(fmaf(x[i + 1], scale_log2, -m_run));
       a2 += ex2(fmaf(x[i + 2], scale_log2, -m_run));
-      a3 += ex2(fmaf(x[i + 3], scale_log2, -m_run));
+      a3 += exp2_mixed(i, fmaf(x[i + 3], scale_log2, -m_run));
     }
     l_run += (a0 + a1) + (a2 + a3);
   } else {
@@ -177,7 +219,7 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
       float p0 = ex2(fmaf(x[i], scale_log2, -L.x));
       float p1 = ex2(fmaf(x[i + 1], scale_log2, -L.y));
       float p2 = ex2(fmaf(x[i + 2], scale_log2, -L.z));
-      float p3 = ex2(fmaf(x[i + 3], scale_log2, -L.w));
+      float p3 = exp2_mixed(i, fmaf(x[i + 3], scale_log2, -L.w));
       if (DIAG) {
         if (c0 + i < row) p0 = 0.f;
         if (c0 + i + 1 < row) p1 = 0.f;
@@ -190,7 +232,7 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
 }
 
 struct TcArgs {
-  int units, heads, T, nt, Tpad;
+  int units, heads, T, nt, np, Tpad;   // nt tiles of 128 tokens, np = ceil(nt / 2) pairs
   float scale_log2;
   const __nv_bfloat16* v;
   int64_t sb, sh, st;       // element strides of v
@@ -202,19 +244,33 @@ struct TcArgs {
   int32_t* dev_status;
 };
 
-// Work items are (unit, fixed tile), longest first and dealt round-robin to the persistent CTAs.
-// PASS 1: fixed = query tile, streamed key tiles 0..tile.  PASS 2: fixed = key tile, streamed
-// query tiles tile..nt-1.
-// id of the n-th item of CTA c: rounds alternate direction so that the longest-first order is dealt
-// like a snake draft (load spread within ~2% instead of ~14% for plain round-robin)
+// Work items are (unit, pair of adjacent fixed tiles = 256 rows), longest first, dealt to the
+// persistent CTAs like a snake draft (rounds alternate direction: load spread within a few percent).
+// Two fixed tiles share every streamed tile, which halves the L2 -> shared-memory traffic per flop;
+// softmax warpgroup f owns fixed tile 2 * pair + f, so nothing is combined across warpgroups.
+//   PASS 1: fixed = query tiles, streamed key tiles 0 .. last fixed tile (fixed tile ft needs st <= ft)
+//   PASS 2: fixed = key tiles, streamed query tiles first fixed tile .. nt-1 (needs st >= ft)
 __device__ __forceinline__ int item_id(int n, int c, int G) { return n * G + ((n & 1) ? G - 1 - c : c); }
 
+struct Item {
+  int u, pair, s_first, s_count;
+};
 template <int PASS>
-__device__ __forceinline__ void item_of(int id, const TcArgs& a, int& u, int& tile, int& s_first, int& s_count) {
+__device__ __forceinline__ Item item_of(int id, const TcArgs& a) {
+  Item it;
   const int r = id / a.units;
-  u = id - r * a.units;
-  if (PASS == 1) { tile = a.nt - 1 - r; s_first = 0; s_count = tile + 1; }
-  else           { tile = r;            s_first = tile; s_count = a.nt - tile; }
+  it.u = id - r * a.units;
+  if (PASS == 1) { it.pair = a.np - 1 - r; it.s_first = 0; it.s_count = min(2 * it.pair + 2, a.nt); }
+  else           { it.pair = r; it.s_first = 2 * r; it.s_count = a.nt - 2 * r; }
+  return it;
+}
+// streamed tiles (as indices s into the item's list) that fixed tile f of the item takes part in
+template <int PASS>
+__device__ __forceinline__ void active_range(const Item& it, int f, int nt, int& s_lo, int& s_hi) {
+  const int ft = 2 * it.pair + f;
+  if (ft >= nt) { s_lo = 0; s_hi = 0; return; }           // odd tail: the second fixed tile does not exist
+  if (PASS == 1) { s_lo = 0; s_hi = min(ft + 1, it.s_count); }
+  else           { s_lo = f; s_hi = it.s_count; }
 }
 
 template <int PASS>
@@ -224,14 +280,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   volatile int* abort_flag = &sm.abort_flag;
-  const int items = a.units * a.nt;
+  const int items = a.units * a.np;
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(&sm.fixed_full[i], 1); mbar_init(&sm.fixed_empty[i], 1);
-      mbar_init(&sm.comb_full[i], 128); mbar_init(&sm.comb_empty[i], 128);
-    }
+    mbar_init(&sm.fixed_full, 1);
+    mbar_init(&sm.fixed_empty, 1);
     for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 4); }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -256,23 +310,32 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       bool ok = true;
       uint32_t n = 0, itl = 0;
       for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
-        int u, tile, s_first, s_count;
-        item_of<PASS>(id, a, u, tile, s_first, s_count);
-        const int b = u / a.heads, h = u - b * a.heads;
-        const int fb = itl & 1;
-        ok = mbar_wait(&sm.fixed_empty[fb], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
-        if (!ok) break;
-        mbar_expect_tx(&sm.fixed_full[fb], TILE_BYTES);
-        tma_load_4d(sm.fixed[fb], tm_fixed, &sm.fixed_full[fb], 0, tile * TILE, h, b);
-        tma_load_4d(sm.fixed[fb] + SLAB_BYTES, tm_fixed, &sm.fixed_full[fb], 64, tile * TILE, h, b);
-        for (int s = 0; s < s_count; ++s, ++n) {
+        const Item it = item_of<PASS>(id, a);
+        const int b = it.u / a.heads, h = it.u - b * a.heads;
+        auto issue_stream = [&](int s) -> bool {
           const int stg = n % NS;
-          ok = mbar_wait(&sm.empty[stg], ((n / NS) & 1) ^ 1, abort_flag, a.dev_status);
-          if (!ok) break;
+          if (!mbar_wait<20>(&sm.empty[stg], ((n / NS) & 1) ^ 1, abort_flag, a.dev_status)) return false;
           mbar_expect_tx(&sm.full[stg], TILE_BYTES);
-          tma_load_4d(sm.stream[stg], tm_stream, &sm.full[stg], 0, (s_first + s) * TILE, h, b);
-          tma_load_4d(sm.stream[stg] + SLAB_BYTES, tm_stream, &sm.full[stg], 64, (s_first + s) * TILE, h, b);
+          tma_load_4d(sm.stream[stg], tm_stream, &sm.full[stg], 0, (it.s_first + s) * TILE, h, b);
+          tma_load_4d(sm.stream[stg] + SLAB_BYTES, tm_stream, &sm.full[stg], 64, (it.s_first + s) * TILE, h, b);
+          ++n;
+          return true;
+        };
+        // the first streamed tiles go out before the fixed tiles: their stages free up while the
+        // previous item's last MMAs (which still read the fixed tiles) are running
+        const int pre = min(NS - 1, it.s_count);
+        int s = 0;
+        for (; ok && s < pre; ++s) ok = issue_stream(s);
+        if (!ok) break;
+        ok = mbar_wait<20>(&sm.fixed_empty, (itl & 1) ^ 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        mbar_expect_tx(&sm.fixed_full, 2 * TILE_BYTES);
+#pragma unroll
+        for (int f = 0; f < 2; ++f) {   // rows beyond T are zero-filled, a tile wholly beyond T too
+          tma_load_4d(sm.fixed[f], tm_fixed, &sm.fixed_full, 0, (2 * it.pair + f) * TILE, h, b);
+          tma_load_4d(sm.fixed[f] + SLAB_BYTES, tm_fixed, &sm.fixed_full, 64, (2 * it.pair + f) * TILE, h, b);
         }
+        for (; ok && s < it.s_count; ++s) ok = issue_stream(s);
       }
     }
   } else if (wid == 1) {
@@ -280,104 +343,118 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (lane == 0) {
       bool ok = true;
       uint32_t n = 0, itl = 0;
+      uint32_t used[2] = {0, 0};        // accumulators handed to warpgroup f so far
+      const uint64_t stage_desc0 = umma_desc(s32(sm.stream[0]));   // stages are TILE_BYTES apart
+      const uint64_t fixed_desc0 = umma_desc(s32(sm.fixed[0]));
       for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
-        int u, tile, s_first, s_count;
-        item_of<PASS>(id, a, u, tile, s_first, s_count);
-        const int fb = itl & 1;
-        ok = mbar_wait(&sm.fixed_full[fb], (itl >> 1) & 1, abort_flag, a.dev_status);
+        const Item it = item_of<PASS>(id, a);
+        int lo[2], hi[2];
+        active_range<PASS>(it, 0, a.nt, lo[0], hi[0]);
+        active_range<PASS>(it, 1, a.nt, lo[1], hi[1]);
+        ok = mbar_wait(&sm.fixed_full, itl & 1, abort_flag, a.dev_status);
         if (!ok) break;
-        const uint32_t fixed_addr = s32(sm.fixed[fb]);
-        for (int s = 0; s < s_count; ++s, ++n) {
-          const int stg = n % NS, ab = n % NACC;
-          ok = mbar_wait(&sm.full[stg], (n / NS) & 1, abort_flag, a.dev_status) &&
-               mbar_wait(&sm.acc_empty[ab], ((n / NACC) & 1) ^ 1, abort_flag, a.dev_status);
+        for (int s = 0; s < it.s_count; ++s, ++n) {
+          const int stg = n % NS;
+          ok = mbar_wait(&sm.full[stg], (n / NS) & 1, abort_flag, a.dev_status);
           if (!ok) break;
-          tc_fence_after();
-          const uint32_t stream_addr = s32(sm.stream[stg]);
-          const uint32_t d_addr = tmem + ab * TILE;
+          const uint64_t stream_desc = stage_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
 #pragma unroll
-          for (int kk = 0; kk < HD / 16; ++kk) {
-            const uint32_t off = (kk / 4) * SLAB_BYTES + (kk % 4) * 32;
-            umma_bf16(d_addr, umma_desc(fixed_addr + off), umma_desc(stream_addr + off), kk > 0 ? 1u : 0u);
+          for (int f = 0; f < 2; ++f) {
+            if (s < lo[f] || s >= hi[f]) continue;
+            const int ab = f * 2 + (used[f] & 1);
+            ok = mbar_wait(&sm.acc_empty[ab], ((used[f] >> 1) & 1) ^ 1, abort_flag, a.dev_status);
+            if (!ok) break;
+            tc_fence_after();
+            umma_tile<0>(tmem + ab * TILE, fixed_desc0 + (uint64_t)f * (TILE_BYTES >> 4), stream_desc);
+            umma_commit(&sm.acc_full[ab]);  // accumulator ready for warpgroup f
+            ++used[f];
           }
+          if (!ok) break;
           umma_commit(&sm.empty[stg]);      // the streamed tile may be overwritten once these MMAs have read it
-          umma_commit(&sm.acc_full[ab]);    // accumulator ready for the softmax warps
         }
-        if (ok) umma_commit(&sm.fixed_empty[fb]);
+        if (ok) umma_commit(&sm.fixed_empty);
       }
     }
   } else if (wid < 10) {
     // ------------------------------------------------------------------ softmax warpgroups
-    const int g = (wid - 2) >> 2;                 // warpgroup 0 or 1: alternate accumulators
+    const int f = (wid - 2) >> 2;                 // warpgroup f owns fixed tile 2 * pair + f
     const int quarter = wid & 3;                  // TMEM lanes this warp may touch
     const int row = quarter * 32 + lane;          // row of the fixed tile = TMEM lane
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    float* lse_w = &sm.lse_s[wid - 2][0][0];
     bool ok = true;
-    uint32_t n = 0, itl = 0;
+    uint32_t used = 0, itl = 0;                   // accumulators consumed so far (same count as the MMA warp keeps)
     for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
-      int u, tile, s_first, s_count;
-      item_of<PASS>(id, a, u, tile, s_first, s_count);
-      const int pi = itl & 1;
-      const uint32_t ipar = (itl >> 1) & 1;
+      const Item it = item_of<PASS>(id, a);
+      const int u = it.u;
+      const int ft = 2 * it.pair + f;             // this warpgroup's fixed tile
+      int s_lo, s_hi;
+      active_range<PASS>(it, f, a.nt, s_lo, s_hi);
+      if (s_lo >= s_hi) continue;                 // tile beyond the sequence: nothing to do, nothing to write
+      const int tok = ft * TILE + row;            // query (pass 1) or key (pass 2) index of this thread
       const float* lse2_u = a.lse2 + (int64_t)u * a.Tpad;
       // pass 2: this key's value norm, written by pass 1; fetched now, used in the item's epilogue
       float n1 = 0.f;
-      if (PASS == 2 && g == 0 && tile * TILE + row < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tile * TILE + row);
+      if (PASS == 2 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tok);
       float m_run = -INFINITY, l_run = 0.f;       // pass 1
       float cs[4] = {0.f, 0.f, 0.f, 0.f};         // pass 2
-      // this warpgroup's tiles of the item: s = s0, s0 + 2, ... (running tile index n0 + s)
-      const uint32_t n0 = n;
-      n += s_count;
-      int s = ((n0 & 1u) == (uint32_t)g) ? 0 : 1;
-      float* lse_w = &sm.lse_s[wid - 2][0][0];
       int buf = 0;
       float xa[32], xb[32];
-      auto acc_of = [&](int ss) { return (int)((n0 + ss) % NACC); };
-      auto tile_wait = [&](int ss) -> bool {
-        bool w = mbar_wait(&sm.acc_full[acc_of(ss)], ((n0 + ss) / NACC) & 1, abort_flag, a.dev_status);
+      auto acc_of = [&](uint32_t k) { return (int)(f * 2 + (k & 1)); };
+      auto tile_wait = [&](uint32_t k) -> bool {
+        bool w = mbar_wait(&sm.acc_full[acc_of(k)], (k >> 1) & 1, abort_flag, a.dev_status);
         w = __all_sync(0xffffffffu, w);
         tc_fence_after();
         return w;
       };
-      if (s < s_count) {
-        ok = tile_wait(s);
-        if (!ok) break;
-        tmem_ld32(lane_addr + acc_of(s) * TILE, xa);
-        if (PASS == 2) {
-          reinterpret_cast<float4*>(lse_w)[lane] = __ldg(reinterpret_cast<const float4*>(lse2_u + (s_first + s) * TILE) + lane);
-          __syncwarp();
-        }
-        tmem_ld_wait();
+      int s = s_lo;
+      ok = tile_wait(used);
+      if (!ok) break;
+      tmem_ld32(lane_addr + acc_of(used) * TILE, xa);
+      if (PASS == 2) {
+        reinterpret_cast<float4*>(lse_w)[lane] = __ldg(reinterpret_cast<const float4*>(lse2_u + (it.s_first + s) * TILE) + lane);
+        __syncwarp();
       }
-      while (s < s_count) {
-        const bool diag = (s_first + s) == tile;
-        const bool has_next = s + 2 < s_count;
-        const uint32_t t_addr = lane_addr + acc_of(s) * TILE;
+      tmem_ld_wait();
+      while (s < s_hi) {
+        const bool diag = (it.s_first + s) == ft;
+        const bool has_next = s + 1 < s_hi;
+        const uint32_t t_addr = lane_addr + acc_of(used) * TILE;
         const float* lse_t = lse_w + buf * TILE;
         float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
         if (PASS == 2 && has_next)
-          lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + (s_first + s + 2) * TILE) + lane);
-        // software pipeline: the TMEM load of the next 32 columns is in flight while these are consumed
-        tmem_ld32(t_addr + 32, xb);
-        if (diag) consume32<PASS, true>(xa, 0, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        else      consume32<PASS, false>(xa, 0, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        tmem_ld_wait();
-        tmem_ld32(t_addr + 64, xa);
-        if (diag) consume32<PASS, true>(xb, 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        else      consume32<PASS, false>(xb, 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        tmem_ld_wait();
-        tmem_ld32(t_addr + 96, xb);
-        if (diag) consume32<PASS, true>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        else      consume32<PASS, false>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        tmem_ld_wait();
+          lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + (it.s_first + s + 1) * TILE) + lane);
+        if (!diag) {
+          // software pipeline: the TMEM load of the next 32 columns is in flight while these are consumed
+          tmem_ld32(t_addr + 32, xb);
+          consume32<PASS, false>(xa, 0, row, a.scale_log2, m_run, l_run, cs, lse_t);
+          tmem_ld_wait();
+          tmem_ld32(t_addr + 64, xa);
+          consume32<PASS, false>(xb, 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
+          tmem_ld_wait();
+          tmem_ld32(t_addr + 96, xb);
+          consume32<PASS, false>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
+          tmem_ld_wait();
+        } else {
+          // the one diagonal tile of an item takes the masked variant, kept compact (not pipelined)
+#pragma unroll 1
+          for (int c0 = 0; c0 < 64; c0 += 32) {
+            consume32<PASS, true>(xa, c0, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            tmem_ld32(t_addr + c0 + 32, xa);
+            tmem_ld_wait();
+          }
+          tmem_ld32(t_addr + 96, xb);
+          consume32<PASS, true>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
+          tmem_ld_wait();
+        }
         // accumulator fully read: hand it back to the MMA warp
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.acc_empty[acc_of(s)]);
+        if (lane == 0) mbar_arrive(&sm.acc_empty[acc_of(used)]);
         if (has_next) {
-          ok = tile_wait(s + 2);
+          ok = tile_wait(used + 1);
           if (!ok) break;
-          tmem_ld32(lane_addr + acc_of(s + 2) * TILE, xa);
+          tmem_ld32(lane_addr + acc_of(used + 1) * TILE, xa);
         }
         if (diag) consume32<PASS, true>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
         else      consume32<PASS, false>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
@@ -386,60 +463,39 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           __syncwarp();
         }
         tmem_ld_wait();
-        s += 2;
+        ++s;
+        ++used;
         buf ^= 1;
       }
       if (!ok) break;
-      const float cs0 = cs[0], cs1 = cs[1], cs2 = cs[2], cs3 = cs[3];
-      // ---- end of item: warpgroup 1 hands its partial to warpgroup 0, which finishes the rows
-      const int tok = tile * TILE + row;           // query (pass 1) or key (pass 2) index of this thread
-      if (g == 1) {
-        ok = mbar_wait(&sm.comb_empty[pi], ipar ^ 1, abort_flag, a.dev_status);
-        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-        if (PASS == 1) { sm.part_a[pi][row] = m_run; sm.part_b[pi][row] = l_run; }
-        else           { sm.part_a[pi][row] = (cs0 + cs1) + (cs2 + cs3); }
-        mbar_arrive(&sm.comb_full[pi]);
-      } else {
-        ok = mbar_wait(&sm.comb_full[pi], ipar, abort_flag, a.dev_status);
-        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-        if (PASS == 1) {
-          const float m1 = sm.part_a[pi][row], l1 = sm.part_b[pi][row];
-          mbar_arrive(&sm.comb_empty[pi]);
-          const float m = fmaxf(m_run, m1);
-          float l = 0.f;
-          if (l_run > 0.f) l += l_run * ex2(m_run - m);
-          if (l1 > 0.f) l += l1 * ex2(m1 - m);
-          const float lse2 = m + log2f(l);
-          a.lse2[(int64_t)u * a.Tpad + tok] = tok < a.T ? lse2 : INFINITY;
-          if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
-        } else {
-          const float tot = ((cs0 + cs1) + (cs2 + cs3)) + sm.part_a[pi][row];
-          mbar_arrive(&sm.comb_empty[pi]);
-          if (tok < a.T) {
-            const int64_t o = (int64_t)u * a.T + tok;
-            a.attn_acc[o] = tot;
-            a.score[o] = tot * n1;
-          }
-        }
+      // ---- end of item: this thread's row is complete
+      if (PASS == 1) {
+        const float lse2 = m_run + log2f(l_run);
+        a.lse2[(int64_t)u * a.Tpad + tok] = tok < a.T ? lse2 : INFINITY;
+        if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
+      } else if (tok < a.T) {
+        const float tot = (cs[0] + cs[1]) + (cs[2] + cs[3]);
+        const int64_t o = (int64_t)u * a.T + tok;
+        a.attn_acc[o] = tot;
+        a.score[o] = tot * n1;
       }
     }
   } else if (PASS == 1) {
     // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
-    // Independent of the attention work of this pass: every (unit, token tile) is an item exactly
-    // once, so this warp covers all tokens.  Pass 2 reads the norms back in its epilogue.
+    // Independent of the attention work of this pass: every (unit, pair of token tiles) is an item
+    // exactly once, so this warp covers all tokens.  Pass 2 reads the norms back in its epilogue.
     uint32_t itl = 0;
     for (int id = item_id(0, blockIdx.x, gridDim.x); id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
-      int u, tile, s_first, s_count;
-      item_of<PASS>(id, a, u, tile, s_first, s_count);
-      const int b = u / a.heads, h = u - b * a.heads;
+      const Item it = item_of<PASS>(id, a);
+      const int b = it.u / a.heads, h = it.u - b * a.heads;
       const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
       // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
       const int sub = lane >> 4, part = lane & 15;
-      for (int r0 = 0; r0 < TILE; r0 += 32) {
+      for (int r0 = 0; r0 < 2 * TILE; r0 += 32) {
         uint4 raw[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const int tok = tile * TILE + r0 + 2 * j + sub;
+          const int tok = it.pair * 2 * TILE + r0 + 2 * j + sub;
           raw[j] = make_uint4(0u, 0u, 0u, 0u);
           if (tok < a.T) raw[j] = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
         }
@@ -452,8 +508,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             acc += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
 #pragma unroll
           for (int o = 8; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-          const int tok = tile * TILE + r0 + 2 * j + sub;
-          if (part == 0 && tok < a.T) a.vnorm[(int64_t)u * a.T + tok] = acc;
+          const int tok = it.pair * 2 * TILE + r0 + 2 * j + sub;
+          if (part == 0 && tok < a.T) a.vnorm[(int64_t)it.u * a.T + tok] = acc;
         }
       }
     }
@@ -528,6 +584,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   TcArgs a;
   a.units = s.units; a.heads = s.heads; a.T = s.T;
   a.nt = (s.T + TILE - 1) / TILE;
+  a.np = (a.nt + 1) / 2;
   a.Tpad = a.nt * TILE;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.v = static_cast<const __nv_bfloat16*>(v);
@@ -541,7 +598,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int items = a.units * a.nt;
+  const int items = a.units * a.np;
   const int grid = items < sms ? items : sms;
   prefill_tc_kernel<1><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   prefill_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
