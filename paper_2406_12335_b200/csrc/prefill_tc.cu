@@ -10,7 +10,7 @@
 // Both operands are [token, d] row-major, i.e. K-major for A and B alike.
 //
 // Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two
-// softmax warpgroups (one per fixed tile of the item, two TMEM accumulators each), warp 10 the
+// softmax warpgroups (each takes one 128-column half of every 256-column accumulator), warp 10 the
 // value-norm reduction (pass 1 only).
 // Every wait is bounded; on expiry the CTA raises a flag, writes VATP_ERR_TIMEOUT to the status
 // word, drains, frees its TMEM and returns.
@@ -24,22 +24,27 @@ namespace {
 constexpr int TC_THREADS = 352;
 constexpr int TILE = 128;          // rows of the fixed tile = columns of a streamed tile
 constexpr int HD = 128;            // head_dim
-constexpr int NS = 4;              // streamed-tile stages in shared memory
-constexpr int NACC = 4;            // TMEM accumulators (128 columns each)
+constexpr int CHUNK = 256;         // streamed tokens per stage = columns of an accumulator
+constexpr int NS = 2;              // streamed-chunk stages in shared memory
+constexpr int NACC = 2;            // TMEM accumulators (256 columns each)
 constexpr int SLAB_BYTES = TILE * 128;        // 128 rows x 64 bf16, 128-byte swizzled
 constexpr int TILE_BYTES = 2 * SLAB_BYTES;    // two K halves
+constexpr int CHUNK_BYTES = 2 * TILE_BYTES;   // 256 rows, two K halves
 constexpr uint64_t WAIT_NS = 1000000000ull;
 #ifndef VATP_POLY_EVERY
 #define VATP_POLY_EVERY 4   // one exponential in this many goes to the FMA pipe (0 = none)
 #endif
 
 struct Smem {
-  alignas(1024) unsigned char fixed[2][TILE_BYTES];      // the item's two fixed tiles
-  alignas(1024) unsigned char stream[NS][TILE_BYTES];
+  alignas(1024) unsigned char fixed[2][TILE_BYTES];      // double-buffered fixed tile
+  alignas(1024) unsigned char stream[NS][CHUNK_BYTES];   // [K half][256 rows][128 bytes] per stage
   alignas(16) float lse_s[8][2][TILE];   // pass 2: per softmax warp, double-buffered normalisers of a query tile
+  float part_a[2][TILE];   // pass 1: running max of warpgroup 1; pass 2: its column sums
+  float part_b[2][TILE];   // pass 1: running sum of warpgroup 1
   alignas(8) uint64_t full[NS], empty[NS];
-  uint64_t fixed_full, fixed_empty;
-  uint64_t acc_full[NACC], acc_empty[NACC];  // accumulators 2f, 2f+1 belong to warpgroup f
+  uint64_t fixed_full[2], fixed_empty[2];
+  uint64_t acc_full[NACC], acc_empty[NACC];
+  uint64_t comb_full[2], comb_empty[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -102,28 +107,33 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
 __device__ __forceinline__ uint64_t umma_desc(uint32_t smem_addr) {
   return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M 128, N 128.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TILE >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M 128, N 128 or 256.
+template <int N>
+__host__ __device__ constexpr uint32_t idesc() {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(TILE >> 4) << 24);
+}
 
-// One 128 x 128 x 16 MMA.  ACC = false overwrites the accumulator, true adds to it.  Issued by a
+// One 128 x N x 16 MMA.  ACC = false overwrites the accumulator, true adds to it.  Issued by a
 // single thread, so every instruction between two MMAs costs tensor-pipe time: the descriptors are
 // built once per tile and advanced by adding compile-time constants.
-template <bool ACC>
+template <bool ACC, int N>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(da), "l"(db), "r"(IDESC), "n"(ACC ? 1 : 0)
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc<N>()), "n"(ACC ? 1 : 0)
       : "memory");
 }
-// descriptor offset (16-byte units) of the kk-th 16-element K step inside a two-slab tile
-__host__ __device__ constexpr uint64_t k_step_offset(int kk) { return (uint64_t)(((kk / 4) * SLAB_BYTES + (kk % 4) * 32) >> 4); }
-template <int KK>
+// Descriptor offsets (16-byte units) of the kk-th 16-element K step.  The fixed tile is two slabs of
+// 128 rows; a streamed chunk is two slabs of 256 rows.
+__host__ __device__ constexpr uint64_t k_off_fixed(int kk) { return (uint64_t)(((kk / 4) * SLAB_BYTES + (kk % 4) * 32) >> 4); }
+__host__ __device__ constexpr uint64_t k_off_stream(int kk) { return (uint64_t)(((kk / 4) * 2 * SLAB_BYTES + (kk % 4) * 32) >> 4); }
+template <int KK, int N>
 __device__ __forceinline__ void umma_tile(uint32_t d_addr, uint64_t da, uint64_t db) {
   if constexpr (KK < HD / 16) {
-    umma_bf16<(KK > 0)>(d_addr, da + k_step_offset(KK), db + k_step_offset(KK));
-    umma_tile<KK + 1>(d_addr, da, db);
+    umma_bf16<(KK > 0), N>(d_addr, da + k_off_fixed(KK), db + k_off_stream(KK));
+    umma_tile<KK + 1, N>(d_addr, da, db);
   }
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
@@ -232,7 +242,7 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
 }
 
 struct TcArgs {
-  int units, heads, T, nt, np, Tpad;   // nt tiles of 128 tokens, np = ceil(nt / 2) pairs
+  int units, heads, T, nt, nch, Tpad;  // nt tiles of 128 tokens, nch = ceil(nt / 2) chunks, Tpad = 256 nch
   float scale_log2;
   const __nv_bfloat16* v;
   int64_t sb, sh, st;       // element strides of v
@@ -244,33 +254,32 @@ struct TcArgs {
   int32_t* dev_status;
 };
 
-// Work items are (unit, pair of adjacent fixed tiles = 256 rows), longest first, dealt to the
-// persistent CTAs like a snake draft (rounds alternate direction: load spread within a few percent).
-// Two fixed tiles share every streamed tile, which halves the L2 -> shared-memory traffic per flop;
-// softmax warpgroup f owns fixed tile 2 * pair + f, so nothing is combined across warpgroups.
-//   PASS 1: fixed = query tiles, streamed key tiles 0 .. last fixed tile (fixed tile ft needs st <= ft)
-//   PASS 2: fixed = key tiles, streamed query tiles first fixed tile .. nt-1 (needs st >= ft)
+// Work items are (unit, fixed tile of 128 rows), longest first, dealt to the persistent CTAs like a
+// snake draft (rounds alternate direction: load spread within a few percent).  The other operand
+// streams in chunks of 256 tokens (two tiles), so that one MMA instruction is 128 x 256 x 16: a
+// single thread issues the MMAs, and at 128 x 128 x 16 the issue cost exceeds the execution time.
+//   PASS 1: fixed = query tile i, streamed key chunks 0 .. i/2       (key tile kt needed iff kt <= i)
+//   PASS 2: fixed = key tile i, streamed query chunks i/2 .. nch-1   (query tile qt needed iff i <= qt < nt)
+// Softmax warpgroup g takes columns [128 g, 128 g + 128) of every accumulator, i.e. streamed tile
+// 2 c + g of chunk c; the two partial results of a row are combined once per item.
 __device__ __forceinline__ int item_id(int n, int c, int G) { return n * G + ((n & 1) ? G - 1 - c : c); }
 
 struct Item {
-  int u, pair, s_first, s_count;
+  int u, tile, c_first, c_count;
 };
 template <int PASS>
 __device__ __forceinline__ Item item_of(int id, const TcArgs& a) {
   Item it;
   const int r = id / a.units;
   it.u = id - r * a.units;
-  if (PASS == 1) { it.pair = a.np - 1 - r; it.s_first = 0; it.s_count = min(2 * it.pair + 2, a.nt); }
-  else           { it.pair = r; it.s_first = 2 * r; it.s_count = a.nt - 2 * r; }
+  if (PASS == 1) { it.tile = a.nt - 1 - r; it.c_first = 0; it.c_count = it.tile / 2 + 1; }
+  else           { it.tile = r; it.c_first = r / 2; it.c_count = a.nch - r / 2; }
   return it;
 }
-// streamed tiles (as indices s into the item's list) that fixed tile f of the item takes part in
+// is streamed tile st (= 2 * chunk + half) needed by the item?
 template <int PASS>
-__device__ __forceinline__ void active_range(const Item& it, int f, int nt, int& s_lo, int& s_hi) {
-  const int ft = 2 * it.pair + f;
-  if (ft >= nt) { s_lo = 0; s_hi = 0; return; }           // odd tail: the second fixed tile does not exist
-  if (PASS == 1) { s_lo = 0; s_hi = min(ft + 1, it.s_count); }
-  else           { s_lo = f; s_hi = it.s_count; }
+__device__ __forceinline__ bool tile_needed(const Item& it, int st, int nt) {
+  return PASS == 1 ? st <= it.tile : (st >= it.tile && st < nt);
 }
 
 template <int PASS>
@@ -280,13 +289,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   volatile int* abort_flag = &sm.abort_flag;
-  const int items = a.units * a.np;
+  const int items = a.units * a.nt;
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
-    mbar_init(&sm.fixed_full, 1);
-    mbar_init(&sm.fixed_empty, 1);
-    for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 4); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&sm.fixed_full[i], 1); mbar_init(&sm.fixed_empty[i], 1);
+      mbar_init(&sm.comb_full[i], 128); mbar_init(&sm.comb_empty[i], 128);
+    }
+    for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 8); }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -312,30 +323,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
         const Item it = item_of<PASS>(id, a);
         const int b = it.u / a.heads, h = it.u - b * a.heads;
-        auto issue_stream = [&](int s) -> bool {
+        const int fb = itl & 1;
+        ok = mbar_wait<20>(&sm.fixed_empty[fb], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        mbar_expect_tx(&sm.fixed_full[fb], TILE_BYTES);
+        tma_load_4d(sm.fixed[fb], tm_fixed, &sm.fixed_full[fb], 0, it.tile * TILE, h, b);
+        tma_load_4d(sm.fixed[fb] + SLAB_BYTES, tm_fixed, &sm.fixed_full[fb], 64, it.tile * TILE, h, b);
+        for (int c = 0; c < it.c_count; ++c, ++n) {
           const int stg = n % NS;
-          if (!mbar_wait<20>(&sm.empty[stg], ((n / NS) & 1) ^ 1, abort_flag, a.dev_status)) return false;
-          mbar_expect_tx(&sm.full[stg], TILE_BYTES);
-          tma_load_4d(sm.stream[stg], tm_stream, &sm.full[stg], 0, (it.s_first + s) * TILE, h, b);
-          tma_load_4d(sm.stream[stg] + SLAB_BYTES, tm_stream, &sm.full[stg], 64, (it.s_first + s) * TILE, h, b);
-          ++n;
-          return true;
-        };
-        // the first streamed tiles go out before the fixed tiles: their stages free up while the
-        // previous item's last MMAs (which still read the fixed tiles) are running
-        const int pre = min(NS - 1, it.s_count);
-        int s = 0;
-        for (; ok && s < pre; ++s) ok = issue_stream(s);
-        if (!ok) break;
-        ok = mbar_wait<20>(&sm.fixed_empty, (itl & 1) ^ 1, abort_flag, a.dev_status);
-        if (!ok) break;
-        mbar_expect_tx(&sm.fixed_full, 2 * TILE_BYTES);
+          ok = mbar_wait<20>(&sm.empty[stg], ((n / NS) & 1) ^ 1, abort_flag, a.dev_status);
+          if (!ok) break;
+          // chunk layout: [K half][256 rows][128 bytes]; rows beyond T arrive as zeros
+          const int tok0 = (it.c_first + c) * CHUNK;
+          mbar_expect_tx(&sm.full[stg], CHUNK_BYTES);
 #pragma unroll
-        for (int f = 0; f < 2; ++f) {   // rows beyond T are zero-filled, a tile wholly beyond T too
-          tma_load_4d(sm.fixed[f], tm_fixed, &sm.fixed_full, 0, (2 * it.pair + f) * TILE, h, b);
-          tma_load_4d(sm.fixed[f] + SLAB_BYTES, tm_fixed, &sm.fixed_full, 64, (2 * it.pair + f) * TILE, h, b);
+          for (int kh = 0; kh < 2; ++kh)
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh)
+              tma_load_4d(sm.stream[stg] + kh * (2 * SLAB_BYTES) + hh * SLAB_BYTES, tm_stream, &sm.full[stg], 64 * kh,
+                          tok0 + hh * TILE, h, b);
         }
-        for (; ok && s < it.s_count; ++s) ok = issue_stream(s);
       }
     }
   } else if (wid == 1) {
@@ -343,87 +350,113 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (lane == 0) {
       bool ok = true;
       uint32_t n = 0, itl = 0;
-      uint32_t used[2] = {0, 0};        // accumulators handed to warpgroup f so far
-      const uint64_t stage_desc0 = umma_desc(s32(sm.stream[0]));   // stages are TILE_BYTES apart
-      const uint64_t fixed_desc0 = umma_desc(s32(sm.fixed[0]));
+      const uint64_t stage_desc0 = umma_desc(s32(sm.stream[0]));   // stages are CHUNK_BYTES apart
+      const uint64_t fixed_desc0 = umma_desc(s32(sm.fixed[0]));    // buffers are TILE_BYTES apart
       for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
         const Item it = item_of<PASS>(id, a);
-        int lo[2], hi[2];
-        active_range<PASS>(it, 0, a.nt, lo[0], hi[0]);
-        active_range<PASS>(it, 1, a.nt, lo[1], hi[1]);
-        ok = mbar_wait(&sm.fixed_full, itl & 1, abort_flag, a.dev_status);
+        const int fb = itl & 1;
+        ok = mbar_wait(&sm.fixed_full[fb], (itl >> 1) & 1, abort_flag, a.dev_status);
         if (!ok) break;
-        for (int s = 0; s < it.s_count; ++s, ++n) {
-          const int stg = n % NS;
-          ok = mbar_wait(&sm.full[stg], (n / NS) & 1, abort_flag, a.dev_status);
+        const uint64_t fixed_desc = fixed_desc0 + (uint64_t)fb * (TILE_BYTES >> 4);
+        for (int c = 0; c < it.c_count; ++c, ++n) {
+          const int stg = n % NS, ab = n % NACC;
+          ok = mbar_wait(&sm.full[stg], (n / NS) & 1, abort_flag, a.dev_status) &&
+               mbar_wait(&sm.acc_empty[ab], ((n / NACC) & 1) ^ 1, abort_flag, a.dev_status);
           if (!ok) break;
-          const uint64_t stream_desc = stage_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
-#pragma unroll
-          for (int f = 0; f < 2; ++f) {
-            if (s < lo[f] || s >= hi[f]) continue;
-            const int ab = f * 2 + (used[f] & 1);
-            ok = mbar_wait(&sm.acc_empty[ab], ((used[f] >> 1) & 1) ^ 1, abort_flag, a.dev_status);
-            if (!ok) break;
-            tc_fence_after();
-            umma_tile<0>(tmem + ab * TILE, fixed_desc0 + (uint64_t)f * (TILE_BYTES >> 4), stream_desc);
-            umma_commit(&sm.acc_full[ab]);  // accumulator ready for warpgroup f
-            ++used[f];
-          }
-          if (!ok) break;
-          umma_commit(&sm.empty[stg]);      // the streamed tile may be overwritten once these MMAs have read it
+          tc_fence_after();
+          const int st0 = 2 * (it.c_first + c);
+          const bool need0 = tile_needed<PASS>(it, st0, a.nt), need1 = tile_needed<PASS>(it, st0 + 1, a.nt);
+          const uint64_t stream_desc = stage_desc0 + (uint64_t)stg * (CHUNK_BYTES >> 4);
+          const uint32_t d_addr = tmem + ab * CHUNK;
+          if (need0 && need1)      umma_tile<0, 256>(d_addr, fixed_desc, stream_desc);
+          else if (need0)          umma_tile<0, 128>(d_addr, fixed_desc, stream_desc);
+          else                     umma_tile<0, 128>(d_addr + TILE, fixed_desc, stream_desc + (SLAB_BYTES >> 4));
+          umma_commit(&sm.empty[stg]);      // the chunk may be overwritten once these MMAs have read it
+          umma_commit(&sm.acc_full[ab]);    // accumulator ready for the softmax warps
         }
-        if (ok) umma_commit(&sm.fixed_empty);
+        if (ok) umma_commit(&sm.fixed_empty[fb]);
       }
     }
   } else if (wid < 10) {
     // ------------------------------------------------------------------ softmax warpgroups
-    const int f = (wid - 2) >> 2;                 // warpgroup f owns fixed tile 2 * pair + f
+    const int g = (wid - 2) >> 2;                 // warpgroup g takes half g of every chunk
     const int quarter = wid & 3;                  // TMEM lanes this warp may touch
     const int row = quarter * 32 + lane;          // row of the fixed tile = TMEM lane
-    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + g * TILE;
     float* lse_w = &sm.lse_s[wid - 2][0][0];
     bool ok = true;
-    uint32_t used = 0, itl = 0;                   // accumulators consumed so far (same count as the MMA warp keeps)
+    uint32_t n = 0, itl = 0;
     for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
       const Item it = item_of<PASS>(id, a);
       const int u = it.u;
-      const int ft = 2 * it.pair + f;             // this warpgroup's fixed tile
-      int s_lo, s_hi;
-      active_range<PASS>(it, f, a.nt, s_lo, s_hi);
-      if (s_lo >= s_hi) continue;                 // tile beyond the sequence: nothing to do, nothing to write
-      const int tok = ft * TILE + row;            // query (pass 1) or key (pass 2) index of this thread
+      const int pi = itl & 1;
+      const uint32_t ipar = (itl >> 1) & 1;
+      const int tok = it.tile * TILE + row;       // query (pass 1) or key (pass 2) index of this thread
       const float* lse2_u = a.lse2 + (int64_t)u * a.Tpad;
       // pass 2: this key's value norm, written by pass 1; fetched now, used in the item's epilogue
       float n1 = 0.f;
-      if (PASS == 2 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tok);
+      if (PASS == 2 && g == 0 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tok);
       float m_run = -INFINITY, l_run = 0.f;       // pass 1
       float cs[4] = {0.f, 0.f, 0.f, 0.f};         // pass 2
+      const uint32_t n0 = n;
+      n += it.c_count;
       int buf = 0;
       float xa[32], xb[32];
-      auto acc_of = [&](uint32_t k) { return (int)(f * 2 + (k & 1)); };
-      auto tile_wait = [&](uint32_t k) -> bool {
-        bool w = mbar_wait(&sm.acc_full[acc_of(k)], (k >> 1) & 1, abort_flag, a.dev_status);
+      // streamed tile of this warpgroup in chunk c, and whether the item needs it
+      auto st_of = [&](int c) { return 2 * (it.c_first + c) + g; };
+      auto needed = [&](int c) { return tile_needed<PASS>(it, st_of(c), a.nt); };
+      auto acc_addr = [&](int c) { return lane_addr + ((n0 + c) % NACC) * CHUNK; };
+      auto chunk_wait = [&](int c) -> bool {
+        bool w = mbar_wait(&sm.acc_full[(n0 + c) % NACC], ((n0 + c) / NACC) & 1, abort_flag, a.dev_status);
         w = __all_sync(0xffffffffu, w);
         tc_fence_after();
         return w;
       };
-      int s = s_lo;
-      ok = tile_wait(used);
-      if (!ok) break;
-      tmem_ld32(lane_addr + acc_of(used) * TILE, xa);
-      if (PASS == 2) {
-        reinterpret_cast<float4*>(lse_w)[lane] = __ldg(reinterpret_cast<const float4*>(lse2_u + (it.s_first + s) * TILE) + lane);
+      auto release = [&](int c) {                 // all TMEM reads of chunk c by this warp are complete
+        tc_fence_before();
         __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.acc_empty[(n0 + c) % NACC]);
+      };
+      // prologue: first chunk
+      ok = chunk_wait(0);
+      if (!ok) break;
+      bool have = needed(0);                      // xa holds columns 0..31 of chunk c (when needed)
+      if (have) {
+        tmem_ld32(acc_addr(0), xa);
+        if (PASS == 2) {
+          reinterpret_cast<float4*>(lse_w)[lane] = __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(0) * TILE) + lane);
+          __syncwarp();
+        }
+        tmem_ld_wait();
       }
-      tmem_ld_wait();
-      while (s < s_hi) {
-        const bool diag = (it.s_first + s) == ft;
-        const bool has_next = s + 1 < s_hi;
-        const uint32_t t_addr = lane_addr + acc_of(used) * TILE;
+      for (int c = 0; c < it.c_count; ++c) {
+        const bool has_next = c + 1 < it.c_count;
+        const bool next_needed = has_next && needed(c + 1);
+        if (!have) {
+          // this half of the chunk is masked for the item: hand the accumulator back at once
+          release(c);
+          if (has_next) {
+            ok = chunk_wait(c + 1);
+            if (!ok) break;
+            if (next_needed) {
+              tmem_ld32(acc_addr(c + 1), xa);
+              if (PASS == 2) {
+                reinterpret_cast<float4*>(lse_w + buf * TILE)[lane] =
+                    __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane);
+                __syncwarp();
+              }
+              tmem_ld_wait();
+            }
+          }
+          have = next_needed;
+          continue;
+        }
+        const bool diag = st_of(c) == it.tile;
+        const uint32_t t_addr = acc_addr(c);
         const float* lse_t = lse_w + buf * TILE;
         float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (PASS == 2 && has_next)
-          lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + (it.s_first + s + 1) * TILE) + lane);
+        if (PASS == 2 && next_needed)
+          lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane);
         if (!diag) {
           // software pipeline: the TMEM load of the next 32 columns is in flight while these are consumed
           tmem_ld32(t_addr + 32, xb);
@@ -447,43 +480,60 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           consume32<PASS, true>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
           tmem_ld_wait();
         }
-        // accumulator fully read: hand it back to the MMA warp
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.acc_empty[acc_of(used)]);
+        release(c);
         if (has_next) {
-          ok = tile_wait(used + 1);
+          ok = chunk_wait(c + 1);
           if (!ok) break;
-          tmem_ld32(lane_addr + acc_of(used + 1) * TILE, xa);
+          if (next_needed) tmem_ld32(acc_addr(c + 1), xa);
         }
         if (diag) consume32<PASS, true>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
         else      consume32<PASS, false>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        if (PASS == 2 && has_next) {
+        if (PASS == 2 && next_needed) {
           reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
           __syncwarp();
         }
         tmem_ld_wait();
-        ++s;
-        ++used;
+        have = next_needed;
         buf ^= 1;
       }
       if (!ok) break;
-      // ---- end of item: this thread's row is complete
-      if (PASS == 1) {
-        const float lse2 = m_run + log2f(l_run);
-        a.lse2[(int64_t)u * a.Tpad + tok] = tok < a.T ? lse2 : INFINITY;
-        if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
-      } else if (tok < a.T) {
-        const float tot = (cs[0] + cs[1]) + (cs[2] + cs[3]);
-        const int64_t o = (int64_t)u * a.T + tok;
-        a.attn_acc[o] = tot;
-        a.score[o] = tot * n1;
+      // ---- end of item: warpgroup 1 hands its partial to warpgroup 0, which finishes the rows
+      if (g == 1) {
+        ok = mbar_wait(&sm.comb_empty[pi], ipar ^ 1, abort_flag, a.dev_status);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        if (PASS == 1) { sm.part_a[pi][row] = m_run; sm.part_b[pi][row] = l_run; }
+        else           { sm.part_a[pi][row] = (cs[0] + cs[1]) + (cs[2] + cs[3]); }
+        mbar_arrive(&sm.comb_full[pi]);
+      } else {
+        ok = mbar_wait(&sm.comb_full[pi], ipar, abort_flag, a.dev_status);
+        if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
+        if (PASS == 1) {
+          const float m1 = sm.part_a[pi][row], l1 = sm.part_b[pi][row];
+          mbar_arrive(&sm.comb_empty[pi]);
+          const float m = fmaxf(m_run, m1);
+          float l = 0.f;
+          if (l_run > 0.f) l += l_run * ex2(m_run - m);
+          if (l1 > 0.f) l += l1 * ex2(m1 - m);
+          const float lse2 = m + log2f(l);
+          a.lse2[(int64_t)u * a.Tpad + tok] = tok < a.T ? lse2 : INFINITY;
+          // an odd tile count leaves half a chunk of padding that pass 2 reads as "no query"
+          if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = INFINITY;
+          if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
+        } else {
+          const float tot = ((cs[0] + cs[1]) + (cs[2] + cs[3])) + sm.part_a[pi][row];
+          mbar_arrive(&sm.comb_empty[pi]);
+          if (tok < a.T) {
+            const int64_t o = (int64_t)u * a.T + tok;
+            a.attn_acc[o] = tot;
+            a.score[o] = tot * n1;
+          }
+        }
       }
     }
   } else if (PASS == 1) {
     // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
-    // Independent of the attention work of this pass: every (unit, pair of token tiles) is an item
-    // exactly once, so this warp covers all tokens.  Pass 2 reads the norms back in its epilogue.
+    // Independent of the attention work of this pass: every (unit, token tile) is an item exactly
+    // once, so this warp covers all tokens.  Pass 2 reads the norms back in its epilogue.
     uint32_t itl = 0;
     for (int id = item_id(0, blockIdx.x, gridDim.x); id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
       const Item it = item_of<PASS>(id, a);
@@ -491,11 +541,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
       // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
       const int sub = lane >> 4, part = lane & 15;
-      for (int r0 = 0; r0 < 2 * TILE; r0 += 32) {
+      for (int r0 = 0; r0 < TILE; r0 += 32) {
         uint4 raw[16];
 #pragma unroll
         for (int j = 0; j < 16; ++j) {
-          const int tok = it.pair * 2 * TILE + r0 + 2 * j + sub;
+          const int tok = it.tile * TILE + r0 + 2 * j + sub;
           raw[j] = make_uint4(0u, 0u, 0u, 0u);
           if (tok < a.T) raw[j] = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
         }
@@ -508,7 +558,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             acc += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
 #pragma unroll
           for (int o = 8; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-          const int tok = it.pair * 2 * TILE + r0 + 2 * j + sub;
+          const int tok = it.tile * TILE + r0 + 2 * j + sub;
           if (part == 0 && tok < a.T) a.vnorm[(int64_t)it.u * a.T + tok] = acc;
         }
       }
@@ -572,7 +622,7 @@ bool vatp_tc_available() {
 }
 
 size_t prefill_tc_workspace_bytes(int units, int T) {
-  const size_t Tpad = (size_t)(T + TILE - 1) / TILE * TILE;
+  const size_t Tpad = (size_t)(T + CHUNK - 1) / CHUNK * CHUNK;
   return (size_t)units * Tpad * sizeof(float);
 }
 
@@ -584,8 +634,8 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   TcArgs a;
   a.units = s.units; a.heads = s.heads; a.T = s.T;
   a.nt = (s.T + TILE - 1) / TILE;
-  a.np = (a.nt + 1) / 2;
-  a.Tpad = a.nt * TILE;
+  a.nch = (a.nt + 1) / 2;
+  a.Tpad = a.nch * CHUNK;
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.v = static_cast<const __nv_bfloat16*>(v);
   a.sb = s.sb; a.sh = s.sh; a.st = s.st;
@@ -598,7 +648,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int items = a.units * a.np;
+  const int items = a.units * a.nt;
   const int grid = items < sms ? items : sms;
   prefill_tc_kernel<1><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   prefill_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
