@@ -207,11 +207,16 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
       for (int i = 0; i < 32; ++i)
         if (c0 + i > row) x[i] = -INFINITY;
     }
-    float cmax = max3(x[0], x[1], x[2]);
-#pragma unroll
-    for (int i = 3; i + 1 < 32; i += 2) cmax = max3(cmax, x[i], x[i + 1]);
-    cmax = fmaxf(cmax, x[31]) * scale_log2;            // scale > 0 keeps the order
-    if (cmax > m_run) { l_run *= ex2(m_run - cmax); m_run = cmax; }
+    // four short max chains instead of one long one, then a branch-free rescale of the running sum
+    float c0m = max3(x[0], x[1], x[2]), c1m = max3(x[8], x[9], x[10]);
+    float c2m = max3(x[16], x[17], x[18]), c3m = max3(x[24], x[25], x[26]);
+    c0m = max3(c0m, x[3], x[4]); c1m = max3(c1m, x[11], x[12]); c2m = max3(c2m, x[19], x[20]); c3m = max3(c3m, x[27], x[28]);
+    c0m = max3(c0m, x[5], x[6]); c1m = max3(c1m, x[13], x[14]); c2m = max3(c2m, x[21], x[22]); c3m = max3(c3m, x[29], x[30]);
+    c0m = max3(c0m, x[7], c1m); c2m = max3(c2m, x[15], c3m);
+    const float cmax = max3(c0m, c2m, fmaxf(x[23], x[31])) * scale_log2;   // scale > 0 keeps the order
+    const float m_new = fmaxf(m_run, cmax);
+    l_run *= ex2(fmaxf(m_run - m_new, -126.f));      // (-inf) - (-inf) = NaN -> -126 -> factor on a zero sum
+    m_run = m_new;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
@@ -457,42 +462,53 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
         if (PASS == 2 && next_needed)
           lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane);
+        // Both paths are rolled loops with few inlined copies of the slice code: the steady-state
+        // body stays small enough for the instruction cache.
         if (!diag) {
           // software pipeline: the TMEM load of the next 32 columns is in flight while these are consumed
-          tmem_ld32(t_addr + 32, xb);
-          consume32<PASS, false>(xa, 0, row, a.scale_log2, m_run, l_run, cs, lse_t);
-          tmem_ld_wait();
-          tmem_ld32(t_addr + 64, xa);
-          consume32<PASS, false>(xb, 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
-          tmem_ld_wait();
-          tmem_ld32(t_addr + 96, xb);
-          consume32<PASS, false>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
-          tmem_ld_wait();
-        } else {
-          // the one diagonal tile of an item takes the masked variant, kept compact (not pipelined)
 #pragma unroll 1
-          for (int c0 = 0; c0 < 64; c0 += 32) {
-            consume32<PASS, true>(xa, c0, row, a.scale_log2, m_run, l_run, cs, lse_t);
-            tmem_ld32(t_addr + c0 + 32, xa);
+          for (int h2 = 0; h2 < 2; ++h2) {
+            tmem_ld32(t_addr + 64 * h2 + 32, xb);
+            consume32<PASS, false>(xa, 64 * h2, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            tmem_ld_wait();
+            if (h2 == 0) {
+              tmem_ld32(t_addr + 64, xa);
+            } else {
+              release(c);
+              if (has_next) {
+                ok = chunk_wait(c + 1);
+                if (ok && next_needed) tmem_ld32(acc_addr(c + 1), xa);
+              }
+            }
+            if (ok) consume32<PASS, false>(xb, 64 * h2 + 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            if (h2 == 1 && PASS == 2 && next_needed) {
+              reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
+              __syncwarp();
+            }
             tmem_ld_wait();
           }
-          tmem_ld32(t_addr + 96, xb);
-          consume32<PASS, true>(xa, 64, row, a.scale_log2, m_run, l_run, cs, lse_t);
+        } else {
+          // the one diagonal tile of an item takes the masked variant (not pipelined)
+#pragma unroll 1
+          for (int c0 = 0; c0 < TILE; c0 += 32) {
+            consume32<PASS, true>(xa, c0, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            if (c0 + 32 < TILE) {
+              tmem_ld32(t_addr + c0 + 32, xa);
+              tmem_ld_wait();
+            }
+          }
+          release(c);
+          if (has_next) {
+            ok = chunk_wait(c + 1);
+            if (ok && next_needed) tmem_ld32(acc_addr(c + 1), xa);
+          }
+          if (PASS == 2 && next_needed) {
+            reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
+            __syncwarp();
+          }
           tmem_ld_wait();
         }
-        release(c);
-        if (has_next) {
-          ok = chunk_wait(c + 1);
-          if (!ok) break;
-          if (next_needed) tmem_ld32(acc_addr(c + 1), xa);
-        }
-        if (diag) consume32<PASS, true>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        else      consume32<PASS, false>(xb, 96, row, a.scale_log2, m_run, l_run, cs, lse_t);
-        if (PASS == 2 && next_needed) {
-          reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
-          __syncwarp();
-        }
-        tmem_ld_wait();
+        if (!ok) break;
         have = next_needed;
         buf ^= 1;
       }
