@@ -41,7 +41,8 @@ typedef enum {
   VATP_ERR_UNSUPPORTED = 2,
   VATP_ERR_WORKSPACE = 3,
   VATP_ERR_CUDA = 4,
-  VATP_ERR_TIMEOUT = 5
+  VATP_ERR_TIMEOUT = 5,
+  VATP_ERR_STATIC_SCRATCH = 6  /* problem needs more scratch than the built-in array holds */
 } vatp_status;
 
 typedef enum { VATP_BF16 = 0, VATP_F32 = 1 } vatp_dtype;
@@ -107,6 +108,35 @@ vatp_status vatp_prefill_scores(const vatp_params* params, const void* q, const 
                                 float* lse_out, float* attn_acc, float* vnorm, float* score,
                                 float* win_rows, void* workspace, size_t workspace_bytes,
                                 int32_t* dev_status, void* cuda_stream);
+
+/*
+ * vatp_prefill_scores for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a packaging variant of the call above and computes exactly the same thing.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option - a plugin inside a host
+ * application that owns all device memory and offers no scratch, a real-time loop that must never
+ * hit the device-wide synchronisation an allocation implies, or a process whose pool was sized up
+ * front.  Such callers still own q, k, v and the outputs, but have nowhere to put the row
+ * normalisers that pass 1 hands to pass 2.  Here that scratch is a fixed device array built into
+ * the library: VATP_STATIC_SCRATCH_BYTES on every GPU that loads the library, held until the
+ * process exits.  The call allocates and frees nothing.
+ *
+ * Arguments are those of vatp_prefill_scores without workspace / workspace_bytes.
+ * Limit: vatp_workspace_bytes(params) <= VATP_STATIC_SCRATCH_BYTES, i.e. batch * heads *
+ * round_up(seq_len, 256) <= 1,048,576 (for example 32 heads x 32768 tokens, or 256 units x 4096);
+ * anything larger returns VATP_ERR_STATIC_SCRATCH before a launch.
+ * First call on a device: looks up the array's device address (once per device, with the current
+ * device) - make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array.  Calls on one stream are ordered and safe;
+ * calls that may overlap on the GPU (different streams, different host threads) race on it and
+ * give wrong scores - serialise them, or use vatp_prefill_scores with separate workspaces.  The
+ * array keeps the previous call's contents; nothing in it needs clearing, because pass 1 writes
+ * every normaliser that pass 2 reads.
+ */
+#define VATP_STATIC_SCRATCH_BYTES (4u << 20)
+vatp_status vatp_prefill_scores_static(const vatp_params* params, const void* q, const void* k, const void* v,
+                                       float* lse_out, float* attn_acc, float* vnorm, float* score,
+                                       float* win_rows, int32_t* dev_status, void* cuda_stream);
 
 /*
  * Budgeted selection (Section 3.2 with Appendix A's budget split): per unit keep the first F

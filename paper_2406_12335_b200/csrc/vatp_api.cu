@@ -67,6 +67,7 @@ const char* vatp_status_string(vatp_status s) {
     case VATP_ERR_WORKSPACE: return "workspace too small or misaligned";
     case VATP_ERR_CUDA: return "CUDA error";
     case VATP_ERR_TIMEOUT: return "device-side wait ran out";
+    case VATP_ERR_STATIC_SCRATCH: return "problem exceeds the library's built-in scratch array";
   }
   return "unknown status";
 }

@@ -18,7 +18,8 @@ lib = C.CDLL(_LIB_PATH)
 OK = 0
 BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
-EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_select", "vatp_compact", "vatp_decode_step",
+STATIC_SCRATCH_BYTES = 4 << 20
+EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
            "vatp_status_string"]
 
 
@@ -42,6 +43,8 @@ lib.vatp_workspace_bytes.restype = C.c_size_t
 lib.vatp_workspace_bytes.argtypes = [C.POINTER(Params)]
 lib.vatp_prefill_scores.restype = C.c_int
 lib.vatp_prefill_scores.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.vatp_prefill_scores_static.restype = C.c_int
+lib.vatp_prefill_scores_static.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.vatp_select.restype = C.c_int
 lib.vatp_select.argtypes = [C.POINTER(Params), _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.vatp_compact.restype = C.c_int
@@ -124,6 +127,17 @@ def vatp_prefill_scores(p: Params, q, k, v, *, lse_out=None, attn_acc, vnorm, sc
     _check(lib.vatp_prefill_scores(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse_out), _ptr(attn_acc), _ptr(vnorm),
                                    _ptr(score), _ptr(win_rows), _ptr(workspace), ws_bytes, _ptr(dev_status),
                                    _stream(stream)), "vatp_prefill_scores")
+
+
+def vatp_prefill_scores_static(p: Params, q, k, v, *, lse_out=None, attn_acc, vnorm, score, win_rows=None,
+                               dev_status=None, stream=None):
+    """vatp_prefill_scores without a workspace argument: for callers that cannot allocate device
+    memory, the scratch is a fixed array inside the library (at most STATIC_SCRATCH_BYTES of row
+    normalisers; larger problems raise VatpError).  All calls on a device share that array, so
+    calls that could overlap on the GPU must be serialised by the caller."""
+    _check(lib.vatp_prefill_scores_static(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse_out), _ptr(attn_acc),
+                                          _ptr(vnorm), _ptr(score), _ptr(win_rows), _ptr(dev_status),
+                                          _stream(stream)), "vatp_prefill_scores_static")
 
 
 def vatp_select(p: Params, score, kept_idx, *, workspace=None, dev_status=None, stream=None):
