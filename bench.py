@@ -158,6 +158,19 @@ def run_reference(args, wl):
 
 
 # ------------------------------------------------------------------------------------ CUDA arm
+def max_over_ranks(values, device, world: int):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the time)."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return t.tolist()
+
+
+def replica_throughput(units_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job units per second when every rank processes `units_per_rank` in `ms` (max over ranks)."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 class LayerState:
     def __init__(self, V, wl, layer, dev):
         from paper_2406_12335_b200 import synth
@@ -264,10 +277,7 @@ def run_cuda(args, wl):
     t_score = [sum(e[0].elapsed_time(e[1]) for e in r[3]) / L for r in recs]    # ms per layer
     t_select = [sum(e[1].elapsed_time(e[2]) for e in r[3]) / L for r in recs]
     t_compact = [sum(e[2].elapsed_time(e[3]) for e in r[3]) / L for r in recs]
-    stats = torch.tensor([sum(t_pre), sum(t_dec), sum(t_all)], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(stats, op=torch.distributed.ReduceOp.MAX)
-    pre_ms, dec_ms, all_ms = (stats / args.steps).tolist()
+    pre_ms, dec_ms, all_ms = (x / args.steps for x in max_over_ranks([sum(t_pre), sum(t_dec), sum(t_all)], dev, world))
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
     host = None if args.no_e2e else [[x.cpu().pin_memory() for x in (ls.q, ls.k, ls.v, ls.dq, ls.dk, ls.dv)] for ls in layers]
@@ -297,10 +307,7 @@ def run_cuda(args, wl):
         e2e_step(); barrier()
         e2e_recs = [e2e_step() for _ in range(max(2, min(args.steps, 5)))]
         barrier()
-        e2e_pre = torch.tensor([statistics.mean(a.elapsed_time(b) for a, b, _ in e2e_recs)], dtype=torch.float64,
-                               device=dev)
-        if world > 1:
-            torch.distributed.all_reduce(e2e_pre, op=torch.distributed.ReduceOp.MAX)
+        e2e_pre_ms = max_over_ranks([statistics.mean(a.elapsed_time(b) for a, b, _ in e2e_recs)], dev, world)[0]
         e2e_dec_ms = statistics.mean(b.elapsed_time(c) for _, b, c in e2e_recs)
 
     if rank != 0:
@@ -308,7 +315,7 @@ def run_cuda(args, wl):
     units = wl.batch * wl.heads
     T, d, B = wl.seq_len, wl.head_dim, wl.budget
     tokens = wl.batch * T * L                                  # layer-tokens scored and pruned per step
-    value = world * tokens / (pre_ms * 1e-3)
+    value = replica_throughput(tokens, pre_ms, world)
     dec_us = dec_ms * 1e3 / (steps_dec * L)
 
     # ---- rooflines (algorithmic work only) ----
@@ -351,7 +358,7 @@ def run_cuda(args, wl):
         "prefill_ms_per_layer": pre_ms / L, "decode_us_per_layer_step": dec_us,
         "roofline": roof, "roofline_all": kernels,
         "e2e": None if host is None else
-               {"value": world * tokens / (float(e2e_pre.item()) * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               {"value": replica_throughput(tokens, e2e_pre_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "decode_us_per_layer_step": e2e_dec_ms * 1e3 / (steps_dec * L)},
         "gpu_launches": args.steps * (L * 4 + steps_dec * L),
         "clocks": clocks,

@@ -16,8 +16,8 @@ def _small(dtype, d, T, B, F, R, b=1, h=2, indicator="h2o", window=0, steps=0, c
     return synth.Workload(cid, f"case_T{T}", dtype, b, h, 1, d, T, B, F, R, indicator, window, steps)
 
 
-def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4):
-    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0):
+    q, k, v = synth.prefill_inputs(wl, layer, "cuda")
     g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink).run()
     P.gpu_invariants(g)
     tol = P.TOL[wl.dtype]
@@ -29,7 +29,7 @@ def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4):
         nb += n_boundary
     adopted = 0
     if decode and wl.decode_steps:
-        dq, dk, dv = synth.decode_inputs(wl, 0, device="cuda")
+        dq, dk, dv = synth.decode_inputs(wl, layer, device="cuda")
         adopted = P.run_decode_and_check(g, refs, dq, dk, dv, wl.decode_steps, tol, check_state_every)
     return g, nb, adopted
 
@@ -137,3 +137,24 @@ def test_config1_llama_layer():
 def test_config1_prefill_all_heads():
     wl = synth.CONFIGS[1].with_(decode_steps=0)
     _run_case(wl, decode=False)
+
+
+@pytest.mark.parametrize("layer,units", [(0, [(0, 0), (7, 31)]), (31, [(3, 17), (5, 2)])])
+def test_config2_stack_layer(layer, units):
+    """Config 2 at its full per-layer size (batch 8, 32 heads, T 8192, budget 1638, recent 256; the
+    value-norm spread grows with the layer): first and last layer, oracle on sampled units, oracle-free
+    invariants on all 256 units of the layer, 128 decode steps."""
+    _run_case(synth.CONFIGS[2], units=units, check_state_every=64, layer=layer)
+
+
+def test_config3_windowed():
+    """Config 3 at full size: last-256-queries indicator (Eq. 3), batch 16, 32 heads, T 2048, budget
+    1024, 512 decode steps with the cache held at budget; oracle on sampled units."""
+    _run_case(synth.CONFIGS[3], units=[(0, 0), (9, 14), (15, 31)], check_state_every=128)
+
+
+def test_config4_long_context_layer():
+    """Config 4 at full size: T 32768, budget 3277, recent 512, 64 boosted-norm tokens per layer.  The
+    oracle materialises the 32768 x 32768 matrix, so it runs on one unit of the last layer; every other
+    unit of that layer is covered by the invariants."""
+    _run_case(synth.CONFIGS[4], units=[(0, 5)], check_state_every=32, layer=31)
