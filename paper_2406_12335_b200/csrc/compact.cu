@@ -6,57 +6,63 @@ namespace vatp {
 namespace {
 
 constexpr int CP_THREADS = 256;
-constexpr int CP_UNROLL = 4;
+constexpr int CP_SLOTS = 64;     // destination slots per CTA
+constexpr int CP_ITERS = CP_SLOTS / (CP_THREADS / 16);
 
-// One "chunk" is 16 bytes of one row of K or V.  Chunks are numbered
-// ((unit * cap + slot) * 2 + which) * cpr + c, so consecutive threads copy consecutive 16-byte
-// pieces of a row and a warp covers whole rows.
+// grid (units, slot groups).  Sixteen lanes copy one row (K and V) in 16-byte pieces; a thread has
+// CP_ITERS rows of K and of V in flight before it stores, and no index needs a division.
 __global__ void __launch_bounds__(CP_THREADS)
 compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict__ k, const char* __restrict__ v,
                const float* __restrict__ attn_acc, const float* __restrict__ vnorm, const int32_t* __restrict__ kept,
                vatp_cache c) {
-  const int cpr = sh.d * elem_bytes / 16;  // chunks per row
-  const int64_t total = (int64_t)sh.units * cap * 2 * cpr;
+  const int u = blockIdx.x;
   const int len = min(sh.T, B);
-  const int64_t base = ((int64_t)blockIdx.x * CP_UNROLL) * CP_THREADS + threadIdx.x;
-  uint4 val[CP_UNROLL];
-  int64_t dst[CP_UNROLL];
+  const int row_bytes = sh.d * elem_bytes;
+  const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
+  const int slot0 = blockIdx.y * CP_SLOTS + hw;
+  const int64_t unit_bytes = unit_offset(sh, u) * elem_bytes;
+  const int64_t tok_bytes = sh.st * elem_bytes;
+
+  int src[CP_ITERS];
 #pragma unroll
-  for (int it = 0; it < CP_UNROLL; ++it) {
-    const int64_t idx = base + (int64_t)it * CP_THREADS;
-    dst[it] = -1;
-    if (idx >= total) continue;
-    const int cc = (int)(idx % cpr);
-    const int64_t row = idx / cpr;
-    const int which = (int)(row & 1);
-    const int64_t us = row >> 1;
-    const int slot = (int)(us % cap);
-    const int u = (int)(us / cap);
-    const int src = slot < len ? kept[(int64_t)u * B + slot] : -1;
-    if (cc == 0 && which == 0) {
-      const int64_t o = (int64_t)u * cap + slot;
-      c.pos[o] = src;
-      c.acc[o] = src >= 0 ? attn_acc[(int64_t)u * sh.T + src] : 0.f;
-      c.vnorm[o] = src >= 0 ? vnorm[(int64_t)u * sh.T + src] : 0.f;
-      if (slot == 0) {
-        c.len[u] = len;
-        c.free_slot[u] = len;
-        c.next_pos[u] = sh.T;
-      }
-    }
-    if (src < 0) continue;
-    const char* in = (which ? v : k) + (unit_offset(sh, u) + (int64_t)src * sh.st) * elem_bytes + (int64_t)cc * 16;
-    val[it] = *reinterpret_cast<const uint4*>(in);
-    dst[it] = (((int64_t)u * cap + slot) * cpr + cc) * 16;
-    if (which) dst[it] = -2 - dst[it];  // tag V destinations
+  for (int i = 0; i < CP_ITERS; ++i) {
+    const int slot = slot0 + i * (CP_THREADS / 16);
+    src[i] = slot < len ? __ldg(kept + (int64_t)u * B + slot) : -1;
   }
+  for (int c0 = l16 * 16; c0 < row_bytes; c0 += 256) {
+    uint4 kv[CP_ITERS], vv[CP_ITERS];
 #pragma unroll
-  for (int it = 0; it < CP_UNROLL; ++it) {
-    if (dst[it] == -1) continue;
-    if (dst[it] >= 0)
-      *reinterpret_cast<uint4*>((char*)c.k_cache + dst[it]) = val[it];
-    else
-      *reinterpret_cast<uint4*>((char*)c.v_cache + (-2 - dst[it])) = val[it];
+    for (int i = 0; i < CP_ITERS; ++i) {
+      if (src[i] < 0) continue;
+      const int64_t o = unit_bytes + (int64_t)src[i] * tok_bytes + c0;
+      kv[i] = __ldg(reinterpret_cast<const uint4*>(k + o));
+      vv[i] = __ldg(reinterpret_cast<const uint4*>(v + o));
+    }
+#pragma unroll
+    for (int i = 0; i < CP_ITERS; ++i) {
+      if (src[i] < 0) continue;
+      const int slot = slot0 + i * (CP_THREADS / 16);
+      const int64_t o = ((int64_t)u * cap + slot) * row_bytes + c0;
+      *reinterpret_cast<uint4*>((char*)c.k_cache + o) = kv[i];
+      *reinterpret_cast<uint4*>((char*)c.v_cache + o) = vv[i];
+    }
+  }
+  // per-slot decode state
+  if (l16 == 0) {
+#pragma unroll
+    for (int i = 0; i < CP_ITERS; ++i) {
+      const int slot = slot0 + i * (CP_THREADS / 16);
+      if (slot >= cap) continue;
+      const int64_t o = (int64_t)u * cap + slot;
+      c.pos[o] = src[i];
+      c.acc[o] = src[i] >= 0 ? __ldg(attn_acc + (int64_t)u * sh.T + src[i]) : 0.f;
+      c.vnorm[o] = src[i] >= 0 ? __ldg(vnorm + (int64_t)u * sh.T + src[i]) : 0.f;
+    }
+  }
+  if (blockIdx.y == 0 && threadIdx.x == 0) {
+    c.len[u] = len;
+    c.free_slot[u] = len;
+    c.next_pos[u] = sh.T;
   }
 }
 
@@ -89,11 +95,8 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            cudaStream_t st) {
   const int eb = dtype == VATP_F32 ? 4 : 2;
   const int cap = cache_capacity(B);
-  const int cpr = s.d * eb / 16;
-  const int64_t total = (int64_t)s.units * cap * 2 * cpr;
-  const int64_t per_block = (int64_t)CP_THREADS * CP_UNROLL;
-  const unsigned blocks = (unsigned)((total + per_block - 1) / per_block);
-  compact_kernel<<<blocks, CP_THREADS, 0, st>>>(s, eb, B, cap, (const char*)k, (const char*)v, attn_acc, vnorm, kept, c);
+  const dim3 grid(s.units, (cap + CP_SLOTS - 1) / CP_SLOTS);
+  compact_kernel<<<grid, CP_THREADS, 0, st>>>(s, eb, B, cap, (const char*)k, (const char*)v, attn_acc, vnorm, kept, c);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   if (s.window > 0) {

@@ -444,6 +444,10 @@ cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const 
                           const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status,
                           cudaStream_t st) {
   const bool win = s.window > 0;
+  if (dtype == VATP_BF16 && s.d == 128) {
+    const cudaError_t e = launch_decode_mma(s, B, F, R, c, q, k, v, out, evicted, dev_status, st);
+    if (e != cudaErrorNotSupported) return e;
+  }
 #define VATP_DISPATCH(T, D)                                                                         \
   return win ? launch_t<T, D, true>(s, B, F, R, c, q, k, v, out, evicted, dev_status, st)           \
              : launch_t<T, D, false>(s, B, F, R, c, q, k, v, out, evicted, dev_status, st)

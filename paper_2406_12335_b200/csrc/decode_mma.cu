@@ -1,0 +1,497 @@
+// Decode step for bf16, head_dim 128 (the LLaMA2-7B shape): append, attend (Eq. 1), indicator
+// update (Eq. 2 / Eq. 3), importance (Eq. 4), release of the lowest-importance unprotected slot.
+//
+// The step is HBM-bound (every cached K and V row is read once) but so short - tens of megabytes -
+// that the latency of each warp's own instruction stream decides its duration.  Hence:
+//   * every warp owns a ring of stages and requests its rows with one bulk copy per row (all 32
+//     lanes issue at once) before anything else happens; rows land on a 272-byte pitch, which makes
+//     ldmatrix conflict-free;
+//   * q.K^T and p.V run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32
+//     accumulate): S^T = q K^T leaves the probabilities of 16 rows in exactly the registers the
+//     A operand of p V wants, so a 16-row group costs about 80 instructions instead of several
+//     hundred.  p is split into two bf16 halves (rows 0-7 / 8-15 of the A tile carry hi / lo), so
+//     the product keeps ~16 bits of p;
+//   * a unit is split over a thread-block cluster when units are few.  CTAs exchange by PUSHING into
+//     each other's shared memory before a cluster barrier (partial max / sum to every rank, partial
+//     output to rank 0, every warp's arg-min candidate to every rank), so nobody reads remote
+//     memory after a barrier: two cluster barriers per step, no global scratch, one launch.
+#include <cooperative_groups.h>
+
+#include "vatp_internal.cuh"
+
+namespace cg = cooperative_groups;
+
+namespace vatp {
+namespace {
+
+constexpr int MW = 8;                 // warps per CTA
+constexpr int MT = MW * 32;
+constexpr int HD = 128;
+constexpr int GROUP = 16;             // rows per MMA group = rows of K (and of V) per stage
+constexpr int ROW_BYTES = HD * 2;
+constexpr int PITCH = ROW_BYTES + 16; // shared-memory row pitch
+constexpr int STAGE_BYTES = 2 * GROUP * PITCH;
+constexpr int MAX_SPLIT = 8;
+constexpr float LOG2E = 1.4426950408889634f;
+constexpr unsigned long long NO_KEY = ~0ull;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait (about one second): false when the copy never signalled.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint64_t t0 = global_ns();
+  while (!mbar_try_wait(bar, parity))
+    if (global_ns() - t0 > 1000000000ull) return false;
+  return true;
+}
+// global -> shared bulk copy; dst, src and bytes are multiples of 16
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+// D (16x8, fp32) += A (16x16, bf16, row) * B (16x8, bf16, col)
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// two floats -> packed bf16 pair (lo in the low half), round to nearest
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// what the CTAs of a unit push to one another
+struct Exch {
+  float m[MAX_SPLIT], l[MAX_SPLIT];       // per rank: max of its logits (log2 domain), sum of exp2(s - m)
+  unsigned long long key[MAX_SPLIT][MW];  // arg-min candidate of every warp of every rank
+  float o[MAX_SPLIT][HD];                 // rank 0 only: partial outputs of every rank
+};
+
+// eviction order as one integer: lower importance first, among equals the higher position first
+__device__ __forceinline__ unsigned long long evict_key(float I, int pos) {
+  return ((unsigned long long)__float_as_uint(I) << 32) | (unsigned)(0x7fffffff - pos);
+}
+
+template <bool WINDOWED>
+__global__ void __launch_bounds__(MT, 1)
+decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
+                  const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
+                  const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
+                  int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
+  extern __shared__ __align__(128) unsigned char dyn[];
+  // [MW][nstage][K rows | V rows] | logits[chunk] | acc[chunk] | vnorm[chunk] | pos[chunk]
+  unsigned char* stage_base = dyn;
+  float* logit_s = reinterpret_cast<float*>(dyn + (size_t)MW * nstage * STAGE_BYTES);
+  float* acc_s = logit_s + chunk;
+  float* vn_s = acc_s + chunk;
+  int* pos_s = reinterpret_cast<int*>(vn_s + chunk);
+
+  __shared__ __align__(8) uint64_t bars[MW * 4 + 1];
+  __shared__ __align__(16) Exch ex;
+  __shared__ __align__(16) float part_o[MW][HD];
+  __shared__ float part_m[MW], part_l[MW];
+
+  cg::cluster_group cluster = cg::this_cluster();
+  const int rank = split > 1 ? (int)cluster.block_rank() : 0;
+  const int u = blockIdx.x / split;
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int j4 = lane & 3;
+
+  // this CTA's slot range inside the allocation
+  const int s0 = min(rank * chunk, cap);
+  const int rows_alloc = min(chunk, cap - s0);
+  const int ngroups = (rows_alloc + GROUP - 1) / GROUP;
+  const __nv_bfloat16* kc = (const __nv_bfloat16*)c.k_cache + ((int64_t)u * cap + s0) * HD;
+  const __nv_bfloat16* vc = (const __nv_bfloat16*)c.v_cache + ((int64_t)u * cap + s0) * HD;
+  uint64_t* my_bars = &bars[wid * 4];
+  uint64_t* state_bar = &bars[MW * 4];
+  unsigned char* my_stages = stage_base + (size_t)wid * nstage * STAGE_BYTES;
+
+  // every warp arms its own barriers: no CTA-wide barrier before the first copy is requested
+  if (lane == 0) {
+    for (int s = 0; s < nstage; ++s) mbar_init(&my_bars[s], 1);
+    if (wid == 1) mbar_init(state_bar, 1);     // armed and used by this same lane
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  // lanes 0-15 fetch the K rows of group g, lanes 16-31 its V rows
+  auto issue = [&](int g, int stage, int limit) {
+    const int r0 = g * GROUP;
+    const int n = min(GROUP, limit - r0);
+    unsigned char* dst = my_stages + stage * STAGE_BYTES;
+    uint64_t* bar = &my_bars[stage];
+    if (lane == 0) mbar_expect_tx(bar, 2u * n * ROW_BYTES);
+    __syncwarp();
+    const int rr = lane & 15;
+    if (rr < n) {
+      const __nv_bfloat16* src = (lane < 16 ? kc : vc) + (int64_t)(r0 + rr) * HD;
+      bulk_g2s(dst + (lane < 16 ? 0 : GROUP * PITCH) + rr * PITCH, src, ROW_BYTES, bar);
+    }
+  };
+  for (int s = 0; s < nstage; ++s)
+    if (wid + s * MW < ngroups) issue(wid + s * MW, s, rows_alloc);
+  if (tid == 32 && rows_alloc > 0) {      // per-slot state of the range
+    const int64_t o = (int64_t)u * cap + s0;
+    mbar_expect_tx(state_bar, 3u * rows_alloc * 4u);
+    bulk_g2s(acc_s, c.acc + o, rows_alloc * 4, state_bar);
+    bulk_g2s(vn_s, c.vnorm + o, rows_alloc * 4, state_bar);
+    bulk_g2s(pos_s, c.pos + o, rows_alloc * 4, state_bar);
+  }
+
+  const int len = c.len[u];
+  const int fs = c.free_slot[u];
+  const int t = c.next_pos[u];
+  const int hi = len + 1;                // slots [0, hi) are live once the new token is in
+  const int cnt = max(min(hi - s0, rows_alloc), 0);
+  const int fs_local = fs - s0;          // row of the incoming token inside this CTA's range (if owned)
+  const bool owns_new = fs_local >= 0 && fs_local < cnt;
+
+  // A operand of q K^T: q replicated over the rows 0-7 of the tile (rows 8-15 zero)
+  const __nv_bfloat16* qn = q_new + (int64_t)u * HD;
+  uint32_t qa[HD / 16][2];
+#pragma unroll
+  for (int ks = 0; ks < HD / 16; ++ks) {
+    qa[ks][0] = __ldg(reinterpret_cast<const uint32_t*>(qn + ks * 16 + 2 * j4));
+    qa[ks][1] = __ldg(reinterpret_cast<const uint32_t*>(qn + ks * 16 + 8 + 2 * j4));
+  }
+  // 16 bytes of the incoming K row (lanes 0-15) or V row (lanes 16-31)
+  const uint4 new_raw = __ldg(reinterpret_cast<const uint4*>((lane < 16 ? k_new : v_new) + (int64_t)u * HD) + (lane & 15));
+
+  // ---- append: the CTA that owns the free slot stores the new row and its l1 norm ----
+  float new_norm = 0.f;
+  {
+    const uint32_t wv[4] = {new_raw.x, new_raw.y, new_raw.z, new_raw.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      new_norm += fabsf(__uint_as_float(wv[i] << 16)) + fabsf(__uint_as_float(wv[i] & 0xffff0000u));
+#pragma unroll
+    for (int o = 8; o; o >>= 1) new_norm += __shfl_xor_sync(0xffffffffu, new_norm, o);
+    new_norm = __shfl_sync(0xffffffffu, new_norm, 16);      // the V half's sum
+  }
+  if (owns_new && wid == 0) {
+    __nv_bfloat16* dst = (__nv_bfloat16*)(lane < 16 ? c.k_cache : c.v_cache) + ((int64_t)u * cap + fs) * HD;
+    reinterpret_cast<uint4*>(dst)[lane & 15] = new_raw;
+    if (lane == 0) {
+      c.vnorm[(int64_t)u * cap + fs] = new_norm;
+      c.pos[(int64_t)u * cap + fs] = t;
+    }
+  }
+
+  // ---- stream the groups: logits, online softmax, partial output ----
+  float m_run = -INFINITY, l_run = 0.f;
+  float o_acc[HD / 8][4];
+#pragma unroll
+  for (int i = 0; i < HD / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
+  bool ok = true;
+  // ldmatrix lane addressing: matrix i = lane / 8, row r = lane % 8
+  const int lm_i = lane >> 3, lm_r = lane & 7;
+  const uint32_t k_lane_off = (uint32_t)(((lm_i >> 1) * 8 + lm_r) * PITCH + (lm_i & 1) * 16);   // K: matrices (rows 0-7, k lo), (rows 0-7, k hi), (rows 8-15, k lo), (rows 8-15, k hi)
+  const uint32_t v_lane_off = (uint32_t)(((lm_i & 1) * 8 + lm_r) * PITCH + (lm_i >> 1) * 16);    // V: (rows 0-7, n lo), (rows 8-15, n lo), (rows 0-7, n hi), (rows 8-15, n hi)
+  int it = 0;
+  for (int g = wid; g < ngroups; g += MW, ++it) {
+    if (it >= nstage && g * GROUP >= cnt) break;     // never requested (see the end of the loop body)
+    const int stage = it % nstage;
+    const uint32_t parity = (it / nstage) & 1;
+    if (ok && !mbar_wait(&my_bars[stage], parity)) ok = false;
+    ok = __all_sync(0xffffffffu, ok);
+    unsigned char* ks = my_stages + stage * STAGE_BYTES;
+    unsigned char* vs = ks + GROUP * PITCH;
+    const int r0 = g * GROUP;
+    bool wrote = false;
+    if (ok && r0 < cnt) {
+      // the incoming token's row is not in the cache yet: patch it in; rows beyond the live range
+      // must not reach the p V product (their probability is 0, but 0 * garbage need not be 0)
+      if (owns_new && fs_local >= r0 && fs_local < r0 + GROUP) {
+        *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (fs_local - r0) * PITCH + (lane & 15) * 16) = new_raw;
+        wrote = true;
+      }
+      if (cnt < r0 + GROUP) {
+        for (int rr = cnt - r0 + (lane >> 4); rr < GROUP; rr += 2)
+          *reinterpret_cast<uint4*>(vs + rr * PITCH + (lane & 15) * 16) = make_uint4(0u, 0u, 0u, 0u);
+        wrote = true;
+      }
+      __syncwarp();
+      // S^T = q K^T: two n-tiles of 8 rows; c[0], c[1] = logits of rows 2 j4, 2 j4 + 1 of the tile
+      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+      const uint32_t kaddr = smem_u32(ks) + k_lane_off;
+#pragma unroll
+      for (int kk = 0; kk < HD / 16; ++kk) {
+        uint32_t bf[4];
+        ldsm_x4(kaddr + kk * 32, bf);
+        mma_bf16(sa, qa[kk][0], 0u, qa[kk][1], 0u, bf[0], bf[1]);
+        mma_bf16(sb, qa[kk][0], 0u, qa[kk][1], 0u, bf[2], bf[3]);
+      }
+      float s[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
+      const int rows[4] = {r0 + 2 * j4, r0 + 2 * j4 + 1, r0 + 8 + 2 * j4, r0 + 9 + 2 * j4};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (rows[i] >= cnt) s[i] = -INFINITY;
+      if (lane < 4) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (rows[i] < cnt) logit_s[rows[i]] = s[i];
+      }
+      float gmax = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+      gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+      gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+      if (gmax > m_run) {          // warp-uniform (r0 < cnt guarantees a live row, so gmax is finite)
+        const float f = ex2(m_run - gmax);   // 0 on the first group
+        l_run *= f;
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i) { o_acc[i][0] *= f; o_acc[i][1] *= f; o_acc[i][2] *= f; o_acc[i][3] *= f; }
+        m_run = gmax;
+      }
+      float p[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) { p[i] = ex2(s[i] - m_run); l_run += p[i]; }
+      // A operand of p V: rows 0-7 carry the high bf16 half of p, rows 8-15 the remainder
+      const uint32_t hi0 = pack_bf16(p[0], p[1]), hi1 = pack_bf16(p[2], p[3]);
+      const uint32_t lo0 = pack_bf16(p[0] - __uint_as_float(hi0 << 16), p[1] - __uint_as_float(hi0 & 0xffff0000u));
+      const uint32_t lo1 = pack_bf16(p[2] - __uint_as_float(hi1 << 16), p[3] - __uint_as_float(hi1 & 0xffff0000u));
+      const uint32_t vaddr = smem_u32(vs) + v_lane_off;
+#pragma unroll
+      for (int nn = 0; nn < HD / 16; ++nn) {
+        uint32_t bf[4];
+        ldsm_x4_t(vaddr + nn * 32, bf);
+        mma_bf16(o_acc[2 * nn], hi0, lo0, hi1, lo1, bf[0], bf[1]);
+        mma_bf16(o_acc[2 * nn + 1], hi0, lo0, hi1, lo1, bf[2], bf[3]);
+      }
+    }
+    // generic-proxy stores into a stage must be ordered before the next bulk copy into it
+    if (wrote) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    const int next = g + nstage * MW;
+    // later requests know the live range: rows beyond it are not fetched
+    if (ok && next < ngroups && next * GROUP < cnt) issue(next, stage, cnt);
+  }
+  if (!ok && lane == 0) {
+    // a copy never completed: flag it and give what is still in flight one more bounded wait
+    if (dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+    for (int s = 0; s < nstage; ++s) mbar_wait(&my_bars[s], 0);
+  }
+  // warp partial: every lane with the same j4 holds the same values; rows 0-7 are the hi part, 8-15 the lo part
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
+  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
+  if (lane < 4) {
+#pragma unroll
+    for (int i = 0; i < HD / 8; ++i)
+      *reinterpret_cast<float2*>(&part_o[wid][i * 8 + 2 * j4]) = make_float2(o_acc[i][0] + o_acc[i][2], o_acc[i][1] + o_acc[i][3]);
+    if (lane == 0) { part_m[wid] = m_run; part_l[wid] = l_run; }
+  }
+  __syncthreads();
+
+  // ---- CTA partial, pushed to the cluster ----
+  {
+    float m_c = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < MW; ++i) m_c = fmaxf(m_c, part_m[i]);
+    float fw[MW], l_c = 0.f;
+#pragma unroll
+    for (int i = 0; i < MW; ++i) {
+      fw[i] = part_m[i] > -INFINITY ? ex2(part_m[i] - m_c) : 0.f;
+      l_c += part_l[i] * fw[i];
+    }
+    if (tid < HD) {
+      float a = 0.f;
+#pragma unroll
+      for (int i = 0; i < MW; ++i) a = fmaf(part_o[i][tid], fw[i], a);
+      float* dst = split > 1 ? cluster.map_shared_rank(&ex.o[rank][tid], 0) : &ex.o[rank][tid];
+      *dst = a;
+    } else if (tid < HD + split) {
+      const int r = tid - HD;
+      Exch* e = split > 1 ? cluster.map_shared_rank(&ex, r) : &ex;
+      e->m[rank] = m_c;
+      e->l[rank] = l_c;
+    }
+  }
+  if (split > 1) cluster.sync(); else __syncthreads();
+
+  // ---- combine the CTAs of the unit (all data is local now) ----
+  float m_all = -INFINITY, L = 0.f;
+  float fr[MAX_SPLIT];
+#pragma unroll
+  for (int r = 0; r < MAX_SPLIT; ++r)
+    if (r < split) m_all = fmaxf(m_all, ex.m[r]);
+#pragma unroll
+  for (int r = 0; r < MAX_SPLIT; ++r) {
+    fr[r] = (r < split && ex.m[r] > -INFINITY) ? ex2(ex.m[r] - m_all) : 0.f;
+    if (r < split) L += ex.l[r] * fr[r];
+  }
+  const float invL = 1.f / L;
+  if (rank == 0 && tid < HD) {
+    float a = 0.f;
+#pragma unroll
+    for (int r = 0; r < MAX_SPLIT; ++r)
+      if (r < split) a = fmaf(ex.o[r][tid], fr[r], a);
+    out[(int64_t)u * HD + tid] = __float2bfloat16(a * invL);
+  }
+
+  // ---- indicator update (Eq. 2 / Eq. 3), importance (Eq. 4), arg-min key ----
+  if (rows_alloc > 0 && !mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+  const bool evicting = hi > B;
+  unsigned long long my_key = NO_KEY;
+  int my_slot = -1, my_pos = -1;
+  for (int r = tid; r < cnt; r += MT) {
+    const int slot = s0 + r;
+    const int64_t o = (int64_t)u * cap + slot;
+    const float p = ex2(logit_s[r] - m_all) * invL;
+    const bool is_new = slot == fs;
+    float S;
+    if (WINDOWED) {
+      float* ring_row = c.ring + ((int64_t)u * w + (t % w)) * cap;
+      long long fx;
+      if (is_new) {
+        // recycled slot: its ring column belongs to the previous occupant
+        for (int rr = 0; rr < w; ++rr) c.ring[((int64_t)u * w + rr) * cap + slot] = 0.f;
+        fx = prob_to_fixed(p);
+      } else {
+        fx = c.acc_fixed[o] + prob_to_fixed(p) - prob_to_fixed(ring_row[slot]);
+      }
+      ring_row[slot] = p;
+      c.acc_fixed[o] = fx;
+      S = fixed_to_prob(fx);
+    } else {
+      S = is_new ? p : acc_s[r] + p;
+    }
+    c.acc[o] = S;
+    if (evicting) {
+      const int ps = is_new ? t : pos_s[r];
+      const float I = S * (is_new ? new_norm : vn_s[r]);
+      if (ps >= F && ps <= t - R) {
+        const unsigned long long key = evict_key(I, ps);
+        if (key < my_key) { my_key = key; my_slot = slot; my_pos = ps; }
+      }
+    }
+  }
+  if (evicting) {
+    // warp minimum of the 64-bit key in two 32-bit steps, pushed to every rank
+    const unsigned hi32 = (unsigned)(my_key >> 32);
+    const unsigned wmin_hi = __reduce_min_sync(0xffffffffu, hi32);
+    const unsigned lo32 = hi32 == wmin_hi ? (unsigned)my_key : 0xffffffffu;
+    const unsigned wmin_lo = __reduce_min_sync(0xffffffffu, lo32);
+    const unsigned long long wkey = ((unsigned long long)wmin_hi << 32) | wmin_lo;
+    if (lane < split) {
+      unsigned long long* dst = split > 1 ? cluster.map_shared_rank(&ex.key[rank][wid], lane) : &ex.key[rank][wid];
+      *dst = wkey;
+    }
+    if (split > 1) cluster.sync(); else __syncthreads();
+    // every warp reduces the split x MW candidates, now local, to the unit's winner
+    unsigned long long win = NO_KEY;
+    {
+      const unsigned long long* all = &ex.key[0][0];
+      const unsigned long long k0 = lane < split * MW ? all[lane] : NO_KEY;
+      const unsigned long long k1 = lane + 32 < split * MW ? all[lane + 32] : NO_KEY;
+      const unsigned long long kk = k0 < k1 ? k0 : k1;
+      const unsigned h = (unsigned)(kk >> 32);
+      const unsigned mh = __reduce_min_sync(0xffffffffu, h);
+      const unsigned ml = __reduce_min_sync(0xffffffffu, h == mh ? (unsigned)kk : 0xffffffffu);
+      win = ((unsigned long long)mh << 32) | ml;
+    }
+    if (win != NO_KEY && my_key == win) {      // positions are unique: exactly one thread of the unit matches
+      c.pos[(int64_t)u * cap + my_slot] = -1;
+      c.free_slot[u] = my_slot;
+      c.len[u] = hi - 1;
+      if (evicted) evicted[u] = my_pos;
+    }
+    if (rank == 0 && tid == 0) {
+      if (win == NO_KEY) {   // nothing eligible (cannot happen when F + R <= B): keep the state consistent
+        c.len[u] = hi;
+        c.free_slot[u] = min(hi, cap - 1);
+        if (evicted) evicted[u] = -1;
+      }
+      c.next_pos[u] = t + 1;
+    }
+  } else if (rank == 0 && tid == 0) {
+    c.len[u] = hi;
+    c.free_slot[u] = hi;
+    c.next_pos[u] = t + 1;
+    if (evicted) evicted[u] = -1;
+  }
+}
+
+}  // namespace
+
+// Returns cudaErrorNotSupported when the shape does not fit this kernel's shared memory (the caller
+// then takes the general kernel).
+cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
+                              const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st) {
+  const int cap = cache_capacity(B);
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  // one CTA per SM: split a unit over a cluster while the grid still fits the machine
+  int split = 1;
+  while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
+  int chunk = (cap + split - 1) / split;
+  chunk = (chunk + GROUP - 1) / GROUP * GROUP;
+  const size_t state_bytes = 4 * sizeof(float) * (size_t)chunk;
+  const size_t budget = 216 * 1024;
+  if (state_bytes + (size_t)MW * STAGE_BYTES > budget) return cudaErrorNotSupported;
+  int nstage = (int)((budget - state_bytes) / ((size_t)MW * STAGE_BYTES));
+  nstage = nstage > 3 ? 3 : nstage;
+  const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
+  if (nstage > groups_per_warp) nstage = groups_per_warp > 0 ? groups_per_warp : 1;
+  const size_t dyn = (size_t)MW * nstage * STAGE_BYTES + state_bytes;
+  const bool win = s.window > 0;
+  auto kern = win ? decode_mma_kernel<true> : decode_mma_kernel<false>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget);
+  if (e != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(s.units * split);
+  cfg.blockDim = dim3(MT);
+  cfg.dynamicSmemBytes = dyn;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = split;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
+                            (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
+                            (__nv_bfloat16*)out, evicted, dev_status);
+}
+
+}  // namespace vatp

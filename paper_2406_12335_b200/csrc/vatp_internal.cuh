@@ -46,6 +46,10 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
                           const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st);
 
+// bf16, head_dim 128 only; cudaErrorNotSupported when the shape does not fit (take launch_decode's general kernel)
+cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
+                              const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st);
+
 // fixed-point image of a probability for the exact window sums (Eq. 3): p in [0, 1] -> p * 2^52
 __host__ __device__ inline long long prob_to_fixed(float p) { return (long long)((double)p * 4503599627370496.0); }
 __host__ __device__ inline float fixed_to_prob(long long x) { return (float)((double)x * (1.0 / 4503599627370496.0)); }
