@@ -81,6 +81,9 @@ typedef struct {
   float   *ring;              /* windowed only: [batch, heads, w, cap] last w probability rows,
                                  row (j mod w) holds query position j; else NULL                */
   int64_t *acc_fixed;         /* windowed only: [batch, heads, cap] exact fixed-point window sum */
+  int32_t *last_slot;         /* [batch, heads] slot the previous step wrote its token to, -1 after
+                                 compaction; lets a step that overlaps the tail of the previous one
+                                 re-read that one row                                            */
 } vatp_cache;
 
 /* Slots per unit of the decode state for a budget of B tokens (see vatp_cache). */
@@ -151,7 +154,8 @@ vatp_status vatp_select(const vatp_params* params, const float* score, int32_t* 
 /*
  * Compaction: gather the surviving K/V rows (bit-exact copies, ascending original index) into
  * the budgeted cache and initialise the decode state: acc <- attn_acc[kept], vnorm <- vnorm[kept],
- * pos <- kept index, len <- min(T, B), free_slot <- len, next_pos <- T; unused slots get pos -1.
+ * pos <- kept index, len <- min(T, B), free_slot <- len, next_pos <- T, last_slot <- -1; unused slots
+ * get pos -1.
  * VATP_IND_WINDOW also gathers win_rows columns into `ring` (row (T - w + r) mod w) and sets
  * acc_fixed to the fixed-point window sums.
  */

@@ -63,6 +63,7 @@ compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict_
     c.len[u] = len;
     c.free_slot[u] = len;
     c.next_pos[u] = sh.T;
+    c.last_slot[u] = -1;
   }
 }
 

@@ -403,6 +403,7 @@ decode_kernel(int split, int chunk, int B, int cap, int F, int R, int w, float s
       c.free_slot[u] = hi;
     }
     c.next_pos[u] = t + 1;
+    c.last_slot[u] = fs;
     if (evicted) evicted[u] = ev_pos;
   }
 }

@@ -2,19 +2,21 @@
 // update (Eq. 2 / Eq. 3), importance (Eq. 4), release of the lowest-importance unprotected slot.
 //
 // The step is HBM-bound (every cached K and V row is read once) but so short - tens of megabytes -
-// that the latency of each warp's own instruction stream decides its duration.  Hence:
-//   * every warp owns a ring of stages and requests its rows with one bulk copy per row (all 32
-//     lanes issue at once) before anything else happens; rows land on a 272-byte pitch, which makes
-//     ldmatrix conflict-free;
+// that fixed latencies decide its duration.  Hence:
+//   * every warp owns a ring of stages and requests its first stages (tiled TMA loads of 16 rows x
+//     128 bytes, 128-byte swizzled so that ldmatrix is conflict-free) before anything else happens;
 //   * q.K^T and p.V run on the warp-level tensor-core path (mma.sync m16n8k16, bf16 in, fp32
 //     accumulate): S^T = q K^T leaves the probabilities of 16 rows in exactly the registers the
-//     A operand of p V wants, so a 16-row group costs about 80 instructions instead of several
-//     hundred.  p is split into two bf16 halves (rows 0-7 / 8-15 of the A tile carry hi / lo), so
-//     the product keeps ~16 bits of p;
-//   * a unit is split over a thread-block cluster when units are few.  CTAs exchange by PUSHING into
-//     each other's shared memory before a cluster barrier (partial max / sum to every rank, partial
-//     output to rank 0, every warp's arg-min candidate to every rank), so nobody reads remote
-//     memory after a barrier: two cluster barriers per step, no global scratch, one launch.
+//     A operand of p V wants, so a 16-row group costs about 80 instructions.  p is split into two
+//     bf16 halves (rows 0-7 / 8-15 of the A tile carry hi / lo): the product keeps ~16 bits of p;
+//   * a unit is split over a thread-block cluster when units are few.  The CTAs PUSH what rank 0
+//     needs (every logit, and per CTA the running max, sum and partial output) into rank 0's shared
+//     memory, meet at ONE cluster barrier and retire; rank 0 alone normalises, updates the
+//     indicators and finds the arg-min.  No global scratch, one launch;
+//   * consecutive steps overlap (programmatic dependent launch): a step requests its first K/V
+//     tiles while the previous step's tail still runs, and reads everything else only after that
+//     step has completed.  The one cache row the previous step may have written - the row of its
+//     incoming token, recorded in last_slot - is re-read after that point and patched in.
 #include <cooperative_groups.h>
 
 #include "vatp_internal.cuh"
@@ -29,8 +31,8 @@ constexpr int MT = MW * 32;
 constexpr int HD = 128;
 constexpr int GROUP = 16;             // rows per MMA group = rows of K (and of V) per stage
 constexpr int ROW_BYTES = HD * 2;
-constexpr int PITCH = ROW_BYTES + 16; // shared-memory row pitch
-constexpr int STAGE_BYTES = 2 * GROUP * PITCH;
+constexpr int TILE_BYTES = GROUP * 128;    // 16 rows x 64 bf16, 128-byte swizzled
+constexpr int STAGE_BYTES = 4 * TILE_BYTES; // K columns 0-63, K 64-127, V 0-63, V 64-127
 constexpr int MAX_SPLIT = 8;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr unsigned long long NO_KEY = ~0ull;
@@ -71,6 +73,12 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
@@ -98,36 +106,47 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// what the CTAs of a unit push to one another
+// what the CTAs of a unit push into rank 0
 struct Exch {
   float m[MAX_SPLIT], l[MAX_SPLIT];       // per rank: max of its logits (log2 domain), sum of exp2(s - m)
-  unsigned long long key[MAX_SPLIT][MW];  // arg-min candidate of every warp of every rank
-  float o[MAX_SPLIT][HD];                 // rank 0 only: partial outputs of every rank
+  float o[MAX_SPLIT][HD];                 // partial outputs of every rank
 };
 
 // eviction order as one integer: lower importance first, among equals the higher position first
 __device__ __forceinline__ unsigned long long evict_key(float I, int pos) {
   return ((unsigned long long)__float_as_uint(I) << 32) | (unsigned)(0x7fffffff - pos);
 }
+// minimum of a 64-bit key over the warp, in two 32-bit steps
+__device__ __forceinline__ unsigned long long warp_min_key(unsigned long long key) {
+  const unsigned h = (unsigned)(key >> 32);
+  const unsigned mh = __reduce_min_sync(0xffffffffu, h);
+  const unsigned ml = __reduce_min_sync(0xffffffffu, h == mh ? (unsigned)key : 0xffffffffu);
+  return ((unsigned long long)mh << 32) | ml;
+}
 
 template <bool WINDOWED>
 __global__ void __launch_bounds__(MT, 1)
-decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
+decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int split,
+                  int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
                   const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
-  extern __shared__ __align__(128) unsigned char dyn[];
-  // [MW][nstage][K rows | V rows] | logits[chunk] | acc[chunk] | vnorm[chunk] | pos[chunk]
+  extern __shared__ unsigned char dyn_raw[];
+  unsigned char* dyn = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dyn_raw) + 1023) & ~uintptr_t(1023));
+  // [MW][nstage] stages | logits[tot] | acc[tot] | vnorm[tot] | pos[tot]; the per-slot arrays span the
+  // whole unit and are used by rank 0 only
+  const int tot = split * chunk;
   unsigned char* stage_base = dyn;
   float* logit_s = reinterpret_cast<float*>(dyn + (size_t)MW * nstage * STAGE_BYTES);
-  float* acc_s = logit_s + chunk;
-  float* vn_s = acc_s + chunk;
-  int* pos_s = reinterpret_cast<int*>(vn_s + chunk);
+  float* acc_s = logit_s + tot;
+  float* vn_s = acc_s + tot;
+  int* pos_s = reinterpret_cast<int*>(vn_s + tot);
 
   __shared__ __align__(8) uint64_t bars[MW * 4 + 1];
   __shared__ __align__(16) Exch ex;
   __shared__ __align__(16) float part_o[MW][HD];
   __shared__ float part_m[MW], part_l[MW];
+  __shared__ unsigned long long warp_key[MW];
 
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = split > 1 ? (int)cluster.block_rank() : 0;
@@ -135,12 +154,15 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   const int j4 = lane & 3;
 
+  // Remote shared memory may only be touched once its CTA runs: everyone arrives here, and waits
+  // (long since satisfied) just before the first remote store.
+  if (split > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+
   // this CTA's slot range inside the allocation
   const int s0 = min(rank * chunk, cap);
   const int rows_alloc = min(chunk, cap - s0);
   const int ngroups = (rows_alloc + GROUP - 1) / GROUP;
-  const __nv_bfloat16* kc = (const __nv_bfloat16*)c.k_cache + ((int64_t)u * cap + s0) * HD;
-  const __nv_bfloat16* vc = (const __nv_bfloat16*)c.v_cache + ((int64_t)u * cap + s0) * HD;
+  const int row_base = u * cap + s0;     // first row of the range in the [units * cap, 128] view of the caches
   uint64_t* my_bars = &bars[wid * 4];
   uint64_t* state_bar = &bars[MW * 4];
   unsigned char* my_stages = stage_base + (size_t)wid * nstage * STAGE_BYTES;
@@ -152,37 +174,38 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncwarp();
-  // lanes 0-15 fetch the K rows of group g, lanes 16-31 its V rows
-  auto issue = [&](int g, int stage, int limit) {
-    const int r0 = g * GROUP;
-    const int n = min(GROUP, limit - r0);
+  // lanes 0-3 fetch the four tiles of group g (rows beyond the caches arrive as zeros)
+  auto issue = [&](int g, int stage) {
     unsigned char* dst = my_stages + stage * STAGE_BYTES;
     uint64_t* bar = &my_bars[stage];
-    if (lane == 0) mbar_expect_tx(bar, 2u * n * ROW_BYTES);
+    if (lane == 0) mbar_expect_tx(bar, STAGE_BYTES);
     __syncwarp();
-    const int rr = lane & 15;
-    if (rr < n) {
-      const __nv_bfloat16* src = (lane < 16 ? kc : vc) + (int64_t)(r0 + rr) * HD;
-      bulk_g2s(dst + (lane < 16 ? 0 : GROUP * PITCH) + rr * PITCH, src, ROW_BYTES, bar);
-    }
+    if (lane < 4) tma_load_2d(dst + lane * TILE_BYTES, lane < 2 ? &tm_k : &tm_v, bar, (lane & 1) * 64, row_base + g * GROUP);
   };
   for (int s = 0; s < nstage; ++s)
-    if (wid + s * MW < ngroups) issue(wid + s * MW, s, rows_alloc);
-  if (tid == 32 && rows_alloc > 0) {      // per-slot state of the range
-    const int64_t o = (int64_t)u * cap + s0;
-    mbar_expect_tx(state_bar, 3u * rows_alloc * 4u);
-    bulk_g2s(acc_s, c.acc + o, rows_alloc * 4, state_bar);
-    bulk_g2s(vn_s, c.vnorm + o, rows_alloc * 4, state_bar);
-    bulk_g2s(pos_s, c.pos + o, rows_alloc * 4, state_bar);
+    if (wid + s * MW < ngroups) issue(wid + s * MW, s);
+  // The next launch in the stream may start now; nothing below this line is read before the previous
+  // launch has completed and its writes are visible.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (rank == 0 && tid == 32) {      // per-slot state of the whole unit
+    const int64_t o = (int64_t)u * cap;
+    mbar_expect_tx(state_bar, 3u * cap * 4u);
+    bulk_g2s(acc_s, c.acc + o, cap * 4, state_bar);
+    bulk_g2s(vn_s, c.vnorm + o, cap * 4, state_bar);
+    bulk_g2s(pos_s, c.pos + o, cap * 4, state_bar);
   }
 
   const int len = c.len[u];
   const int fs = c.free_slot[u];
   const int t = c.next_pos[u];
+  const int ls = c.last_slot[u];
   const int hi = len + 1;                // slots [0, hi) are live once the new token is in
   const int cnt = max(min(hi - s0, rows_alloc), 0);
   const int fs_local = fs - s0;          // row of the incoming token inside this CTA's range (if owned)
   const bool owns_new = fs_local >= 0 && fs_local < cnt;
+  const int ls_local = ls - s0;          // row the previous step appended (its tile may predate that store)
+  const bool owns_last = ls >= 0 && ls != fs && ls_local >= 0 && ls_local < cnt;
 
   // A operand of q K^T: q replicated over the rows 0-7 of the tile (rows 8-15 zero)
   const __nv_bfloat16* qn = q_new + (int64_t)u * HD;
@@ -194,6 +217,11 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
   }
   // 16 bytes of the incoming K row (lanes 0-15) or V row (lanes 16-31)
   const uint4 new_raw = __ldg(reinterpret_cast<const uint4*>((lane < 16 ? k_new : v_new) + (int64_t)u * HD) + (lane & 15));
+
+  uint4 last_raw = make_uint4(0u, 0u, 0u, 0u);
+  if (owns_last)
+    last_raw = *(reinterpret_cast<const uint4*>((const __nv_bfloat16*)(lane < 16 ? c.k_cache : c.v_cache) +
+                                                ((int64_t)u * cap + ls) * HD) + (lane & 15));
 
   // ---- append: the CTA that owns the free slot stores the new row and its l1 norm ----
   float new_norm = 0.f;
@@ -214,6 +242,8 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
       c.pos[(int64_t)u * cap + fs] = t;
     }
   }
+  if (split > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  float* logit_r0 = split > 1 ? cluster.map_shared_rank(logit_s, 0) : logit_s;
 
   // ---- stream the groups: logits, online softmax, partial output ----
   float m_run = -INFINITY, l_run = 0.f;
@@ -221,10 +251,13 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
 #pragma unroll
   for (int i = 0; i < HD / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
   bool ok = true;
-  // ldmatrix lane addressing: matrix i = lane / 8, row r = lane % 8
+  // ldmatrix lane addressing: matrix i = lane / 8, row r = lane % 8.  A tile row is 128 bytes and its
+  // 16-byte chunk c sits at position c ^ (row % 8).
+  //   K (plain):  matrices (rows 0-7, k lo), (rows 0-7, k hi), (rows 8-15, k lo), (rows 8-15, k hi)
+  //   V (trans):  matrices (rows 0-7, n lo), (rows 8-15, n lo), (rows 0-7, n hi), (rows 8-15, n hi)
   const int lm_i = lane >> 3, lm_r = lane & 7;
-  const uint32_t k_lane_off = (uint32_t)(((lm_i >> 1) * 8 + lm_r) * PITCH + (lm_i & 1) * 16);   // K: matrices (rows 0-7, k lo), (rows 0-7, k hi), (rows 8-15, k lo), (rows 8-15, k hi)
-  const uint32_t v_lane_off = (uint32_t)(((lm_i & 1) * 8 + lm_r) * PITCH + (lm_i >> 1) * 16);    // V: (rows 0-7, n lo), (rows 8-15, n lo), (rows 0-7, n hi), (rows 8-15, n hi)
+  const uint32_t k_row_off = (uint32_t)(((lm_i >> 1) * 8 + lm_r) * 128), k_x = (uint32_t)((lm_i & 1) ^ lm_r);
+  const uint32_t v_row_off = (uint32_t)(((lm_i & 1) * 8 + lm_r) * 128), v_x = (uint32_t)((lm_i >> 1) ^ lm_r);
   int it = 0;
   for (int g = wid; g < ngroups; g += MW, ++it) {
     if (it >= nstage && g * GROUP >= cnt) break;     // never requested (see the end of the loop body)
@@ -233,29 +266,35 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
     if (ok && !mbar_wait(&my_bars[stage], parity)) ok = false;
     ok = __all_sync(0xffffffffu, ok);
     unsigned char* ks = my_stages + stage * STAGE_BYTES;
-    unsigned char* vs = ks + GROUP * PITCH;
+    unsigned char* vs = ks + 2 * TILE_BYTES;
     const int r0 = g * GROUP;
     bool wrote = false;
     if (ok && r0 < cnt) {
       // the incoming token's row is not in the cache yet: patch it in; rows beyond the live range
       // must not reach the p V product (their probability is 0, but 0 * garbage need not be 0)
       if (owns_new && fs_local >= r0 && fs_local < r0 + GROUP) {
-        *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (fs_local - r0) * PITCH + (lane & 15) * 16) = new_raw;
+        const int rr = fs_local - r0, ch = lane & 15;
+        *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = new_raw;
+        wrote = true;
+      }
+      if (owns_last && ls_local >= r0 && ls_local < r0 + GROUP) {
+        const int rr = ls_local - r0, ch = lane & 15;
+        *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = last_raw;
         wrote = true;
       }
       if (cnt < r0 + GROUP) {
         for (int rr = cnt - r0 + (lane >> 4); rr < GROUP; rr += 2)
-          *reinterpret_cast<uint4*>(vs + rr * PITCH + (lane & 15) * 16) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(vs + ((lane >> 3) & 1) * TILE_BYTES + rr * 128 + ((lane & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
         wrote = true;
       }
       __syncwarp();
       // S^T = q K^T: two n-tiles of 8 rows; c[0], c[1] = logits of rows 2 j4, 2 j4 + 1 of the tile
       float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-      const uint32_t kaddr = smem_u32(ks) + k_lane_off;
+      const uint32_t kaddr = smem_u32(ks) + k_row_off;
 #pragma unroll
       for (int kk = 0; kk < HD / 16; ++kk) {
         uint32_t bf[4];
-        ldsm_x4(kaddr + kk * 32, bf);
+        ldsm_x4(kaddr + (kk >> 2) * TILE_BYTES + ((k_x ^ ((2 * kk) & 7)) << 4), bf);
         mma_bf16(sa, qa[kk][0], 0u, qa[kk][1], 0u, bf[0], bf[1]);
         mma_bf16(sb, qa[kk][0], 0u, qa[kk][1], 0u, bf[2], bf[3]);
       }
@@ -267,7 +306,7 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
       if (lane < 4) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          if (rows[i] < cnt) logit_s[rows[i]] = s[i];
+          if (rows[i] < cnt) logit_r0[s0 + rows[i]] = s[i];
       }
       float gmax = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
       gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
@@ -286,11 +325,11 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
       const uint32_t hi0 = pack_bf16(p[0], p[1]), hi1 = pack_bf16(p[2], p[3]);
       const uint32_t lo0 = pack_bf16(p[0] - __uint_as_float(hi0 << 16), p[1] - __uint_as_float(hi0 & 0xffff0000u));
       const uint32_t lo1 = pack_bf16(p[2] - __uint_as_float(hi1 << 16), p[3] - __uint_as_float(hi1 & 0xffff0000u));
-      const uint32_t vaddr = smem_u32(vs) + v_lane_off;
+      const uint32_t vaddr = smem_u32(vs) + v_row_off;
 #pragma unroll
       for (int nn = 0; nn < HD / 16; ++nn) {
         uint32_t bf[4];
-        ldsm_x4_t(vaddr + nn * 32, bf);
+        ldsm_x4_t(vaddr + (nn >> 2) * TILE_BYTES + ((v_x ^ ((2 * nn) & 7)) << 4), bf);
         mma_bf16(o_acc[2 * nn], hi0, lo0, hi1, lo1, bf[0], bf[1]);
         mma_bf16(o_acc[2 * nn + 1], hi0, lo0, hi1, lo1, bf[2], bf[3]);
       }
@@ -299,8 +338,8 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
     if (wrote) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     __syncwarp();
     const int next = g + nstage * MW;
-    // later requests know the live range: rows beyond it are not fetched
-    if (ok && next < ngroups && next * GROUP < cnt) issue(next, stage, cnt);
+    // later requests know the live range: groups beyond it are not fetched
+    if (ok && next < ngroups && next * GROUP < cnt) issue(next, stage);
   }
   if (!ok && lane == 0) {
     // a copy never completed: flag it and give what is still in flight one more bounded wait
@@ -318,8 +357,8 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
   }
   __syncthreads();
 
-  // ---- CTA partial, pushed to the cluster ----
-  {
+  // ---- CTA partial, pushed into rank 0 ----
+  if (tid <= HD) {
     float m_c = -INFINITY;
 #pragma unroll
     for (int i = 0; i < MW; ++i) m_c = fmaxf(m_c, part_m[i]);
@@ -329,22 +368,21 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
       fw[i] = part_m[i] > -INFINITY ? ex2(part_m[i] - m_c) : 0.f;
       l_c += part_l[i] * fw[i];
     }
+    Exch* e0 = split > 1 ? cluster.map_shared_rank(&ex, 0) : &ex;
     if (tid < HD) {
       float a = 0.f;
 #pragma unroll
       for (int i = 0; i < MW; ++i) a = fmaf(part_o[i][tid], fw[i], a);
-      float* dst = split > 1 ? cluster.map_shared_rank(&ex.o[rank][tid], 0) : &ex.o[rank][tid];
-      *dst = a;
-    } else if (tid < HD + split) {
-      const int r = tid - HD;
-      Exch* e = split > 1 ? cluster.map_shared_rank(&ex, r) : &ex;
-      e->m[rank] = m_c;
-      e->l[rank] = l_c;
+      e0->o[rank][tid] = a;
+    } else {
+      e0->m[rank] = m_c;
+      e0->l[rank] = l_c;
     }
   }
   if (split > 1) cluster.sync(); else __syncthreads();
+  if (rank != 0) return;      // nothing of this CTA's shared memory is read by others
 
-  // ---- combine the CTAs of the unit (all data is local now) ----
+  // ---- rank 0: combine the CTAs of the unit (all data is local now) ----
   float m_all = -INFINITY, L = 0.f;
   float fr[MAX_SPLIT];
 #pragma unroll
@@ -356,7 +394,7 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
     if (r < split) L += ex.l[r] * fr[r];
   }
   const float invL = 1.f / L;
-  if (rank == 0 && tid < HD) {
+  if (tid < HD) {
     float a = 0.f;
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r)
@@ -364,15 +402,15 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
     out[(int64_t)u * HD + tid] = __float2bfloat16(a * invL);
   }
 
-  // ---- indicator update (Eq. 2 / Eq. 3), importance (Eq. 4), arg-min key ----
-  if (rows_alloc > 0 && !mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+  // ---- indicator update (Eq. 2 / Eq. 3), importance (Eq. 4), arg-min ----
+  if (!mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
   const bool evicting = hi > B;
   unsigned long long my_key = NO_KEY;
   int my_slot = -1, my_pos = -1;
-  for (int r = tid; r < cnt; r += MT) {
-    const int slot = s0 + r;
+#pragma unroll 4
+  for (int slot = tid; slot < hi; slot += MT) {
     const int64_t o = (int64_t)u * cap + slot;
-    const float p = ex2(logit_s[r] - m_all) * invL;
+    const float p = ex2(logit_s[slot] - m_all) * invL;
     const bool is_new = slot == fs;
     float S;
     if (WINDOWED) {
@@ -389,12 +427,12 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
       c.acc_fixed[o] = fx;
       S = fixed_to_prob(fx);
     } else {
-      S = is_new ? p : acc_s[r] + p;
+      S = is_new ? p : acc_s[slot] + p;
     }
     c.acc[o] = S;
     if (evicting) {
-      const int ps = is_new ? t : pos_s[r];
-      const float I = S * (is_new ? new_norm : vn_s[r]);
+      const int ps = is_new ? t : pos_s[slot];
+      const float I = S * (is_new ? new_norm : vn_s[slot]);
       if (ps >= F && ps <= t - R) {
         const unsigned long long key = evict_key(I, ps);
         if (key < my_key) { my_key = key; my_slot = slot; my_pos = ps; }
@@ -402,47 +440,30 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
     }
   }
   if (evicting) {
-    // warp minimum of the 64-bit key in two 32-bit steps, pushed to every rank
-    const unsigned hi32 = (unsigned)(my_key >> 32);
-    const unsigned wmin_hi = __reduce_min_sync(0xffffffffu, hi32);
-    const unsigned lo32 = hi32 == wmin_hi ? (unsigned)my_key : 0xffffffffu;
-    const unsigned wmin_lo = __reduce_min_sync(0xffffffffu, lo32);
-    const unsigned long long wkey = ((unsigned long long)wmin_hi << 32) | wmin_lo;
-    if (lane < split) {
-      unsigned long long* dst = split > 1 ? cluster.map_shared_rank(&ex.key[rank][wid], lane) : &ex.key[rank][wid];
-      *dst = wkey;
-    }
-    if (split > 1) cluster.sync(); else __syncthreads();
-    // every warp reduces the split x MW candidates, now local, to the unit's winner
-    unsigned long long win = NO_KEY;
-    {
-      const unsigned long long* all = &ex.key[0][0];
-      const unsigned long long k0 = lane < split * MW ? all[lane] : NO_KEY;
-      const unsigned long long k1 = lane + 32 < split * MW ? all[lane + 32] : NO_KEY;
-      const unsigned long long kk = k0 < k1 ? k0 : k1;
-      const unsigned h = (unsigned)(kk >> 32);
-      const unsigned mh = __reduce_min_sync(0xffffffffu, h);
-      const unsigned ml = __reduce_min_sync(0xffffffffu, h == mh ? (unsigned)kk : 0xffffffffu);
-      win = ((unsigned long long)mh << 32) | ml;
-    }
-    if (win != NO_KEY && my_key == win) {      // positions are unique: exactly one thread of the unit matches
+    const unsigned long long wkey = warp_min_key(my_key);
+    if (lane == 0) warp_key[wid] = wkey;
+    __syncthreads();
+    const unsigned long long win = warp_min_key(lane < MW ? warp_key[lane] : NO_KEY);
+    if (win != NO_KEY && my_key == win) {      // positions are unique: exactly one thread matches
       c.pos[(int64_t)u * cap + my_slot] = -1;
       c.free_slot[u] = my_slot;
       c.len[u] = hi - 1;
       if (evicted) evicted[u] = my_pos;
     }
-    if (rank == 0 && tid == 0) {
+    if (tid == 0) {
       if (win == NO_KEY) {   // nothing eligible (cannot happen when F + R <= B): keep the state consistent
         c.len[u] = hi;
         c.free_slot[u] = min(hi, cap - 1);
         if (evicted) evicted[u] = -1;
       }
       c.next_pos[u] = t + 1;
+      c.last_slot[u] = fs;
     }
-  } else if (rank == 0 && tid == 0) {
+  } else if (tid == 0) {
     c.len[u] = hi;
     c.free_slot[u] = hi;
     c.next_pos[u] = t + 1;
+    c.last_slot[u] = fs;
     if (evicted) evicted[u] = -1;
   }
 }
@@ -454,6 +475,7 @@ decode_mma_kernel(int split, int chunk, int nstage, int B, int cap, int F, int R
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
                               const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st) {
   const int cap = cache_capacity(B);
+  if (!vatp_tc_available()) return cudaErrorNotSupported;
   static int sms = 0;
   if (!sms) {
     int dev = 0;
@@ -465,14 +487,18 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
   int chunk = (cap + split - 1) / split;
   chunk = (chunk + GROUP - 1) / GROUP * GROUP;
-  const size_t state_bytes = 4 * sizeof(float) * (size_t)chunk;
-  const size_t budget = 216 * 1024;
-  if (state_bytes + (size_t)MW * STAGE_BYTES > budget) return cudaErrorNotSupported;
-  int nstage = (int)((budget - state_bytes) / ((size_t)MW * STAGE_BYTES));
+  const size_t state_bytes = 4 * sizeof(float) * (size_t)chunk * split;
+  const size_t budget = 215 * 1024;     // dynamic shared memory, of which 1 KB is alignment slack
+  if (state_bytes + (size_t)MW * STAGE_BYTES + 1024 > budget) return cudaErrorNotSupported;
+  int nstage = (int)((budget - 1024 - state_bytes) / ((size_t)MW * STAGE_BYTES));
   nstage = nstage > 3 ? 3 : nstage;
   const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
   if (nstage > groups_per_warp) nstage = groups_per_warp > 0 ? groups_per_warp : 1;
-  const size_t dyn = (size_t)MW * nstage * STAGE_BYTES + state_bytes;
+  const size_t dyn = (size_t)MW * nstage * STAGE_BYTES + state_bytes + 1024;
+  CUtensorMap tm_k, tm_v;
+  if (!make_rows_map_bf16(&tm_k, c.k_cache, (uint64_t)s.units * cap, GROUP) ||
+      !make_rows_map_bf16(&tm_v, c.v_cache, (uint64_t)s.units * cap, GROUP))
+    return cudaErrorInvalidValue;
   const bool win = s.window > 0;
   auto kern = win ? decode_mma_kernel<true> : decode_mma_kernel<false>;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget);
@@ -482,14 +508,16 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   cfg.blockDim = dim3(MT);
   cfg.dynamicSmemBytes = dyn;
   cfg.stream = st;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = split;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // may start before the previous launch has drained
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
+  cfg.numAttrs = 2;
+  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
                             (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                             (__nv_bfloat16*)out, evicted, dev_status);
 }

@@ -47,7 +47,8 @@ inline size_t lse_bytes(const vatp_params* p) {
 }
 
 bool cache_ok(const vatp_cache* c, bool windowed) {
-  if (!c || !c->k_cache || !c->v_cache || !c->acc || !c->vnorm || !c->pos || !c->len || !c->free_slot || !c->next_pos)
+  if (!c || !c->k_cache || !c->v_cache || !c->acc || !c->vnorm || !c->pos || !c->len || !c->free_slot || !c->next_pos ||
+      !c->last_slot)
     return false;
   if (!aligned16(c->k_cache) || !aligned16(c->v_cache) || !aligned16(c->acc) || !aligned16(c->vnorm) || !aligned16(c->pos))
     return false;

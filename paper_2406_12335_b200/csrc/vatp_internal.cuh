@@ -1,5 +1,6 @@
 // Internal declarations shared by the kernels of libvatp (not part of the public C ABI).
 #pragma once
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -31,6 +32,10 @@ __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162flo
 
 // true once the tensor-core prefill kernel is usable on the current device (sm_100, driver entry points found)
 bool vatp_tc_available();
+
+// 2-D tensor map over `rows` contiguous rows of 128 bf16: box = 64 columns x box_rows rows, 128-byte
+// swizzle, rows beyond the end read as zeros.  False when the driver entry point is missing.
+bool make_rows_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint32_t box_rows);
 
 // ---- launchers (each returns cudaGetLastError()) ----
 cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const void* k, const void* v, float* lse,

@@ -33,7 +33,7 @@ class Params(C.Structure):
 class CacheStruct(C.Structure):
     _fields_ = [("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("acc", C.c_void_p), ("vnorm", C.c_void_p),
                 ("pos", C.c_void_p), ("len", C.c_void_p), ("free_slot", C.c_void_p), ("next_pos", C.c_void_p),
-                ("ring", C.c_void_p), ("acc_fixed", C.c_void_p)]
+                ("ring", C.c_void_p), ("acc_fixed", C.c_void_p), ("last_slot", C.c_void_p)]
 
 
 _vp = C.c_void_p
@@ -109,13 +109,14 @@ class Cache:
         self.len = torch.zeros(b, h, dtype=torch.int32, device=device)
         self.free_slot = torch.zeros(b, h, dtype=torch.int32, device=device)
         self.next_pos = torch.zeros(b, h, dtype=torch.int32, device=device)
+        self.last_slot = torch.full((b, h), -1, dtype=torch.int32, device=device)
         self.ring = self.acc_fixed = None
         if p.indicator == IND_WINDOW:
             self.ring = torch.zeros(b, h, p.window_w, cap, dtype=torch.float32, device=device)
             self.acc_fixed = torch.zeros(b, h, cap, dtype=torch.int64, device=device)
         self.struct = CacheStruct(*[_ptr(t) for t in (self.k_cache, self.v_cache, self.acc, self.vnorm, self.pos,
                                                        self.len, self.free_slot, self.next_pos, self.ring,
-                                                       self.acc_fixed)])
+                                                       self.acc_fixed, self.last_slot)])
 
     def nbytes(self) -> int:
         return sum(t.numel() * t.element_size() for t in (self.k_cache, self.v_cache, self.acc, self.vnorm, self.pos))

@@ -29,7 +29,7 @@ def test_exports_every_declared_symbol(V):
 def test_struct_layout_matches_header(V):
     assert C.sizeof(V.Params) == 72       # 7 int32 + float + 3 int32 + pad + 3 int64
     assert V.Params.stride_b.offset == 48
-    assert C.sizeof(V.CacheStruct) == 80
+    assert C.sizeof(V.CacheStruct) == 88
 
 
 def test_status_strings(V):
