@@ -13,11 +13,19 @@
 //     needs (every logit, and per CTA the running max, sum and partial output) into rank 0's shared
 //     memory, meet at ONE cluster barrier and retire; rank 0 alone normalises, updates the
 //     indicators and finds the arg-min.  No global scratch, one launch;
-//   * consecutive steps overlap (programmatic dependent launch): a step requests its first K/V
-//     tiles while the previous step's tail still runs, and reads everything else only after that
-//     step has completed.  The one cache row the previous step may have written - the row of its
-//     incoming token, recorded in last_slot - is re-read after that point and patched in.
+//   * consecutive steps overlap (programmatic dependent launch).  A control warp releases the next
+//     launch in the stream at once and then waits for the previous one, so launches complete in
+//     order and every CTA stays resident until its predecessor has completed: the number of
+//     launches in flight is bounded by what fits on the machine, and two CTAs fit on an SM.  The
+//     host keeps, per stream, the buffers of the last launches; a launch that shares no buffer with
+//     any launch that can still be in flight (another layer's or another sequence's cache) runs
+//     without waiting for anything.  Otherwise (same cache, or unknown) a step requests its first
+//     K/V tiles early and reads everything else only after the previous launch has completed; the
+//     one cache row that launch may have written - the row of its incoming token, recorded in
+//     last_slot - is re-read after that point and patched in.
 #include <cooperative_groups.h>
+
+#include <mutex>
 
 #include "vatp_internal.cuh"
 
@@ -26,8 +34,9 @@ namespace cg = cooperative_groups;
 namespace vatp {
 namespace {
 
-constexpr int MW = 8;                 // warps per CTA
-constexpr int MT = MW * 32;
+constexpr int MW = 4;                 // streaming warps per CTA
+constexpr int WT = MW * 32;           // their threads
+constexpr int MT = WT + 32;           // plus one control warp
 constexpr int HD = 128;
 constexpr int GROUP = 16;             // rows per MMA group = rows of K (and of V) per stage
 constexpr int ROW_BYTES = HD * 2;
@@ -106,11 +115,18 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
+// barrier over the streaming warps only (the control warp does not take part)
+__device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" ::"n"(WT) : "memory"); }
+__device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
 // what the CTAs of a unit push into rank 0
 struct Exch {
   float m[MAX_SPLIT], l[MAX_SPLIT];       // per rank: max of its logits (log2 domain), sum of exp2(s - m)
   float o[MAX_SPLIT][HD];                 // partial outputs of every rank
 };
+
+static_assert(WT == HD, "one streaming thread per output channel");
 
 // eviction order as one integer: lower importance first, among equals the higher position first
 __device__ __forceinline__ unsigned long long evict_key(float I, int pos) {
@@ -125,9 +141,9 @@ __device__ __forceinline__ unsigned long long warp_min_key(unsigned long long ke
 }
 
 template <bool WINDOWED>
-__global__ void __launch_bounds__(MT, 1)
-decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int split,
-                  int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
+__global__ void __launch_bounds__(MT, 2)
+decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int independent,
+                  int split, int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
                   const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
@@ -156,7 +172,20 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
   // Remote shared memory may only be touched once its CTA runs: everyone arrives here, and waits
   // (long since satisfied) just before the first remote store.
-  if (split > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+  if (split > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");   // all five warps
+
+  if (wid == MW) {
+    // ---- control warp: release the next launch, then hold this CTA until the previous launch has completed
+    // (it arrives at the unit's barrier at once, so that the streaming warps never wait for it)
+    if (split > 1) { cluster_wait_acquire(); cluster_arrive_release(); }
+    if (lane == 0) {
+      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+    __syncwarp();
+    if (split > 1) cluster_wait_acquire();
+    return;
+  }
 
   // this CTA's slot range inside the allocation
   const int s0 = min(rank * chunk, cap);
@@ -186,8 +215,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (wid + s * MW < ngroups) issue(wid + s * MW, s);
   // The next launch in the stream may start now; nothing below this line is read before the previous
   // launch has completed and its writes are visible.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (!independent) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (rank == 0 && tid == 32) {      // per-slot state of the whole unit
     const int64_t o = (int64_t)u * cap;
     mbar_expect_tx(state_bar, 3u * cap * 4u);
@@ -205,7 +233,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int fs_local = fs - s0;          // row of the incoming token inside this CTA's range (if owned)
   const bool owns_new = fs_local >= 0 && fs_local < cnt;
   const int ls_local = ls - s0;          // row the previous step appended (its tile may predate that store)
-  const bool owns_last = ls >= 0 && ls != fs && ls_local >= 0 && ls_local < cnt;
+  const bool owns_last = !independent && ls >= 0 && ls != fs && ls_local >= 0 && ls_local < cnt;
 
   // A operand of q K^T: q replicated over the rows 0-7 of the tile (rows 8-15 zero)
   const __nv_bfloat16* qn = q_new + (int64_t)u * HD;
@@ -242,7 +270,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       c.pos[(int64_t)u * cap + fs] = t;
     }
   }
-  if (split > 1) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  if (split > 1) cluster_wait_acquire();
   float* logit_r0 = split > 1 ? cluster.map_shared_rank(logit_s, 0) : logit_s;
 
   // ---- stream the groups: logits, online softmax, partial output ----
@@ -355,10 +383,10 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       *reinterpret_cast<float2*>(&part_o[wid][i * 8 + 2 * j4]) = make_float2(o_acc[i][0] + o_acc[i][2], o_acc[i][1] + o_acc[i][3]);
     if (lane == 0) { part_m[wid] = m_run; part_l[wid] = l_run; }
   }
-  __syncthreads();
+  workers_sync();
 
   // ---- CTA partial, pushed into rank 0 ----
-  if (tid <= HD) {
+  {
     float m_c = -INFINITY;
 #pragma unroll
     for (int i = 0; i < MW; ++i) m_c = fmaxf(m_c, part_m[i]);
@@ -374,12 +402,13 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 #pragma unroll
       for (int i = 0; i < MW; ++i) a = fmaf(part_o[i][tid], fw[i], a);
       e0->o[rank][tid] = a;
-    } else {
+    }
+    if (tid == 0) {
       e0->m[rank] = m_c;
       e0->l[rank] = l_c;
     }
   }
-  if (split > 1) cluster.sync(); else __syncthreads();
+  if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync();
   if (rank != 0) return;      // nothing of this CTA's shared memory is read by others
 
   // ---- rank 0: combine the CTAs of the unit (all data is local now) ----
@@ -408,7 +437,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   unsigned long long my_key = NO_KEY;
   int my_slot = -1, my_pos = -1;
 #pragma unroll 4
-  for (int slot = tid; slot < hi; slot += MT) {
+  for (int slot = tid; slot < hi; slot += WT) {
     const int64_t o = (int64_t)u * cap + slot;
     const float p = ex2(logit_s[slot] - m_all) * invL;
     const bool is_new = slot == fs;
@@ -442,7 +471,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   if (evicting) {
     const unsigned long long wkey = warp_min_key(my_key);
     if (lane == 0) warp_key[wid] = wkey;
-    __syncthreads();
+    workers_sync();
     const unsigned long long win = warp_min_key(lane < MW ? warp_key[lane] : NO_KEY);
     if (win != NO_KEY && my_key == win) {      // positions are unique: exactly one thread matches
       c.pos[(int64_t)u * cap + my_slot] = -1;
@@ -468,6 +497,67 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   }
 }
 
+
+// Host-side record, per stream, of the buffers the last launches write and of the share of the
+// machine each occupies.  Every CTA of a launch stays resident until the previous launch has
+// completed, so launch M - j can still be running when M starts only if the launches between them fit
+// on the machine together: M may skip all waiting when it touches nothing that those launches write.
+struct Range {
+  const char* p;
+  size_t n;
+};
+constexpr int HIST = 8, NRANGE = 13;
+struct LaunchRecord {
+  Range w[NRANGE];
+  double share;        // CTAs / (resident CTAs the machine holds of this launch's kind)
+};
+struct StreamHistory {
+  cudaStream_t stream;
+  bool valid;
+  int count, head;     // records held, index of the newest
+  LaunchRecord rec[HIST];
+};
+std::mutex g_hist_mutex;
+StreamHistory g_hist[8];
+int g_hist_next = 0;
+
+inline bool overlaps(const Range& a, const Range& b) {
+  return a.p && b.p && a.n && b.n && a.p < b.p + b.n && b.p < a.p + a.n;
+}
+
+// true when `touched` overlaps nothing that a launch possibly still in flight on `st` writes; records this launch
+bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, const Range* written, double share) {
+  std::lock_guard<std::mutex> lock(g_hist_mutex);
+  StreamHistory* h = nullptr;
+  for (auto& x : g_hist)
+    if (x.valid && x.stream == st) h = &x;
+  if (!h) {
+    h = &g_hist[g_hist_next];
+    g_hist_next = (g_hist_next + 1) % 8;
+    h->stream = st;
+    h->valid = true;
+    h->count = 0;
+    h->head = -1;
+  }
+  // the first recorded launch followed a kernel that releases nothing early: everything before it had completed
+  bool indep = h->count > 0;
+  double between = 0.0;      // machine share of the launches between the candidate and this one
+  for (int j = 0; indep && j < h->count && between < 1.0; ++j) {
+    const LaunchRecord& r = h->rec[(h->head - j + HIST) % HIST];
+    for (int i = 0; i < nt && indep; ++i)
+      for (int k = 0; k < NRANGE; ++k)
+        if (overlaps(touched[i], r.w[k])) { indep = false; break; }
+    between += r.share;
+    if (j == HIST - 1 && between < 1.0 && h->count == HIST) indep = false;   // history too short to tell
+  }
+  h->head = (h->head + 1) % HIST;
+  if (h->count < HIST) ++h->count;
+  LaunchRecord& r = h->rec[h->head];
+  for (int k = 0; k < NRANGE; ++k) r.w[k] = written[k];
+  r.share = share;
+  return indep;
+}
+
 }  // namespace
 
 // Returns cudaErrorNotSupported when the shape does not fit this kernel's shared memory (the caller
@@ -482,16 +572,20 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     cudaGetDevice(&dev);
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
   }
-  // one CTA per SM: split a unit over a cluster while the grid still fits the machine
+  // split a unit over a cluster while the grid still fits on the SMs once (a second launch can then be resident too)
   int split = 1;
   while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
   int chunk = (cap + split - 1) / split;
   chunk = (chunk + GROUP - 1) / GROUP * GROUP;
   const size_t state_bytes = 4 * sizeof(float) * (size_t)chunk * split;
-  const size_t budget = 215 * 1024;     // dynamic shared memory, of which 1 KB is alignment slack
-  if (state_bytes + (size_t)MW * STAGE_BYTES + 1024 > budget) return cudaErrorNotSupported;
-  int nstage = (int)((budget - 1024 - state_bytes) / ((size_t)MW * STAGE_BYTES));
-  nstage = nstage > 3 ? 3 : nstage;
+  // Two CTAs per SM (so that consecutive launches can both be resident) when at least two stages per
+  // warp fit in half an SM's shared memory, otherwise one CTA with up to four stages.
+  const size_t half_sm = 104 * 1024, whole_sm = 215 * 1024;     // dynamic bytes, 1 KB of it alignment slack
+  if (state_bytes + (size_t)MW * STAGE_BYTES + 1024 > whole_sm) return cudaErrorNotSupported;
+  int nstage = state_bytes + 1024 + 2 * (size_t)MW * STAGE_BYTES <= half_sm
+                   ? (int)((half_sm - 1024 - state_bytes) / ((size_t)MW * STAGE_BYTES))
+                   : (int)((whole_sm - 1024 - state_bytes) / ((size_t)MW * STAGE_BYTES));
+  nstage = nstage > 4 ? 4 : nstage;
   const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
   if (nstage > groups_per_warp) nstage = groups_per_warp > 0 ? groups_per_warp : 1;
   const size_t dyn = (size_t)MW * nstage * STAGE_BYTES + state_bytes + 1024;
@@ -500,9 +594,23 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
       !make_rows_map_bf16(&tm_v, c.v_cache, (uint64_t)s.units * cap, GROUP))
     return cudaErrorInvalidValue;
   const bool win = s.window > 0;
+  const size_t units = (size_t)s.units, slots = units * cap;
+  Range written[16] = {{(const char*)c.k_cache, slots * ROW_BYTES}, {(const char*)c.v_cache, slots * ROW_BYTES},
+                       {(const char*)c.acc, slots * 4}, {(const char*)c.vnorm, slots * 4}, {(const char*)c.pos, slots * 4},
+                       {(const char*)c.len, units * 4}, {(const char*)c.free_slot, units * 4},
+                       {(const char*)c.next_pos, units * 4}, {(const char*)c.last_slot, units * 4},
+                       {(const char*)out, units * ROW_BYTES}, {(const char*)evicted, evicted ? units * 4 : 0},
+                       {win ? (const char*)c.ring : nullptr, win ? slots * s.window * 4 : 0},
+                       {win ? (const char*)c.acc_fixed : nullptr, win ? slots * 8 : 0},
+                       {(const char*)q, units * ROW_BYTES}, {(const char*)k, units * ROW_BYTES}, {(const char*)v, units * ROW_BYTES}};
   auto kern = win ? decode_mma_kernel<true> : decode_mma_kernel<false>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
   if (e != cudaSuccess) return e;
+  // share of the machine this launch holds while resident (every CTA waits for the previous launch before it retires)
+  int occ = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, MT, dyn) != cudaSuccess || occ < 1) occ = 1;
+  const double share = (double)(s.units * split) / ((double)occ * sms);
+  const int independent = independent_of_in_flight(st, written, 16, written, share) ? 1 : 0;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(s.units * split);
   cfg.blockDim = dim3(MT);
@@ -517,7 +625,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
+  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
                             (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                             (__nv_bfloat16*)out, evicted, dev_status);
 }

@@ -31,14 +31,14 @@ constexpr int SLAB_BYTES = TILE * 128;        // 128 rows x 64 bf16, 128-byte sw
 constexpr int TILE_BYTES = 2 * SLAB_BYTES;    // two K halves
 constexpr int CHUNK_BYTES = 2 * TILE_BYTES;   // 256 rows, two K halves
 constexpr uint64_t WAIT_NS = 1000000000ull;
-#ifndef VATP_POLY_EVERY
-#define VATP_POLY_EVERY 4   // one exponential in this many goes to the FMA pipe (0 = none)
+#ifndef VATP_POLY_MASK
+#define VATP_POLY_MASK 0x1111   // bit p set: pair p (of the 16 pairs of a 32-column slice) takes the FMA-pipe exponential
 #endif
 
 struct Smem {
   alignas(1024) unsigned char fixed[2][TILE_BYTES];      // double-buffered fixed tile
   alignas(1024) unsigned char stream[NS][CHUNK_BYTES];   // [K half][256 rows][128 bytes] per stage
-  alignas(16) float lse_s[8][2][TILE];   // pass 2: per softmax warp, double-buffered normalisers of a query tile
+  alignas(16) float lse_s[8][2][TILE];   // pass 2: per softmax warp, double-buffered NEGATED normalisers of a query tile
   float part_a[2][TILE];   // pass 1: running max of warpgroup 1; pass 2: its column sums
   float part_b[2][TILE];   // pass 1: running sum of warpgroup 1
   alignas(8) uint64_t full[NS], empty[NS];
@@ -166,26 +166,65 @@ __device__ __forceinline__ float ex2(float x) {
   return y;
 }
 
-// exp2 on the FMA pipe for x <= 0: round-to-nearest split x = n + f with f in [-0.5, 0.5] (adding
+// Packed fp32 pairs (fma.rn.f32x2 / add.rn.f32x2): one issue slot does two lanes' worth of FMA work.
+// The softmax warps are bound by instruction issue, not by the FMA pipe, so packing halves the cost
+// of everything around the exponential.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk2(float lo, float hi) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void upk2(f32x2 v, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v)); }
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float hsum2(f32x2 v) {
+  float a, b;
+  upk2(v, a, b);
+  return a + b;
+}
+
+// exp2 of a pair on the special-function unit (16 results per clock per SM)
+__device__ __forceinline__ f32x2 ex2_sfu2(f32x2 v) {
+  float a, b;
+  upk2(v, a, b);
+  return pk2(ex2(a), ex2(b));
+}
+// exp2 of a pair on the FMA pipe: round-to-nearest split x = n + f with f in [-0.5, 0.5] (adding
 // 1.5 * 2^23 leaves n in the low mantissa bits), a degree-3 minimax polynomial for 2^f (relative
-// error 7.5e-5) and an exponent-field add for 2^n.  The special-function unit issues 16 exp2 per
-// clock per SM, which bounds this kernel before the tensor pipe does; sending one element in four
-// here moves that share of the exponentials onto otherwise idle FMA issue slots.
-__device__ __forceinline__ float ex2_fma(float x) {
-  x = fmaxf(x, -126.f);
-  const float t = x + 12582912.f;
-  const float f = x - (t - 12582912.f);
-  const float p = fmaf(fmaf(fmaf(0.05517164617776871f, f, 0.2426111251115799f), f, 0.6932609677314758f), f,
-                       0.9999280571937561f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+// error 7.5e-5) and an exponent-field add for 2^n.  The special-function unit alone would bound the
+// kernel below the tensor pipe; a share of the pairs (VATP_POLY_MASK) goes here instead.
+__device__ __forceinline__ f32x2 ex2_fma2(f32x2 v) {
+  float a, b;
+  upk2(v, a, b);
+  v = pk2(fmaxf(a, -126.f), fmaxf(b, -126.f));
+  const f32x2 t = add2(v, pk2(12582912.f, 12582912.f));
+  const f32x2 r = add2(t, pk2(-12582912.f, -12582912.f));
+  const f32x2 f = fma2(r, pk2(-1.f, -1.f), v);
+  f32x2 p = fma2(pk2(0.05517164617776871f, 0.05517164617776871f), f, pk2(0.2426111251115799f, 0.2426111251115799f));
+  p = fma2(p, f, pk2(0.6932609677314758f, 0.6932609677314758f));
+  p = fma2(p, f, pk2(0.9999280571937561f, 0.9999280571937561f));
+  float tl, th, pl, ph;
+  upk2(t, tl, th);
+  upk2(p, pl, ph);
+  return pk2(__int_as_float(__float_as_int(pl) + (__float_as_int(tl) << 23)),
+             __int_as_float(__float_as_int(ph) + (__float_as_int(th) << 23)));
+}
+// pair index p in 0..15 of a slice: compile-time choice of the pipe
+__device__ __forceinline__ f32x2 exp2_pair(int p, f32x2 v) {
+  if ((VATP_POLY_MASK >> p) & 1) return ex2_fma2(v);
+  return ex2_sfu2(v);
 }
 
-// i is the unrolled element index (a multiple of 4): compile-time choice of the pipe
-__device__ __forceinline__ float exp2_mixed(int i, float x) {
-  if (VATP_POLY_EVERY > 0 && ((i + 4) % VATP_POLY_EVERY) == 0) return ex2_fma(x);
-  return ex2(x);
-}
-
+__device__ __forceinline__ float4 neg4(float4 v) { return make_float4(-v.x, -v.y, -v.z, -v.w); }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -197,10 +236,12 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 //   PASS 1 (row = query, columns = keys): online max / sum of exp2(scale_log2 * s); on the diagonal
 //           tile keys beyond the query are masked.
 //   PASS 2 (row = key, columns = queries): cs += exp2(scale_log2 * s - lse2[query]); on the diagonal
-//           tile queries before the key are masked.  lse_t: the tile's 128 normalisers in shared memory.
+//           tile queries before the key are masked.  nlse_t: the tile's 128 NEGATED normalisers in
+//           shared memory.  cs: two packed pairs of running sums.
 template <int PASS, bool DIAG>
 __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float scale_log2, float& m_run, float& l_run,
-                                          float (&cs)[4], const float* lse_t) {
+                                          f32x2 (&cs)[2], const float* nlse_t) {
+  const f32x2 c2 = pk2(scale_log2, scale_log2);
   if (PASS == 1) {
     if (DIAG) {
 #pragma unroll
@@ -217,32 +258,40 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
     const float m_new = fmaxf(m_run, cmax);
     l_run *= ex2(fmaxf(m_run - m_new, -126.f));      // (-inf) - (-inf) = NaN -> -126 -> factor on a zero sum
     m_run = m_new;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    const f32x2 nm2 = pk2(-m_run, -m_run);
+    f32x2 a0 = pk2(0.f, 0.f), a1 = a0;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
-      a0 += ex2(fmaf(x[i], scale_log2, -m_run));
-      a1 += ex2(fmaf(x[i + 1], scale_log2, -m_run));
-      a2 += ex2(fmaf(x[i + 2], scale_log2, -m_run));
-      a3 += exp2_mixed(i, fmaf(x[i + 3], scale_log2, -m_run));
+      a0 = add2(a0, exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, nm2)));
+      a1 = add2(a1, exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, nm2)));
     }
-    l_run += (a0 + a1) + (a2 + a3);
+    l_run += hsum2(add2(a0, a1));
+  } else if (!DIAG) {
+    const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(nlse_t + c0);
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+      const ulonglong2 L = lp[i >> 2];
+      cs[0] = add2(cs[0], exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, L.x)));
+      cs[1] = add2(cs[1], exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, L.y)));
+    }
   } else {
-    const float4* lp = reinterpret_cast<const float4*>(lse_t + c0);
+    const float4* lp = reinterpret_cast<const float4*>(nlse_t + c0);
+    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
       const float4 L = lp[i >> 2];
-      float p0 = ex2(fmaf(x[i], scale_log2, -L.x));
-      float p1 = ex2(fmaf(x[i + 1], scale_log2, -L.y));
-      float p2 = ex2(fmaf(x[i + 2], scale_log2, -L.z));
-      float p3 = exp2_mixed(i, fmaf(x[i + 3], scale_log2, -L.w));
-      if (DIAG) {
-        if (c0 + i < row) p0 = 0.f;
-        if (c0 + i + 1 < row) p1 = 0.f;
-        if (c0 + i + 2 < row) p2 = 0.f;
-        if (c0 + i + 3 < row) p3 = 0.f;
-      }
-      cs[0] += p0; cs[1] += p1; cs[2] += p2; cs[3] += p3;
+      float p0 = ex2(fmaf(x[i], scale_log2, L.x));
+      float p1 = ex2(fmaf(x[i + 1], scale_log2, L.y));
+      float p2 = ex2(fmaf(x[i + 2], scale_log2, L.z));
+      float p3 = ex2(fmaf(x[i + 3], scale_log2, L.w));
+      if (c0 + i < row) p0 = 0.f;
+      if (c0 + i + 1 < row) p1 = 0.f;
+      if (c0 + i + 2 < row) p2 = 0.f;
+      if (c0 + i + 3 < row) p3 = 0.f;
+      s0 += p0; s1 += p1; s2 += p2; s3 += p3;
     }
+    cs[0] = add2(cs[0], pk2(s0, s1));
+    cs[1] = add2(cs[1], pk2(s2, s3));
   }
 }
 
@@ -402,7 +451,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       float n1 = 0.f;
       if (PASS == 2 && g == 0 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tok);
       float m_run = -INFINITY, l_run = 0.f;       // pass 1
-      float cs[4] = {0.f, 0.f, 0.f, 0.f};         // pass 2
+      f32x2 cs[2] = {pk2(0.f, 0.f), pk2(0.f, 0.f)};   // pass 2: four running sums, packed
       const uint32_t n0 = n;
       n += it.c_count;
       int buf = 0;
@@ -429,7 +478,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       if (have) {
         tmem_ld32(acc_addr(0), xa);
         if (PASS == 2) {
-          reinterpret_cast<float4*>(lse_w)[lane] = __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(0) * TILE) + lane);
+          reinterpret_cast<float4*>(lse_w)[lane] = neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(0) * TILE) + lane));
           __syncwarp();
         }
         tmem_ld_wait();
@@ -447,7 +496,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
               tmem_ld32(acc_addr(c + 1), xa);
               if (PASS == 2) {
                 reinterpret_cast<float4*>(lse_w + buf * TILE)[lane] =
-                    __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane);
+                    neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane));
                 __syncwarp();
               }
               tmem_ld_wait();
@@ -461,7 +510,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         const float* lse_t = lse_w + buf * TILE;
         float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
         if (PASS == 2 && next_needed)
-          lnext = __ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane);
+          lnext = neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane));
         // Both paths are rolled loops with few inlined copies of the slice code: the steady-state
         // body stays small enough for the instruction cache.
         if (!diag) {
@@ -518,7 +567,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         ok = mbar_wait(&sm.comb_empty[pi], ipar ^ 1, abort_flag, a.dev_status);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         if (PASS == 1) { sm.part_a[pi][row] = m_run; sm.part_b[pi][row] = l_run; }
-        else           { sm.part_a[pi][row] = (cs[0] + cs[1]) + (cs[2] + cs[3]); }
+        else           { sm.part_a[pi][row] = hsum2(add2(cs[0], cs[1])); }
         mbar_arrive(&sm.comb_full[pi]);
       } else {
         ok = mbar_wait(&sm.comb_full[pi], ipar, abort_flag, a.dev_status);
@@ -536,7 +585,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = INFINITY;
           if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
         } else {
-          const float tot = ((cs[0] + cs[1]) + (cs[2] + cs[3])) + sm.part_a[pi][row];
+          const float tot = hsum2(add2(cs[0], cs[1])) + sm.part_a[pi][row];
           mbar_arrive(&sm.comb_empty[pi]);
           if (tok < a.T) {
             const int64_t o = (int64_t)u * a.T + tok;
