@@ -149,7 +149,7 @@ def run_reference(args, wl):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": (statistics.mean(pre) + statistics.mean(dec)) * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"config1 {wl.name} (oracle on a sample)", "sample": sample},
+            "config": {"workload": f"config{wl.cid} {wl.name} (oracle on a sample)", "sample": sample},
             "decode_us_per_layer_step": dec_us,
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -182,6 +182,7 @@ class LayerState:
         self.attn_acc = torch.empty(b, h, T, **f32)
         self.vnorm = torch.empty(b, h, T, **f32)
         self.score = torch.empty(b, h, T, **f32)
+        self.win_rows = torch.empty(b, h, wl.window, T, **f32) if wl.indicator == "window" else None
         self.kept = torch.empty(b, h, wl.budget, dtype=torch.int32, device=dev)
         self.ws = torch.empty(max(V.vatp_workspace_bytes(self.p), 256), dtype=torch.uint8, device=dev)
         self.cache = V.Cache(self.p, device=dev)
@@ -213,11 +214,12 @@ def run_cuda(args, wl):
         for i, ls in enumerate(layers):
             if ev: ev[i][0].record()
             V.vatp_prefill_scores(ls.p, ls.q, ls.k, ls.v, attn_acc=ls.attn_acc, vnorm=ls.vnorm, score=ls.score,
-                                  workspace=ls.ws, dev_status=status)
+                                  win_rows=ls.win_rows, workspace=ls.ws, dev_status=status)
             if ev: ev[i][1].record()
             V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
             if ev: ev[i][2].record()
-            V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, dev_status=status)
+            V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows,
+                           dev_status=status)
             if ev: ev[i][3].record()
 
     def decode_all():
@@ -319,9 +321,14 @@ def run_cuda(args, wl):
     dec_us = dec_ms * 1e3 / (steps_dec * L)
 
     # ---- rooflines (algorithmic work only) ----
-    flops_score = 2 * (2.0 * d) * T * (T + 1) / 2 * units      # two passes of the causal half of QK^T
+    if wl.indicator == "window":                               # only the last w query rows (Eq. 3)
+        w = min(wl.window, T)
+        pairs = w * T - w * (w - 1) / 2
+    else:
+        pairs = T * (T + 1) / 2
+    flops_score = 2 * (2.0 * d) * pairs * units                # two passes of the causal part of QK^T
     bytes_compact = units * (2 * 2 * B * d * 2 + 12 * B)       # K,V rows read + written, 12 B of state per slot
-    bytes_decode = units * (B + 1) * (2 * d * 2 + 16)          # K,V rows once, acc r+w, vnorm, pos
+    bytes_decode = units * (B + 1) * (2 * d * 2 + 16 + (8 if wl.indicator == "window" else 0))  # K,V rows once, acc r+w, vnorm, pos (+ ring row r+w)
     bytes_select = units * (4 * T + 4 * B)
     ms = statistics.mean
     kernels = {
@@ -348,11 +355,11 @@ def run_cuda(args, wl):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": all_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 inputs, f32 accumulate", "data": "synthetic",
-        "config": {"workload": f"config1 {wl.name}: b{wl.batch} h{wl.heads} d{d} T{T} budget{B} recent{wl.n_recent} "
-                               f"sinkF{wl.n_sink} h2o, {steps_dec} decode steps, x{L} independently seeded layers",
+        "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": f"config{wl.cid} {wl.name}: b{wl.batch} h{wl.heads} d{d} T{T} budget{B} recent{wl.n_recent} "
+                               f"sinkF{wl.n_sink} {wl.indicator}, {steps_dec} decode steps, x{L} independently seeded layers",
                    "layers": L,
-                   "l2": "256 MB flush write between steps; layer rotation keeps the decode state (277 MB) out of L2",
+                   "l2": f"256 MB flush write between steps; layer rotation over {L} decode states ({L * bytes_decode / 1e6:.0f} MB per visit of all layers)",
                    "replicas": "each GPU runs the whole workload (path does not shard within a call)",
                    "decode_graph": graph is not None},
         "prefill_ms_per_layer": pre_ms / L, "decode_us_per_layer_step": dec_us,
@@ -364,7 +371,7 @@ def run_cuda(args, wl):
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
-        cu, cs = 2, 16
+        cu, cs = 24, 64      # about 10-20 s of CPU work
         a, b = oracle_sample(wl, cu, cs)
         v = wl.batch * T / (a / cu * units)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
@@ -386,10 +393,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--layers", type=int, default=LAYERS, help="independently seeded layers held on the device")
+    ap.add_argument("--config", type=int, default=1, choices=sorted([0, 1, 2, 3, 4]),
+                    help="workload to time; 1 is the benchmark, the others are for the per-config roofline tables "
+                         "(choose --layers so that the inputs fit: config 2 and 4 hold 1.6 GB per layer)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps (profiling runs)")
     args = ap.parse_args()
     from paper_2406_12335_b200 import synth
-    wl = synth.CONFIGS[1]
+    wl = synth.CONFIGS[args.config]
     if args.decode_steps is not None:
         wl = wl.with_(decode_steps=args.decode_steps)
     if args.impl == "reference":

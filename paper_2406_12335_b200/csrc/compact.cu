@@ -11,7 +11,7 @@ constexpr int CP_ITERS = CP_SLOTS / (CP_THREADS / 16);
 
 // grid (units, slot groups).  Sixteen lanes copy one row (K and V) in 16-byte pieces; a thread has
 // CP_ITERS rows of K and of V in flight before it stores, and no index needs a division.
-__global__ void __launch_bounds__(CP_THREADS)
+__global__ void __launch_bounds__(CP_THREADS, 4)
 compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict__ k, const char* __restrict__ v,
                const float* __restrict__ attn_acc, const float* __restrict__ vnorm, const int32_t* __restrict__ kept,
                vatp_cache c) {

@@ -238,9 +238,16 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 //   PASS 2 (row = key, columns = queries): cs += exp2(scale_log2 * s - lse2[query]); on the diagonal
 //           tile queries before the key are masked.  nlse_t: the tile's 128 NEGATED normalisers in
 //           shared memory.  cs: two packed pairs of running sums.
-template <int PASS, bool DIAG>
+//   WIN (pass 2, Eq. 3): the probabilities themselves are also written out, column i of the slice to
+//           wo.p[i * wo.T] for wo.lo <= i < wo.hi (the rows of the last-w-queries window).
+struct WinOut {
+  float* p;
+  int lo, hi;
+  int64_t T;
+};
+template <int PASS, bool DIAG, bool WIN>
 __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float scale_log2, float& m_run, float& l_run,
-                                          f32x2 (&cs)[2], const float* nlse_t) {
+                                          f32x2 (&cs)[2], const float* nlse_t, const WinOut& wo) {
   const f32x2 c2 = pk2(scale_log2, scale_log2);
   if (PASS == 1) {
     if (DIAG) {
@@ -271,8 +278,19 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
       const ulonglong2 L = lp[i >> 2];
-      cs[0] = add2(cs[0], exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, L.x)));
-      cs[1] = add2(cs[1], exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, L.y)));
+      const f32x2 e0 = exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, L.x));
+      const f32x2 e1 = exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, L.y));
+      cs[0] = add2(cs[0], e0);
+      cs[1] = add2(cs[1], e1);
+      if (WIN) {
+        float p0, p1, p2, p3;
+        upk2(e0, p0, p1);
+        upk2(e1, p2, p3);
+        if (i >= wo.lo && i < wo.hi) wo.p[i * wo.T] = p0;
+        if (i + 1 >= wo.lo && i + 1 < wo.hi) wo.p[(i + 1) * wo.T] = p1;
+        if (i + 2 >= wo.lo && i + 2 < wo.hi) wo.p[(i + 2) * wo.T] = p2;
+        if (i + 3 >= wo.lo && i + 3 < wo.hi) wo.p[(i + 3) * wo.T] = p3;
+      }
     }
   } else {
     const float4* lp = reinterpret_cast<const float4*>(nlse_t + c0);
@@ -289,6 +307,12 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
       if (c0 + i + 2 < row) p2 = 0.f;
       if (c0 + i + 3 < row) p3 = 0.f;
       s0 += p0; s1 += p1; s2 += p2; s3 += p3;
+      if (WIN) {
+        if (i >= wo.lo && i < wo.hi) wo.p[i * wo.T] = p0;
+        if (i + 1 >= wo.lo && i + 1 < wo.hi) wo.p[(i + 1) * wo.T] = p1;
+        if (i + 2 >= wo.lo && i + 2 < wo.hi) wo.p[(i + 2) * wo.T] = p2;
+        if (i + 3 >= wo.lo && i + 3 < wo.hi) wo.p[(i + 3) * wo.T] = p3;
+      }
     }
     cs[0] = add2(cs[0], pk2(s0, s1));
     cs[1] = add2(cs[1], pk2(s2, s3));
@@ -306,44 +330,51 @@ struct TcArgs {
   float* vnorm;
   float* score;
   int32_t* dev_status;
+  // Eq. 3 (last w queries): only query rows >= first_row count; ft = first_row / 128; win_rows row r is
+  // query wrow0 + r (wrow0 = T - w, negative when the prompt is shorter than the window).  H2O: all zero.
+  int first_row, ft, wrow0, window;
+  float* win_rows;
 };
 
 // Work items are (unit, fixed tile of 128 rows), longest first, dealt to the persistent CTAs like a
 // snake draft (rounds alternate direction: load spread within a few percent).  The other operand
 // streams in chunks of 256 tokens (two tiles), so that one MMA instruction is 128 x 256 x 16: a
 // single thread issues the MMAs, and at 128 x 128 x 16 the issue cost exceeds the execution time.
-//   PASS 1: fixed = query tile i, streamed key chunks 0 .. i/2       (key tile kt needed iff kt <= i)
-//   PASS 2: fixed = key tile i, streamed query chunks i/2 .. nch-1   (query tile qt needed iff i <= qt < nt)
+//   PASS 1: fixed = query tile i, streamed key chunks 0 .. i/2       (key tile kt needed iff kt <= i);
+//           with a history window only the query tiles that reach into it are items
+//   PASS 2: fixed = key tile i, streamed query chunks lo/2 .. nch-1  (query tile qt needed iff lo <= qt < nt,
+//           lo = max(i, first tile of the window))
 // Softmax warpgroup g takes columns [128 g, 128 g + 128) of every accumulator, i.e. streamed tile
 // 2 c + g of chunk c; the two partial results of a row are combined once per item.
 __device__ __forceinline__ int item_id(int n, int c, int G) { return n * G + ((n & 1) ? G - 1 - c : c); }
 
 struct Item {
   int u, tile, c_first, c_count;
+  int lo;   // pass 2: first query tile that counts for this key tile
 };
 template <int PASS>
 __device__ __forceinline__ Item item_of(int id, const TcArgs& a) {
   Item it;
   const int r = id / a.units;
   it.u = id - r * a.units;
-  if (PASS == 1) { it.tile = a.nt - 1 - r; it.c_first = 0; it.c_count = it.tile / 2 + 1; }
-  else           { it.tile = r; it.c_first = r / 2; it.c_count = a.nch - r / 2; }
+  if (PASS == 1) { it.tile = a.nt - 1 - r; it.c_first = 0; it.c_count = it.tile / 2 + 1; it.lo = 0; }
+  else           { it.tile = r; it.lo = max(r, a.ft); it.c_first = it.lo / 2; it.c_count = a.nch - it.c_first; }
   return it;
 }
 // is streamed tile st (= 2 * chunk + half) needed by the item?
 template <int PASS>
 __device__ __forceinline__ bool tile_needed(const Item& it, int st, int nt) {
-  return PASS == 1 ? st <= it.tile : (st >= it.tile && st < nt);
+  return PASS == 1 ? st <= it.tile : (st >= it.lo && st < nt);
 }
 
-template <int PASS>
+template <int PASS, bool WIN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k, TcArgs a) {
   extern __shared__ unsigned char smem_raw[];
   Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
   volatile int* abort_flag = &sm.abort_flag;
-  const int items = a.units * a.nt;
+  const int items = a.units * (PASS == 1 ? a.nt - a.ft : a.nt);
 
   if (tid == 0) {
     for (int i = 0; i < NS; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
@@ -460,6 +491,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       auto st_of = [&](int c) { return 2 * (it.c_first + c) + g; };
       auto needed = [&](int c) { return tile_needed<PASS>(it, st_of(c), a.nt); };
       auto acc_addr = [&](int c) { return lane_addr + ((n0 + c) % NACC) * CHUNK; };
+      // where the probabilities of the 32 query columns starting at column c0 of streamed tile stile go (Eq. 3 rows)
+      auto wout = [&](int stile, int c0) {
+        WinOut wo{nullptr, 0, 0, 0};
+        if (WIN && PASS == 2) {
+          const int q0 = stile * TILE + c0;
+          wo.T = a.T;
+          wo.lo = min(max(a.first_row - q0, 0), 32);
+          wo.hi = tok < a.T ? min(max(a.T - q0, 0), 32) : 0;
+          wo.p = a.win_rows + ((int64_t)u * a.window + (q0 - a.wrow0)) * a.T + tok;
+        }
+        return wo;
+      };
       auto chunk_wait = [&](int c) -> bool {
         bool w = mbar_wait(&sm.acc_full[(n0 + c) % NACC], ((n0 + c) / NACC) & 1, abort_flag, a.dev_status);
         w = __all_sync(0xffffffffu, w);
@@ -518,7 +561,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll 1
           for (int h2 = 0; h2 < 2; ++h2) {
             tmem_ld32(t_addr + 64 * h2 + 32, xb);
-            consume32<PASS, false>(xa, 64 * h2, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            consume32<PASS, false, WIN>(xa, 64 * h2, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(st_of(c), 64 * h2));
             tmem_ld_wait();
             if (h2 == 0) {
               tmem_ld32(t_addr + 64, xa);
@@ -529,7 +572,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
                 if (ok && next_needed) tmem_ld32(acc_addr(c + 1), xa);
               }
             }
-            if (ok) consume32<PASS, false>(xb, 64 * h2 + 32, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            if (ok) consume32<PASS, false, WIN>(xb, 64 * h2 + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(st_of(c), 64 * h2 + 32));
             if (h2 == 1 && PASS == 2 && next_needed) {
               reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
               __syncwarp();
@@ -540,7 +583,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           // the one diagonal tile of an item takes the masked variant (not pipelined)
 #pragma unroll 1
           for (int c0 = 0; c0 < TILE; c0 += 32) {
-            consume32<PASS, true>(xa, c0, row, a.scale_log2, m_run, l_run, cs, lse_t);
+            consume32<PASS, true, WIN>(xa, c0, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(st_of(c), c0));
             if (c0 + 32 < TILE) {
               tmem_ld32(t_addr + c0 + 32, xa);
               tmem_ld_wait();
@@ -580,7 +623,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (l_run > 0.f) l += l_run * ex2(m_run - m);
           if (l1 > 0.f) l += l1 * ex2(m1 - m);
           const float lse2 = m + log2f(l);
-          a.lse2[(int64_t)u * a.Tpad + tok] = tok < a.T ? lse2 : INFINITY;
+          // queries outside the prompt or before the history window contribute nothing to pass 2
+          a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? lse2 : INFINITY;
           // an odd tile count leaves half a chunk of padding that pass 2 reads as "no query"
           if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = INFINITY;
           if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
@@ -597,11 +641,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
   } else if (PASS == 1) {
     // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
-    // Independent of the attention work of this pass: every (unit, token tile) is an item exactly
-    // once, so this warp covers all tokens.  Pass 2 reads the norms back in its epilogue.
-    uint32_t itl = 0;
-    for (int id = item_id(0, blockIdx.x, gridDim.x); id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
-      const Item it = item_of<PASS>(id, a);
+    // Independent of the attention work of this pass: the CTAs share out all (unit, token tile) pairs,
+    // so these warps cover every token.  Pass 2 reads the norms back in its epilogue.
+    for (int id = blockIdx.x; id < a.units * a.nt; id += gridDim.x) {
+      Item it;
+      it.tile = id / a.units;
+      it.u = id - it.tile * a.units;
       const int b = it.u / a.heads, h = it.u - b * a.heads;
       const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
       // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
@@ -627,6 +672,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (part == 0 && tok < a.T) a.vnorm[(int64_t)it.u * a.T + tok] = acc;
         }
       }
+    }
+  } else if (WIN) {
+    // ------------------------------------------------------------------ pass 2, Eq. 3: window rows nobody visits
+    // For key tile i the query tiles before it are never streamed (causal), and when the prompt is
+    // shorter than the window its first rows belong to no query: those entries of win_rows are zero.
+    uint32_t itl = 0;
+    for (int id = item_id(0, blockIdx.x, gridDim.x); id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
+      const Item it = item_of<PASS>(id, a);
+      float* wr = a.win_rows + (int64_t)it.u * a.window * a.T;
+      const int k0 = it.tile * TILE;
+      const int r_end = min(it.tile * TILE, a.T) - a.wrow0;      // rows of queries before this key tile
+      for (int r = 0; r < min(r_end, a.window); ++r)
+        for (int kk = lane; kk < TILE; kk += 32)
+          if (k0 + kk < a.T) wr[(int64_t)r * a.T + k0 + kk] = 0.f;
     }
   }
 
@@ -703,8 +762,8 @@ size_t prefill_tc_workspace_bytes(int units, int T) {
 }
 
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
-                              float* lse_out, float* attn_acc, float* vnorm, float* score, int32_t* dev_status,
-                              cudaStream_t st) {
+                              float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
+                              int32_t* dev_status, cudaStream_t st) {
   CUtensorMap tm_q, tm_k;
   if (!make_map(&tm_q, q, s) || !make_map(&tm_k, k, s)) return cudaErrorInvalidValue;
   TcArgs a;
@@ -717,17 +776,24 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.sb = s.sb; a.sh = s.sh; a.st = s.st;
   a.lse2 = lse_ws; a.lse_out = lse_out; a.attn_acc = attn_acc; a.vnorm = vnorm; a.score = score;
   a.dev_status = dev_status;
+  const bool win = s.window > 0;
+  a.window = win ? s.window : 0;
+  a.first_row = win && s.T > s.window ? s.T - s.window : 0;
+  a.ft = a.first_row / TILE;
+  a.wrow0 = win ? s.T - s.window : 0;
+  a.win_rows = win ? win_rows : nullptr;
   const size_t smem = sizeof(Smem) + 1024;
   cudaError_t e;
-  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+  if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const int items = a.units * a.nt;
-  const int grid = items < sms ? items : sms;
-  prefill_tc_kernel<1><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
-  prefill_tc_kernel<2><<<grid, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
+  prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  if (win) prefill_tc_kernel<2, true><<<items2 < sms ? items2 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  else     prefill_tc_kernel<2, false><<<items2 < sms ? items2 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   return cudaGetLastError();
 }
 

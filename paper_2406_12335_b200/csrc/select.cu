@@ -24,7 +24,6 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
   __shared__ uint32_t hist[256];
   __shared__ uint32_t sh_prefix, sh_need;
   __shared__ uint32_t warp_keep[SEL_WARPS], warp_eq[SEL_WARPS];
-  __shared__ uint32_t run_keep, run_eq;
 
   const int u = blockIdx.x;
   const float* sc = score + (int64_t)u * T;
@@ -47,14 +46,23 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
   }
   auto key_at = [&](int i) -> uint32_t { return STAGED ? keys_s[i] : order_key(sc[F + i]); };
 
-  // radix select, most significant byte first: find the key value tau of rank ksel (descending)
+  // radix select, most significant byte first: find the key value tau of rank ksel (descending).
+  // Scores of one head share a few exponents, so most keys of a pass fall into a handful of bins:
+  // lanes with the same digit are counted by one of them (match + one atomic per distinct digit).
   uint32_t prefix = 0, mask = 0, need = (uint32_t)ksel;
+  const int lane = tid & 31, wid = tid >> 5;
   for (int shift = 24; shift >= 0; shift -= 8) {
     for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0;
     __syncthreads();
-    for (int i = tid; i < n; i += SEL_THREADS) {
-      const uint32_t key = key_at(i);
-      if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+    for (int base = 0; base < n; base += SEL_THREADS) {
+      const int i = base + tid;
+      uint32_t digit = 256u;                       // lanes without a candidate share a dummy digit
+      if (i < n) {
+        const uint32_t key = key_at(i);
+        if ((key & mask) == prefix) digit = (key >> shift) & 255u;
+      }
+      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
+      if (digit < 256u && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
     }
     __syncthreads();
     if (tid < 32) {
@@ -85,42 +93,50 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
     prefix = sh_prefix;
     need = sh_need;
     mask |= 255u << shift;
-    __syncthreads();
   }
   const uint32_t tau = prefix;     // the ksel-th largest key; `need` of the keys equal to tau survive
   const uint32_t need_eq = need;
 
-  // ordered compaction: keep key > tau, and the first need_eq (lowest index) keys equal to tau
-  if (tid == 0) { run_keep = 0; run_eq = 0; }
+  // ordered compaction: keep key > tau, and the first need_eq (lowest index) keys equal to tau.
+  // Thread t owns the contiguous range [t * per, (t + 1) * per); one block-wide exclusive scan of
+  // (kept, equal) counts gives every thread its output offset and the rank of its first tie.
+  const int per = (n + SEL_THREADS - 1) / SEL_THREADS;
+  const int lo = min(tid * per, n), hi_i = min(lo + per, n);
+  uint32_t n_gt = 0, n_eq = 0;
+  for (int i = lo; i < hi_i; ++i) {
+    const uint32_t key = key_at(i);
+    n_gt += key > tau;
+    n_eq += key == tau;
+  }
+  // inclusive scan inside the warp, then over the warp totals
+  uint32_t s_gt = n_gt, s_eq = n_eq;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const uint32_t a = __shfl_up_sync(0xffffffffu, s_gt, off), b = __shfl_up_sync(0xffffffffu, s_eq, off);
+    if (lane >= off) { s_gt += a; s_eq += b; }
+  }
+  if (lane == 31) { warp_keep[wid] = s_gt; warp_eq[wid] = s_eq; }
   __syncthreads();
-  const int lane = tid & 31, wid = tid >> 5;
-  for (int base = 0; base < n; base += SEL_THREADS) {
-    const int i = base + tid;
-    uint32_t key = 0;
-    bool gt = false, eq = false;
-    if (i < n) { key = key_at(i); gt = key > tau; eq = key == tau; }
-    const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) warp_eq[wid] = __popc(eq_ballot);
-    __syncthreads();
-    uint32_t eq_before = run_eq;
-    for (int w = 0; w < wid; ++w) eq_before += warp_eq[w];
-    eq_before += __popc(eq_ballot & ((1u << lane) - 1u));
-    const bool keep = gt || (eq && eq_before < need_eq);
-    const uint32_t keep_ballot = __ballot_sync(0xffffffffu, keep);
-    if (lane == 0) warp_keep[wid] = __popc(keep_ballot);
-    __syncthreads();
-    uint32_t keep_before = run_keep;
-    for (int w = 0; w < wid; ++w) keep_before += warp_keep[w];
-    keep_before += __popc(keep_ballot & ((1u << lane) - 1u));
-    if (keep) out[F + keep_before] = F + i;
-    __syncthreads();
-    if (tid == 0) {
-      uint32_t a = 0, b = 0;
-      for (int w = 0; w < SEL_WARPS; ++w) { a += warp_keep[w]; b += warp_eq[w]; }
-      run_keep += a;
-      run_eq += b;
+  if (wid == 0) {
+    uint32_t a = warp_keep[lane], b = warp_eq[lane];
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const uint32_t x = __shfl_up_sync(0xffffffffu, a, off), y = __shfl_up_sync(0xffffffffu, b, off);
+      if (lane >= off) { a += x; b += y; }
     }
-    __syncthreads();
+    warp_keep[lane] = a;      // inclusive totals up to and including warp `lane`
+    warp_eq[lane] = b;
+  }
+  __syncthreads();
+  const uint32_t gt_before = s_gt - n_gt + (wid ? warp_keep[wid - 1] : 0u);
+  uint32_t eq_rank = s_eq - n_eq + (wid ? warp_eq[wid - 1] : 0u);
+  // ties before index i that survive = min(eq_rank, need_eq)
+  uint32_t o = gt_before + min(eq_rank, need_eq);
+  for (int i = lo; i < hi_i; ++i) {
+    const uint32_t key = key_at(i);
+    const bool keep = key > tau || (key == tau && eq_rank < need_eq);
+    eq_rank += key == tau;
+    if (keep) out[F + o++] = F + i;
   }
 }
 

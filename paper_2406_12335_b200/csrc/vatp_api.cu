@@ -97,8 +97,8 @@ vatp_status vatp_prefill_scores(const vatp_params* p, const void* q, const void*
   float* ws = static_cast<float*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e;
-  if (p->dtype == VATP_BF16 && p->head_dim == 128 && !windowed && vatp_tc_available())
-    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, dev_status, st);
+  if (p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available())
+    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st);
   else
     e = launch_prefill_simt(sh, p->dtype, q, k, v, lse_out ? lse_out : ws, attn_acc, vnorm, score, win_rows, st);
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;

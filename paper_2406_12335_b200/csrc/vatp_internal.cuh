@@ -41,8 +41,8 @@ bool make_rows_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint32_
 cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const void* k, const void* v, float* lse,
                                 float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st);
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
-                              float* lse_out, float* attn_acc, float* vnorm, float* score, int32_t* dev_status,
-                              cudaStream_t st);
+                              float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
+                              int32_t* dev_status, cudaStream_t st);
 size_t prefill_tc_workspace_bytes(int units, int T);  // padded log2-domain row normalisers
 cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st);
 cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, const void* v, const float* attn_acc,

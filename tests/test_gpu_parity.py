@@ -205,3 +205,20 @@ def test_interleaved_caches_match_separate_runs(b, h):
     units = [(0, 0), (b - 1, h - 1), (b // 2, h // 2)]
     refs = {u: P.check_prefill_unit(g, u[0], u[1], P.TOL["bf16"])[:2] for u in units}
     P.run_decode_and_check(g, refs, *ins[1], steps, P.TOL["bf16"], check_state_every=4)
+
+
+@pytest.mark.parametrize("T,w,B,F,R", [
+    (1000, 300, 400, 2, 10),     # window start inside a tile, ragged prompt
+    (200, 256, 80, 0, 10),       # prompt shorter than the window: Eq. 3 is Eq. 2, leading rows of the history are empty
+    (768, 128, 300, 4, 10),      # window = exactly the last tile
+    (513, 1, 200, 0, 0),         # a window of one query
+    (640, 640, 256, 2, 16),      # window = whole prompt
+])
+def test_windowed_indicator_shapes(T, w, B, F, R):
+    """Eq. 3 on the tensor-core path (bf16, d 128) for windows that start anywhere, with decode steps that
+    roll the history ring."""
+    _run_case(_small("bf16", 128, T, B, F, R, b=1, h=2, indicator="window", window=w, steps=8, cid=60))
+
+
+def test_windowed_indicator_fp32_path():
+    _run_case(_small("f32", 64, 300, 120, 2, 10, b=1, h=2, indicator="window", window=77, steps=6, cid=61))
