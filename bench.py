@@ -328,6 +328,8 @@ def run_cuda(args, wl):
         pairs = T * (T + 1) / 2
     flops_score = 2 * (2.0 * d) * pairs * units                # two passes of the causal part of QK^T
     bytes_compact = units * (2 * 2 * B * d * 2 + 12 * B)       # K,V rows read + written, 12 B of state per slot
+    if wl.indicator == "window":
+        bytes_compact += units * 2 * 4 * B * min(wl.window, T)  # kept columns of the last-w rows read, ring written
     bytes_decode = units * (B + 1) * (2 * d * 2 + 16 + (8 if wl.indicator == "window" else 0))  # K,V rows once, acc r+w, vnorm, pos (+ ring row r+w)
     bytes_select = units * (4 * T + 4 * B)
     ms = statistics.mean

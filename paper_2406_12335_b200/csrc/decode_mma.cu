@@ -143,20 +143,23 @@ __device__ __forceinline__ unsigned long long warp_min_key(unsigned long long ke
 template <bool WINDOWED>
 __global__ void __launch_bounds__(MT, 2)
 decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int independent,
-                  int split, int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
+                  int state_in_smem, int split, int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
                   const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
   extern __shared__ unsigned char dyn_raw[];
   unsigned char* dyn = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dyn_raw) + 1023) & ~uintptr_t(1023));
   // [MW][nstage] stages | logits[tot] | acc[tot] | vnorm[tot] | pos[tot]; the per-slot arrays span the
-  // whole unit and are used by rank 0 only
+  // whole unit and are used by rank 0 only.  For large caches only the logits are held here, which keeps
+  // the CTA small enough for two launches to be resident together; acc, vnorm and pos are then copied
+  // into the stage memory once the streaming is over (state_in_smem == 2) or, if even that is too
+  // small, read from global memory in the tail (state_in_smem == 0).
   const int tot = split * chunk;
   unsigned char* stage_base = dyn;
   float* logit_s = reinterpret_cast<float*>(dyn + (size_t)MW * nstage * STAGE_BYTES);
-  float* acc_s = logit_s + tot;
-  float* vn_s = acc_s + tot;
-  int* pos_s = reinterpret_cast<int*>(vn_s + tot);
+  float* acc_s = state_in_smem == 2 ? reinterpret_cast<float*>(stage_base) : logit_s + tot;
+  float* vn_s = acc_s + (state_in_smem == 2 ? cap : tot);
+  int* pos_s = reinterpret_cast<int*>(vn_s + (state_in_smem == 2 ? cap : tot));
 
   __shared__ __align__(8) uint64_t bars[MW * 4 + 1];
   __shared__ __align__(16) Exch ex;
@@ -218,10 +221,16 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   if (!independent) asm volatile("griddepcontrol.wait;" ::: "memory");
   if (rank == 0 && tid == 32) {      // per-slot state of the whole unit
     const int64_t o = (int64_t)u * cap;
-    mbar_expect_tx(state_bar, 3u * cap * 4u);
-    bulk_g2s(acc_s, c.acc + o, cap * 4, state_bar);
-    bulk_g2s(vn_s, c.vnorm + o, cap * 4, state_bar);
-    bulk_g2s(pos_s, c.pos + o, cap * 4, state_bar);
+    if (state_in_smem == 1) {
+      mbar_expect_tx(state_bar, 3u * cap * 4u);
+      bulk_g2s(acc_s, c.acc + o, cap * 4, state_bar);
+      bulk_g2s(vn_s, c.vnorm + o, cap * 4, state_bar);
+      bulk_g2s(pos_s, c.pos + o, cap * 4, state_bar);
+    } else if (state_in_smem == 0) {
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.acc + o), "r"(cap * 4) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.vnorm + o), "r"(cap * 4) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.pos + o), "r"(cap * 4) : "memory");
+    }
   }
 
   const int len = c.len[u];
@@ -232,6 +241,11 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int cnt = max(min(hi - s0, rows_alloc), 0);
   const int fs_local = fs - s0;          // row of the incoming token inside this CTA's range (if owned)
   const bool owns_new = fs_local >= 0 && fs_local < cnt;
+  if (WINDOWED && rank == 0 && tid == 64) {
+    // the tail reads the ring row that leaves the window and the exact sums: have them in L2 by then
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.ring + ((int64_t)u * w + (t % w)) * cap), "r"(cap * 4) : "memory");
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.acc_fixed + (int64_t)u * cap), "r"(cap * 8) : "memory");
+  }
   const int ls_local = ls - s0;          // row the previous step appended (its tile may predate that store)
   const bool owns_last = !independent && ls >= 0 && ls != fs && ls_local >= 0 && ls_local < cnt;
 
@@ -384,6 +398,16 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (lane == 0) { part_m[wid] = m_run; part_l[wid] = l_run; }
   }
   workers_sync();
+  if (state_in_smem == 2 && rank == 0 && tid == 32) {
+    // every stage of this CTA has been consumed: the per-slot state of the unit lands there while the
+    // cluster gathers (the stages were last written by bulk copies and read by ldmatrix; warps that
+    // stored into them have fenced)
+    const int64_t o = (int64_t)u * cap;
+    mbar_expect_tx(state_bar, 3u * cap * 4u);
+    bulk_g2s(acc_s, c.acc + o, cap * 4, state_bar);
+    bulk_g2s(vn_s, c.vnorm + o, cap * 4, state_bar);
+    bulk_g2s(pos_s, c.pos + o, cap * 4, state_bar);
+  }
 
   // ---- CTA partial, pushed into rank 0 ----
   {
@@ -432,7 +456,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   }
 
   // ---- indicator update (Eq. 2 / Eq. 3), importance (Eq. 4), arg-min ----
-  if (!mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+  if (state_in_smem && !mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
   const bool evicting = hi > B;
   unsigned long long my_key = NO_KEY;
   int my_slot = -1, my_pos = -1;
@@ -446,9 +470,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       float* ring_row = c.ring + ((int64_t)u * w + (t % w)) * cap;
       long long fx;
       if (is_new) {
-        // recycled slot: its ring column belongs to the previous occupant
-        for (int rr = 0; rr < w; ++rr) c.ring[((int64_t)u * w + rr) * cap + slot] = 0.f;
-        fx = prob_to_fixed(p);
+        fx = prob_to_fixed(p);     // (the recycled slot's ring column is cleared below)
       } else {
         fx = c.acc_fixed[o] + prob_to_fixed(p) - prob_to_fixed(ring_row[slot]);
       }
@@ -456,17 +478,22 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       c.acc_fixed[o] = fx;
       S = fixed_to_prob(fx);
     } else {
-      S = is_new ? p : acc_s[slot] + p;
+      S = is_new ? p : (state_in_smem ? acc_s[slot] : c.acc[o]) + p;
     }
     c.acc[o] = S;
     if (evicting) {
-      const int ps = is_new ? t : pos_s[slot];
-      const float I = S * (is_new ? new_norm : vn_s[slot]);
+      const int ps = is_new ? t : (state_in_smem ? pos_s[slot] : c.pos[o]);
+      const float I = S * (is_new ? new_norm : (state_in_smem ? vn_s[slot] : c.vnorm[o]));
       if (ps >= F && ps <= t - R) {
         const unsigned long long key = evict_key(I, ps);
         if (key < my_key) { my_key = key; my_slot = slot; my_pos = ps; }
       }
     }
+  }
+  if (WINDOWED) {
+    // recycled slot: the other rows of its ring column belong to the previous occupant
+    for (int rr = tid; rr < w; rr += WT)
+      if (rr != t % w) c.ring[((int64_t)u * w + rr) * cap + fs] = 0.f;
   }
   if (evicting) {
     const unsigned long long wkey = warp_min_key(my_key);
@@ -577,17 +604,25 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
   int chunk = (cap + split - 1) / split;
   chunk = (chunk + GROUP - 1) / GROUP * GROUP;
-  const size_t state_bytes = 4 * sizeof(float) * (size_t)chunk * split;
   // Two CTAs per SM (so that consecutive launches can both be resident) when at least two stages per
-  // warp fit in half an SM's shared memory, otherwise one CTA with up to four stages.
+  // warp fit in half an SM's shared memory beside the per-slot state; large caches leave acc / vnorm /
+  // pos in global memory (L2-prefetched) to get there; otherwise one CTA with up to four stages.
   const size_t half_sm = 104 * 1024, whole_sm = 215 * 1024;     // dynamic bytes, 1 KB of it alignment slack
-  if (state_bytes + (size_t)MW * STAGE_BYTES + 1024 > whole_sm) return cudaErrorNotSupported;
-  int nstage = state_bytes + 1024 + 2 * (size_t)MW * STAGE_BYTES <= half_sm
-                   ? (int)((half_sm - 1024 - state_bytes) / ((size_t)MW * STAGE_BYTES))
-                   : (int)((whole_sm - 1024 - state_bytes) / ((size_t)MW * STAGE_BYTES));
+  const size_t stage_set = (size_t)MW * STAGE_BYTES;
+  const size_t tot = (size_t)chunk * split;
+  size_t state_bytes = 4 * sizeof(float) * tot;
+  int state_in_smem = 1;
+  if (state_bytes + 1024 + 2 * stage_set > half_sm && sizeof(float) * tot + 1024 + 2 * stage_set <= half_sm) {
+    state_bytes = sizeof(float) * tot;
+    state_in_smem = (size_t)cap * 12 <= 2 * stage_set ? 2 : 0;
+  }
+  if (state_bytes + stage_set + 1024 > whole_sm) return cudaErrorNotSupported;
+  int nstage = state_bytes + 1024 + 2 * stage_set <= half_sm ? (int)((half_sm - 1024 - state_bytes) / stage_set)
+                                                             : (int)((whole_sm - 1024 - state_bytes) / stage_set);
   nstage = nstage > 4 ? 4 : nstage;
   const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
   if (nstage > groups_per_warp) nstage = groups_per_warp > 0 ? groups_per_warp : 1;
+  if (state_in_smem == 2 && (size_t)cap * 12 > (size_t)MW * nstage * STAGE_BYTES) state_in_smem = 0;
   const size_t dyn = (size_t)MW * nstage * STAGE_BYTES + state_bytes + 1024;
   CUtensorMap tm_k, tm_v;
   if (!make_rows_map_bf16(&tm_k, c.k_cache, (uint64_t)s.units * cap, GROUP) ||
@@ -625,7 +660,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
+  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, state_in_smem, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
                             (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                             (__nv_bfloat16*)out, evicted, dev_status);
 }

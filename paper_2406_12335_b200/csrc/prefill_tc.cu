@@ -333,11 +333,13 @@ struct TcArgs {
   // Eq. 3 (last w queries): only query rows >= first_row count; ft = first_row / 128; win_rows row r is
   // query wrow0 + r (wrow0 = T - w, negative when the prompt is shorter than the window).  H2O: all zero.
   int first_row, ft, wrow0, window;
+  int gu;                   // units per scheduling group (their K and Q fit in L2 together)
   float* win_rows;
 };
 
-// Work items are (unit, fixed tile of 128 rows), longest first, dealt to the persistent CTAs like a
-// snake draft (rounds alternate direction: load spread within a few percent).  The other operand
+// Work items are (unit, fixed tile of 128 rows), longest first within a group of units whose K and Q
+// share the L2 (with hundreds of units the streamed operand would otherwise come from HBM every
+// time), dealt to the persistent CTAs like a snake draft (rounds alternate direction).  The other operand
 // streams in chunks of 256 tokens (two tiles), so that one MMA instruction is 128 x 256 x 16: a
 // single thread issues the MMAs, and at 128 x 128 x 16 the issue cost exceeds the execution time.
 //   PASS 1: fixed = query tile i, streamed key chunks 0 .. i/2       (key tile kt needed iff kt <= i);
@@ -355,8 +357,14 @@ struct Item {
 template <int PASS>
 __device__ __forceinline__ Item item_of(int id, const TcArgs& a) {
   Item it;
-  const int r = id / a.units;
-  it.u = id - r * a.units;
+  // units are taken in groups whose K and Q stay in L2 together; inside a group, longest items first
+  const int ntp = PASS == 1 ? a.nt - a.ft : a.nt;
+  const int grp = id / (a.gu * ntp);
+  const int rem = id - grp * (a.gu * ntp);
+  const int u0 = grp * a.gu;
+  const int nu = min(a.gu, a.units - u0);
+  const int r = rem / nu;
+  it.u = u0 + (rem - r * nu);
   if (PASS == 1) { it.tile = a.nt - 1 - r; it.c_first = 0; it.c_count = it.tile / 2 + 1; it.lo = 0; }
   else           { it.tile = r; it.lo = max(r, a.ft); it.c_first = it.lo / 2; it.c_count = a.nch - it.c_first; }
   return it;
@@ -782,6 +790,16 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.ft = a.first_row / TILE;
   a.wrow0 = win ? s.T - s.window : 0;
   a.win_rows = win ? win_rows : nullptr;
+  // K and Q of one unit are 2 * T * 256 bytes; keep a group's working set near 48 MB (L2 is 126 MB),
+  // or take all units at once when everything fits anyway
+  {
+    const size_t unit_bytes = (size_t)2 * s.T * HD * 2;
+    if ((size_t)s.units * unit_bytes <= ((size_t)96 << 20)) a.gu = s.units;
+    else {
+      const size_t g = ((size_t)48 << 20) / unit_bytes;
+      a.gu = g < 1 ? 1 : (g > (size_t)s.units ? s.units : (int)g);
+    }
+  }
   const size_t smem = sizeof(Smem) + 1024;
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(prefill_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;

@@ -222,3 +222,10 @@ def test_windowed_indicator_shapes(T, w, B, F, R):
 
 def test_windowed_indicator_fp32_path():
     _run_case(_small("f32", 64, 300, 120, 2, 10, b=1, h=2, indicator="window", window=77, steps=6, cid=61))
+
+
+def test_decode_large_cache_state_paths():
+    """Caches too large for the per-slot state to sit beside the streaming stages: the state is copied
+    into the stage memory after the streaming (budget 3000) or read from global memory (budget 6000)."""
+    for T, B in ((3400, 3000), (6500, 6000)):
+        _run_case(_small("bf16", 128, T, B, 2, 64, b=1, h=2, steps=5, cid=62), check_state_every=5)
