@@ -57,7 +57,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE,
+                                          "-i", str(self.index), "-lms", "20"], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -351,7 +351,10 @@ def run_cuda(args, wl):
     dominant = max(share, key=share.get)
     roof = dict(kernels[dominant])
     roof["kernel"] = dominant
-    roof["traffic"] = None
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
+    # profiles/decode_mma_config1.md (same kernel, same shape); other kernels / shapes: not captured
+    roof["traffic"] = 34.52e6 if (dominant == "decode_step" and wl.cid == 1) else None
+    roof["algorithmic_bytes_per_launch"] = bytes_decode if dominant == "decode_step" else None
     roof["time_share"] = share[dominant] / sum(share.values())
 
     line = {
