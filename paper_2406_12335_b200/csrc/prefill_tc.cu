@@ -274,10 +274,12 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
     }
     l_run += hsum2(add2(a0, a1));
   } else if (!DIAG) {
-    const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(nlse_t + c0);
+    // explicit shared-memory loads: through the generic pointer they would take the slower generic path
+    const uint32_t lp = s32(nlse_t + c0);
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
-      const ulonglong2 L = lp[i >> 2];
+      ulonglong2 L;
+      asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(L.x), "=l"(L.y) : "r"(lp + 4 * i));
       const f32x2 e0 = exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, L.x));
       const f32x2 e1 = exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, L.y));
       cs[0] = add2(cs[0], e0);
@@ -293,11 +295,12 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
       }
     }
   } else {
-    const float4* lp = reinterpret_cast<const float4*>(nlse_t + c0);
+    const uint32_t lp = s32(nlse_t + c0);
     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
     for (int i = 0; i < 32; i += 4) {
-      const float4 L = lp[i >> 2];
+      float4 L;
+      asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(L.x), "=f"(L.y), "=f"(L.z), "=f"(L.w) : "r"(lp + 4 * i));
       float p0 = ex2(fmaf(x[i], scale_log2, L.x));
       float p1 = ex2(fmaf(x[i + 1], scale_log2, L.y));
       float p2 = ex2(fmaf(x[i + 2], scale_log2, L.z));
