@@ -104,7 +104,7 @@ size_t vatp_workspace_bytes(const vatp_params* params);
  * win_rows: VATP_IND_WINDOW only: [batch, heads, w, T] fp32 output, row r = probabilities of
  *           query T - w + r (zero where masked or where T - w + r < 0); NULL for H2O.
  * workspace: >= vatp_workspace_bytes(params) bytes of device scratch, 256-byte aligned; holds the
- *           row normalisers between the two passes.
+ *           row normalisers between the two passes and two work-item counters.
  * bf16 with head_dim 128 runs on the tensor cores; other combinations use an fp32 FMA kernel.
  */
 vatp_status vatp_prefill_scores(const vatp_params* params, const void* q, const void* k, const void* v,
@@ -136,7 +136,7 @@ vatp_status vatp_prefill_scores(const vatp_params* params, const void* q, const 
  * array keeps the previous call's contents; nothing in it needs clearing, because pass 1 writes
  * every normaliser that pass 2 reads.
  */
-#define VATP_STATIC_SCRATCH_BYTES (4u << 20)
+#define VATP_STATIC_SCRATCH_BYTES ((4u << 20) + 256u)
 vatp_status vatp_prefill_scores_static(const vatp_params* params, const void* q, const void* k, const void* v,
                                        float* lse_out, float* attn_acc, float* vnorm, float* score,
                                        float* win_rows, int32_t* dev_status, void* cuda_stream);

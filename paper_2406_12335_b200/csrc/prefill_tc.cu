@@ -45,6 +45,8 @@ struct Smem {
   uint64_t fixed_full[2], fixed_empty[2];
   uint64_t acc_full[NACC], acc_empty[NACC];
   uint64_t comb_full[2], comb_empty[2];
+  uint64_t item_full[4], item_empty[4];   // FIFO of work-item ids from the producer to the other roles
+  int item_ring[4];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -337,12 +339,14 @@ struct TcArgs {
   // query wrow0 + r (wrow0 = T - w, negative when the prompt is shorter than the window).  H2O: all zero.
   int first_row, ft, wrow0, window;
   int gu;                   // units per scheduling group (their K and Q fit in L2 together)
+  unsigned* counters;       // [2] next work item of pass 1 / pass 2 (zeroed before pass 1 is launched)
   float* win_rows;
 };
 
 // Work items are (unit, fixed tile of 128 rows), longest first within a group of units whose K and Q
 // share the L2 (with hundreds of units the streamed operand would otherwise come from HBM every
-// time), dealt to the persistent CTAs like a snake draft (rounds alternate direction).  The other operand
+// time).  The persistent CTAs draw them from a global counter, so a CTA that finishes early takes
+// the next item instead of idling (a static deal left the average CTA idle for a tenth of a pass).  The other operand
 // streams in chunks of 256 tokens (two tiles), so that one MMA instruction is 128 x 256 x 16: a
 // single thread issues the MMAs, and at 128 x 128 x 16 the issue cost exceeds the execution time.
 //   PASS 1: fixed = query tile i, streamed key chunks 0 .. i/2       (key tile kt needed iff kt <= i);
@@ -351,7 +355,6 @@ struct TcArgs {
 //           lo = max(i, first tile of the window))
 // Softmax warpgroup g takes columns [128 g, 128 g + 128) of every accumulator, i.e. streamed tile
 // 2 c + g of chunk c; the two partial results of a row are combined once per item.
-__device__ __forceinline__ int item_id(int n, int c, int G) { return n * G + ((n & 1) ? G - 1 - c : c); }
 
 struct Item {
   int u, tile, c_first, c_count;
@@ -394,6 +397,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       mbar_init(&sm.comb_full[i], 128); mbar_init(&sm.comb_empty[i], 128);
     }
     for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 8); }
+    // consumers of the item FIFO: the MMA warp, eight softmax warps and, for Eq. 3's pass 2, the side warp
+    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 9 + ((PASS == 2 && WIN) ? 1 : 0)); }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -407,6 +412,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
+  // Consumer side of the item FIFO: the itl-th item of this CTA (an id >= items ends the pass).
+  // The slot is handed back as soon as the id has been read.
+  auto next_item = [&](uint32_t itl, bool whole_warp) -> int {
+    const int slot = itl & 3;
+    bool got = mbar_wait(&sm.item_full[slot], (itl >> 2) & 1, abort_flag, a.dev_status);
+    if (whole_warp) got = __all_sync(0xffffffffu, got);
+    const int id = got ? *reinterpret_cast<volatile int*>(&sm.item_ring[slot]) : -1;
+    if (whole_warp) __syncwarp();
+    if (got && (!whole_warp || lane == 0)) mbar_arrive(&sm.item_empty[slot]);
+    return id;     // -1: the CTA is aborting
+  };
+
   // the operand that stays fixed per item and the one that streams
   const CUtensorMap* tm_fixed = PASS == 1 ? &tm_q : &tm_k;
   const CUtensorMap* tm_stream = PASS == 1 ? &tm_k : &tm_q;
@@ -415,8 +432,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       bool ok = true;
-      uint32_t n = 0, itl = 0;
-      for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
+      uint32_t n = 0;
+      int next = (int)atomicAdd(&a.counters[PASS - 1], 1u);
+      for (uint32_t itl = 0; ok; ++itl) {
+        const int id = next;
+        const int slot = itl & 3;
+        ok = mbar_wait<20>(&sm.item_empty[slot], ((itl >> 2) & 1) ^ 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        *reinterpret_cast<volatile int*>(&sm.item_ring[slot]) = id;
+        mbar_arrive(&sm.item_full[slot]);
+        if (id >= items) break;
+        next = (int)atomicAdd(&a.counters[PASS - 1], 1u);     // in flight while this item's tiles are requested
         const Item it = item_of<PASS>(id, a);
         const int b = it.u / a.heads, h = it.u - b * a.heads;
         const int fb = itl & 1;
@@ -445,10 +471,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       bool ok = true;
-      uint32_t n = 0, itl = 0;
+      uint32_t n = 0;
       const uint64_t stage_desc0 = umma_desc(s32(sm.stream[0]));   // stages are CHUNK_BYTES apart
       const uint64_t fixed_desc0 = umma_desc(s32(sm.fixed[0]));    // buffers are TILE_BYTES apart
-      for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
+      for (uint32_t itl = 0; ok; ++itl) {
+        const int id = next_item(itl, false);
+        if (id < 0 || id >= items) break;
         const Item it = item_of<PASS>(id, a);
         const int fb = itl & 1;
         ok = mbar_wait(&sm.fixed_full[fb], (itl >> 1) & 1, abort_flag, a.dev_status);
@@ -481,8 +509,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + g * TILE;
     float* lse_w = &sm.lse_s[wid - 2][0][0];
     bool ok = true;
-    uint32_t n = 0, itl = 0;
-    for (int id = item_id(0, blockIdx.x, gridDim.x); ok && id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
+    uint32_t n = 0;
+    for (uint32_t itl = 0; ok; ++itl) {
+      const int id = next_item(itl, true);
+      if (id < 0 || id >= items) break;
       const Item it = item_of<PASS>(id, a);
       const int u = it.u;
       const int pi = itl & 1;
@@ -688,8 +718,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ------------------------------------------------------------------ pass 2, Eq. 3: window rows nobody visits
     // For key tile i the query tiles before it are never streamed (causal), and when the prompt is
     // shorter than the window its first rows belong to no query: those entries of win_rows are zero.
-    uint32_t itl = 0;
-    for (int id = item_id(0, blockIdx.x, gridDim.x); id < items; id = item_id(++itl, blockIdx.x, gridDim.x)) {
+    for (uint32_t itl = 0;; ++itl) {
+      const int id = next_item(itl, true);
+      if (id < 0 || id >= items) break;
       const Item it = item_of<PASS>(id, a);
       float* wr = a.win_rows + (int64_t)it.u * a.window * a.T;
       const int k0 = it.tile * TILE;
@@ -769,7 +800,7 @@ bool vatp_tc_available() {
 
 size_t prefill_tc_workspace_bytes(int units, int T) {
   const size_t Tpad = (size_t)(T + CHUNK - 1) / CHUNK * CHUNK;
-  return (size_t)units * Tpad * sizeof(float);
+  return ((size_t)units * Tpad * sizeof(float) + 255) / 256 * 256 + 256;   // normalisers, then the work-item counters
 }
 
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
@@ -787,6 +818,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.sb = s.sb; a.sh = s.sh; a.st = s.st;
   a.lse2 = lse_ws; a.lse_out = lse_out; a.attn_acc = attn_acc; a.vnorm = vnorm; a.score = score;
   a.dev_status = dev_status;
+  a.counters = reinterpret_cast<unsigned*>(reinterpret_cast<char*>(lse_ws) + ((size_t)a.units * a.Tpad * sizeof(float) + 255) / 256 * 256);
   const bool win = s.window > 0;
   a.window = win ? s.window : 0;
   a.first_row = win && s.T > s.window ? s.T - s.window : 0;
@@ -812,6 +844,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
+  if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
   prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   if (win) prefill_tc_kernel<2, true><<<items2 < sms ? items2 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   else     prefill_tc_kernel<2, false><<<items2 < sms ? items2 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);

@@ -18,7 +18,7 @@ lib = C.CDLL(_LIB_PATH)
 OK = 0
 BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
-STATIC_SCRATCH_BYTES = 4 << 20
+STATIC_SCRATCH_BYTES = (4 << 20) + 256
 EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
            "vatp_status_string"]
 

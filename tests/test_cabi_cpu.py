@@ -39,7 +39,7 @@ def test_status_strings(V):
 
 def test_host_side_validation(V):
     ok = dict(batch=1, heads=2, seq_len=64, head_dim=64, dtype="f32", budget=16, n_sink=2, n_recent=4)
-    assert V.vatp_workspace_bytes(V.make_params(**ok)) == 2048   # 2 units x one padded 256-token chunk x 4 bytes
+    assert V.vatp_workspace_bytes(V.make_params(**ok)) == 2048 + 256   # 2 units x one padded 256-token chunk x 4 bytes, then the work-item counters
     assert V.vatp_workspace_bytes(V.make_params(**{**ok, "head_dim": 96})) == 0
     assert V.vatp_workspace_bytes(V.make_params(**{**ok, "n_recent": 15})) == 0     # F + R > B
     p = V.make_params(**ok)
