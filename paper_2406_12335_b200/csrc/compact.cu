@@ -9,8 +9,9 @@ constexpr int CP_THREADS = 256;
 constexpr int CP_SLOTS = 64;     // destination slots per CTA
 constexpr int CP_ITERS = CP_SLOTS / (CP_THREADS / 16);
 
-// grid (units, slot groups).  Sixteen lanes copy one row (K and V) in 16-byte pieces; a thread has
-// CP_ITERS rows of K and of V in flight before it stores, and no index needs a division.
+// grid (units, y), each CTA walking slot groups y, y + gridDim.y, ... so that the whole grid is one
+// resident wave.  Sixteen lanes copy one row (K and V) in 16-byte pieces; a thread has CP_ITERS rows of
+// K and of V in flight before it stores, and no index needs a division.
 __global__ void __launch_bounds__(CP_THREADS, 4)
 compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict__ k, const char* __restrict__ v,
                const float* __restrict__ attn_acc, const float* __restrict__ vnorm, const int32_t* __restrict__ kept,
@@ -19,10 +20,11 @@ compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict_
   const int len = min(sh.T, B);
   const int row_bytes = sh.d * elem_bytes;
   const int hw = threadIdx.x >> 4, l16 = threadIdx.x & 15;
-  const int slot0 = blockIdx.y * CP_SLOTS + hw;
   const int64_t unit_bytes = unit_offset(sh, u) * elem_bytes;
   const int64_t tok_bytes = sh.st * elem_bytes;
 
+  for (int grp = blockIdx.y; grp * CP_SLOTS < cap; grp += gridDim.y) {
+  const int slot0 = grp * CP_SLOTS + hw;
   int src[CP_ITERS];
 #pragma unroll
   for (int i = 0; i < CP_ITERS; ++i) {
@@ -58,6 +60,7 @@ compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict_
       c.acc[o] = src[i] >= 0 ? __ldg(attn_acc + (int64_t)u * sh.T + src[i]) : 0.f;
       c.vnorm[o] = src[i] >= 0 ? __ldg(vnorm + (int64_t)u * sh.T + src[i]) : 0.f;
     }
+  }
   }
   if (blockIdx.y == 0 && threadIdx.x == 0) {
     c.len[u] = len;
@@ -96,7 +99,16 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            cudaStream_t st) {
   const int eb = dtype == VATP_F32 ? 4 : 2;
   const int cap = cache_capacity(B);
-  const dim3 grid(s.units, (cap + CP_SLOTS - 1) / CP_SLOTS);
+  static int sms = 0;
+  if (!sms) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
+  }
+  const int groups = (cap + CP_SLOTS - 1) / CP_SLOTS;
+  int gy = 4 * sms / s.units;        // four CTAs fit on an SM
+  gy = gy < 1 ? 1 : (gy > groups ? groups : gy);
+  const dim3 grid(s.units, gy);
   compact_kernel<<<grid, CP_THREADS, 0, st>>>(s, eb, B, cap, (const char*)k, (const char*)v, attn_acc, vnorm, kept, c);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
