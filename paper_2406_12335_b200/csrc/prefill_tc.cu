@@ -21,7 +21,8 @@
 namespace vatp {
 namespace {
 
-constexpr int TC_THREADS = 352;
+constexpr int NSW = 16;            // softmax warps
+constexpr int TC_THREADS = (2 + NSW + 1) * 32;
 constexpr int TILE = 128;          // rows of the fixed tile = columns of a streamed tile
 constexpr int HD = 128;            // head_dim
 constexpr int CHUNK = 256;         // streamed tokens per stage = columns of an accumulator
@@ -32,15 +33,15 @@ constexpr int TILE_BYTES = 2 * SLAB_BYTES;    // two K halves
 constexpr int CHUNK_BYTES = 2 * TILE_BYTES;   // 256 rows, two K halves
 constexpr uint64_t WAIT_NS = 1000000000ull;
 #ifndef VATP_POLY_MASK
-#define VATP_POLY_MASK 0x1111   // bit p set: pair p (of the 16 pairs of a 32-column slice) takes the FMA-pipe exponential
+#define VATP_POLY_MASK 0x0101   // bit p set: pair p (of the 16 pairs of a 32-column slice) takes the FMA-pipe exponential
 #endif
 
 struct Smem {
   alignas(1024) unsigned char fixed[2][TILE_BYTES];      // double-buffered fixed tile
   alignas(1024) unsigned char stream[NS][CHUNK_BYTES];   // [K half][256 rows][128 bytes] per stage
-  alignas(16) float lse_s[8][2][TILE];   // pass 2: per softmax warp, double-buffered NEGATED normalisers of a query tile
-  float part_a[2][TILE];   // pass 1: running max of warpgroup 1; pass 2: its column sums
-  float part_b[2][TILE];   // pass 1: running sum of warpgroup 1
+  alignas(16) float lse_s[NSW][2][64];   // pass 2: per softmax warp, double-buffered NEGATED normalisers of its 64 query columns
+  float part_a[2][3][TILE];   // pass 1: running max of warpgroups 1-3; pass 2: their column sums
+  float part_b[2][3][TILE];   // pass 1: running sum of warpgroups 1-3
   alignas(8) uint64_t full[NS], empty[NS];
   uint64_t fixed_full[2], fixed_empty[2];
   uint64_t acc_full[NACC], acc_empty[NACC];
@@ -394,11 +395,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     for (int i = 0; i < NS; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(&sm.fixed_full[i], 1); mbar_init(&sm.fixed_empty[i], 1);
-      mbar_init(&sm.comb_full[i], 128); mbar_init(&sm.comb_empty[i], 128);
+      mbar_init(&sm.comb_full[i], 3 * 128); mbar_init(&sm.comb_empty[i], 128);
     }
-    for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], 8); }
+    for (int i = 0; i < NACC; ++i) { mbar_init(&sm.acc_full[i], 1); mbar_init(&sm.acc_empty[i], NSW); }
     // consumers of the item FIFO: the MMA warp, eight softmax warps and, for Eq. 3's pass 2, the side warp
-    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 9 + ((PASS == 2 && WIN) ? 1 : 0)); }
+    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 1 + NSW + ((PASS == 2 && WIN) ? 1 : 0)); }
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -427,6 +428,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   // the operand that stays fixed per item and the one that streams
   const CUtensorMap* tm_fixed = PASS == 1 ? &tm_q : &tm_k;
   const CUtensorMap* tm_stream = PASS == 1 ? &tm_k : &tm_q;
+
+  // Pass 2 is launched as a programmatic dependent of pass 1: its CTAs start as pass-1 CTAs retire and
+  // set up, fetch items and stream Q / K tiles at once; only what pass 1 writes (normalisers, value
+  // norms) is read after griddepcontrol.wait, i.e. once pass 1 has completed.
+  if (PASS == 1 && tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (wid == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -501,15 +507,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (ok) umma_commit(&sm.fixed_empty[fb]);
       }
     }
-  } else if (wid < 10) {
+  } else if (wid < 2 + NSW) {
     // ------------------------------------------------------------------ softmax warpgroups
-    const int g = (wid - 2) >> 2;                 // warpgroup g takes half g of every chunk
+    const int sw = wid - 2;
+    const int g = sw >> 2;                        // warpgroup g takes columns [64 g, 64 g + 64) of every accumulator
     const int quarter = wid & 3;                  // TMEM lanes this warp may touch
     const int row = quarter * 32 + lane;          // row of the fixed tile = TMEM lane
-    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + g * TILE;
-    float* lse_w = &sm.lse_s[wid - 2][0][0];
+    const int half = g >> 1;                      // which 128-token tile of a chunk those columns belong to
+    const int cbase = (g & 1) * 64;               // and where they start inside that tile
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + half * TILE + cbase;
+    float* lse_w = &sm.lse_s[sw][0][0];
     bool ok = true;
     uint32_t n = 0;
+    if (PASS == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (uint32_t itl = 0; ok; ++itl) {
       const int id = next_item(itl, true);
       if (id < 0 || id >= items) break;
@@ -527,11 +537,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const uint32_t n0 = n;
       n += it.c_count;
       int buf = 0;
-      float xa[32], xb[32];
-      // streamed tile of this warpgroup in chunk c, and whether the item needs it
-      auto st_of = [&](int c) { return 2 * (it.c_first + c) + g; };
+      // streamed tile this warp's columns belong to in chunk c, and whether the item needs it
+      auto st_of = [&](int c) { return 2 * (it.c_first + c) + half; };
       auto needed = [&](int c) { return tile_needed<PASS>(it, st_of(c), a.nt); };
-      auto acc_addr = [&](int c) { return lane_addr + ((n0 + c) % NACC) * CHUNK; };
       // where the probabilities of the 32 query columns starting at column c0 of streamed tile stile go (Eq. 3 rows)
       auto wout = [&](int stile, int c0) {
         WinOut wo{nullptr, 0, 0, 0};
@@ -544,125 +552,83 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
         return wo;
       };
-      auto chunk_wait = [&](int c) -> bool {
-        bool w = mbar_wait(&sm.acc_full[(n0 + c) % NACC], ((n0 + c) / NACC) & 1, abort_flag, a.dev_status);
-        w = __all_sync(0xffffffffu, w);
-        tc_fence_after();
-        return w;
+      // pass 2: this warp's 64 normalisers of chunk c (negated), one float4 per lane 0-15
+      auto lse_fetch = [&](int c) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (lane < 16) v = neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c) * TILE + cbase) + lane));
+        return v;
       };
-      auto release = [&](int c) {                 // all TMEM reads of chunk c by this warp are complete
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.acc_empty[(n0 + c) % NACC]);
-      };
-      // prologue: first chunk
-      ok = chunk_wait(0);
-      if (!ok) break;
-      bool have = needed(0);                      // xa holds columns 0..31 of chunk c (when needed)
-      if (have) {
-        tmem_ld32(acc_addr(0), xa);
-        if (PASS == 2) {
-          reinterpret_cast<float4*>(lse_w)[lane] = neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(0) * TILE) + lane));
-          __syncwarp();
+      if (PASS == 2) {
+        int c1 = 0;
+        while (c1 < it.c_count && !needed(c1)) ++c1;
+        if (c1 < it.c_count) {
+          const float4 v = lse_fetch(c1);
+          if (lane < 16) reinterpret_cast<float4*>(lse_w)[lane] = v;
         }
-        tmem_ld_wait();
+        __syncwarp();
       }
       for (int c = 0; c < it.c_count; ++c) {
-        const bool has_next = c + 1 < it.c_count;
-        const bool next_needed = has_next && needed(c + 1);
-        if (!have) {
-          // this half of the chunk is masked for the item: hand the accumulator back at once
-          release(c);
-          if (has_next) {
-            ok = chunk_wait(c + 1);
-            if (!ok) break;
-            if (next_needed) {
-              tmem_ld32(acc_addr(c + 1), xa);
-              if (PASS == 2) {
-                reinterpret_cast<float4*>(lse_w + buf * TILE)[lane] =
-                    neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane));
-                __syncwarp();
-              }
-              tmem_ld_wait();
-            }
-          }
-          have = next_needed;
+        const uint32_t ab = (n0 + c) % NACC;
+        bool w = mbar_wait(&sm.acc_full[ab], ((n0 + c) / NACC) & 1, abort_flag, a.dev_status);
+        w = __all_sync(0xffffffffu, w);
+        if (!w) { ok = false; break; }
+        tc_fence_after();
+        if (!needed(c)) {
+          // this tile of the chunk is masked for the item: hand the accumulator back at once
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
           continue;
         }
-        const bool diag = st_of(c) == it.tile;
-        const uint32_t t_addr = acc_addr(c);
-        const float* lse_t = lse_w + buf * TILE;
+        float xa[32], xb[32];
+        const uint32_t t_addr = lane_addr + ab * CHUNK;
+        tmem_ld32(t_addr, xa);
+        tmem_ld32(t_addr + 32, xb);
+        // normalisers of the next needed chunk travel while this one is consumed
+        const bool next_needed = c + 1 < it.c_count && needed(c + 1);
         float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (PASS == 2 && next_needed)
-          lnext = neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c + 1) * TILE) + lane));
-        // Both paths are rolled loops with few inlined copies of the slice code: the steady-state
-        // body stays small enough for the instruction cache.
-        if (!diag) {
-          // software pipeline: the TMEM load of the next 32 columns is in flight while these are consumed
-#pragma unroll 1
-          for (int h2 = 0; h2 < 2; ++h2) {
-            tmem_ld32(t_addr + 64 * h2 + 32, xb);
-            consume32<PASS, false, WIN>(xa, 64 * h2, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(st_of(c), 64 * h2));
-            tmem_ld_wait();
-            if (h2 == 0) {
-              tmem_ld32(t_addr + 64, xa);
-            } else {
-              release(c);
-              if (has_next) {
-                ok = chunk_wait(c + 1);
-                if (ok && next_needed) tmem_ld32(acc_addr(c + 1), xa);
-              }
-            }
-            if (ok) consume32<PASS, false, WIN>(xb, 64 * h2 + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(st_of(c), 64 * h2 + 32));
-            if (h2 == 1 && PASS == 2 && next_needed) {
-              reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
-              __syncwarp();
-            }
-            tmem_ld_wait();
-          }
+        if (PASS == 2 && next_needed) lnext = lse_fetch(c + 1);
+        tmem_ld_wait();
+        // this warp's columns are in registers: the MMA warp may overwrite them
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
+        const float* lse_t = lse_w + buf * 64 - cbase;     // indexed by the column inside the tile
+        const int stile = st_of(c);
+        if (stile == it.tile) {
+          consume32<PASS, true, WIN>(xa, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
+          consume32<PASS, true, WIN>(xb, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
         } else {
-          // the one diagonal tile of an item takes the masked variant (not pipelined)
-#pragma unroll 1
-          for (int c0 = 0; c0 < TILE; c0 += 32) {
-            consume32<PASS, true, WIN>(xa, c0, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(st_of(c), c0));
-            if (c0 + 32 < TILE) {
-              tmem_ld32(t_addr + c0 + 32, xa);
-              tmem_ld_wait();
-            }
-          }
-          release(c);
-          if (has_next) {
-            ok = chunk_wait(c + 1);
-            if (ok && next_needed) tmem_ld32(acc_addr(c + 1), xa);
-          }
-          if (PASS == 2 && next_needed) {
-            reinterpret_cast<float4*>(lse_w + (buf ^ 1) * TILE)[lane] = lnext;
-            __syncwarp();
-          }
-          tmem_ld_wait();
+          consume32<PASS, false, WIN>(xa, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
+          consume32<PASS, false, WIN>(xb, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
         }
-        if (!ok) break;
-        have = next_needed;
-        buf ^= 1;
+        if (PASS == 2 && next_needed) {
+          if (lane < 16) reinterpret_cast<float4*>(lse_w + (buf ^ 1) * 64)[lane] = lnext;
+          __syncwarp();
+          buf ^= 1;
+        }
       }
       if (!ok) break;
-      // ---- end of item: warpgroup 1 hands its partial to warpgroup 0, which finishes the rows
-      if (g == 1) {
+      // ---- end of item: warpgroups 1-3 hand their partials to warpgroup 0, which finishes the rows
+      if (g > 0) {
         ok = mbar_wait(&sm.comb_empty[pi], ipar ^ 1, abort_flag, a.dev_status);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
-        if (PASS == 1) { sm.part_a[pi][row] = m_run; sm.part_b[pi][row] = l_run; }
-        else           { sm.part_a[pi][row] = hsum2(add2(cs[0], cs[1])); }
+        if (PASS == 1) { sm.part_a[pi][g - 1][row] = m_run; sm.part_b[pi][g - 1][row] = l_run; }
+        else           { sm.part_a[pi][g - 1][row] = hsum2(add2(cs[0], cs[1])); }
         mbar_arrive(&sm.comb_full[pi]);
       } else {
         ok = mbar_wait(&sm.comb_full[pi], ipar, abort_flag, a.dev_status);
         if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
         if (PASS == 1) {
-          const float m1 = sm.part_a[pi][row], l1 = sm.part_b[pi][row];
+          const float m1 = sm.part_a[pi][0][row], m2 = sm.part_a[pi][1][row], m3 = sm.part_a[pi][2][row];
+          const float l1 = sm.part_b[pi][0][row], l2 = sm.part_b[pi][1][row], l3 = sm.part_b[pi][2][row];
           mbar_arrive(&sm.comb_empty[pi]);
-          const float m = fmaxf(m_run, m1);
+          const float m = fmaxf(fmaxf(m_run, m1), fmaxf(m2, m3));
           float l = 0.f;
           if (l_run > 0.f) l += l_run * ex2(m_run - m);
           if (l1 > 0.f) l += l1 * ex2(m1 - m);
+          if (l2 > 0.f) l += l2 * ex2(m2 - m);
+          if (l3 > 0.f) l += l3 * ex2(m3 - m);
           const float lse2 = m + log2f(l);
           // queries outside the prompt or before the history window contribute nothing to pass 2
           a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? lse2 : INFINITY;
@@ -670,7 +636,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = INFINITY;
           if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
         } else {
-          const float tot = hsum2(add2(cs[0], cs[1])) + sm.part_a[pi][row];
+          const float tot = hsum2(add2(cs[0], cs[1])) + (sm.part_a[pi][0][row] + sm.part_a[pi][1][row]) + sm.part_a[pi][2][row];
           mbar_arrive(&sm.comb_empty[pi]);
           if (tok < a.T) {
             const int64_t o = (int64_t)u * a.T + tok;
@@ -846,9 +812,19 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
   if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
   prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
-  if (win) prefill_tc_kernel<2, true><<<items2 < sms ? items2 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
-  else     prefill_tc_kernel<2, false><<<items2 < sms ? items2 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
-  return cudaGetLastError();
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(items2 < sms ? items2 : sms);
+  cfg.blockDim = dim3(TC_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return win ? cudaLaunchKernelEx(&cfg, prefill_tc_kernel<2, true>, tm_q, tm_k, a)
+             : cudaLaunchKernelEx(&cfg, prefill_tc_kernel<2, false>, tm_q, tm_k, a);
 }
 
 }  // namespace vatp
