@@ -9,9 +9,15 @@
 //           multiplies by the value l1 norm (Eq. 4), which a side warp of pass 1 has reduced.
 // Both operands are [token, d] row-major, i.e. K-major for A and B alike.
 //
-// Warp roles (352 threads): warp 0 TMA producer, warp 1 MMA issuer and TMEM owner, warps 2-9 two
-// softmax warpgroups (each takes one 128-column half of every 256-column accumulator), warp 10 the
-// value-norm reduction (pass 1 only).
+// With a history window (Eq. 3) only the last w query rows count: pass 1 covers the query tiles that
+// reach into the window, pass 2 streams from the window's first tile on and also writes the
+// probabilities of those rows (win_rows); a side warp zeroes the entries nobody visits.
+//
+// Warp roles (608 threads): warp 0 TMA producer (it also draws the work items from a global counter
+// and passes them on), warp 1 MMA issuer and TMEM owner, warps 2-17 four softmax warpgroups (each takes
+// one 64-column quarter of every 256-column accumulator, loads it into registers and hands the
+// accumulator back at once; four warps per scheduler keep the exponential unit busy where two could
+// not), warp 18 the value-norm reduction (pass 1) / window zero fill (pass 2 with Eq. 3).
 // Every wait is bounded; on expiry the CTA raises a flag, writes VATP_ERR_TIMEOUT to the status
 // word, drains, frees its TMEM and returns.
 #include <cuda.h>
@@ -234,6 +240,33 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
   return d;
 }
 
+// pass 1 building blocks for one 32-column slice (x: raw dot products of this thread's query row)
+__device__ __forceinline__ void mask_after_diagonal(float (&x)[32], int c0, int row) {
+#pragma unroll
+  for (int i = 0; i < 32; ++i)
+    if (c0 + i > row) x[i] = -INFINITY;
+}
+__device__ __forceinline__ float slice_max(const float (&x)[32]) {
+  // four short max chains instead of one long one
+  float c0m = max3(x[0], x[1], x[2]), c1m = max3(x[8], x[9], x[10]);
+  float c2m = max3(x[16], x[17], x[18]), c3m = max3(x[24], x[25], x[26]);
+  c0m = max3(c0m, x[3], x[4]); c1m = max3(c1m, x[11], x[12]); c2m = max3(c2m, x[19], x[20]); c3m = max3(c3m, x[27], x[28]);
+  c0m = max3(c0m, x[5], x[6]); c1m = max3(c1m, x[13], x[14]); c2m = max3(c2m, x[21], x[22]); c3m = max3(c3m, x[29], x[30]);
+  c0m = max3(c0m, x[7], c1m); c2m = max3(c2m, x[15], c3m);
+  return max3(c0m, c2m, fmaxf(x[23], x[31]));
+}
+// sum over the slice of exp2(scale_log2 * x - m)
+__device__ __forceinline__ float slice_exp_sum(const float (&x)[32], float scale_log2, float m) {
+  const f32x2 c2 = pk2(scale_log2, scale_log2), nm2 = pk2(-m, -m);
+  f32x2 a0 = pk2(0.f, 0.f), a1 = a0;
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    a0 = add2(a0, exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, nm2)));
+    a1 = add2(a1, exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, nm2)));
+  }
+  return hsum2(add2(a0, a1));
+}
+
 // One 32-column slice of an accumulator row.  x holds raw dot products; c0 is the slice's first
 // column inside the tile, row the thread's row.
 //   PASS 1 (row = query, columns = keys): online max / sum of exp2(scale_log2 * s); on the diagonal
@@ -253,29 +286,12 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
                                           f32x2 (&cs)[2], const float* nlse_t, const WinOut& wo) {
   const f32x2 c2 = pk2(scale_log2, scale_log2);
   if (PASS == 1) {
-    if (DIAG) {
-#pragma unroll
-      for (int i = 0; i < 32; ++i)
-        if (c0 + i > row) x[i] = -INFINITY;
-    }
-    // four short max chains instead of one long one, then a branch-free rescale of the running sum
-    float c0m = max3(x[0], x[1], x[2]), c1m = max3(x[8], x[9], x[10]);
-    float c2m = max3(x[16], x[17], x[18]), c3m = max3(x[24], x[25], x[26]);
-    c0m = max3(c0m, x[3], x[4]); c1m = max3(c1m, x[11], x[12]); c2m = max3(c2m, x[19], x[20]); c3m = max3(c3m, x[27], x[28]);
-    c0m = max3(c0m, x[5], x[6]); c1m = max3(c1m, x[13], x[14]); c2m = max3(c2m, x[21], x[22]); c3m = max3(c3m, x[29], x[30]);
-    c0m = max3(c0m, x[7], c1m); c2m = max3(c2m, x[15], c3m);
-    const float cmax = max3(c0m, c2m, fmaxf(x[23], x[31])) * scale_log2;   // scale > 0 keeps the order
+    if (DIAG) mask_after_diagonal(x, c0, row);
+    const float cmax = slice_max(x) * scale_log2;   // scale > 0 keeps the order
     const float m_new = fmaxf(m_run, cmax);
     l_run *= ex2(fmaxf(m_run - m_new, -126.f));      // (-inf) - (-inf) = NaN -> -126 -> factor on a zero sum
     m_run = m_new;
-    const f32x2 nm2 = pk2(-m_run, -m_run);
-    f32x2 a0 = pk2(0.f, 0.f), a1 = a0;
-#pragma unroll
-    for (int i = 0; i < 32; i += 4) {
-      a0 = add2(a0, exp2_pair(i >> 1, fma2(pk2(x[i], x[i + 1]), c2, nm2)));
-      a1 = add2(a1, exp2_pair((i >> 1) + 1, fma2(pk2(x[i + 2], x[i + 3]), c2, nm2)));
-    }
-    l_run += hsum2(add2(a0, a1));
+    l_run += slice_exp_sum(x, scale_log2, m_run);
   } else if (!DIAG) {
     // explicit shared-memory loads: through the generic pointer they would take the slower generic path
     const uint32_t lp = s32(nlse_t + c0);
@@ -595,7 +611,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
         const float* lse_t = lse_w + buf * 64 - cbase;     // indexed by the column inside the tile
         const int stile = st_of(c);
-        if (stile == it.tile) {
+        if (PASS == 1) {
+          // both slices share one row maximum and one rescale of the running sum
+          if (stile == it.tile) { mask_after_diagonal(xa, cbase, row); mask_after_diagonal(xb, cbase + 32, row); }
+          const float m_new = fmaxf(m_run, fmaxf(slice_max(xa), slice_max(xb)) * a.scale_log2);
+          l_run *= ex2(fmaxf(m_run - m_new, -126.f));
+          m_run = m_new;
+          l_run += slice_exp_sum(xa, a.scale_log2, m_run) + slice_exp_sum(xb, a.scale_log2, m_run);
+        } else if (stile == it.tile) {
           consume32<PASS, true, WIN>(xa, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
           consume32<PASS, true, WIN>(xb, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
         } else {
