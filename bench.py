@@ -351,8 +351,8 @@ def run_cuda(args, wl):
     dominant = max(share, key=share.get)
     roof = dict(kernels[dominant])
     roof["kernel"] = dominant
-    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu capture summarised in
-    # profiles/decode_mma_config1.md (same kernel, same shape); other kernels / shapes: not captured
+    # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of this kernel at
+    # this shape (profiles/); other kernels / shapes: not captured
     roof["traffic"] = 34.52e6 if (dominant == "decode_step" and wl.cid == 1) else None
     roof["algorithmic_bytes_per_launch"] = bytes_decode if dominant == "decode_step" else None
     roof["time_share"] = share[dominant] / sum(share.values())
