@@ -178,6 +178,15 @@ vatp_status vatp_decode_step(const vatp_params* params, const vatp_cache* cache,
                              const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
                              int32_t* dev_status, void* cuda_stream);
 
+/*
+ * Self-test of the bounded device-side waits (every pipeline wait in this library gives up after a
+ * time limit, writes VATP_ERR_TIMEOUT to *dev_status and lets the kernel return; nothing traps).
+ * Launches one CTA that waits on a barrier nobody arms for `limit_ns` nanoseconds (1 .. 1e8).
+ * dev_status: device int32, set to VATP_ERR_TIMEOUT by the kernel; waited_ns: device uint64,
+ * nullable, receives the time actually waited.  The paper has no counterpart.
+ */
+vatp_status vatp_selftest_bounded_wait(uint64_t limit_ns, int32_t* dev_status, uint64_t* waited_ns, void* cuda_stream);
+
 const char* vatp_status_string(vatp_status status);
 
 #ifdef __cplusplus

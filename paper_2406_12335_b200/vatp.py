@@ -20,7 +20,7 @@ BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
 STATIC_SCRATCH_BYTES = (4 << 20) + 256
 EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
-           "vatp_status_string"]
+           "vatp_selftest_bounded_wait", "vatp_status_string"]
 
 
 class Params(C.Structure):
@@ -51,6 +51,8 @@ lib.vatp_compact.restype = C.c_int
 lib.vatp_compact.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(CacheStruct), _vp, _vp]
 lib.vatp_decode_step.restype = C.c_int
 lib.vatp_decode_step.argtypes = [C.POINTER(Params), C.POINTER(CacheStruct), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.vatp_selftest_bounded_wait.restype = C.c_int
+lib.vatp_selftest_bounded_wait.argtypes = [C.c_uint64, _vp, _vp, _vp]
 lib.vatp_status_string.restype = C.c_char_p
 lib.vatp_status_string.argtypes = [C.c_int]
 
@@ -157,3 +159,10 @@ def vatp_decode_step(p: Params, cache: Cache, q_new, k_new, v_new, out, *, evict
                      stream=None):
     _check(lib.vatp_decode_step(C.byref(p), C.byref(cache.struct), _ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(out),
                                 _ptr(evicted_pos), _ptr(dev_status), _stream(stream)), "vatp_decode_step")
+
+
+def vatp_selftest_bounded_wait(limit_ns: int, dev_status, waited_ns=None, *, stream=None):
+    """Launches the one-CTA kernel that waits `limit_ns` on a barrier nobody arms and then reports
+    VATP_ERR_TIMEOUT (5) in dev_status: shows that an expired device-side wait ends cleanly."""
+    _check(lib.vatp_selftest_bounded_wait(int(limit_ns), _ptr(dev_status), _ptr(waited_ns), _stream(stream)),
+           "vatp_selftest_bounded_wait")

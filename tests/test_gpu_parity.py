@@ -229,3 +229,18 @@ def test_decode_large_cache_state_paths():
     into the stage memory after the streaming (budget 3000) or read from global memory (budget 6000)."""
     for T, B in ((3400, 3000), (6500, 6000)):
         _run_case(_small("bf16", 128, T, B, 2, 64, b=1, h=2, steps=5, cid=62), check_state_every=5)
+
+
+def test_expired_device_wait_reports_timeout_and_context_survives():
+    """Failure detection without a fault: a wait that nothing satisfies runs out after its limit, the
+    kernel writes VATP_ERR_TIMEOUT to the status word and returns; the next launch works as usual."""
+    V = P.vatp()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    waited = torch.zeros(1, dtype=torch.int64, device="cuda")
+    V.vatp_selftest_bounded_wait(2_000_000, status, waited)          # 2 ms
+    torch.cuda.synchronize()
+    assert int(status.item()) == 5
+    assert 2_000_000 <= int(waited.item()) < 50_000_000
+    with pytest.raises(V.VatpError):
+        V.vatp_selftest_bounded_wait(10**9, status)                   # limits above 0.1 s are refused on the host
+    _run_case(_small("bf16", 128, 300, 100, 2, 10, steps=3, cid=63))  # the context is intact
