@@ -669,7 +669,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
       }
     }
-  } else if (PASS == 1) {
+  } else if (PASS == 1 && a.ft == 0) {
     // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
     // Independent of the attention work of this pass: the CTAs share out all (unit, token tile) pairs,
     // so these warps cover every token.  Pass 2 reads the norms back in its epilogue.
@@ -731,6 +731,35 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   if (wid == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
+// Value l1 norms as a kernel of their own (Eq. 4): used with a history window, where pass 1 covers only
+// the window's query tiles and is too short to hide one warp per SM walking all of V.  Sixteen lanes
+// per row, eight rows in flight per lane.
+__global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a) {
+  const int u = blockIdx.x;
+  const int b = u / a.heads, h = u - b * a.heads;
+  const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
+  const int sub = threadIdx.x >> 4, part = threadIdx.x & 15;       // 16 rows per pass of the CTA
+  const int row0 = blockIdx.y * 128 + sub;
+  uint4 raw[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int tok = row0 + 16 * j;
+    raw[j] = make_uint4(0u, 0u, 0u, 0u);
+    if (tok < a.T) raw[j] = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
+#pragma unroll
+    for (int o = 8; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    const int tok = row0 + 16 * j;
+    if (part == 0 && tok < a.T) a.vnorm[(int64_t)u * a.T + tok] = acc;
   }
 }
 
@@ -834,6 +863,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
   if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
+  if (a.ft > 0) vnorm_kernel<<<dim3(a.units, (s.T + 127) / 128), 256, 0, st>>>(a);
   prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
