@@ -244,3 +244,51 @@ def test_expired_device_wait_reports_timeout_and_context_survives():
     with pytest.raises(V.VatpError):
         V.vatp_selftest_bounded_wait(10**9, status)                   # limits above 0.1 s are refused on the host
     _run_case(_small("bf16", 128, 300, 100, 2, 10, steps=3, cid=63))  # the context is intact
+
+
+def test_config1_layers_interleaved_in_a_graph_match_stepping_alone():
+    """The launch configuration the benchmark times: several independently seeded config-1 layers, their
+    decode steps interleaved and replayed from a CUDA graph (consecutive launches overlap on the GPU).
+    Outputs, evictions and final state must equal, bit for bit, each layer stepped alone with a
+    synchronisation after every step."""
+    V = P.vatp()
+    wl = synth.CONFIGS[1].with_(decode_steps=12)
+    L, steps = 3, wl.decode_steps
+
+    def prefilled():
+        gs = []
+        for layer in range(L):
+            q, k, v = synth.prefill_inputs(wl, layer, "cuda")
+            gs.append(P.GpuPrefill(wl, q, k, v).run())
+        return gs
+
+    ins = [synth.decode_inputs(wl, layer, device="cuda") for layer in range(L)]
+    shape = (steps, wl.batch, wl.heads, wl.head_dim)
+    alone = prefilled()
+    outs_a = [torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
+    evs_a = [torch.empty(shape[:3], dtype=torch.int32, device="cuda") for _ in range(L)]
+    for g, (dq, dk, dv), o, e in zip(alone, ins, outs_a, evs_a):
+        for s in range(steps):
+            V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
+            torch.cuda.synchronize()
+    inter = prefilled()
+    outs_b = [torch.empty_like(o) for o in outs_a]
+    evs_b = [torch.empty_like(e) for e in evs_a]
+
+    def all_steps(first, last):
+        for s in range(first, last):
+            for g, (dq, dk, dv), o, e in zip(inter, ins, outs_b, evs_b):
+                V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
+
+    all_steps(0, 2)                     # first calls outside the capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        all_steps(2, steps)
+    graph.replay()
+    torch.cuda.synchronize()
+    for ga, gb, oa, ob, ea, eb in zip(alone, inter, outs_a, outs_b, evs_a, evs_b):
+        assert int(gb.status.item()) == 0
+        assert torch.equal(oa, ob) and torch.equal(ea, eb)
+        for name in ("k_cache", "v_cache", "acc", "vnorm", "pos", "len", "free_slot", "next_pos"):
+            assert torch.equal(getattr(ga.cache, name), getattr(gb.cache, name)), name
