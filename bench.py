@@ -381,7 +381,7 @@ def run_cuda(args, wl):
         v = wl.batch * T / (a / cu * units)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
                                 "sample": f"{cu} of {units} heads of one layer (full prompt {T}, {cs} decode steps), "
-                                          f"{a + b:.1f} s of CPU work, per-layer figure extrapolated x{units // cu}",
+                                          f"{a + b:.1f} s of CPU work, per-layer figure extrapolated x{units / cu:.2f}",
                                 "decode_us_per_layer_step": b / (cu * cs) * units * 1e6}
     print(json.dumps(line), flush=True)
     if world > 1:
