@@ -293,3 +293,29 @@ def test_config1_layers_interleaved_in_a_graph_match_stepping_alone():
         assert torch.equal(oa, ob) and torch.equal(ea, eb)
         for name in ("k_cache", "v_cache", "acc", "vnorm", "pos", "len", "free_slot", "next_pos"):
             assert torch.equal(getattr(ga.cache, name), getattr(gb.cache, name)), name
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
+def test_optional_outputs_may_be_null(dtype, d):
+    """lse_out and evicted_pos are nullable: leaving them out changes nothing else."""
+    V = P.vatp()
+    wl = _small(dtype, d, 400, 150, 2, 12, b=1, h=3, steps=4, cid=64)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    full = P.GpuPrefill(wl, q, k, v).run()
+    bare = P.GpuPrefill(wl, q, k, v)
+    V.vatp_prefill_scores(bare.p, q, k, v, attn_acc=bare.attn_acc, vnorm=bare.vnorm, score=bare.score,
+                          workspace=bare.ws, dev_status=bare.status)                      # no lse_out
+    V.vatp_select(bare.p, bare.score, bare.kept)
+    V.vatp_compact(bare.p, k, v, bare.attn_acc, bare.vnorm, bare.kept, bare.cache)
+    torch.cuda.synchronize()
+    assert torch.equal(full.score, bare.score) and torch.equal(full.kept, bare.kept)
+    dq, dk, dv = synth.decode_inputs(wl, 0, device="cuda")
+    o1 = torch.empty(1, 3, d, dtype=q.dtype, device="cuda")
+    o2 = torch.empty_like(o1)
+    ev = torch.empty(1, 3, dtype=torch.int32, device="cuda")
+    for s in range(wl.decode_steps):
+        V.vatp_decode_step(full.p, full.cache, dq[s], dk[s], dv[s], o1, evicted_pos=ev, dev_status=full.status)
+        V.vatp_decode_step(bare.p, bare.cache, dq[s], dk[s], dv[s], o2)                     # no evicted_pos, no status word
+        torch.cuda.synchronize()
+        assert torch.equal(o1, o2)
+    assert torch.equal(full.cache.pos, bare.cache.pos) and torch.equal(full.cache.acc, bare.cache.acc)
