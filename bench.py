@@ -252,9 +252,11 @@ def run_cuda(args, wl):
 
     E = lambda: torch.cuda.Event(enable_timing=True)
 
-    def one_step(timed):
+    def one_step(per_kernel_events):
+        """One step.  The timed steps record three events only: an event between two kernels would break
+        the programmatic dependency that lets a launch set up while its predecessor drains."""
         flush.fill_(rank + 1)                       # evict L2 between iterations
-        ev = [[E() for _ in range(4)] for _ in range(L)]
+        ev = [[E() for _ in range(4)] for _ in range(L)] if per_kernel_events else None
         e0, e1, e2 = E(), E(), E()
         e0.record()
         prefill_all(ev)
@@ -268,17 +270,20 @@ def run_cuda(args, wl):
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    recs = [one_step(True) for _ in range(args.steps)]
+    recs = [one_step(False) for _ in range(args.steps)]
     barrier()
     clocks = sampler.stop()
+    # per-kernel breakdown of the prefill side: a few extra steps with an event after every call
+    brk = [one_step(True) for _ in range(max(2, min(args.steps, 5)))]
+    barrier()
     assert int(status.item()) == 0, "device status word set"
 
     t_pre = [a.elapsed_time(b) for a, b, _, _ in recs]               # ms, all layers
     t_dec = [b.elapsed_time(c) for _, b, c, _ in recs]
     t_all = [a.elapsed_time(c) for a, _, c, _ in recs]
-    t_score = [sum(e[0].elapsed_time(e[1]) for e in r[3]) / L for r in recs]    # ms per layer
-    t_select = [sum(e[1].elapsed_time(e[2]) for e in r[3]) / L for r in recs]
-    t_compact = [sum(e[2].elapsed_time(e[3]) for e in r[3]) / L for r in recs]
+    t_score = [sum(e[0].elapsed_time(e[1]) for e in r[3]) / L for r in brk]     # ms per layer
+    t_select = [sum(e[1].elapsed_time(e[2]) for e in r[3]) / L for r in brk]
+    t_compact = [sum(e[2].elapsed_time(e[3]) for e in r[3]) / L for r in brk]
     pre_ms, dec_ms, all_ms = (x / args.steps for x in max_over_ranks([sum(t_pre), sum(t_dec), sum(t_all)], dev, world))
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region

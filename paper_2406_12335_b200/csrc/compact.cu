@@ -16,6 +16,8 @@ __global__ void __launch_bounds__(CP_THREADS, 4)
 compact_kernel(Shape sh, int elem_bytes, int B, int cap, const char* __restrict__ k, const char* __restrict__ v,
                const float* __restrict__ attn_acc, const float* __restrict__ vnorm, const int32_t* __restrict__ kept,
                vatp_cache c) {
+  // launched as a programmatic dependent of the selection: nothing is read before that has completed
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int u = blockIdx.x;
   const int len = min(sh.T, B);
   const int row_bytes = sh.d * elem_bytes;
@@ -109,8 +111,9 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
   int gy = 4 * sms / s.units;        // four CTAs fit on an SM
   gy = gy < 1 ? 1 : (gy > groups ? groups : gy);
   const dim3 grid(s.units, gy);
-  compact_kernel<<<grid, CP_THREADS, 0, st>>>(s, eb, B, cap, (const char*)k, (const char*)v, attn_acc, vnorm, kept, c);
-  cudaError_t e = cudaGetLastError();
+  DependentLaunch dl(grid, dim3(CP_THREADS), 0, st);
+  cudaError_t e = cudaLaunchKernelEx(&dl.cfg, compact_kernel, s, eb, B, cap, (const char*)k, (const char*)v, attn_acc, vnorm,
+                                     kept, c);
   if (e != cudaSuccess) return e;
   if (s.window > 0) {
     ring_kernel<<<dim3((cap + 127) / 128, s.units), 128, 0, st>>>(s.units, s.T, s.window, B, cap, win_rows, kept, c);

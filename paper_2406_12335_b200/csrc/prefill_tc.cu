@@ -448,7 +448,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   // Pass 2 is launched as a programmatic dependent of pass 1: its CTAs start as pass-1 CTAs retire and
   // set up, fetch items and stream Q / K tiles at once; only what pass 1 writes (normalisers, value
   // norms) is read after griddepcontrol.wait, i.e. once pass 1 has completed.
-  if (PASS == 1 && tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  // (Pass 2 in turn releases whatever follows it; vatp_select, launched the same way, reads the scores
+  // only after its own griddepcontrol.wait.)
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (wid == 0) {
     // ------------------------------------------------------------------ TMA producer

@@ -25,6 +25,10 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
   __shared__ uint32_t sh_prefix, sh_need;
   __shared__ uint32_t warp_keep[SEL_WARPS], warp_eq[SEL_WARPS];
 
+  // Launched as a programmatic dependent: the next launch (the compaction) may set up now, and the
+  // scores are read only once the launch that produced them has completed.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int u = blockIdx.x;
   const float* sc = score + (int64_t)u * T;
   int32_t* out = kept + (int64_t)u * B;
@@ -148,11 +152,11 @@ cudaError_t launch_select(int units, int T, int B, int F, int R, const float* sc
   if (bytes <= 200 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
     if (e != cudaSuccess) return e;
-    select_kernel<true><<<units, SEL_THREADS, bytes, st>>>(T, B, F, R, score, kept);
-  } else {
-    select_kernel<false><<<units, SEL_THREADS, 0, st>>>(T, B, F, R, score, kept);
+    DependentLaunch dl(dim3(units), dim3(SEL_THREADS), bytes, st);
+    return cudaLaunchKernelEx(&dl.cfg, select_kernel<true>, T, B, F, R, score, kept);
   }
-  return cudaGetLastError();
+  DependentLaunch dl(dim3(units), dim3(SEL_THREADS), 0, st);
+  return cudaLaunchKernelEx(&dl.cfg, select_kernel<false>, T, B, F, R, score, kept);
 }
 
 }  // namespace vatp

@@ -37,6 +37,24 @@ bool vatp_tc_available();
 // swizzle, rows beyond the end read as zeros.  False when the driver entry point is missing.
 bool make_rows_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint32_t box_rows);
 
+// Launch configuration of a kernel that may be scheduled before the previous launch in the stream has
+// drained (programmatic dependent launch).  Such a kernel executes griddepcontrol.wait before it reads
+// anything an earlier launch wrote.
+struct DependentLaunch {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  DependentLaunch(dim3 grid, dim3 block, size_t smem, cudaStream_t st) : cfg{} {
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+  }
+};
+
 // ---- launchers (each returns cudaGetLastError()) ----
 cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const void* k, const void* v, float* lse,
                                 float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st);
