@@ -187,6 +187,17 @@ vatp_status vatp_decode_step(const vatp_params* params, const vatp_cache* cache,
  */
 vatp_status vatp_selftest_bounded_wait(uint64_t limit_ns, int32_t* dev_status, uint64_t* waited_ns, void* cuda_stream);
 
+/*
+ * Host-only probe of the rule that lets consecutive vatp_decode_step launches overlap on the GPU (no
+ * device work, usable without a GPU).  Pretends that a launch on `stream` reads and writes the n
+ * (<= 13) host-described byte ranges [begin[i], begin[i] + bytes[i]) and keeps `share` of the
+ * machine's CTA slots until the launch before it has completed.  Returns 1 when that launch would
+ * run without waiting for its predecessors - it overlaps none of the recorded launches that can
+ * still be resident - else 0, and records it; -1 on bad arguments.  `stream` is only a key (use
+ * values no real stream has).  The paper has no counterpart.
+ */
+int32_t vatp_selftest_overlap_policy(void* stream, const uint64_t* begin, const uint64_t* bytes, int32_t n, double share);
+
 const char* vatp_status_string(vatp_status status);
 
 #ifdef __cplusplus

@@ -587,6 +587,15 @@ bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, con
 
 }  // namespace
 
+// Host-only probe of the overlap policy (no device work): feeds one pretend launch that touches and
+// writes the `n` byte ranges [begin[i], begin[i] + bytes[i]) on `stream` and occupies `share` of the
+// machine; returns whether it would have been allowed to run beside the launches before it.
+bool decode_overlap_policy_probe(void* stream, const uint64_t* begin, const uint64_t* bytes, int n, double share) {
+  Range r[NRANGE] = {};
+  for (int i = 0; i < n && i < NRANGE; ++i) r[i] = Range{reinterpret_cast<const char*>(begin[i]), (size_t)bytes[i]};
+  return independent_of_in_flight(static_cast<cudaStream_t>(stream), r, NRANGE, r, share);
+}
+
 // Returns cudaErrorNotSupported when the shape does not fit this kernel's shared memory (the caller
 // then takes the general kernel).
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,

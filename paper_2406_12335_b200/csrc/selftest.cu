@@ -38,6 +38,12 @@ __global__ void bounded_wait_kernel(unsigned long long limit_ns, int32_t* dev_st
 
 }  // namespace
 
+extern "C" int32_t vatp_selftest_overlap_policy(void* stream, const uint64_t* begin, const uint64_t* bytes, int32_t n,
+                                                double share) {
+  if (!begin || !bytes || n <= 0) return -1;
+  return vatp::decode_overlap_policy_probe(stream, begin, bytes, n, share) ? 1 : 0;
+}
+
 extern "C" vatp_status vatp_selftest_bounded_wait(uint64_t limit_ns, int32_t* dev_status, uint64_t* waited_ns,
                                                   void* cuda_stream) {
   if (!dev_status) return VATP_ERR_INVALID_ARG;

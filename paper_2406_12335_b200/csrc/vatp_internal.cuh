@@ -73,6 +73,8 @@ cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const 
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
                               const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st);
 
+bool decode_overlap_policy_probe(void* stream, const uint64_t* begin, const uint64_t* bytes, int n, double share);
+
 // fixed-point image of a probability for the exact window sums (Eq. 3): p in [0, 1] -> p * 2^52
 __host__ __device__ inline long long prob_to_fixed(float p) { return (long long)((double)p * 4503599627370496.0); }
 __host__ __device__ inline float fixed_to_prob(long long x) { return (float)((double)x * (1.0 / 4503599627370496.0)); }

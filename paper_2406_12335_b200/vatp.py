@@ -20,7 +20,7 @@ BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
 STATIC_SCRATCH_BYTES = (4 << 20) + 256
 EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
-           "vatp_selftest_bounded_wait", "vatp_status_string"]
+           "vatp_selftest_bounded_wait", "vatp_selftest_overlap_policy", "vatp_status_string"]
 
 
 class Params(C.Structure):
@@ -53,6 +53,8 @@ lib.vatp_decode_step.restype = C.c_int
 lib.vatp_decode_step.argtypes = [C.POINTER(Params), C.POINTER(CacheStruct), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.vatp_selftest_bounded_wait.restype = C.c_int
 lib.vatp_selftest_bounded_wait.argtypes = [C.c_uint64, _vp, _vp, _vp]
+lib.vatp_selftest_overlap_policy.restype = C.c_int32
+lib.vatp_selftest_overlap_policy.argtypes = [_vp, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64), C.c_int32, C.c_double]
 lib.vatp_status_string.restype = C.c_char_p
 lib.vatp_status_string.argtypes = [C.c_int]
 

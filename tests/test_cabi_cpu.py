@@ -64,3 +64,42 @@ def test_host_side_validation(V):
     assert V.lib.vatp_prefill_scores(C.byref(sp), 16, 16, 16, 16, 16, 16, 16, null, null, 0, null, null) == 1
     # decode: null cache
     assert V.lib.vatp_decode_step(C.byref(p), null, 16, 16, 16, 16, null, null, null) == 1
+
+
+def _probe(V, stream, caches, share):
+    """One pretend decode launch touching the given (begin, bytes) ranges."""
+    n = len(caches)
+    begin = (C.c_uint64 * n)(*[c[0] for c in caches])
+    size = (C.c_uint64 * n)(*[c[1] for c in caches])
+    return V.lib.vatp_selftest_overlap_policy(C.c_void_p(stream), begin, size, n, share)
+
+
+def test_decode_overlap_policy(V):
+    """Host logic that decides whether a decode launch may run beside its predecessors: it must share no
+    buffer with any recorded launch that can still be resident (every launch stays resident until the one
+    before it has completed, so the shares of the launches in between bound how far back to look)."""
+    MB = 1 << 20
+    cache = lambda i: [(0x10_0000_0000 + i * 64 * MB, 32 * MB), (0x90_0000_0000 + i * MB, 4096)]
+    # four caches in rotation, each launch holding 43% of the machine: the same cache comes back after
+    # three others, whose shares add up to more than the machine -> its previous step has retired
+    s = 0xA001
+    assert _probe(V, s, cache(0), 0.43) == 0            # nothing known about what ran before the first launch
+    assert [_probe(V, s, cache(i), 0.43) for i in (1, 2, 3)] == [1, 1, 1]
+    assert [_probe(V, s, cache(i % 4), 0.43) for i in range(4, 12)] == [1] * 8
+    # three caches in rotation: only two launches (86%) lie between a cache's steps -> it must wait
+    s = 0xA002
+    assert _probe(V, s, cache(0), 0.43) == 0
+    assert [_probe(V, s, cache(i % 3), 0.43) for i in range(1, 9)] == [1, 1, 0, 0, 0, 0, 0, 0]
+    # the same cache twice in a row always waits; a partial overlap of one buffer is enough
+    s = 0xA003
+    _probe(V, s, cache(0), 0.9)
+    assert _probe(V, s, cache(0), 0.9) == 0
+    assert _probe(V, s, [(0x10_0000_0000 + 31 * MB, 2 * MB)], 0.9) == 0
+    assert _probe(V, s, cache(5), 0.9) == 1
+    # tiny launches: more than the recorded history could still be resident -> never assume independence
+    s = 0xA004
+    got = [_probe(V, s, cache(i), 0.01) for i in range(12)]
+    assert got[0] == 0 and got[1:8] == [1] * 7 and got[8:] == [0] * 4
+    # streams do not see each other's launches
+    assert _probe(V, 0xA005, cache(0), 0.43) == 0 and _probe(V, 0xA005, cache(1), 0.43) == 1
+    assert _probe(V, 0xA005, [], 0.5) == -1
