@@ -553,7 +553,8 @@ inline bool overlaps(const Range& a, const Range& b) {
 }
 
 // true when `touched` overlaps nothing that a launch possibly still in flight on `st` writes; records this launch
-bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, const Range* written, double share) {
+bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, const Range* written, double share_if_indep,
+                               double share_if_not) {
   std::lock_guard<std::mutex> lock(g_hist_mutex);
   StreamHistory* h = nullptr;
   for (auto& x : g_hist)
@@ -581,7 +582,7 @@ bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, con
   if (h->count < HIST) ++h->count;
   LaunchRecord& r = h->rec[h->head];
   for (int k = 0; k < NRANGE; ++k) r.w[k] = written[k];
-  r.share = share;
+  r.share = indep ? share_if_indep : share_if_not;
   return indep;
 }
 
@@ -593,7 +594,7 @@ bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, con
 bool decode_overlap_policy_probe(void* stream, const uint64_t* begin, const uint64_t* bytes, int n, double share) {
   Range r[NRANGE] = {};
   for (int i = 0; i < n && i < NRANGE; ++i) r[i] = Range{reinterpret_cast<const char*>(begin[i]), (size_t)bytes[i]};
-  return independent_of_in_flight(static_cast<cudaStream_t>(stream), r, NRANGE, r, share);
+  return independent_of_in_flight(static_cast<cudaStream_t>(stream), r, NRANGE, r, share, share);
 }
 
 // Returns cudaErrorNotSupported when the shape does not fit this kernel's shared memory (the caller
@@ -613,26 +614,41 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
   int chunk = (cap + split - 1) / split;
   chunk = (chunk + GROUP - 1) / GROUP * GROUP;
-  // Two CTAs per SM (so that consecutive launches can both be resident) when at least two stages per
-  // warp fit in half an SM's shared memory beside the per-slot state; large caches leave acc / vnorm /
-  // pos in global memory (L2-prefetched) to get there; otherwise one CTA with up to four stages.
+  // Shared-memory plan.  A launch that may run beside its neighbours stays within half an SM (two CTAs
+  // per SM, so that consecutive launches can both be resident) when at least two stages per warp fit
+  // there beside the per-slot state; large caches leave acc / vnorm / pos out of shared memory to get
+  // there.  A launch that has to wait for its predecessor anyway runs alone: it takes the whole SM and
+  // up to four stages per warp, which doubles the bytes it keeps in flight.
+  struct Plan {
+    int state_in_smem, nstage;
+    size_t dyn;
+    bool ok;
+  };
   const size_t half_sm = 104 * 1024, whole_sm = 215 * 1024;     // dynamic bytes, 1 KB of it alignment slack
   const size_t stage_set = (size_t)MW * STAGE_BYTES;
   const size_t tot = (size_t)chunk * split;
-  size_t state_bytes = 4 * sizeof(float) * tot;
-  int state_in_smem = 1;
-  if (state_bytes + 1024 + 2 * stage_set > half_sm && sizeof(float) * tot + 1024 + 2 * stage_set <= half_sm) {
-    state_bytes = sizeof(float) * tot;
-    state_in_smem = (size_t)cap * 12 <= 2 * stage_set ? 2 : 0;
-  }
-  if (state_bytes + stage_set + 1024 > whole_sm) return cudaErrorNotSupported;
-  int nstage = state_bytes + 1024 + 2 * stage_set <= half_sm ? (int)((half_sm - 1024 - state_bytes) / stage_set)
-                                                             : (int)((whole_sm - 1024 - state_bytes) / stage_set);
-  nstage = nstage > 4 ? 4 : nstage;
-  const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
-  if (nstage > groups_per_warp) nstage = groups_per_warp > 0 ? groups_per_warp : 1;
-  if (state_in_smem == 2 && (size_t)cap * 12 > (size_t)MW * nstage * STAGE_BYTES) state_in_smem = 0;
-  const size_t dyn = (size_t)MW * nstage * STAGE_BYTES + state_bytes + 1024;
+  auto make_plan = [&](bool alone) {
+    Plan p{};
+    size_t state_bytes = 4 * sizeof(float) * tot;
+    p.state_in_smem = 1;
+    const bool fits_half = !alone && state_bytes + 1024 + 2 * stage_set <= half_sm;
+    if (!alone && !fits_half && sizeof(float) * tot + 1024 + 2 * stage_set <= half_sm) {
+      state_bytes = sizeof(float) * tot;
+      p.state_in_smem = (size_t)cap * 12 <= 2 * stage_set ? 2 : 0;
+    }
+    p.ok = state_bytes + stage_set + 1024 <= whole_sm;
+    if (!p.ok) return p;
+    const bool half = !alone && state_bytes + 1024 + 2 * stage_set <= half_sm;
+    p.nstage = (int)(((half ? half_sm : whole_sm) - 1024 - state_bytes) / stage_set);
+    p.nstage = p.nstage > 4 ? 4 : p.nstage;
+    const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
+    if (p.nstage > groups_per_warp) p.nstage = groups_per_warp > 0 ? groups_per_warp : 1;
+    if (p.state_in_smem == 2 && (size_t)cap * 12 > (size_t)MW * p.nstage * STAGE_BYTES) p.state_in_smem = 0;
+    p.dyn = (size_t)MW * p.nstage * STAGE_BYTES + state_bytes + 1024;
+    return p;
+  };
+  const Plan beside = make_plan(false), lone = make_plan(true);
+  if (!beside.ok || !lone.ok) return cudaErrorNotSupported;
   CUtensorMap tm_k, tm_v;
   if (!make_rows_map_bf16(&tm_k, c.k_cache, (uint64_t)s.units * cap, GROUP) ||
       !make_rows_map_bf16(&tm_v, c.v_cache, (uint64_t)s.units * cap, GROUP))
@@ -651,10 +667,15 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
   if (e != cudaSuccess) return e;
   // share of the machine this launch holds while resident (every CTA waits for the previous launch before it retires)
-  int occ = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, MT, dyn) != cudaSuccess || occ < 1) occ = 1;
-  const double share = (double)(s.units * split) / ((double)occ * sms);
-  const int independent = independent_of_in_flight(st, written, 16, written, share) ? 1 : 0;
+  auto share_of = [&](const Plan& p) {
+    int occ = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, MT, p.dyn) != cudaSuccess || occ < 1) occ = 1;
+    return (double)(s.units * split) / ((double)occ * sms);
+  };
+  const int independent = independent_of_in_flight(st, written, 16, written, share_of(beside), share_of(lone)) ? 1 : 0;
+  const Plan& pl = independent ? beside : lone;
+  const int nstage = pl.nstage, state_in_smem = pl.state_in_smem;
+  const size_t dyn = pl.dyn;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(s.units * split);
   cfg.blockDim = dim3(MT);

@@ -161,16 +161,11 @@ def test_config4_long_context_layer():
     _run_case(synth.CONFIGS[4], units=[(0, 5)], check_state_every=32, layer=31)
 
 
-@pytest.mark.parametrize("b,h", [(1, 3), (5, 32)])
-def test_interleaved_caches_match_separate_runs(b, h):
-    """Decode steps of three independent caches issued back to back on one stream (launches that share
-    no buffer may overlap on the GPU) give bit for bit what each cache gives when stepped alone, and
-    the result agrees with the oracle.  With 3 units per cache every launch could still be in flight
-    when the same cache comes round again, so the steps wait for one another; with 160 units a launch
-    fills half the machine and the steps of different caches run side by side."""
+def _interleaved_equals_alone(wls, steps):
+    """Steps the caches of `wls` (a) one after the other, each alone with a synchronisation after every
+    step, and (b) round robin with no synchronisation; outputs, evictions and final state must be equal
+    bit for bit.  Returns a function that prefills fresh caches and the decode inputs."""
     V = P.vatp()
-    steps = 12
-    wls = [_small("bf16", 128, 900, 300, 2, 30, b=b, h=h, steps=steps, cid=70 + i) for i in range(3)]
 
     def prefilled():
         gs = []
@@ -180,15 +175,13 @@ def test_interleaved_caches_match_separate_runs(b, h):
         return gs
 
     ins = [synth.decode_inputs(wl, 0, device="cuda") for wl in wls]
-    # (a) each cache alone, synchronising after every step
     alone = prefilled()
-    outs_a = [torch.empty(steps, b, h, 128, dtype=torch.bfloat16, device="cuda") for _ in wls]
-    evs_a = [torch.empty(steps, b, h, dtype=torch.int32, device="cuda") for _ in wls]
+    outs_a = [torch.empty(steps, wl.batch, wl.heads, wl.head_dim, dtype=torch.bfloat16, device="cuda") for wl in wls]
+    evs_a = [torch.empty(steps, wl.batch, wl.heads, dtype=torch.int32, device="cuda") for wl in wls]
     for g, (dq, dk, dv), o, e in zip(alone, ins, outs_a, evs_a):
         for s in range(steps):
             V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
             torch.cuda.synchronize()
-    # (b) interleaved, no synchronisation in between
     inter = prefilled()
     outs_b = [torch.empty_like(o) for o in outs_a]
     evs_b = [torch.empty_like(e) for e in evs_a]
@@ -197,10 +190,23 @@ def test_interleaved_caches_match_separate_runs(b, h):
             V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
     torch.cuda.synchronize()
     for ga, gb, oa, ob, ea, eb in zip(alone, inter, outs_a, outs_b, evs_a, evs_b):
-        assert int(gb.status.item()) == 0
+        assert int(ga.status.item()) == 0 and int(gb.status.item()) == 0
         assert torch.equal(oa, ob) and torch.equal(ea, eb)
         for name in ("k_cache", "v_cache", "acc", "vnorm", "pos", "len", "free_slot", "next_pos"):
             assert torch.equal(getattr(ga.cache, name), getattr(gb.cache, name)), name
+    return prefilled, ins
+
+
+@pytest.mark.parametrize("b,h", [(1, 3), (5, 32)])
+def test_interleaved_caches_match_separate_runs(b, h):
+    """Decode steps of three independent caches issued back to back on one stream (launches that share
+    no buffer may overlap on the GPU) give bit for bit what each cache gives when stepped alone, and
+    the result agrees with the oracle.  With 3 units per cache every launch could still be in flight
+    when the same cache comes round again, so the steps wait for one another; with 160 units a launch
+    fills half the machine and the steps of different caches run side by side."""
+    steps = 12
+    wls = [_small("bf16", 128, 900, 300, 2, 30, b=b, h=h, steps=steps, cid=70 + i) for i in range(3)]
+    prefilled, ins = _interleaved_equals_alone(wls, steps)
     # (c) and the trajectory of some units of one cache against the oracle
     g = prefilled()[1]
     units = [(0, 0), (b - 1, h - 1), (b // 2, h // 2)]
@@ -226,10 +232,15 @@ def test_windowed_indicator_fp32_path():
 
 
 def test_decode_large_cache_state_paths():
-    """Caches too large for the per-slot state to sit beside the streaming stages: the state is copied
-    into the stage memory after the streaming (budget 3000) or read from global memory (budget 6000)."""
+    """Caches too large for the per-slot state to sit beside the streaming stages.  Stepped alone, a
+    launch waits for its predecessor and takes a whole SM, state included (checked against the
+    oracle).  Five such caches of 40 units stepped round robin run side by side, two CTAs per SM: there
+    the state is copied into the stage memory after the streaming (budget 3000) or read from global
+    memory (budget 6000), and the results must equal those of stepping alone."""
     for T, B in ((3400, 3000), (6500, 6000)):
         _run_case(_small("bf16", 128, T, B, 2, 64, b=1, h=2, steps=5, cid=62), check_state_every=5)
+        wls = [_small("bf16", 128, T, B, 2, 64, b=1, h=40, steps=4, cid=64 + i) for i in range(5)]
+        _interleaved_equals_alone(wls, 4)
 
 
 def test_expired_device_wait_reports_timeout_and_context_survives():
