@@ -32,6 +32,7 @@ __all__ = [
     "indicator_h2o",
     "indicator_window",
     "value_l1_norm",
+    "value_norm",
     "importance",
     "select_keep",
     "compact_rows",
@@ -99,6 +100,23 @@ def value_l1_norm(v) -> np.ndarray:
     return np.abs(_f64(v)).sum(axis=1)
 
 
+def value_norm(v, kind: str = "l1") -> np.ndarray:
+    """Norm of every value row over the head's d channels, for the three kinds
+    the Ablation Study compares (its table of norms): "l1" = sum of |v_c| (the
+    one Eq. 4 uses), "l2" = square root of the sum of v_c^2, "linf" = the
+    largest |v_c|."""
+    x = np.abs(_f64(v))
+    if x.ndim == 1:
+        x = x[None, :]
+    if kind == "l1":
+        return x.sum(axis=1)
+    if kind == "l2":
+        return np.sqrt((x * x).sum(axis=1))
+    if kind == "linf":
+        return x.max(axis=1)
+    raise ValueError("norm kind must be 'l1', 'l2' or 'linf'")
+
+
 def importance(S: np.ndarray, n1: np.ndarray) -> np.ndarray:
     """Eq. 4: I_k = S_k * ||v_k||_1."""
     return _f64(S) * _f64(n1)
@@ -133,9 +151,11 @@ def compact_rows(x: np.ndarray, kept: np.ndarray) -> np.ndarray:
     return np.ascontiguousarray(np.asarray(x)[np.asarray(kept, dtype=np.int64)])
 
 
-def prefill(q, k, v, scale: float, *, window: int | None = None, inclusive_extra: int = 0):
+def prefill(q, k, v, scale: float, *, window: int | None = None, inclusive_extra: int = 0, norm: str = "l1"):
     """One unit's prefill quantities: dict with a, lse, S, n1, I (and the
-    window rows a[T-w:, :] when the indicator is Eq. 3)."""
+    window rows a[T-w:, :] when the indicator is Eq. 3).  norm: which value
+    norm Eq. 4 multiplies by ("l1" is the method; "l2" / "linf" are the
+    ablation's variants); the key stays "n1" for all kinds."""
     a = attention_probs(q, k, scale)
     if window is None:
         S = indicator_h2o(a)
@@ -144,7 +164,7 @@ def prefill(q, k, v, scale: float, *, window: int | None = None, inclusive_extra
         S = indicator_window(a, window, inclusive_extra)
         first = max(a.shape[0] - (window + inclusive_extra), 0)
         rows = a[first:, :].copy()
-    n1 = value_l1_norm(v)
+    n1 = value_l1_norm(v) if norm == "l1" else value_norm(v, norm)
     return {
         "a": a,
         "lse": row_logsumexp(q, k, scale),
@@ -160,7 +180,8 @@ class DecodeState:
 
     pos[i]   original token position of cache entry i (ascending)
     K, V     rows of the cached keys / values (float64 copies of input bits)
-    n1       ||v||_1 per entry
+    n1       value norm per entry (||v||_1 unless norm says otherwise)
+    norm     kind of the value norm taken of tokens appended by decode steps
     S        H2O indicator per entry (Eq. 2), maintained incrementally
     hist     windowed mode only: the last <= w probability rows as a matrix
              [rows, entries] whose columns follow pos; Eq. 3 is re-summed from
@@ -171,8 +192,9 @@ class DecodeState:
     """
 
     def __init__(self, k, v, S, n1, kept, T: int, *, window: int | None = None,
-                 window_rows: np.ndarray | None = None, inclusive_extra: int = 0):
+                 window_rows: np.ndarray | None = None, inclusive_extra: int = 0, norm: str = "l1"):
         kept = np.asarray(kept, dtype=np.int64)
+        self.norm = norm
         self.pos = [int(p) for p in kept]
         self.K = [_f64(k)[p].copy() for p in kept]
         self.V = [_f64(v)[p].copy() for p in kept]
@@ -224,7 +246,7 @@ def decode_step(state: DecodeState, q, k, v, scale: float, B: int, F: int, R: in
     state.pos.append(t)
     state.K.append(_f64(k).copy())
     state.V.append(_f64(v).copy())
-    state.n1.append(float(np.abs(_f64(v)).sum()))
+    state.n1.append(float(value_norm(v, state.norm)[0]))
     state.S.append(0.0)
     if state.window is not None:
         state.hist = np.concatenate([state.hist, np.zeros((state.hist.shape[0], 1))], axis=1)

@@ -203,6 +203,57 @@ def test_l1_norm_closed_forms():
     assert O.value_l1_norm(np.array([[3.0, -4.0]]))[0] == 7.0
 
 
+def test_norm_kinds_closed_forms_and_orderings():
+    """The Ablation Study's three norms: closed forms on sign vectors and a 3-4-12 row, the textbook
+    chain linf <= l2 <= l1 <= sqrt(d) l2 <= d linf, brute force by loops, homogeneity, and the fact
+    that "l1" is the norm Eq. 4 uses."""
+    d = 128
+    rng = np.random.default_rng(5)
+    sign = rng.choice([-1.0, 1.0], size=(6, d))
+    np.testing.assert_array_equal(O.value_norm(sign, "l1"), np.full(6, float(d)))
+    np.testing.assert_allclose(O.value_norm(sign, "l2"), math.sqrt(d), rtol=1e-15)
+    np.testing.assert_array_equal(O.value_norm(sign, "linf"), np.ones(6))
+    row = np.array([[3.0, -4.0, 12.0]])
+    assert O.value_norm(row, "l1")[0] == 19.0 and O.value_norm(row, "l2")[0] == 13.0 and O.value_norm(row, "linf")[0] == 12.0
+    v = rng.normal(size=(50, d)) * np.exp(rng.normal(size=(50, 1)))
+    l1, l2, li = (O.value_norm(v, kd) for kd in ("l1", "l2", "linf"))
+    eps = 1e-12
+    assert np.all(li <= l2 * (1 + eps)) and np.all(l2 <= l1 * (1 + eps))
+    assert np.all(l1 <= math.sqrt(d) * l2 * (1 + eps)) and np.all(l2 <= math.sqrt(d) * li * (1 + eps))
+    for r in range(5):   # brute force
+        assert abs(math.fsum(abs(x) for x in v[r]) - l1[r]) <= 1e-12 * l1[r]
+        assert abs(math.sqrt(math.fsum(x * x for x in v[r])) - l2[r]) <= 1e-12 * l2[r]
+        assert max(abs(x) for x in v[r]) == li[r]
+    for kd in ("l1", "l2", "linf"):   # |c| comes out; a one-hot row has all three norms equal
+        np.testing.assert_allclose(O.value_norm(-2.5 * v, kd), 2.5 * O.value_norm(v, kd), rtol=1e-14)
+        onehot = np.zeros((1, d)); onehot[0, 17] = -0.75
+        assert O.value_norm(onehot, kd)[0] == 0.75
+    np.testing.assert_array_equal(O.value_norm(v, "l1"), O.value_l1_norm(v))
+    with pytest.raises(ValueError):
+        O.value_norm(v, "l3")
+
+
+def test_norm_kind_reaches_prefill_and_decode():
+    """prefill(norm=...) multiplies Eq. 4 by the chosen norm and decode steps take the same norm of
+    the tokens they append; a value row with one large channel ranks differently under l1 and linf."""
+    rng = np.random.default_rng(9)
+    T, d = 12, 8
+    q, k, v = rng.normal(size=(T, d)), rng.normal(size=(T, d)), rng.normal(size=(T, d))
+    for kd in ("l1", "l2", "linf"):
+        r = O.prefill(q, k, v, 0.3, norm=kd)
+        np.testing.assert_array_equal(r["n1"], O.value_norm(v, kd))
+        np.testing.assert_array_equal(r["I"], r["S"] * O.value_norm(v, kd))
+        st = O.DecodeState(k, v, r["S"], r["n1"], np.arange(T), T, norm=kd)
+        vn = rng.normal(size=d)
+        O.decode_step(st, rng.normal(size=d), rng.normal(size=d), vn, 0.3, B=T + 1, F=0, R=1)
+        assert st.n1[-1] == O.value_norm(vn, kd)[0]
+    spike = np.zeros(d); spike[0] = 3.0           # l1 3, linf 3
+    flat = np.full(d, 1.0)                        # l1 8, linf 1
+    both = np.stack([spike, flat])
+    assert O.value_norm(both, "l1")[0] < O.value_norm(both, "l1")[1]
+    assert O.value_norm(both, "linf")[0] > O.value_norm(both, "linf")[1]
+
+
 def test_importance_is_product():
     S = np.array([0.5, 2.0, 0.0])
     n = np.array([4.0, 0.25, 9.0])
