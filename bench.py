@@ -104,10 +104,10 @@ def oracle_sample(wl, units: int, decode_steps: int):
     t_pre = t_dec = 0.0
     for h in range(units):
         t0 = time.perf_counter()
-        r = O.prefill(q[0, h], k[0, h], v[0, h], wl.scale)
+        r = O.prefill(q[0, h], k[0, h], v[0, h], wl.scale, norm=wl.norm)
         kept = O.select_keep(r["I"], wl.budget, wl.n_sink, wl.n_recent)
         O.compact_rows(k[0, h], kept); O.compact_rows(v[0, h], kept)
-        st = O.DecodeState(k[0, h], v[0, h], r["S"], r["n1"], kept, wl.seq_len)
+        st = O.DecodeState(k[0, h], v[0, h], r["S"], r["n1"], kept, wl.seq_len, norm=wl.norm)
         t1 = time.perf_counter()
         for s in range(decode_steps):
             O.decode_step(st, dq[s, 0, h], dk[s, 0, h], dv[s, 0, h], wl.scale, wl.budget, wl.n_sink, wl.n_recent)
@@ -176,7 +176,7 @@ class LayerState:
         from paper_2406_12335_b200 import synth
         self.q, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
         self.p = V.params_for(self.q, budget=wl.budget, n_sink=wl.n_sink, n_recent=wl.n_recent, scale=wl.scale,
-                              indicator=wl.indicator, window=wl.window)
+                              indicator=wl.indicator, window=wl.window, norm=wl.norm)
         b, h, T = wl.batch, wl.heads, wl.seq_len
         f32 = dict(dtype=torch.float32, device=dev)
         self.attn_acc = torch.empty(b, h, T, **f32)
@@ -407,11 +407,15 @@ def main():
                     help="workload to time; 1 is the benchmark, the others are for the per-config roofline tables "
                          "(choose --layers so that the inputs fit: config 2 and 4 hold 1.6 GB per layer)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps (profiling runs)")
+    ap.add_argument("--norm", default="l1", choices=["l1", "l2", "linf"],
+                    help="value norm of Eq. 4: l1 is the method (and the benchmark), l2 / linf the Ablation Study's variants")
     args = ap.parse_args()
     from paper_2406_12335_b200 import synth
     wl = synth.CONFIGS[args.config]
     if args.decode_steps is not None:
         wl = wl.with_(decode_steps=args.decode_steps)
+    if args.norm != "l1":
+        wl = wl.with_(norm=args.norm, name=f"{wl.name} norm={args.norm}")
     if args.impl == "reference":
         run_reference(args, wl)
     else:

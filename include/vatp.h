@@ -47,6 +47,10 @@ typedef enum {
 
 typedef enum { VATP_BF16 = 0, VATP_F32 = 1 } vatp_dtype;
 typedef enum { VATP_IND_H2O = 0, VATP_IND_WINDOW = 1 } vatp_indicator;
+/* Which norm of the value row Eq. 4 multiplies the indicator by.  L1 is the method; L2 and LINF are
+ * the variants the Ablation Study compares it with (its table of norms).  The per-slot `vnorm`
+ * arrays hold whichever kind the parameters name. */
+typedef enum { VATP_NORM_L1 = 0, VATP_NORM_L2 = 1, VATP_NORM_LINF = 2 } vatp_norm_kind;
 
 /* Problem description shared by the four calls (host struct). */
 typedef struct {
@@ -60,6 +64,7 @@ typedef struct {
   int32_t budget;            /* B: tokens kept per unit                                        */
   int32_t n_sink;            /* F: leading tokens always kept                                  */
   int32_t n_recent;          /* R: most recent tokens always kept; F + R <= B                  */
+  int32_t norm_kind;         /* vatp_norm_kind of the value norm in Eq. 4; 0 = the paper's l1   */
   int64_t stride_b, stride_h, stride_t; /* element strides of q, k, v; 0 = contiguous          */
 } vatp_params;
 

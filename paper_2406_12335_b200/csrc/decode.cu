@@ -97,7 +97,7 @@ __device__ __forceinline__ bool evicts_before(float Ia, int pa, float Ib, int pb
 
 template <typename T, int D, bool WINDOWED>
 __global__ void __launch_bounds__(DEC_THREADS)
-decode_kernel(int split, int chunk, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
+decode_kernel(int split, int chunk, int B, int cap, int F, int R, int w, int norm, float scale_log2, vatp_cache c,
               const T* __restrict__ q_new, const T* __restrict__ k_new, const T* __restrict__ v_new,
               T* __restrict__ out, int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
   constexpr int EPV = Vec16<T>::N;       // elements per 16-byte vector
@@ -183,16 +183,17 @@ decode_kernel(int split, int chunk, int B, int cap, int F, int R, int w, float s
 #pragma unroll
   for (int i = 0; i < EPV; ++i) qx[i] *= scale_log2;
 
-  // ---- append: the CTA that owns the free slot stores the new row and its l1 norm ----
+  // ---- append: the CTA that owns the free slot stores the new row and its norm (Eq. 4) ----
   const bool owns_new = fs >= s0 && fs < s0 + cnt;
   float new_norm = 0.f;
   {
     float vx[EPV];
     Vec16<T>::unpack(vn_raw, vx);
 #pragma unroll
-    for (int i = 0; i < EPV; ++i) new_norm += fabsf(vx[i]);
+    for (int i = 0; i < EPV; ++i) new_norm = norm_fold(norm, new_norm, vx[i]);
 #pragma unroll
-    for (int o = LPR / 2; o; o >>= 1) new_norm += __shfl_xor_sync(0xffffffffu, new_norm, o);
+    for (int o = LPR / 2; o; o >>= 1) new_norm = norm_merge(norm, new_norm, __shfl_xor_sync(0xffffffffu, new_norm, o));
+    new_norm = norm_finish(norm, new_norm);
   }
   if (owns_new && wid == 0 && sub == 0) {
     *reinterpret_cast<uint4*>((T*)c.k_cache + ((int64_t)u * cap + fs) * D + col) = kn_raw;
@@ -435,7 +436,7 @@ cudaError_t launch_t(const Shape& s, int B, int F, int R, const vatp_cache& c, c
   attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, kern, split, chunk, B, cap, F, R, s.window, s.scale * LOG2E, c, (const T*)q,
+  return cudaLaunchKernelEx(&cfg, kern, split, chunk, B, cap, F, R, s.window, s.norm, s.scale * LOG2E, c, (const T*)q,
                             (const T*)k, (const T*)v, (T*)out, evicted, dev_status);
 }
 

@@ -143,7 +143,8 @@ __device__ __forceinline__ unsigned long long warp_min_key(unsigned long long ke
 template <bool WINDOWED>
 __global__ void __launch_bounds__(MT, 2)
 decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int independent,
-                  int state_in_smem, int split, int chunk, int nstage, int B, int cap, int F, int R, int w, float scale_log2, vatp_cache c,
+                  int state_in_smem, int split, int chunk, int nstage, int B, int cap, int F, int R, int w, int norm, float scale_log2,
+                  vatp_cache c,
                   const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
@@ -265,16 +266,16 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     last_raw = *(reinterpret_cast<const uint4*>((const __nv_bfloat16*)(lane < 16 ? c.k_cache : c.v_cache) +
                                                 ((int64_t)u * cap + ls) * HD) + (lane & 15));
 
-  // ---- append: the CTA that owns the free slot stores the new row and its l1 norm ----
+  // ---- append: the CTA that owns the free slot stores the new row and its norm (Eq. 4) ----
   float new_norm = 0.f;
   {
     const uint32_t wv[4] = {new_raw.x, new_raw.y, new_raw.z, new_raw.w};
 #pragma unroll
     for (int i = 0; i < 4; ++i)
-      new_norm += fabsf(__uint_as_float(wv[i] << 16)) + fabsf(__uint_as_float(wv[i] & 0xffff0000u));
+      new_norm = norm_fold(norm, norm_fold(norm, new_norm, __uint_as_float(wv[i] << 16)), __uint_as_float(wv[i] & 0xffff0000u));
 #pragma unroll
-    for (int o = 8; o; o >>= 1) new_norm += __shfl_xor_sync(0xffffffffu, new_norm, o);
-    new_norm = __shfl_sync(0xffffffffu, new_norm, 16);      // the V half's sum
+    for (int o = 8; o; o >>= 1) new_norm = norm_merge(norm, new_norm, __shfl_xor_sync(0xffffffffu, new_norm, o));
+    new_norm = norm_finish(norm, __shfl_sync(0xffffffffu, new_norm, 16));      // the V half's partial
   }
   if (owns_new && wid == 0) {
     __nv_bfloat16* dst = (__nv_bfloat16*)(lane < 16 ? c.k_cache : c.v_cache) + ((int64_t)u * cap + fs) * HD;
@@ -690,7 +691,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, state_in_smem, split, chunk, nstage, B, cap, F, R, s.window, s.scale * LOG2E, c,
+  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, state_in_smem, split, chunk, nstage, B, cap, F, R, s.window, s.norm, s.scale * LOG2E, c,
                             (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                             (__nv_bfloat16*)out, evicted, dev_status);
 }

@@ -178,7 +178,7 @@ colsum_kernel(Shape sh, const T* __restrict__ q, const T* __restrict__ k, const 
   __syncthreads();
 #pragma unroll
   for (int j = 0; j < 4; ++j) red[ty * TILE + tx + 16 * j] = cs[j];
-  // value l1 norms: 4 threads per row
+  // value norms (Eq. 4): 4 threads per row
   float* vn_s = Qs;  // reuse
   __syncthreads();
   {
@@ -186,11 +186,11 @@ colsum_kernel(Shape sh, const T* __restrict__ q, const T* __restrict__ k, const 
     float acc = 0.f;
     if (r < keys_valid) {
       const T* p = vu + (int64_t)(k0 + r) * sh.st;
-      for (int c = part; c < sh.d; c += 4) acc += fabsf(to_f32(p[c]));
+      for (int c = part; c < sh.d; c += 4) acc = norm_fold(sh.norm, acc, to_f32(p[c]));
     }
-    acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-    acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-    if (part == 0) vn_s[r] = acc;
+    acc = norm_merge(sh.norm, acc, __shfl_xor_sync(0xffffffffu, acc, 1));
+    acc = norm_merge(sh.norm, acc, __shfl_xor_sync(0xffffffffu, acc, 2));
+    if (part == 0) vn_s[r] = norm_finish(sh.norm, acc);
   }
   __syncthreads();
   if (threadIdx.x < keys_valid) {

@@ -6,7 +6,7 @@
 //   pass 2  rows = 128 keys (fixed tile), streamed tiles = queries diagonal..end: S^T = K Q^T is
 //           recomputed, every thread owns one key and adds exp2(s - lse_j) over the query columns
 //           of its TMEM lane (Eq. 2) - a per-thread running sum, no shuffles, no atomics - then
-//           multiplies by the value l1 norm (Eq. 4), which a side warp of pass 1 has reduced.
+//           multiplies by the value norm (Eq. 4: l1), which a side warp of pass 1 has reduced.
 // Both operands are [token, d] row-major, i.e. K-major for A and B alike.
 //
 // With a history window (Eq. 3) only the last w query rows count: pass 1 covers the query tiles that
@@ -356,6 +356,8 @@ struct TcArgs {
   // query wrow0 + r (wrow0 = T - w, negative when the prompt is shorter than the window).  H2O: all zero.
   int first_row, ft, wrow0, window;
   int gu;                   // units per scheduling group (their K and Q fit in L2 together)
+  int norm;                 // vatp_norm_kind of the value norm
+  int side_norm;            // pass 1 reduces the value norms in its side warp (else vnorm_kernel has, before it)
   unsigned* counters;       // [2] next work item of pass 1 / pass 2 (zeroed before pass 1 is launched)
   float* win_rows;
 };
@@ -396,6 +398,41 @@ __device__ __forceinline__ Item item_of(int id, const TcArgs& a) {
 template <int PASS>
 __device__ __forceinline__ bool tile_needed(const Item& it, int st, int nt) {
   return PASS == 1 ? st <= it.tile : (st >= it.lo && st < nt);
+}
+
+// Value norms of all (unit, token tile) pairs, shared out over the CTAs: the work of pass 1's side warp.
+template <int KIND>
+__device__ __forceinline__ void side_value_norms(const TcArgs& a, int lane) {
+  for (int id = blockIdx.x; id < a.units * a.nt; id += gridDim.x) {
+    Item it;
+    it.tile = id / a.units;
+    it.u = id - it.tile * a.units;
+    const int b = it.u / a.heads, h = it.u - b * a.heads;
+    const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
+    // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
+    const int sub = lane >> 4, part = lane & 15;
+    for (int r0 = 0; r0 < TILE; r0 += 32) {
+      uint4 raw[16];
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const int tok = it.tile * TILE + r0 + 2 * j + sub;
+        raw[j] = make_uint4(0u, 0u, 0u, 0u);
+        if (tok < a.T) raw[j] = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
+      }
+#pragma unroll
+      for (int j = 0; j < 16; ++j) {
+        const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
+        float acc = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          acc = norm_fold(KIND, norm_fold(KIND, acc, __uint_as_float(w[i] << 16)), __uint_as_float(w[i] & 0xffff0000u));
+#pragma unroll
+        for (int o = 8; o; o >>= 1) acc = norm_merge(KIND, acc, __shfl_xor_sync(0xffffffffu, acc, o));
+        const int tok = it.tile * TILE + r0 + 2 * j + sub;
+        if (part == 0 && tok < a.T) a.vnorm[(int64_t)it.u * a.T + tok] = norm_finish(KIND, acc);
+      }
+    }
+  }
 }
 
 template <int PASS, bool WIN>
@@ -671,40 +708,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
       }
     }
-  } else if (PASS == 1 && a.ft == 0) {
-    // ------------------------------------------------------------------ value l1 norms (Eq. 4), warp 10
+  } else if (PASS == 1 && a.side_norm) {
+    // ------------------------------------------------------------------ value norms (Eq. 4), the side warp
     // Independent of the attention work of this pass: the CTAs share out all (unit, token tile) pairs,
     // so these warps cover every token.  Pass 2 reads the norms back in its epilogue.
-    for (int id = blockIdx.x; id < a.units * a.nt; id += gridDim.x) {
-      Item it;
-      it.tile = id / a.units;
-      it.u = id - it.tile * a.units;
-      const int b = it.u / a.heads, h = it.u - b * a.heads;
-      const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
-      // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
-      const int sub = lane >> 4, part = lane & 15;
-      for (int r0 = 0; r0 < TILE; r0 += 32) {
-        uint4 raw[16];
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int tok = it.tile * TILE + r0 + 2 * j + sub;
-          raw[j] = make_uint4(0u, 0u, 0u, 0u);
-          if (tok < a.T) raw[j] = __ldg(reinterpret_cast<const uint4*>(vu + (int64_t)tok * a.st) + part);
-        }
-#pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
-          float acc = 0.f;
-#pragma unroll
-          for (int i = 0; i < 4; ++i)
-            acc += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
-#pragma unroll
-          for (int o = 8; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-          const int tok = it.tile * TILE + r0 + 2 * j + sub;
-          if (part == 0 && tok < a.T) a.vnorm[(int64_t)it.u * a.T + tok] = acc;
-        }
-      }
-    }
+    // Only Eq. 4's own l1 norm is taken here.  This warp shares a scheduler with four softmax warps and
+    // gets few issue slots: with the square and root of the l2 variant it became the last thing to
+    // finish in every CTA and the whole pass a fifth longer, so the ablation's variants go to the
+    // kernel below instead.
+    side_value_norms<VATP_NORM_L1>(a, lane);
   } else if (WIN) {
     // ------------------------------------------------------------------ pass 2, Eq. 3: window rows nobody visits
     // For key tile i the query tiles before it are never streamed (causal), and when the prompt is
@@ -736,9 +748,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   }
 }
 
-// Value l1 norms as a kernel of their own (Eq. 4): used with a history window, where pass 1 covers only
-// the window's query tiles and is too short to hide one warp per SM walking all of V.  Sixteen lanes
+// Value norms as a kernel of their own (Eq. 4): used with a history window, where pass 1 covers only
+// the window's query tiles and is too short to hide one warp per SM walking all of V, and for the
+// l2 / l-infinity variants.  Sixteen lanes
 // per row, eight rows in flight per lane.
+template <int KIND>
 __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a) {
   const int u = blockIdx.x;
   const int b = u / a.heads, h = u - b * a.heads;
@@ -757,11 +771,12 @@ __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a) {
     const uint32_t w[4] = {raw[j].x, raw[j].y, raw[j].z, raw[j].w};
     float acc = 0.f;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) acc += fabsf(__uint_as_float(w[i] << 16)) + fabsf(__uint_as_float(w[i] & 0xffff0000u));
+    for (int i = 0; i < 4; ++i)
+      acc = norm_fold(KIND, norm_fold(KIND, acc, __uint_as_float(w[i] << 16)), __uint_as_float(w[i] & 0xffff0000u));
 #pragma unroll
-    for (int o = 8; o; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    for (int o = 8; o; o >>= 1) acc = norm_merge(KIND, acc, __shfl_xor_sync(0xffffffffu, acc, o));
     const int tok = row0 + 16 * j;
-    if (part == 0 && tok < a.T) a.vnorm[(int64_t)u * a.T + tok] = acc;
+    if (part == 0 && tok < a.T) a.vnorm[(int64_t)u * a.T + tok] = norm_finish(KIND, acc);
   }
 }
 
@@ -838,6 +853,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.sb = s.sb; a.sh = s.sh; a.st = s.st;
   a.lse2 = lse_ws; a.lse_out = lse_out; a.attn_acc = attn_acc; a.vnorm = vnorm; a.score = score;
   a.dev_status = dev_status;
+  a.norm = s.norm;
   a.counters = reinterpret_cast<unsigned*>(reinterpret_cast<char*>(lse_ws) + ((size_t)a.units * a.Tpad * sizeof(float) + 255) / 256 * 256);
   const bool win = s.window > 0;
   a.window = win ? s.window : 0;
@@ -865,7 +881,13 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
   if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
-  if (a.ft > 0) vnorm_kernel<<<dim3(a.units, (s.T + 127) / 128), 256, 0, st>>>(a);
+  a.side_norm = a.ft == 0 && a.norm == VATP_NORM_L1;
+  if (!a.side_norm) {
+    const dim3 grid(a.units, (s.T + 127) / 128);
+    if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a);
+    else if (a.norm == VATP_NORM_L2) vnorm_kernel<VATP_NORM_L2><<<grid, 256, 0, st>>>(a);
+    else vnorm_kernel<VATP_NORM_LINF><<<grid, 256, 0, st>>>(a);
+  }
   prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};

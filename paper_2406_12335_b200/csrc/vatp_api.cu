@@ -17,6 +17,7 @@ vatp_status check_params(const vatp_params* p, bool need_T) {
   if (p->dtype != VATP_BF16 && p->dtype != VATP_F32) return VATP_ERR_UNSUPPORTED;
   if (p->indicator != VATP_IND_H2O && p->indicator != VATP_IND_WINDOW) return VATP_ERR_UNSUPPORTED;
   if (p->indicator == VATP_IND_WINDOW && p->window_w <= 0) return VATP_ERR_INVALID_ARG;
+  if (p->norm_kind != VATP_NORM_L1 && p->norm_kind != VATP_NORM_L2 && p->norm_kind != VATP_NORM_LINF) return VATP_ERR_UNSUPPORTED;
   if (p->budget <= 0 || p->n_sink < 0 || p->n_recent < 0) return VATP_ERR_INVALID_ARG;
   if ((int64_t)p->n_sink + p->n_recent > p->budget) return VATP_ERR_INVALID_ARG;
   if (!(p->scale > 0.f)) return VATP_ERR_INVALID_ARG;
@@ -34,6 +35,7 @@ vatp_status make_shape(const vatp_params* p, Shape* s) {
   s->sb = p->stride_b ? p->stride_b : (int64_t)p->heads * s->sh;
   s->scale = p->scale;
   s->window = p->indicator == VATP_IND_WINDOW ? p->window_w : 0;
+  s->norm = p->norm_kind;
   const int eb = p->dtype == VATP_F32 ? 4 : 2;
   if (s->st < s->d) return VATP_ERR_INVALID_ARG;
   if ((s->st * eb) % 16 || (s->sh * eb) % 16 || (s->sb * eb) % 16) return VATP_ERR_INVALID_ARG;
@@ -148,6 +150,7 @@ vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, cons
   sh.d = p->head_dim;
   sh.scale = p->scale;
   sh.window = windowed ? p->window_w : 0;
+  sh.norm = p->norm_kind;
   cudaError_t e = launch_decode(sh, p->dtype, p->budget, p->n_sink, p->n_recent, *cache, q_new, k_new, v_new, out,
                                 evicted_pos, dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;

@@ -16,7 +16,17 @@ struct Shape {
   int64_t sb, sh, st;  // element strides of q/k/v
   float scale;
   int window;          // 0 = accumulate over all queries (Eq. 2); >0 = last `window` queries (Eq. 3)
+  int norm;            // vatp_norm_kind of the value norm in Eq. 4
 };
+
+// Value-row norms (Eq. 4 uses l1; the Ablation Study's variants are l2 and l-infinity).  A row is
+// folded element by element into a partial, partials of different lanes are merged, and the merged
+// partial is finished: l1 sums |x|, l2 sums x^2 and takes the root, l-infinity takes the largest |x|.
+__device__ __forceinline__ float norm_fold(int kind, float part, float x) {
+  return kind == VATP_NORM_L1 ? part + fabsf(x) : kind == VATP_NORM_L2 ? fmaf(x, x, part) : fmaxf(part, fabsf(x));
+}
+__device__ __forceinline__ float norm_merge(int kind, float a, float b) { return kind == VATP_NORM_LINF ? fmaxf(a, b) : a + b; }
+__device__ __forceinline__ float norm_finish(int kind, float part) { return kind == VATP_NORM_L2 ? sqrtf(part) : part; }
 
 // slots per unit in the decode state: budget + 1, rounded up to a multiple of 8 so that every
 // per-slot array of a unit starts on a 32-byte boundary (bulk copies need 16)

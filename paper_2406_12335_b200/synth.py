@@ -48,6 +48,7 @@ class Workload:
     sigma_lo: float = 1.0
     sigma_hi: float = 1.0
     boost: int = 0
+    norm: str = "l1"      # value norm of Eq. 4: "l1" (the method) | "l2" | "linf" (the Ablation Study's variants)
 
     @property
     def scale(self) -> float:

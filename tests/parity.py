@@ -34,7 +34,7 @@ class GpuPrefill:
         b, h, T = wl.batch, wl.heads, wl.seq_len
         self.q, self.k, self.v = q, k, v
         self.p = V.params_for(q, budget=wl.budget, n_sink=self.F, n_recent=wl.n_recent, scale=wl.scale,
-                              indicator=wl.indicator, window=wl.window)
+                              indicator=wl.indicator, window=wl.window, norm=wl.norm)
         f32 = dict(dtype=torch.float32, device=dev)
         self.lse = torch.empty(b, h, T, **f32)
         self.attn_acc = torch.empty(b, h, T, **f32)
@@ -70,7 +70,7 @@ def check_prefill_unit(g: GpuPrefill, b: int, h: int, tol: float):
     T, B, F, R = wl.seq_len, wl.budget, g.F, wl.n_recent
     qn, kn, vn = (to_np64(x[b, h]) for x in (g.q, g.k, g.v))
     window = wl.window if wl.indicator == "window" else None
-    ref = O.prefill(qn, kn, vn, wl.scale, window=window)
+    ref = O.prefill(qn, kn, vn, wl.scale, window=window, norm=wl.norm)
 
     first = max(T - wl.window, 0) if window else 0
     lse = to_np64(g.lse[b, h])
@@ -150,7 +150,7 @@ def run_decode_and_check(g: GpuPrefill, ref_by_unit: dict, dq, dk, dv, steps: in
     states = {}
     for (b, h), (ref, kept) in ref_by_unit.items():
         states[(b, h)] = O.DecodeState(to_np64(g.k[b, h]), to_np64(g.v[b, h]), ref["S"], ref["n1"], kept, wl.seq_len,
-                                       window=window, window_rows=ref["window_rows"])
+                                       window=window, window_rows=ref["window_rows"], norm=wl.norm)
     out = torch.empty(wl.batch, wl.heads, wl.head_dim, dtype=g.q.dtype, device=dev)
     evicted = torch.empty(wl.batch, wl.heads, dtype=torch.int32, device=dev)
     adopted = 0

@@ -64,6 +64,15 @@ def test_host_side_validation(V):
     assert V.lib.vatp_prefill_scores(C.byref(sp), 16, 16, 16, 16, 16, 16, 16, null, null, 0, null, null) == 1
     # decode: null cache
     assert V.lib.vatp_decode_step(C.byref(p), null, 16, 16, 16, 16, null, null, null) == 1
+    # value norm kinds: l1 / l2 / linf are accepted, anything else is unsupported; the field fills what
+    # used to be padding before the 64-bit strides, so the struct keeps its size
+    assert C.sizeof(V.Params) == 72 and V.Params.norm_kind.offset == 44 and V.Params.stride_b.offset == 48
+    for kind in ("l1", "l2", "linf"):
+        assert V.vatp_workspace_bytes(V.make_params(**ok, norm=kind)) == 2048 + 256
+    odd = V.make_params(**ok)
+    odd.norm_kind = 3
+    assert V.vatp_workspace_bytes(odd) == 0
+    assert V.lib.vatp_select(C.byref(odd), 16, 16, null, 0, null, null) == 2
 
 
 def _probe(V, stream, caches, share):

@@ -231,6 +231,24 @@ def test_windowed_indicator_fp32_path():
     _run_case(_small("f32", 64, 300, 120, 2, 10, b=1, h=2, indicator="window", window=77, steps=6, cid=61))
 
 
+@pytest.mark.parametrize("norm", ["l2", "linf"])
+@pytest.mark.parametrize("dtype,d,T,B,indicator,window", [
+    ("bf16", 128, 700, 300, "h2o", 0),        # tensor-core prefill (side warp) + tensor-core decode
+    ("bf16", 128, 600, 250, "window", 200),   # windowed: the norm kernel of its own
+    ("f32", 64, 333, 100, "h2o", 0),          # general kernels
+])
+def test_value_norm_kinds(norm, dtype, d, T, B, indicator, window):
+    """The Ablation Study's l2 and l-infinity norms in place of Eq. 4's l1: prefill norms, scores,
+    kept sets, and the norms of tokens appended by decode steps (which decide later evictions)."""
+    wl = _small(dtype, d, T, B, 2, 10, b=1, h=3, indicator=indicator, window=window, steps=12, cid=66).with_(norm=norm)
+    g, _, _ = _run_case(wl)
+    v0 = g.v[0, 0].double()
+    ref = v0.pow(2).sum(-1).sqrt() if norm == "l2" else v0.abs().amax(-1)
+    assert torch.allclose(g.vnorm[0, 0].double(), ref, rtol=1e-5, atol=0)
+    l1 = v0.abs().sum(-1)
+    assert torch.all(g.vnorm[0, 0].double() < l1)     # a different norm really was taken
+
+
 def test_decode_large_cache_state_paths():
     """Caches too large for the per-slot state to sit beside the streaming stages.  Stepped alone, a
     launch waits for its predecessor and takes a whole SM, state included (checked against the
