@@ -35,6 +35,7 @@ __all__ = [
     "value_norm",
     "importance",
     "select_keep",
+    "appendix_a_split",
     "compact_rows",
     "prefill",
     "DecodeState",
@@ -144,6 +145,37 @@ def select_keep(I, B: int, F: int, R: int) -> np.ndarray:
     kept = np.concatenate([np.arange(0, F), top, np.arange(T - R, T)]).astype(np.int64)
     kept.sort()
     return kept
+
+
+def appendix_a_split(method: str, prompt_len: int, ratio: float = 0.5, model: str = "llama2-7b-chat",
+                     vatp: bool = True) -> dict:
+    """Hyper-parameters of Appendix A ("Implementation Details") for one prompt.
+
+    The KV budget k is a fraction of the prompt length (50% in the accuracy
+    tables; 100/50/25% in the throughput table of "Inference Efficiency"),
+    the same for every head and layer.  With H2O, k/2 tokens are chosen by
+    importance and k/2 form the local window.  With Scissorhands, k-10 tokens
+    are chosen by importance, the local window is 10 tokens and the history
+    window is w = 400 queries.  VATP additionally keeps the first F tokens,
+    F = 20 for LLaMA2-7B-chat and 40 for Vicuna-v1.5-7B-16k; the plain
+    baselines (vatp=False) keep none.
+    reading: k is rounded half up; for odd k the local window takes the
+    floor; the F kept tokens count inside the importance-chosen share, so
+    exactly k tokens survive; when the shares do not fit, the window is cut
+    first to k and F to what is left.
+    Returns B (= k), F, R, w (None for H2O) and n_scored = B - F - R.
+    """
+    k = int(np.floor(ratio * prompt_len + 0.5))
+    if method == "h2o":
+        R, w = k // 2, None
+    elif method == "scissorhands":
+        R, w = 10, 400
+    else:
+        raise ValueError("method must be 'h2o' or 'scissorhands'")
+    F = {"llama2-7b-chat": 20, "vicuna-v1.5-7b-16k": 40}[model] if vatp else 0
+    R = min(R, k)
+    F = min(F, k - R)
+    return {"B": k, "F": F, "R": R, "w": w, "n_scored": k - F - R}
 
 
 def compact_rows(x: np.ndarray, kept: np.ndarray) -> np.ndarray:

@@ -5,7 +5,7 @@ synthetic-workload module can be imported on machines without the library.
 """
 from importlib import import_module
 
-__all__ = ["synth", "vatp", "build"]
+__all__ = ["synth", "vatp", "build", "presets"]
 
 
 def __getattr__(name):

@@ -457,3 +457,52 @@ def test_forced_eviction_only_within_tolerance():
     res = O.decode_step(st, q[T], k[T], v[T], 0.5, B, F, R)
     with pytest.raises(ValueError):
         O.decode_step(st2, q[T], k[T], v[T], 0.5, B, F, R, force_evict=res["runner_up"], tie_tol=1e-12)
+
+
+# ------------------------------------------------------------------ Appendix A hyper-parameters
+def _appendix_a_rows():
+    rows = []
+    with open(os.path.join(GOLD, "appendix_a_presets.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            left, right = line.split("|")
+            method, model, vatp, T, ratio = left.split()
+            rows.append((method, model, bool(int(vatp)), int(T), float(ratio), [int(x) for x in right.split()]))
+    return rows
+
+
+def test_appendix_a_split_matches_the_papers_values():
+    """tests/golden/appendix_a_presets.txt holds what Appendix A states (k/2 + k/2 for H2O; k-10, 10 and
+    w = 400 for Scissorhands; F = 20 / 40), written out by hand for the budgets of the throughput table."""
+    rows = _appendix_a_rows()
+    assert len(rows) >= 9
+    for method, model, vatp, T, ratio, (k, F, R, w, chosen) in rows:
+        s = O.appendix_a_split(method, T, ratio, model, vatp=vatp)
+        assert (s["B"], s["F"], s["R"], s["w"] or 0) == (k, F, R, w), (method, model, ratio)
+        assert s["n_scored"] + s["F"] == chosen and s["n_scored"] + s["F"] + s["R"] == k
+
+
+def test_appendix_a_split_invariants_and_the_product_presets():
+    """Every split is a valid argument of select_keep (F + R <= B, kept count = B), tiny budgets
+    included; the product's own preset table (written separately) gives the same numbers."""
+    from paper_2406_12335_b200 import presets
+    rng = np.random.default_rng(5)
+    for method in ("h2o", "scissorhands"):
+        for model in ("llama2-7b-chat", "vicuna-v1.5-7b-16k"):
+            for T in (7, 33, 100, 1001, 4096, 18409):
+                for ratio in (0.1, 0.25, 0.5, 1.0):
+                    for vatp in (True, False):
+                        s = O.appendix_a_split(method, T, ratio, model, vatp=vatp)
+                        assert 0 <= s["F"] and 0 <= s["R"] and s["F"] + s["R"] <= s["B"] <= T
+                        assert s["n_scored"] == s["B"] - s["F"] - s["R"] >= 0
+                        kept = O.select_keep(rng.random(T), s["B"], s["F"], s["R"])
+                        assert len(kept) == s["B"]
+                        assert set(range(s["F"])) <= set(kept.tolist())
+                        assert set(range(T - s["R"], T)) <= set(kept.tolist()) or s["B"] >= T
+                        p = presets.appendix_a(method, T, ratio, model, sinks=vatp)
+                        assert (p["budget"], p["n_sink"], p["n_recent"], p["window"]) == \
+                            (s["B"], s["F"], s["R"], s["w"] or 0)
+                        assert p["indicator"] == ("window" if s["w"] else "h2o")
+    with pytest.raises(ValueError):
+        O.appendix_a_split("fastgen", 100)
