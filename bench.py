@@ -102,12 +102,14 @@ def oracle_sample(wl, units: int, decode_steps: int):
     q, k, v = (x.double().numpy() for x in synth.prefill_inputs(sub, 0, "cpu"))
     dq, dk, dv = (x.double().numpy() for x in synth.decode_inputs(sub, 0, decode_steps, "cpu"))
     t_pre = t_dec = 0.0
+    window = wl.window if wl.indicator == "window" else None      # Eq. 3 instead of Eq. 2
     for h in range(units):
         t0 = time.perf_counter()
-        r = O.prefill(q[0, h], k[0, h], v[0, h], wl.scale, norm=wl.norm)
+        r = O.prefill(q[0, h], k[0, h], v[0, h], wl.scale, window=window, norm=wl.norm)
         kept = O.select_keep(r["I"], wl.budget, wl.n_sink, wl.n_recent)
         O.compact_rows(k[0, h], kept); O.compact_rows(v[0, h], kept)
-        st = O.DecodeState(k[0, h], v[0, h], r["S"], r["n1"], kept, wl.seq_len, norm=wl.norm)
+        st = O.DecodeState(k[0, h], v[0, h], r["S"], r["n1"], kept, wl.seq_len, window=window,
+                           window_rows=r["window_rows"], norm=wl.norm)
         t1 = time.perf_counter()
         for s in range(decode_steps):
             O.decode_step(st, dq[s, 0, h], dk[s, 0, h], dv[s, 0, h], wl.scale, wl.budget, wl.n_sink, wl.n_recent)
@@ -403,9 +405,15 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--layers", type=int, default=LAYERS, help="independently seeded layers held on the device")
-    ap.add_argument("--config", type=int, default=1, choices=sorted([0, 1, 2, 3, 4]),
+    ap.add_argument("--config", type=int, default=1, choices=sorted([0, 1, 2, 3, 4, 5]),
                     help="workload to time; 1 is the benchmark, the others are for the per-config roofline tables "
-                         "(choose --layers so that the inputs fit: config 2 and 4 hold 1.6 GB per layer)")
+                         "(choose --layers so that the inputs fit: config 2 and 4 hold 1.6 GB per layer, config 5 "
+                         "6.3 GB); 5 is the shape of the paper's throughput table (batch 12, prompt 4096, 128 steps)")
+    ap.add_argument("--budget-ratio", type=float, default=None,
+                    help="KV budget as a fraction of the prompt (the throughput table's 1.0 / 0.5 / 0.25), split as "
+                         "Appendix A states for --method")
+    ap.add_argument("--method", default=None, choices=["h2o", "scissorhands"],
+                    help="host method whose Appendix A split --budget-ratio applies (default: the workload's indicator)")
     ap.add_argument("--decode-steps", type=int, default=None, help="override the workload's decode steps (profiling runs)")
     ap.add_argument("--norm", default="l1", choices=["l1", "l2", "linf"],
                     help="value norm of Eq. 4: l1 is the method (and the benchmark), l2 / linf the Ablation Study's variants")
@@ -414,6 +422,12 @@ def main():
     wl = synth.CONFIGS[args.config]
     if args.decode_steps is not None:
         wl = wl.with_(decode_steps=args.decode_steps)
+    if args.budget_ratio is not None:
+        from paper_2406_12335_b200 import presets
+        method = args.method or ("scissorhands" if wl.indicator == "window" else "h2o")
+        pr = presets.appendix_a(method, wl.seq_len, args.budget_ratio)
+        wl = wl.with_(budget=pr["budget"], n_sink=pr["n_sink"], n_recent=pr["n_recent"], indicator=pr["indicator"],
+                      window=pr["window"], name=f"{wl.name} {method} budget {args.budget_ratio:g}")
     if args.norm != "l1":
         wl = wl.with_(norm=args.norm, name=f"{wl.name} norm={args.norm}")
     if args.impl == "reference":

@@ -118,6 +118,27 @@ vatp_status vatp_prefill_scores(const vatp_params* params, const void* q, const 
                                 int32_t* dev_status, void* cuda_stream);
 
 /*
+ * Prefill scoring when the row normalisers of Eq. 1 already exist.  The Limitations section
+ * ("FlashAttention Support for H2O") names the cost this removes: a fused attention kernel does not
+ * return the attention matrix, so accumulated attention (Eq. 2) seemed to need the O(n^2) matrix.
+ * Such a kernel does return, per query row j, lse[j] = log sum_{i<=j} exp(scale * <q_j, k_i>);
+ * given those, pass 1 above is skipped and the indicator costs ONE recomputation of QK^T:
+ *   attn_acc[k] = sum_j exp(scale * <q_j, k_k> - lse_in[j])   (Eq. 2, or Eq. 3 over the last w rows)
+ *   vnorm, score as in vatp_prefill_scores (Eq. 4).
+ * lse_in:  [batch, heads, T] fp32 device array, natural log, 16-byte aligned, read only; it must
+ *          be the causal row normaliser for the same q, k and scale (the result is as accurate as
+ *          lse_in is: an error e in lse_in[j] scales row j's probabilities by exp(-e)).  With
+ *          VATP_IND_WINDOW only rows j >= T - w are read.
+ * lse_out: nullable; receives a copy of lse_in.  All other arguments, the workspace requirement
+ *          and the error behaviour are those of vatp_prefill_scores; NULL lse_in is
+ *          VATP_ERR_INVALID_ARG.
+ */
+vatp_status vatp_prefill_scores_from_lse(const vatp_params* params, const void* q, const void* k, const void* v,
+                                         const float* lse_in, float* lse_out, float* attn_acc, float* vnorm,
+                                         float* score, float* win_rows, void* workspace, size_t workspace_bytes,
+                                         int32_t* dev_status, void* cuda_stream);
+
+/*
  * vatp_prefill_scores for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a packaging variant of the call above and computes exactly the same thing.)
  *

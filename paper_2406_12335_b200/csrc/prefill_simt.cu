@@ -207,7 +207,7 @@ colsum_kernel(Shape sh, const T* __restrict__ q, const T* __restrict__ k, const 
 
 template <typename T>
 cudaError_t launch_t(const Shape& s, const T* q, const T* k, const T* v, float* lse, float* attn_acc, float* vnorm,
-                     float* score, float* win_rows, cudaStream_t st) {
+                     float* score, float* win_rows, cudaStream_t st, bool lse_given) {
   const int ld = s.d + 1;
   const size_t smem1 = sizeof(float) * 2 * TILE * ld;
   const size_t smem2 = smem1 + sizeof(float) * (TILE + 16 * TILE);
@@ -219,7 +219,7 @@ cudaError_t launch_t(const Shape& s, const T* q, const T* k, const T* v, float* 
   const int first_row = s.window > 0 ? max(s.T - s.window, 0) : 0;
   const int qtiles = (s.T - first_row + TILE - 1) / TILE;
   const int ktiles = (s.T + TILE - 1) / TILE;
-  rowstats_kernel<T><<<dim3(qtiles, s.units), NTHREADS, smem1, st>>>(s, q, k, lse, first_row);
+  if (!lse_given) rowstats_kernel<T><<<dim3(qtiles, s.units), NTHREADS, smem1, st>>>(s, q, k, lse, first_row);
   colsum_kernel<T><<<dim3(ktiles, s.units), NTHREADS, smem2, st>>>(s, q, k, v, lse, attn_acc, vnorm, score,
                                                                     s.window > 0 ? win_rows : nullptr, first_row);
   return cudaGetLastError();
@@ -228,11 +228,13 @@ cudaError_t launch_t(const Shape& s, const T* q, const T* k, const T* v, float* 
 }  // namespace
 
 cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const void* k, const void* v, float* lse,
-                                float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st) {
+                                float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st,
+                                bool lse_given) {
   if (dtype == VATP_F32)
-    return launch_t<float>(s, (const float*)q, (const float*)k, (const float*)v, lse, attn_acc, vnorm, score, win_rows, st);
+    return launch_t<float>(s, (const float*)q, (const float*)k, (const float*)v, lse, attn_acc, vnorm, score, win_rows, st,
+                           lse_given);
   return launch_t<__nv_bfloat16>(s, (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v, lse,
-                                 attn_acc, vnorm, score, win_rows, st);
+                                 attn_acc, vnorm, score, win_rows, st, lse_given);
 }
 
 }  // namespace vatp

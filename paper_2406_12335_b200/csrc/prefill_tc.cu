@@ -780,6 +780,22 @@ __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a) {
   }
 }
 
+// Row normalisers supplied by the caller (an attention forward that ran earlier produces them) brought
+// into the layout pass 2 reads: log2 domain, padded to whole chunks, +inf where a query contributes
+// nothing (beyond the prompt, before the history window).  Stands in for pass 1.
+__global__ void __launch_bounds__(256) lse_import_kernel(TcArgs a, const float* __restrict__ lse_in) {
+  const int u = blockIdx.x;
+  const int i = blockIdx.y * 256 + threadIdx.x;
+  if (i >= a.Tpad) return;
+  float x = INFINITY;
+  if (i < a.T) {
+    const float l = __ldg(lse_in + (int64_t)u * a.T + i);
+    if (i >= a.first_row) x = l * 1.4426950408889634f;
+    if (a.lse_out && a.lse_out != lse_in) a.lse_out[(int64_t)u * a.T + i] = l;
+  }
+  a.lse2[(int64_t)u * a.Tpad + i] = x;
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -840,7 +856,7 @@ size_t prefill_tc_workspace_bytes(int units, int T) {
 
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
-                              int32_t* dev_status, cudaStream_t st) {
+                              int32_t* dev_status, cudaStream_t st, const float* lse_in) {
   CUtensorMap tm_q, tm_k;
   if (!make_map(&tm_q, q, s) || !make_map(&tm_k, k, s)) return cudaErrorInvalidValue;
   TcArgs a;
@@ -881,14 +897,17 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
   if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
-  a.side_norm = a.ft == 0 && a.norm == VATP_NORM_L1;
+  a.side_norm = a.ft == 0 && a.norm == VATP_NORM_L1 && !lse_in;   // the side warp belongs to pass 1
   if (!a.side_norm) {
     const dim3 grid(a.units, (s.T + 127) / 128);
     if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a);
     else if (a.norm == VATP_NORM_L2) vnorm_kernel<VATP_NORM_L2><<<grid, 256, 0, st>>>(a);
     else vnorm_kernel<VATP_NORM_LINF><<<grid, 256, 0, st>>>(a);
   }
-  prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  if (lse_in)
+    lse_import_kernel<<<dim3(a.units, a.Tpad / 256), 256, 0, st>>>(a, lse_in);
+  else
+    prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(items2 < sms ? items2 : sms);

@@ -58,6 +58,37 @@ bool cache_ok(const vatp_cache* c, bool windowed) {
   return true;
 }
 
+// Both prefill entry points: lse_in == nullptr runs pass 1, otherwise the caller's normalisers replace it.
+vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, const void* v, const float* lse_in,
+                         float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows, void* workspace,
+                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  vatp_status s = check_params(p, true);
+  if (s != VATP_OK) return s;
+  if (!q || !k || !v || !attn_acc || !vnorm || !score) return VATP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
+  const bool windowed = p->indicator == VATP_IND_WINDOW;
+  if (windowed && !win_rows) return VATP_ERR_INVALID_ARG;
+  Shape sh;
+  s = make_shape(p, &sh);
+  if (s != VATP_OK) return s;
+  if (!workspace || workspace_bytes < lse_bytes(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+    return VATP_ERR_WORKSPACE;
+  float* ws = static_cast<float*>(workspace);
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e;
+  if (p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available()) {
+    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st, lse_in);
+  } else if (lse_in) {
+    // pass 2 of the general kernel reads natural-log normalisers [units][T] directly
+    e = launch_prefill_simt(sh, p->dtype, q, k, v, const_cast<float*>(lse_in), attn_acc, vnorm, score, win_rows, st, true);
+    if (e == cudaSuccess && lse_out && lse_out != lse_in)
+      e = cudaMemcpyAsync(lse_out, lse_in, sizeof(float) * (size_t)sh.units * sh.T, cudaMemcpyDeviceToDevice, st);
+  } else {
+    e = launch_prefill_simt(sh, p->dtype, q, k, v, lse_out ? lse_out : ws, attn_acc, vnorm, score, win_rows, st);
+  }
+  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -85,25 +116,17 @@ size_t vatp_workspace_bytes(const vatp_params* p) {
 vatp_status vatp_prefill_scores(const vatp_params* p, const void* q, const void* k, const void* v, float* lse_out,
                                 float* attn_acc, float* vnorm, float* score, float* win_rows, void* workspace,
                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
-  vatp_status s = check_params(p, true);
-  if (s != VATP_OK) return s;
-  if (!q || !k || !v || !attn_acc || !vnorm || !score) return VATP_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
-  const bool windowed = p->indicator == VATP_IND_WINDOW;
-  if (windowed && !win_rows) return VATP_ERR_INVALID_ARG;
-  Shape sh;
-  s = make_shape(p, &sh);
-  if (s != VATP_OK) return s;
-  if (!workspace || workspace_bytes < lse_bytes(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
-    return VATP_ERR_WORKSPACE;
-  float* ws = static_cast<float*>(workspace);
-  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e;
-  if (p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available())
-    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st);
-  else
-    e = launch_prefill_simt(sh, p->dtype, q, k, v, lse_out ? lse_out : ws, attn_acc, vnorm, score, win_rows, st);
-  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+  return prefill_impl(p, q, k, v, nullptr, lse_out, attn_acc, vnorm, score, win_rows, workspace, workspace_bytes,
+                      dev_status, cuda_stream);
+}
+
+vatp_status vatp_prefill_scores_from_lse(const vatp_params* p, const void* q, const void* k, const void* v,
+                                         const float* lse_in, float* lse_out, float* attn_acc, float* vnorm,
+                                         float* score, float* win_rows, void* workspace, size_t workspace_bytes,
+                                         int32_t* dev_status, void* cuda_stream) {
+  if (!lse_in || !aligned16(lse_in)) return VATP_ERR_INVALID_ARG;
+  return prefill_impl(p, q, k, v, lse_in, lse_out, attn_acc, vnorm, score, win_rows, workspace, workspace_bytes,
+                      dev_status, cuda_stream);
 }
 
 vatp_status vatp_select(const vatp_params* p, const float* score, int32_t* kept_idx, void* workspace,

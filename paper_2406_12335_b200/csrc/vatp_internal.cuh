@@ -66,11 +66,14 @@ struct DependentLaunch {
 };
 
 // ---- launchers (each returns cudaGetLastError()) ----
+// lse_given: `lse` already holds the row normalisers (natural log), pass 1 is skipped
 cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const void* k, const void* v, float* lse,
-                                float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st);
+                                float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st,
+                                bool lse_given = false);
+// lse_in: row normalisers [units][T] (natural log) from the caller; non-null skips pass 1
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
-                              int32_t* dev_status, cudaStream_t st);
+                              int32_t* dev_status, cudaStream_t st, const float* lse_in = nullptr);
 size_t prefill_tc_workspace_bytes(int units, int T);  // padded log2-domain row normalisers
 cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st);
 cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, const void* v, const float* attn_acc,

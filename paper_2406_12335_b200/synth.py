@@ -79,6 +79,10 @@ CONFIGS = {
     3: Workload(3, "windowed_2k_b16", "bf16", 16, 32, 1, 128, 2048, 1024, 0, 10, "window", 256, 512),
     4: Workload(4, "long_32k", "bf16", 1, 32, 32, 128, 32768, _round_half_up(0.1 * 32768), 0, 512, "h2o", 0, 64,
                 boost=64),
+    # the shape of the paper's throughput measurements ("Inference Efficiency": prompt 4096, 128 generated tokens,
+    # batch 12) with Appendix A's Scissorhands split at a 50% budget (10 local tokens, history window 400) and
+    # F = 20 kept leading tokens; other budgets of that table: see presets.appendix_a
+    5: Workload(5, "throughput_table_b12_4k", "bf16", 12, 32, 1, 128, 4096, 2048, 20, 10, "window", 400, 128),
 }
 
 

@@ -20,7 +20,7 @@ BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
 NORM_KINDS = {"l1": 0, "l2": 1, "linf": 2}
 STATIC_SCRATCH_BYTES = (4 << 20) + 256
-EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
+EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_from_lse", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
            "vatp_selftest_bounded_wait", "vatp_selftest_overlap_policy", "vatp_status_string"]
 
 
@@ -44,6 +44,8 @@ lib.vatp_workspace_bytes.restype = C.c_size_t
 lib.vatp_workspace_bytes.argtypes = [C.POINTER(Params)]
 lib.vatp_prefill_scores.restype = C.c_int
 lib.vatp_prefill_scores.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.vatp_prefill_scores_from_lse.restype = C.c_int
+lib.vatp_prefill_scores_from_lse.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.vatp_prefill_scores_static.restype = C.c_int
 lib.vatp_prefill_scores_static.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.vatp_select.restype = C.c_int
@@ -134,6 +136,16 @@ def vatp_prefill_scores(p: Params, q, k, v, *, lse_out=None, attn_acc, vnorm, sc
     _check(lib.vatp_prefill_scores(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse_out), _ptr(attn_acc), _ptr(vnorm),
                                    _ptr(score), _ptr(win_rows), _ptr(workspace), ws_bytes, _ptr(dev_status),
                                    _stream(stream)), "vatp_prefill_scores")
+
+
+def vatp_prefill_scores_from_lse(p: Params, q, k, v, lse_in, *, lse_out=None, attn_acc, vnorm, score, win_rows=None,
+                                 workspace=None, dev_status=None, stream=None):
+    """vatp_prefill_scores with the row normalisers (natural-log lse of the causal softmax rows, as an
+    attention forward returns them) given: pass 1 is skipped, QK^T is recomputed once."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vatp_prefill_scores_from_lse(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse_in), _ptr(lse_out),
+                                            _ptr(attn_acc), _ptr(vnorm), _ptr(score), _ptr(win_rows), _ptr(workspace),
+                                            ws_bytes, _ptr(dev_status), _stream(stream)), "vatp_prefill_scores_from_lse")
 
 
 def vatp_prefill_scores_static(p: Params, q, k, v, *, lse_out=None, attn_acc, vnorm, score, win_rows=None,

@@ -249,6 +249,34 @@ def test_value_norm_kinds(norm, dtype, d, T, B, indicator, window):
     assert torch.all(g.vnorm[0, 0].double() < l1)     # a different norm really was taken
 
 
+@pytest.mark.parametrize("method,ratio", [("scissorhands", 1.0), ("scissorhands", 0.5), ("scissorhands", 0.25),
+                                           ("h2o", 0.5), ("h2o", 0.25)])
+def test_appendix_a_presets(method, ratio):
+    """Appendix A's hyper-parameters through the product's preset table: H2O (half the budget chosen by
+    importance, half local window) and Scissorhands (10 local tokens, history window 400) with the first
+    20 tokens kept, at the throughput table's budgets.  At 100% nothing is pruned at prefill and the first
+    decode step already evicts.  The oracle takes its split from its own Appendix A function."""
+    from oracle import vatp_oracle as O
+    from paper_2406_12335_b200 import presets
+    T = 900
+    pr = presets.appendix_a(method, T, ratio)
+    sp = O.appendix_a_split(method, T, ratio)
+    assert (pr["budget"], pr["n_sink"], pr["n_recent"], pr["window"]) == (sp["B"], sp["F"], sp["R"], sp["w"] or 0)
+    wl = synth.Workload(67, f"preset_{method}_{ratio}", "bf16", 1, 3, 1, 128, T, sp["B"], sp["F"], sp["R"],
+                        "window" if sp["w"] else "h2o", sp["w"] or 0, 10)
+    g, _, _ = _run_case(wl, check_state_every=5)
+    assert int(g.cache.len[0, 0]) == sp["B"]                    # held at budget: 10 appended, 10 evicted
+    assert torch.all(g.cache.pos[0, 0, : sp["F"]].cpu() == torch.arange(sp["F"]))
+
+
+def test_config5_throughput_table_shape():
+    """The shape of the paper's throughput measurements (batch 12, prompt 4096, Scissorhands split with
+    w = 400, F = 20) at the 50% budget, full per-layer size: oracle on sampled units with decode steps,
+    oracle-free invariants on all 384 units."""
+    wl = synth.CONFIGS[5].with_(decode_steps=24)
+    _run_case(wl, units=[(0, 0), (11, 31)], check_state_every=12)
+
+
 def test_decode_large_cache_state_paths():
     """Caches too large for the per-slot state to sit beside the streaming stages.  Stepped alone, a
     launch waits for its predecessor and takes a whole SM, state included (checked against the
