@@ -23,12 +23,26 @@ def to_np64(x: torch.Tensor) -> np.ndarray:
     return x.detach().to("cpu", torch.float64).numpy()
 
 
+def attention_forward_lse(q: torch.Tensor, k: torch.Tensor, scale: float) -> torch.Tensor:
+    """Stand-in for the log-sum-exp output of an attention forward: plain torch, float64 on the
+    inputs' device, one unit at a time; [batch, heads, T] fp32."""
+    b, h, T, _ = q.shape
+    out = torch.empty(b, h, T, dtype=torch.float32, device=q.device)
+    mask = torch.ones(T, T, dtype=torch.bool, device=q.device).triu(1)
+    for i in range(b):
+        for j in range(h):
+            s = (q[i, j].double() @ k[i, j].double().T) * scale
+            out[i, j] = torch.logsumexp(s.masked_fill(mask, float("-inf")), dim=-1).float()
+    return out
+
+
 class GpuPrefill:
     """Device buffers and the three prefill-side calls for one layer of a workload."""
 
-    def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None):
+    def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None, lse_given=False):
         V = vatp()
         self.wl = wl
+        self.lse_given = lse_given
         self.F = wl.n_sink if n_sink is None else n_sink
         dev = q.device
         b, h, T = wl.batch, wl.heads, wl.seq_len
@@ -48,9 +62,16 @@ class GpuPrefill:
 
     def run(self):
         V = vatp()
-        V.vatp_prefill_scores(self.p, self.q, self.k, self.v, lse_out=self.lse, attn_acc=self.attn_acc,
-                              vnorm=self.vnorm, score=self.score, win_rows=self.win_rows, workspace=self.ws,
-                              dev_status=self.status)
+        if self.lse_given:
+            # the row normalisers arrive from outside, as from an attention forward that ran before
+            self.lse_in = attention_forward_lse(self.q, self.k, self.wl.scale)
+            V.vatp_prefill_scores_from_lse(self.p, self.q, self.k, self.v, self.lse_in, lse_out=self.lse,
+                                           attn_acc=self.attn_acc, vnorm=self.vnorm, score=self.score,
+                                           win_rows=self.win_rows, workspace=self.ws, dev_status=self.status)
+        else:
+            V.vatp_prefill_scores(self.p, self.q, self.k, self.v, lse_out=self.lse, attn_acc=self.attn_acc,
+                                  vnorm=self.vnorm, score=self.score, win_rows=self.win_rows, workspace=self.ws,
+                                  dev_status=self.status)
         V.vatp_select(self.p, self.score, self.kept, workspace=self.ws, dev_status=self.status)
         V.vatp_compact(self.p, self.k, self.v, self.attn_acc, self.vnorm, self.kept, self.cache,
                        win_rows=self.win_rows, dev_status=self.status)

@@ -55,6 +55,10 @@ def test_host_side_validation(V):
     assert V.lib.vatp_prefill_scores(C.byref(p), 8, 16, 16, null, 16, 16, 16, null, null, 0, null, null) == 1
     assert V.lib.vatp_prefill_scores(C.byref(p), 16, 16, 16, null, 16, 16, 16, null, null, 0, null, null) == 3
     assert V.lib.vatp_prefill_scores(C.byref(p), 16, 16, 16, null, 16, 16, 16, null, 256, 8, null, null) == 3
+    # given-normaliser variant: lse_in is required and 16-byte aligned; then the usual checks apply
+    assert V.lib.vatp_prefill_scores_from_lse(C.byref(p), 16, 16, 16, null, null, 16, 16, 16, null, 256, 4096, null, null) == 1
+    assert V.lib.vatp_prefill_scores_from_lse(C.byref(p), 16, 16, 16, 8, null, 16, 16, 16, null, 256, 4096, null, null) == 1
+    assert V.lib.vatp_prefill_scores_from_lse(C.byref(p), 16, 16, 16, 16, null, 16, 16, 16, null, null, 0, null, null) == 3
     wp = V.make_params(**{**ok, "indicator": "window", "window": 0})
     assert V.lib.vatp_select(C.byref(wp), 16, 16, null, 0, null, null) == 1
     wp = V.make_params(**{**ok, "indicator": "window", "window": 8})

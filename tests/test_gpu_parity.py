@@ -16,9 +16,9 @@ def _small(dtype, d, T, B, F, R, b=1, h=2, indicator="h2o", window=0, steps=0, c
     return synth.Workload(cid, f"case_T{T}", dtype, b, h, 1, d, T, B, F, R, indicator, window, steps)
 
 
-def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0):
+def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0, lse_given=False):
     q, k, v = synth.prefill_inputs(wl, layer, "cuda")
-    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink).run()
+    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink, lse_given=lse_given).run()
     P.gpu_invariants(g)
     tol = P.TOL[wl.dtype]
     units = units or [(b, h) for b in range(wl.batch) for h in range(wl.heads)]
@@ -275,6 +275,35 @@ def test_config5_throughput_table_shape():
     oracle-free invariants on all 384 units."""
     wl = synth.CONFIGS[5].with_(decode_steps=24)
     _run_case(wl, units=[(0, 0), (11, 31)], check_state_every=12)
+
+
+@pytest.mark.parametrize("dtype,d,T,B,indicator,window,norm", [
+    ("bf16", 128, 1000, 300, "h2o", 0, "l1"),       # tensor-core pass 2 alone, ragged against 128 and 256
+    ("bf16", 128, 640, 200, "h2o", 0, "linf"),      # odd tile count (half a chunk of padding)
+    ("bf16", 128, 900, 450, "window", 400, "l1"),   # Eq. 3: only the last 400 normalisers are read
+    ("f32", 64, 333, 100, "h2o", 0, "l1"),          # general kernel
+    ("f32", 64, 300, 120, "window", 77, "l2"),
+    ("bf16", 64, 257, 128, "h2o", 0, "l1"),
+])
+def test_prefill_from_given_row_normalisers(dtype, d, T, B, indicator, window, norm):
+    """vatp_prefill_scores_from_lse: the normalisers of Eq. 1 come from outside (a float64 torch
+    computation standing in for an attention forward), pass 1 is skipped; indicator, norms, scores, kept
+    sets, compaction and decode steps are checked against the oracle as for the two-pass call, and the
+    outputs agree with the two-pass call within the score tolerance."""
+    wl = _small(dtype, d, T, B, 2, 10, b=2, h=2, indicator=indicator, window=window, steps=4, cid=68).with_(norm=norm)
+    g, _, _ = _run_case(wl, lse_given=True)
+    assert torch.equal(g.lse, g.lse_in)                      # lse_out receives a copy
+    two = P.GpuPrefill(wl, g.q, g.k, g.v).run()
+    tol = P.TOL[dtype]
+    for name in ("attn_acc", "vnorm", "score"):
+        a, b_ = getattr(g, name).double(), getattr(two, name).double()
+        assert torch.all((a - b_).abs() <= 2 * tol * b_.abs() + 1e-30), name
+
+
+def test_prefill_from_given_row_normalisers_config1():
+    """Config 1's shape (32 heads, prompt 4096) with given normalisers: oracle on sampled heads."""
+    wl = synth.CONFIGS[1].with_(decode_steps=0)
+    _run_case(wl, decode=False, units=[(0, 0), (0, 17)], lse_given=True)
 
 
 def test_decode_large_cache_state_paths():
