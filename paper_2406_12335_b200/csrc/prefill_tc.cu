@@ -280,7 +280,26 @@ struct WinOut {
   float* p;
   int lo, hi;
   int64_t T;
+  char* base;      // all 32 columns live (lo == 0, hi == 32): this unit's window block (same for the whole warp) ...
+  uint32_t off;    // ... and this thread's byte offset of column 0 in it; columns are row4 bytes apart
+  uint32_t row4;
+  bool full;
 };
+// Four consecutive window rows of one key.  The common case (whole slice inside the window and the prompt) is one
+// 32-bit multiply-add and one store per value on a warp-uniform base; ragged slices test every column.
+__device__ __forceinline__ void win_store4(const WinOut& wo, int i, float p0, float p1, float p2, float p3) {
+  if (wo.full) {
+    *reinterpret_cast<float*>(wo.base + (wo.off + (uint32_t)i * wo.row4)) = p0;
+    *reinterpret_cast<float*>(wo.base + (wo.off + (uint32_t)(i + 1) * wo.row4)) = p1;
+    *reinterpret_cast<float*>(wo.base + (wo.off + (uint32_t)(i + 2) * wo.row4)) = p2;
+    *reinterpret_cast<float*>(wo.base + (wo.off + (uint32_t)(i + 3) * wo.row4)) = p3;
+  } else {
+    if (i >= wo.lo && i < wo.hi) wo.p[i * wo.T] = p0;
+    if (i + 1 >= wo.lo && i + 1 < wo.hi) wo.p[(i + 1) * wo.T] = p1;
+    if (i + 2 >= wo.lo && i + 2 < wo.hi) wo.p[(i + 2) * wo.T] = p2;
+    if (i + 3 >= wo.lo && i + 3 < wo.hi) wo.p[(i + 3) * wo.T] = p3;
+  }
+}
 template <int PASS, bool DIAG, bool WIN>
 __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float scale_log2, float& m_run, float& l_run,
                                           f32x2 (&cs)[2], const float* nlse_t, const WinOut& wo) {
@@ -307,10 +326,7 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
         float p0, p1, p2, p3;
         upk2(e0, p0, p1);
         upk2(e1, p2, p3);
-        if (i >= wo.lo && i < wo.hi) wo.p[i * wo.T] = p0;
-        if (i + 1 >= wo.lo && i + 1 < wo.hi) wo.p[(i + 1) * wo.T] = p1;
-        if (i + 2 >= wo.lo && i + 2 < wo.hi) wo.p[(i + 2) * wo.T] = p2;
-        if (i + 3 >= wo.lo && i + 3 < wo.hi) wo.p[(i + 3) * wo.T] = p3;
+        win_store4(wo, i, p0, p1, p2, p3);
       }
     }
   } else {
@@ -330,10 +346,7 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
       if (c0 + i + 3 < row) p3 = 0.f;
       s0 += p0; s1 += p1; s2 += p2; s3 += p3;
       if (WIN) {
-        if (i >= wo.lo && i < wo.hi) wo.p[i * wo.T] = p0;
-        if (i + 1 >= wo.lo && i + 1 < wo.hi) wo.p[(i + 1) * wo.T] = p1;
-        if (i + 2 >= wo.lo && i + 2 < wo.hi) wo.p[(i + 2) * wo.T] = p2;
-        if (i + 3 >= wo.lo && i + 3 < wo.hi) wo.p[(i + 3) * wo.T] = p3;
+        win_store4(wo, i, p0, p1, p2, p3);
       }
     }
     cs[0] = add2(cs[0], pk2(s0, s1));
@@ -597,13 +610,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       auto needed = [&](int c) { return tile_needed<PASS>(it, st_of(c), a.nt); };
       // where the probabilities of the 32 query columns starting at column c0 of streamed tile stile go (Eq. 3 rows)
       auto wout = [&](int stile, int c0) {
-        WinOut wo{nullptr, 0, 0, 0};
+        WinOut wo{nullptr, 0, 0, 0, nullptr, 0u, 0u, false};
         if (WIN && PASS == 2) {
           const int q0 = stile * TILE + c0;
           wo.T = a.T;
           wo.lo = min(max(a.first_row - q0, 0), 32);
           wo.hi = tok < a.T ? min(max(a.T - q0, 0), 32) : 0;
           wo.p = a.win_rows + ((int64_t)u * a.window + (q0 - a.wrow0)) * a.T + tok;
+          // a unit's window block is window * T * 4 bytes: 32-bit offsets while that stays below 4 GB
+          wo.full = wo.lo == 0 && wo.hi == 32 && (uint64_t)a.window * a.T < (1ull << 30);
+          wo.base = reinterpret_cast<char*>(a.win_rows + (int64_t)u * a.window * a.T);
+          wo.off = wo.full ? ((uint32_t)(q0 - a.wrow0) * (uint32_t)a.T + (uint32_t)tok) * 4u : 0u;
+          wo.row4 = (uint32_t)a.T * 4u;
         }
         return wo;
       };
