@@ -770,9 +770,28 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // the window's query tiles and is too short to hide one warp per SM walking all of V, and for the
 // l2 / l-infinity variants.  Sixteen lanes
 // per row, eight rows in flight per lane.
+// When the caller supplies the row normalisers (lse_in, natural log, [units][T]) the same launch brings them
+// into the layout pass 2 reads and so stands in for pass 1: log2 domain, padded to whole chunks, +inf where a
+// query contributes nothing (beyond the prompt, before the history window).
 template <int KIND>
-__global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a) {
+__global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a, const float* __restrict__ lse_in) {
+  // pass 2, a programmatic dependent, may set up while this kernel runs; it reads what is written here
+  // only after its griddepcontrol.wait
+  if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int u = blockIdx.x;
+  if (lse_in) {
+    // this CTA's 128 tokens; the last CTA of the unit also fills the padding up to Tpad
+    const int last = blockIdx.y == gridDim.y - 1 ? a.Tpad : (blockIdx.y + 1) * 128;
+    for (int i = blockIdx.y * 128 + threadIdx.x; i < last; i += 256) {
+      float x = INFINITY;
+      if (i < a.T) {
+        const float l = __ldg(lse_in + (int64_t)u * a.T + i);
+        if (i >= a.first_row) x = l * 1.4426950408889634f;
+        if (a.lse_out && a.lse_out != lse_in) a.lse_out[(int64_t)u * a.T + i] = l;
+      }
+      a.lse2[(int64_t)u * a.Tpad + i] = x;
+    }
+  }
   const int b = u / a.heads, h = u - b * a.heads;
   const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
   const int sub = threadIdx.x >> 4, part = threadIdx.x & 15;       // 16 rows per pass of the CTA
@@ -796,22 +815,6 @@ __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a) {
     const int tok = row0 + 16 * j;
     if (part == 0 && tok < a.T) a.vnorm[(int64_t)u * a.T + tok] = norm_finish(KIND, acc);
   }
-}
-
-// Row normalisers supplied by the caller (an attention forward that ran earlier produces them) brought
-// into the layout pass 2 reads: log2 domain, padded to whole chunks, +inf where a query contributes
-// nothing (beyond the prompt, before the history window).  Stands in for pass 1.
-__global__ void __launch_bounds__(256) lse_import_kernel(TcArgs a, const float* __restrict__ lse_in) {
-  const int u = blockIdx.x;
-  const int i = blockIdx.y * 256 + threadIdx.x;
-  if (i >= a.Tpad) return;
-  float x = INFINITY;
-  if (i < a.T) {
-    const float l = __ldg(lse_in + (int64_t)u * a.T + i);
-    if (i >= a.first_row) x = l * 1.4426950408889634f;
-    if (a.lse_out && a.lse_out != lse_in) a.lse_out[(int64_t)u * a.T + i] = l;
-  }
-  a.lse2[(int64_t)u * a.Tpad + i] = x;
 }
 
 // ---- host side -------------------------------------------------------------------------------
@@ -918,14 +921,11 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.side_norm = a.ft == 0 && a.norm == VATP_NORM_L1 && !lse_in;   // the side warp belongs to pass 1
   if (!a.side_norm) {
     const dim3 grid(a.units, (s.T + 127) / 128);
-    if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a);
-    else if (a.norm == VATP_NORM_L2) vnorm_kernel<VATP_NORM_L2><<<grid, 256, 0, st>>>(a);
-    else vnorm_kernel<VATP_NORM_LINF><<<grid, 256, 0, st>>>(a);
+    if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a, lse_in);
+    else if (a.norm == VATP_NORM_L2) vnorm_kernel<VATP_NORM_L2><<<grid, 256, 0, st>>>(a, lse_in);
+    else vnorm_kernel<VATP_NORM_LINF><<<grid, 256, 0, st>>>(a, lse_in);
   }
-  if (lse_in)
-    lse_import_kernel<<<dim3(a.units, a.Tpad / 256), 256, 0, st>>>(a, lse_in);
-  else
-    prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  if (!lse_in) prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(items2 < sms ? items2 : sms);
