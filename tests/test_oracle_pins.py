@@ -506,3 +506,15 @@ def test_appendix_a_split_invariants_and_the_product_presets():
                         assert p["indicator"] == ("window" if s["w"] else "h2o")
     with pytest.raises(ValueError):
         O.appendix_a_split("fastgen", 100)
+
+
+def test_workload5_is_the_scissorhands_split_at_half_budget():
+    """The added timing workload (prompt 4096, batch 12, 128 steps: the paper's throughput measurements) carries
+    Appendix A's Scissorhands split at 50%, as both the oracle's and the product's tables give it."""
+    from paper_2406_12335_b200 import presets, synth
+    wl = synth.CONFIGS[5]
+    s = O.appendix_a_split("scissorhands", wl.seq_len, 0.5, "llama2-7b-chat")
+    assert (wl.budget, wl.n_sink, wl.n_recent, wl.window, wl.indicator) == (s["B"], s["F"], s["R"], s["w"], "window")
+    assert (wl.batch, wl.heads, wl.head_dim, wl.seq_len, wl.decode_steps) == (12, 32, 128, 4096, 128)
+    p = presets.appendix_a("scissorhands", wl.seq_len, 0.5)
+    assert (p["budget"], p["n_sink"], p["n_recent"], p["window"]) == (wl.budget, wl.n_sink, wl.n_recent, wl.window)
