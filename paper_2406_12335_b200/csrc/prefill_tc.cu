@@ -13,8 +13,9 @@
 // reach into the window, pass 2 streams from the window's first tile on and also writes the
 // probabilities of those rows (win_rows); a side warp zeroes the entries nobody visits.
 //
-// Warp roles (608 threads): warp 0 TMA producer (it also draws the work items from a global counter
-// and passes them on), warp 1 MMA issuer and TMEM owner, warps 2-17 four softmax warpgroups (each takes
+// Warp roles (608 threads): warp 0 TMA producer (it also draws the work items from a global counter,
+// works out what they cover and passes that on, and in pass 2 copies the row normalisers of every
+// chunk into shared memory beside its tiles), warp 1 MMA issuer and TMEM owner, warps 2-17 four softmax warpgroups (each takes
 // one 64-column quarter of every 256-column accumulator, loads it into registers and hands the
 // accumulator back at once; four warps per scheduler keep the exponential unit busy where two could
 // not), warp 18 the value-norm reduction (pass 1) / window zero fill (pass 2 with Eq. 3).
@@ -34,6 +35,7 @@ constexpr int HD = 128;            // head_dim
 constexpr int CHUNK = 256;         // streamed tokens per stage = columns of an accumulator
 constexpr int NS = 2;              // streamed-chunk stages in shared memory
 constexpr int NACC = 2;            // TMEM accumulators (256 columns each)
+constexpr int NLSE = 8;            // ring of per-chunk normaliser rows in shared memory (pass 2)
 constexpr int SLAB_BYTES = TILE * 128;        // 128 rows x 64 bf16, 128-byte swizzled
 constexpr int TILE_BYTES = 2 * SLAB_BYTES;    // two K halves
 constexpr int CHUNK_BYTES = 2 * TILE_BYTES;   // 256 rows, two K halves
@@ -45,15 +47,15 @@ constexpr uint64_t WAIT_NS = 1000000000ull;
 struct Smem {
   alignas(1024) unsigned char fixed[2][TILE_BYTES];      // double-buffered fixed tile
   alignas(1024) unsigned char stream[NS][CHUNK_BYTES];   // [K half][256 rows][128 bytes] per stage
-  alignas(16) float lse_s[NSW][2][64];   // pass 2: per softmax warp, double-buffered NEGATED normalisers of its 64 query columns
+  alignas(128) float nlse[NLSE][CHUNK];  // pass 2: ring of the NEGATED normalisers of the streamed chunks (bulk copies by the producer)
   float part_a[2][3][TILE];   // pass 1: running max of warpgroups 1-3; pass 2: their column sums
   float part_b[2][3][TILE];   // pass 1: running sum of warpgroups 1-3
   alignas(8) uint64_t full[NS], empty[NS];
   uint64_t fixed_full[2], fixed_empty[2];
   uint64_t acc_full[NACC], acc_empty[NACC];
   uint64_t comb_full[2], comb_empty[2];
-  uint64_t item_full[4], item_empty[4];   // FIFO of work-item ids from the producer to the other roles
-  int item_ring[4];
+  uint64_t item_full[4], item_empty[4];   // FIFO of work items from the producer to the other roles
+  int item_ring[4][8];                    // u, tile, c_first, c_count, lo (u < 0: no more items)
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -110,6 +112,13 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(s32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(s32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
+}
+
+// untiled global -> shared bulk copy; both addresses and the size are multiples of 16 bytes
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(s32(dst)), "l"(src), "r"(bytes), "r"(s32(bar))
+               : "memory");
 }
 
 // Shared-memory matrix descriptor: K-major operand, 128-byte swizzle, 8-row groups 1024 bytes apart.
@@ -233,7 +242,6 @@ __device__ __forceinline__ f32x2 exp2_pair(int p, f32x2 v) {
   return ex2_sfu2(v);
 }
 
-__device__ __forceinline__ float4 neg4(float4 v) { return make_float4(-v.x, -v.y, -v.z, -v.w); }
 __device__ __forceinline__ float max3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -359,7 +367,7 @@ struct TcArgs {
   float scale_log2;
   const __nv_bfloat16* v;
   int64_t sb, sh, st;       // element strides of v
-  float* lse2;              // [units][Tpad] log2-domain row normalisers (+inf beyond T)
+  float* lse2;              // [units][Tpad] NEGATED log2-domain row normalisers (-inf where no query counts)
   float* lse_out;           // [units][T] natural-log copy, nullable
   float* attn_acc;
   float* vnorm;
@@ -479,16 +487,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
 
-  // Consumer side of the item FIFO: the itl-th item of this CTA (an id >= items ends the pass).
-  // The slot is handed back as soon as the id has been read.
-  auto next_item = [&](uint32_t itl, bool whole_warp) -> int {
+  // Consumer side of the item FIFO: the itl-th item of this CTA (u < 0 ends the pass, also when the CTA
+  // is aborting).  The producer has worked out what the item covers, once for the whole CTA (the index
+  // arithmetic takes several integer divisions).  The slot is handed back as soon as it has been read.
+  auto next_item = [&](uint32_t itl, bool whole_warp) -> Item {
     const int slot = itl & 3;
     bool got = mbar_wait(&sm.item_full[slot], (itl >> 2) & 1, abort_flag, a.dev_status);
     if (whole_warp) got = __all_sync(0xffffffffu, got);
-    const int id = got ? *reinterpret_cast<volatile int*>(&sm.item_ring[slot]) : -1;
+    Item it{-1, 0, 0, 0, 0};
+    if (got) {
+      const volatile int* f = &sm.item_ring[slot][0];
+      it.u = f[0]; it.tile = f[1]; it.c_first = f[2]; it.c_count = f[3]; it.lo = f[4];
+    }
     if (whole_warp) __syncwarp();
     if (got && (!whole_warp || lane == 0)) mbar_arrive(&sm.item_empty[slot]);
-    return id;     // -1: the CTA is aborting
+    return it;
   };
 
   // the operand that stays fixed per item and the one that streams
@@ -506,18 +519,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       bool ok = true;
+      bool waited_for_pass1 = false;
       uint32_t n = 0;
       int next = (int)atomicAdd(&a.counters[PASS - 1], 1u);
       for (uint32_t itl = 0; ok; ++itl) {
         const int id = next;
         const int slot = itl & 3;
+        Item it{-1, 0, 0, 0, 0};
+        if (id < items) it = item_of<PASS>(id, a);
         ok = mbar_wait<20>(&sm.item_empty[slot], ((itl >> 2) & 1) ^ 1, abort_flag, a.dev_status);
         if (!ok) break;
-        *reinterpret_cast<volatile int*>(&sm.item_ring[slot]) = id;
+        {
+          volatile int* f = &sm.item_ring[slot][0];
+          f[0] = it.u; f[1] = it.tile; f[2] = it.c_first; f[3] = it.c_count; f[4] = it.lo;
+        }
         mbar_arrive(&sm.item_full[slot]);
         if (id >= items) break;
         next = (int)atomicAdd(&a.counters[PASS - 1], 1u);     // in flight while this item's tiles are requested
-        const Item it = item_of<PASS>(id, a);
         const int b = it.u / a.heads, h = it.u - b * a.heads;
         const int fb = itl & 1;
         ok = mbar_wait<20>(&sm.fixed_empty[fb], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
@@ -531,13 +549,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (!ok) break;
           // chunk layout: [K half][256 rows][128 bytes]; rows beyond T arrive as zeros
           const int tok0 = (it.c_first + c) * CHUNK;
-          mbar_expect_tx(&sm.full[stg], CHUNK_BYTES);
+          mbar_expect_tx(&sm.full[stg], CHUNK_BYTES + (PASS == 2 ? CHUNK * 4 : 0));
 #pragma unroll
           for (int kh = 0; kh < 2; ++kh)
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh)
               tma_load_4d(sm.stream[stg] + kh * (2 * SLAB_BYTES) + hh * SLAB_BYTES, tm_stream, &sm.full[stg], 64 * kh,
                           tok0 + hh * TILE, h, b);
+          if (PASS == 2) {
+            // The chunk's 256 normalisers travel with its tiles and are complete when its MMAs are.  Ring slot
+            // n % NLSE: the MMAs of chunk n - 2 have completed (that freed this stage), so every softmax warp
+            // has handed back accumulator n - 4 and is past the normalisers of chunk n - 5 and of all before it.
+            // They are pass 1's output: nothing of it is read before that launch has completed.
+            if (!waited_for_pass1) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited_for_pass1 = true; }
+            bulk_load(sm.nlse[n % NLSE], a.lse2 + (int64_t)it.u * a.Tpad + tok0, CHUNK * 4, &sm.full[stg]);
+          }
         }
       }
     }
@@ -549,9 +575,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const uint64_t stage_desc0 = umma_desc(s32(sm.stream[0]));   // stages are CHUNK_BYTES apart
       const uint64_t fixed_desc0 = umma_desc(s32(sm.fixed[0]));    // buffers are TILE_BYTES apart
       for (uint32_t itl = 0; ok; ++itl) {
-        const int id = next_item(itl, false);
-        if (id < 0 || id >= items) break;
-        const Item it = item_of<PASS>(id, a);
+        const Item it = next_item(itl, false);
+        if (it.u < 0) break;
         const int fb = itl & 1;
         ok = mbar_wait(&sm.fixed_full[fb], (itl >> 1) & 1, abort_flag, a.dev_status);
         if (!ok) break;
@@ -584,19 +609,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int half = g >> 1;                      // which 128-token tile of a chunk those columns belong to
     const int cbase = (g & 1) * 64;               // and where they start inside that tile
     const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + half * TILE + cbase;
-    float* lse_w = &sm.lse_s[sw][0][0];
     bool ok = true;
     uint32_t n = 0;
     if (PASS == 2) asm volatile("griddepcontrol.wait;" ::: "memory");
     for (uint32_t itl = 0; ok; ++itl) {
-      const int id = next_item(itl, true);
-      if (id < 0 || id >= items) break;
-      const Item it = item_of<PASS>(id, a);
+      const Item it = next_item(itl, true);
+      if (it.u < 0) break;
       const int u = it.u;
       const int pi = itl & 1;
       const uint32_t ipar = (itl >> 1) & 1;
       const int tok = it.tile * TILE + row;       // query (pass 1) or key (pass 2) index of this thread
-      const float* lse2_u = a.lse2 + (int64_t)u * a.Tpad;
       // pass 2: this key's value norm, written by pass 1; fetched now, used in the item's epilogue
       float n1 = 0.f;
       if (PASS == 2 && g == 0 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tok);
@@ -604,7 +626,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       f32x2 cs[2] = {pk2(0.f, 0.f), pk2(0.f, 0.f)};   // pass 2: four running sums, packed
       const uint32_t n0 = n;
       n += it.c_count;
-      int buf = 0;
       // streamed tile this warp's columns belong to in chunk c, and whether the item needs it
       auto st_of = [&](int c) { return 2 * (it.c_first + c) + half; };
       auto needed = [&](int c) { return tile_needed<PASS>(it, st_of(c), a.nt); };
@@ -625,21 +646,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
         return wo;
       };
-      // pass 2: this warp's 64 normalisers of chunk c (negated), one float4 per lane 0-15
-      auto lse_fetch = [&](int c) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (lane < 16) v = neg4(__ldg(reinterpret_cast<const float4*>(lse2_u + st_of(c) * TILE + cbase) + lane));
-        return v;
-      };
-      if (PASS == 2) {
-        int c1 = 0;
-        while (c1 < it.c_count && !needed(c1)) ++c1;
-        if (c1 < it.c_count) {
-          const float4 v = lse_fetch(c1);
-          if (lane < 16) reinterpret_cast<float4*>(lse_w)[lane] = v;
-        }
-        __syncwarp();
-      }
       for (int c = 0; c < it.c_count; ++c) {
         const uint32_t ab = (n0 + c) % NACC;
         bool w = mbar_wait(&sm.acc_full[ab], ((n0 + c) / NACC) & 1, abort_flag, a.dev_status);
@@ -653,40 +659,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
           continue;
         }
-        float xa[32], xb[32];
+        // The warp's 64 columns are taken as two waves of 32: with one wave of accumulator values live
+        // the compiler has registers left to keep several exponentials in flight.
+        float x[32];
         const uint32_t t_addr = lane_addr + ab * CHUNK;
-        tmem_ld32(t_addr, xa);
-        tmem_ld32(t_addr + 32, xb);
-        // normalisers of the next needed chunk travel while this one is consumed
-        const bool next_needed = c + 1 < it.c_count && needed(c + 1);
-        float4 lnext = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (PASS == 2 && next_needed) lnext = lse_fetch(c + 1);
+        const int stile = st_of(c);
+        // pass 2: the chunk's negated normalisers arrived with its tiles (the accumulator being complete
+        // implies that those copies are); indexed by the column inside this warp's tile
+        const float* lse_t = sm.nlse[(n0 + c) % NLSE] + half * TILE;
+        tmem_ld32(t_addr, x);
         tmem_ld_wait();
-        // this warp's columns are in registers: the MMA warp may overwrite them
+        if (stile == it.tile) consume32<PASS, true, WIN>(x, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
+        else                  consume32<PASS, false, WIN>(x, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
+        tmem_ld32(t_addr + 32, x);
+        tmem_ld_wait();
+        // all of this warp's columns have been read: the MMA warp may overwrite them
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(&sm.acc_empty[ab]);
-        const float* lse_t = lse_w + buf * 64 - cbase;     // indexed by the column inside the tile
-        const int stile = st_of(c);
-        if (PASS == 1) {
-          // both slices share one row maximum and one rescale of the running sum
-          if (stile == it.tile) { mask_after_diagonal(xa, cbase, row); mask_after_diagonal(xb, cbase + 32, row); }
-          const float m_new = fmaxf(m_run, fmaxf(slice_max(xa), slice_max(xb)) * a.scale_log2);
-          l_run *= ex2(fmaxf(m_run - m_new, -126.f));
-          m_run = m_new;
-          l_run += slice_exp_sum(xa, a.scale_log2, m_run) + slice_exp_sum(xb, a.scale_log2, m_run);
-        } else if (stile == it.tile) {
-          consume32<PASS, true, WIN>(xa, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
-          consume32<PASS, true, WIN>(xb, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
-        } else {
-          consume32<PASS, false, WIN>(xa, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
-          consume32<PASS, false, WIN>(xb, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
-        }
-        if (PASS == 2 && next_needed) {
-          if (lane < 16) reinterpret_cast<float4*>(lse_w + (buf ^ 1) * 64)[lane] = lnext;
-          __syncwarp();
-          buf ^= 1;
-        }
+        if (stile == it.tile) consume32<PASS, true, WIN>(x, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
+        else                  consume32<PASS, false, WIN>(x, cbase + 32, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase + 32));
       }
       if (!ok) break;
       // ---- end of item: warpgroups 1-3 hand their partials to warpgroup 0, which finishes the rows
@@ -711,9 +703,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           if (l3 > 0.f) l += l3 * ex2(m3 - m);
           const float lse2 = m + log2f(l);
           // queries outside the prompt or before the history window contribute nothing to pass 2
-          a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? lse2 : INFINITY;
+          // (stored negated: pass 2 adds it to the scaled dot product)
+          a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? -lse2 : -INFINITY;
           // an odd tile count leaves half a chunk of padding that pass 2 reads as "no query"
-          if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = INFINITY;
+          if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
           if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
         } else {
           const float tot = hsum2(add2(cs[0], cs[1])) + (sm.part_a[pi][0][row] + sm.part_a[pi][1][row]) + sm.part_a[pi][2][row];
@@ -740,9 +733,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     // For key tile i the query tiles before it are never streamed (causal), and when the prompt is
     // shorter than the window its first rows belong to no query: those entries of win_rows are zero.
     for (uint32_t itl = 0;; ++itl) {
-      const int id = next_item(itl, true);
-      if (id < 0 || id >= items) break;
-      const Item it = item_of<PASS>(id, a);
+      const Item it = next_item(itl, true);
+      if (it.u < 0) break;
       float* wr = a.win_rows + (int64_t)it.u * a.window * a.T;
       const int k0 = it.tile * TILE;
       const int r_end = min(it.tile * TILE, a.T) - a.wrow0;      // rows of queries before this key tile
@@ -771,8 +763,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 // l2 / l-infinity variants.  Sixteen lanes
 // per row, eight rows in flight per lane.
 // When the caller supplies the row normalisers (lse_in, natural log, [units][T]) the same launch brings them
-// into the layout pass 2 reads and so stands in for pass 1: log2 domain, padded to whole chunks, +inf where a
-// query contributes nothing (beyond the prompt, before the history window).
+// into the layout pass 2 reads and so stands in for pass 1: log2 domain and negated, padded to whole chunks,
+// -inf where a query contributes nothing (beyond the prompt, before the history window).
 template <int KIND>
 __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a, const float* __restrict__ lse_in) {
   // pass 2, a programmatic dependent, may set up while this kernel runs; it reads what is written here
@@ -783,10 +775,10 @@ __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a, const float* __res
     // this CTA's 128 tokens; the last CTA of the unit also fills the padding up to Tpad
     const int last = blockIdx.y == gridDim.y - 1 ? a.Tpad : (blockIdx.y + 1) * 128;
     for (int i = blockIdx.y * 128 + threadIdx.x; i < last; i += 256) {
-      float x = INFINITY;
+      float x = -INFINITY;
       if (i < a.T) {
         const float l = __ldg(lse_in + (int64_t)u * a.T + i);
-        if (i >= a.first_row) x = l * 1.4426950408889634f;
+        if (i >= a.first_row) x = -l * 1.4426950408889634f;
         if (a.lse_out && a.lse_out != lse_in) a.lse_out[(int64_t)u * a.T + i] = l;
       }
       a.lse2[(int64_t)u * a.Tpad + i] = x;
