@@ -153,7 +153,8 @@ def run_reference(args, wl):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": f"config{wl.cid} {wl.name} (oracle on a sample)", "sample": sample},
             "decode_us_per_layer_step": dec_us,
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cpu_threads(),
+                             "kind": "oracle", "form": "float64 numpy, Python lists for the decode state", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -178,7 +179,10 @@ class LayerState:
         from paper_2406_12335_b200 import synth
         self.q, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
         self.p = V.params_for(self.q, budget=wl.budget, n_sink=wl.n_sink, n_recent=wl.n_recent, scale=wl.scale,
-                              indicator=wl.indicator, window=wl.window, norm=wl.norm)
+                              indicator=wl.indicator, window=wl.window, norm=wl.norm, decode_overlap=True)
+        # the same parameters without the opt-in: every decode step then waits for all earlier work in the stream
+        self.p_wait = type(self.p).from_buffer_copy(self.p)
+        self.p_wait.flags = 0
         b, h, T = wl.batch, wl.heads, wl.seq_len
         f32 = dict(dtype=torch.float32, device=dev)
         self.attn_acc = torch.empty(b, h, T, **f32)
@@ -232,22 +236,26 @@ def run_cuda(args, wl):
                            dev_status=status)
             if ev: ev[i][3].record()
 
-    def decode_all():
+    def decode_all(overlap=True):
         for s in range(steps_dec):
             for ls in layers:
-                V.vatp_decode_step(ls.p, ls.cache, ls.dq[s], ls.dk[s], ls.dv[s], ls.out[s], evicted_pos=ls.evicted[s],
-                                   dev_status=status)
+                V.vatp_decode_step(ls.p if overlap else ls.p_wait, ls.cache, ls.dq[s], ls.dk[s], ls.dv[s], ls.out[s],
+                                   evicted_pos=ls.evicted[s], dev_status=status)
 
     # warm up once outside any capture (first calls set kernel attributes), then capture the
     # launch-bound decode loop in a CUDA graph
     prefill_all(); decode_all(); torch.cuda.synchronize()
     lse_given[0], fill_lse[0] = args.lse_given, False
-    graph = None
+    graph = graph_wait = None
     if not args.no_graph:
         prefill_all(); torch.cuda.synchronize()
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph):
             decode_all()
+        torch.cuda.synchronize()
+        graph_wait = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph_wait):
+            decode_all(overlap=False)
         torch.cuda.synchronize()
 
     def run_decode():
@@ -287,6 +295,26 @@ def run_cuda(args, wl):
     # per-kernel breakdown of the prefill side: a few extra steps with an event after every call
     brk = [one_step(True) for _ in range(max(2, min(args.steps, 5)))]
     barrier()
+
+    # the same decode steps with every launch waiting for all earlier work in the stream (no opt-in to
+    # overlapping launches): what a chain of dependent steps costs - in a model, layer l + 1's q/k/v come
+    # from layer l's output
+    def wait_step():
+        flush.fill_(rank + 1)
+        prefill_all()
+        e1, e2 = E(), E()
+        e1.record()
+        if graph_wait is not None:
+            graph_wait.replay()
+        else:
+            decode_all(overlap=False)
+        e2.record()
+        return e1, e2
+
+    wait_step()
+    wrecs = [wait_step() for _ in range(max(2, min(args.steps, 5)))]
+    barrier()
+    dec_wait_ms = max_over_ranks([statistics.mean(a.elapsed_time(b) for a, b in wrecs)], dev, world)[0]
     assert int(status.item()) == 0, "device status word set"
 
     t_pre = [a.elapsed_time(b) for a, b, _, _ in recs]               # ms, all layers
@@ -335,6 +363,7 @@ def run_cuda(args, wl):
     tokens = wl.batch * T * L                                  # layer-tokens scored and pruned per step
     value = replica_throughput(tokens, pre_ms, world)
     dec_us = dec_ms * 1e3 / (steps_dec * L)
+    dec_wait_us = dec_wait_ms * 1e3 / (steps_dec * L)
 
     # ---- rooflines (algorithmic work only) ----
     if wl.indicator == "window":                               # only the last w query rows (Eq. 3)
@@ -358,19 +387,25 @@ def run_cuda(args, wl):
         "compact": {"bound": "hbm", "achieved": bytes_compact / (ms(t_compact) * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                     "unit": "GB/s", "us_per_launch": ms(t_compact) * 1e3},
         "decode_step": {"bound": "hbm", "achieved": bytes_decode / (dec_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"],
-                        "unit": "GB/s", "us_per_launch": dec_us},
+                        "unit": "GB/s", "us_per_launch": dec_us,
+                        "launches": f"steps of {L} independent layer caches in rotation, overlap flag set: consecutive launches run side by side"},
+        # same steps, every launch waiting for all earlier work in the stream (the default of vatp_decode_step)
+        "decode_step_dependent": {"bound": "hbm", "achieved": bytes_decode / (dec_wait_us * 1e-6) / 1e9,
+                                  "peak": peaks["hbm_gbs"], "unit": "GB/s", "us_per_launch": dec_wait_us},
     }
     for kd in kernels.values():
         kd["frac"] = kd["achieved"] / kd["peak"]
         kd["peak_source"] = peaks["source"]
     share = {"prefill_scores": ms(t_score) * L, "select": ms(t_select) * L, "compact": ms(t_compact) * L,
-             "decode_step": dec_ms}
+             "decode_step": dec_ms}          # (decode_step_dependent is an extra measurement, not part of the timed step)
     dominant = max(share, key=share.get)
     roof = dict(kernels[dominant])
     roof["kernel"] = dominant
     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of this kernel at
     # this shape (profiles/); other kernels / shapes: not captured
     roof["traffic"] = 34.52e6 if (dominant == "decode_step" and wl.cid == 1) else None
+    roof["traffic_source"] = ("ncu capture of this kernel at this shape, summarised in profiles/decode_mma_config1.md "
+                              "(not measured in this run)") if roof["traffic"] else None
     roof["algorithmic_bytes_per_launch"] = bytes_decode if dominant == "decode_step" else None
     roof["time_share"] = share[dominant] / sum(share.values())
 
@@ -385,6 +420,7 @@ def run_cuda(args, wl):
                    "replicas": "each GPU runs the whole workload (path does not shard within a call)",
                    "decode_graph": graph is not None},
         "prefill_ms_per_layer": pre_ms / L, "decode_us_per_layer_step": dec_us,
+        "decode_us_per_layer_step_dependent": dec_wait_us,
         "roofline": roof, "roofline_all": kernels,
         "e2e": None if host is None else
                {"value": replica_throughput(tokens, e2e_pre_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
@@ -396,7 +432,7 @@ def run_cuda(args, wl):
         cu, cs = 24, 64      # about 10-20 s of CPU work
         a, b = oracle_sample(wl, cu, cs)
         v = wl.batch * T / (a / cu * units)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle",
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cpu_threads(), "kind": "oracle", "form": "float64 numpy, Python lists for the decode state",
                                 "sample": f"{cu} of {units} heads of one layer (full prompt {T}, {cs} decode steps), "
                                           f"{a + b:.1f} s of CPU work, per-layer figure extrapolated x{units / cu:.2f}",
                                 "decode_us_per_layer_step": b / (cu * cs) * units * 1e6}

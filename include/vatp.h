@@ -51,6 +51,8 @@ typedef enum { VATP_IND_H2O = 0, VATP_IND_WINDOW = 1 } vatp_indicator;
  * the variants the Ablation Study compares it with (its table of norms).  The per-slot `vnorm`
  * arrays hold whichever kind the parameters name. */
 typedef enum { VATP_NORM_L1 = 0, VATP_NORM_L2 = 1, VATP_NORM_LINF = 2 } vatp_norm_kind;
+/* Bits of vatp_params.flags.  VATP_FLAG_DECODE_OVERLAP: see vatp_decode_step. */
+typedef enum { VATP_FLAG_DECODE_OVERLAP = 1 } vatp_flags;
 
 /* Problem description shared by the four calls (host struct). */
 typedef struct {
@@ -65,6 +67,7 @@ typedef struct {
   int32_t n_sink;            /* F: leading tokens always kept                                  */
   int32_t n_recent;          /* R: most recent tokens always kept; F + R <= B                  */
   int32_t norm_kind;         /* vatp_norm_kind of the value norm in Eq. 4; 0 = the paper's l1   */
+  int32_t flags;             /* OR of vatp_flags; 0 = none                                     */
   int64_t stride_b, stride_h, stride_t; /* element strides of q, k, v; 0 = contiguous          */
 } vatp_params;
 
@@ -199,6 +202,26 @@ vatp_status vatp_compact(const vatp_params* params, const void* k, const void* v
  * q_new, k_new, v_new: [batch, heads, head_dim]; out: same shape and dtype.
  * evicted_pos: [batch, heads] int32, nullable; position released this step or -1.
  * State arrays are updated in place.  seq_len in params is ignored.
+ *
+ * Ordering on the stream.  The step is enqueued as a launch that may begin while the work before it
+ * in the stream is still draining.  By default that is invisible: before anything else, the step only
+ * requests K/V cache tiles; it reads q_new, k_new, v_new and the state, and writes anything, only after
+ * all earlier work in the stream has completed, and it re-reads the one cache row the previous step
+ * appended.  The only assumption is about those early tile reads: between the compaction (or the
+ * previous step) and this step, cache rows are written by calls of this library only, or by kernels of
+ * the caller that do not release their dependents before they finish (ordinary launches do not).
+ *
+ * VATP_FLAG_DECODE_OVERLAP in params->flags opts in to more.  The library then keeps, per stream, the
+ * buffers of its recent decode launches; a step whose buffers (cache arrays, q_new, k_new, v_new, out,
+ * evicted_pos) overlap none of the launches that can still be running starts reading at once and runs
+ * beside them - steps of different layers' or sequences' caches issued back to back.  Steps that share a
+ * buffer with such a launch behave as in the default.  The caller then guarantees that every input of a
+ * flagged step was complete in memory before the previous vatp_decode_step on the stream was enqueued,
+ * or was written by an earlier vatp_decode_step; put differently: after enqueueing other work that
+ * produces a step's inputs, make the first step call without the flag.  Any other call of this library
+ * on the stream (prefill, selection, compaction) ends the record by itself.  Under stream capture the
+ * record is kept per capture, and the first step recorded into a graph always waits, so a replay is
+ * valid whatever ran before it.
  */
 vatp_status vatp_decode_step(const vatp_params* params, const vatp_cache* cache, const void* q_new,
                              const void* k_new, const void* v_new, void* out, int32_t* evicted_pos,
@@ -219,8 +242,10 @@ vatp_status vatp_selftest_bounded_wait(uint64_t limit_ns, int32_t* dev_status, u
  * (<= 13) host-described byte ranges [begin[i], begin[i] + bytes[i]) and keeps `share` of the
  * machine's CTA slots until the launch before it has completed.  Returns 1 when that launch would
  * run without waiting for its predecessors - it overlaps none of the recorded launches that can
- * still be resident - else 0, and records it; -1 on bad arguments.  `stream` is only a key (use
- * values no real stream has).  The paper has no counterpart.
+ * still be resident - else 0, and records it; -1 on bad arguments.  A negative `share` instead ends
+ * the stream's record, as every other call of this library on a stream does (the next launch then
+ * waits), and returns 0.  `stream` is only a key (use values no real stream has).  The launches
+ * probed here count as having opted in (VATP_FLAG_DECODE_OVERLAP).  The paper has no counterpart.
  */
 int32_t vatp_selftest_overlap_policy(void* stream, const uint64_t* begin, const uint64_t* bytes, int32_t n, double share);
 

@@ -107,12 +107,7 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            cudaStream_t st) {
   const int eb = dtype == VATP_F32 ? 4 : 2;
   const int cap = cache_capacity(B);
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
+  const int sms = device_sm_count();
   if ((int64_t)s.units * cap >= ((int64_t)1 << 32)) return cudaErrorInvalidValue;
   const int64_t steps = ((int64_t)s.units * cap + CP_ROWS - 1) / CP_ROWS;
   const int64_t wave = 4 * (int64_t)sms;        // four CTAs fit on an SM

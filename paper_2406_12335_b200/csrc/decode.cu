@@ -444,12 +444,13 @@ cudaError_t launch_t(const Shape& s, int B, int F, int R, const vatp_cache& c, c
 
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
                           const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status,
-                          cudaStream_t st) {
+                          cudaStream_t st, bool may_overlap) {
   const bool win = s.window > 0;
   if (dtype == VATP_BF16 && s.d == 128) {
-    const cudaError_t e = launch_decode_mma(s, B, F, R, c, q, k, v, out, evicted, dev_status, st);
+    const cudaError_t e = launch_decode_mma(s, B, F, R, c, q, k, v, out, evicted, dev_status, st, may_overlap);
     if (e != cudaErrorNotSupported) return e;
   }
+  decode_history_forget(st);     // the general kernel is an ordinary launch: the record of overlapping launches ends here
 #define VATP_DISPATCH(T, D)                                                                         \
   return win ? launch_t<T, D, true>(s, B, F, R, c, q, k, v, out, evicted, dev_status, st)           \
              : launch_t<T, D, false>(s, B, F, R, c, q, k, v, out, evicted, dev_status, st)

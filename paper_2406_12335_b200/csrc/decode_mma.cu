@@ -13,16 +13,18 @@
 //     needs (every logit, and per CTA the running max, sum and partial output) into rank 0's shared
 //     memory, meet at ONE cluster barrier and retire; rank 0 alone normalises, updates the
 //     indicators and finds the arg-min.  No global scratch, one launch;
-//   * consecutive steps overlap (programmatic dependent launch).  A control warp releases the next
-//     launch in the stream at once and then waits for the previous one, so launches complete in
-//     order and every CTA stays resident until its predecessor has completed: the number of
-//     launches in flight is bounded by what fits on the machine, and two CTAs fit on an SM.  The
-//     host keeps, per stream, the buffers of the last launches; a launch that shares no buffer with
-//     any launch that can still be in flight (another layer's or another sequence's cache) runs
-//     without waiting for anything.  Otherwise (same cache, or unknown) a step requests its first
-//     K/V tiles early and reads everything else only after the previous launch has completed; the
-//     one cache row that launch may have written - the row of its incoming token, recorded in
-//     last_slot - is re-read after that point and patched in.
+//   * consecutive steps overlap (programmatic dependent launch).  By default a step requests its
+//     first K/V tiles early and reads everything else only after all earlier work in the stream has
+//     completed; its control warp releases the next launch once that wait is over, so at most one
+//     unfinished predecessor exists while a step sets up, and the one cache row that predecessor
+//     may have written - the row of its incoming token, recorded in last_slot - is re-read after
+//     the wait and patched in.  A caller that steps several independent caches on one stream may
+//     opt in (VATP_FLAG_DECODE_OVERLAP) to more: the host keeps, per stream, the buffers of the
+//     last launches, and a launch that shares no buffer with any launch that can still be in
+//     flight (another layer's or another sequence's cache) never waits: its control warp releases
+//     the next launch at once and only holds the CTA until the previous launch has completed, so
+//     launches still complete in order and the number in flight is bounded by what fits on the
+//     machine (two CTAs fit on an SM).
 #include <cooperative_groups.h>
 
 #include <mutex>
@@ -183,8 +185,12 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     // (it arrives at the unit's barrier at once, so that the streaming warps never wait for it)
     if (split > 1) { cluster_wait_acquire(); cluster_arrive_release(); }
     if (lane == 0) {
-      asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+      // An independent launch lets its successor start at once.  A launch that waits for its
+      // predecessor releases its successor only after that wait: the successor's early tile
+      // requests then race with this launch alone, never with launches before it.
+      if (independent) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
       asm volatile("griddepcontrol.wait;" ::: "memory");
+      if (!independent) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
     __syncwarp();
     if (split > 1) cluster_wait_acquire();
@@ -541,6 +547,7 @@ struct LaunchRecord {
 };
 struct StreamHistory {
   cudaStream_t stream;
+  unsigned long long capture;   // 0: launches issued for execution; else the id of the stream capture that recorded them
   bool valid;
   int count, head;     // records held, index of the newest
   LaunchRecord rec[HIST];
@@ -553,23 +560,39 @@ inline bool overlaps(const Range& a, const Range& b) {
   return a.p && b.p && a.n && b.n && a.p < b.p + b.n && b.p < a.p + a.n;
 }
 
-// true when `touched` overlaps nothing that a launch possibly still in flight on `st` writes; records this launch
-bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, const Range* written, double share_if_indep,
-                               double share_if_not) {
-  std::lock_guard<std::mutex> lock(g_hist_mutex);
-  StreamHistory* h = nullptr;
+// Id of the capture `st` is recording into, 0 when it is not capturing.  Launches recorded into a graph
+// keep a history of their own: what was issued for execution before the capture says nothing about what
+// precedes a node when the graph is replayed, and the recorded launches are not in flight afterwards.
+unsigned long long capture_of(cudaStream_t st) {
+  cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+  unsigned long long id = 0;
+  if (cudaStreamGetCaptureInfo(st, &status, &id) != cudaSuccess) { cudaGetLastError(); return 0; }
+  return status == cudaStreamCaptureStatusActive ? (id ? id : ~0ull) : 0;
+}
+
+StreamHistory* history_of(cudaStream_t st, unsigned long long capture, bool create) {
   for (auto& x : g_hist)
-    if (x.valid && x.stream == st) h = &x;
-  if (!h) {
-    h = &g_hist[g_hist_next];
-    g_hist_next = (g_hist_next + 1) % 8;
-    h->stream = st;
-    h->valid = true;
-    h->count = 0;
-    h->head = -1;
-  }
-  // the first recorded launch followed a kernel that releases nothing early: everything before it had completed
-  bool indep = h->count > 0;
+    if (x.valid && x.stream == st && x.capture == capture) return &x;
+  if (!create) return nullptr;
+  StreamHistory* h = &g_hist[g_hist_next];
+  g_hist_next = (g_hist_next + 1) % 8;
+  h->stream = st;
+  h->capture = capture;
+  h->valid = true;
+  h->count = 0;
+  h->head = -1;
+  return h;
+}
+
+// True when `touched` overlaps nothing that a launch possibly still in flight on `st` writes; records this
+// launch.  may_overlap false (the caller did not opt in): records it and answers false.
+bool independent_of_in_flight(cudaStream_t st, unsigned long long capture, bool may_overlap, const Range* touched, int nt,
+                               const Range* written, double share_if_indep, double share_if_not) {
+  std::lock_guard<std::mutex> lock(g_hist_mutex);
+  StreamHistory* h = history_of(st, capture, true);
+  // The first recorded launch follows work this table knows nothing about (another kernel, the start of a
+  // graph): it waits, and by the time it lets its successor start everything before it has completed.
+  bool indep = may_overlap && h->count > 0;
   double between = 0.0;      // machine share of the launches between the candidate and this one
   for (int j = 0; indep && j < h->count && between < 1.0; ++j) {
     const LaunchRecord& r = h->rec[(h->head - j + HIST) % HIST];
@@ -595,21 +618,28 @@ bool independent_of_in_flight(cudaStream_t st, const Range* touched, int nt, con
 bool decode_overlap_policy_probe(void* stream, const uint64_t* begin, const uint64_t* bytes, int n, double share) {
   Range r[NRANGE] = {};
   for (int i = 0; i < n && i < NRANGE; ++i) r[i] = Range{reinterpret_cast<const char*>(begin[i]), (size_t)bytes[i]};
-  return independent_of_in_flight(static_cast<cudaStream_t>(stream), r, NRANGE, r, share, share);
+  return independent_of_in_flight(static_cast<cudaStream_t>(stream), 0, true, r, NRANGE, r, share, share);
+}
+
+// Any other work this library enqueues on `st` (prefill, selection, compaction, the general decode kernel)
+// ends the record: the decode launch after it waits for everything before it.
+void decode_history_forget(cudaStream_t st, bool probe_only) {
+  const unsigned long long capture = probe_only ? 0 : capture_of(st);
+  std::lock_guard<std::mutex> lock(g_hist_mutex);
+  if (StreamHistory* h = history_of(st, capture, false)) {
+    h->count = 0;
+    h->head = -1;
+  }
 }
 
 // Returns cudaErrorNotSupported when the shape does not fit this kernel's shared memory (the caller
 // then takes the general kernel).
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
-                              const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st) {
+                              const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
+                              bool may_overlap) {
   const int cap = cache_capacity(B);
   if (!vatp_tc_available()) return cudaErrorNotSupported;
-  static int sms = 0;
-  if (!sms) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) sms = 148;
-  }
+  const int sms = device_sm_count();
   // split a unit over a cluster while the grid still fits on the SMs once (a second launch can then be resident too)
   int split = 1;
   while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
@@ -673,7 +703,8 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, MT, p.dyn) != cudaSuccess || occ < 1) occ = 1;
     return (double)(s.units * split) / ((double)occ * sms);
   };
-  const int independent = independent_of_in_flight(st, written, 16, written, share_of(beside), share_of(lone)) ? 1 : 0;
+  const int independent =
+      independent_of_in_flight(st, capture_of(st), may_overlap, written, 16, written, share_of(beside), share_of(lone)) ? 1 : 0;
   const Plan& pl = independent ? beside : lone;
   const int nstage = pl.nstage, state_in_smem = pl.state_in_smem;
   const size_t dyn = pl.dyn;

@@ -23,6 +23,8 @@
 // word, drains, frees its TMEM and returns.
 #include <cuda.h>
 
+#include <mutex>
+
 #include "vatp_internal.cuh"
 
 namespace vatp {
@@ -851,16 +853,33 @@ bool make_rows_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint32_
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool vatp_tc_available() {
-  static int cached = -1;
-  if (cached < 0) {
-    int dev = 0, major = 0;
-    cached = cudaGetDevice(&dev) == cudaSuccess &&
-             cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10 &&
-             encode_fn() != nullptr;
+// Per-device facts, looked up on first use with that device current (a process may drive several GPUs).
+namespace {
+constexpr int kMaxDevices = 64;
+struct DeviceFacts {
+  int known, tc, sms;
+};
+DeviceFacts g_facts[kMaxDevices];
+std::mutex g_facts_mutex;
+
+DeviceFacts device_facts() {
+  int dev = 0;
+  DeviceFacts f{1, 0, 148};
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return f;
+  std::lock_guard<std::mutex> lock(g_facts_mutex);
+  if (!g_facts[dev].known) {
+    int major = 0, sms = 0;
+    f.tc = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) == cudaSuccess && major == 10 &&
+           encode_fn() != nullptr;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0) f.sms = sms;
+    g_facts[dev] = f;
   }
-  return cached == 1;
+  return g_facts[dev];
 }
+}  // namespace
+
+bool vatp_tc_available() { return device_facts().tc == 1; }
+int device_sm_count() { return device_facts().sms; }
 
 size_t prefill_tc_workspace_bytes(int units, int T) {
   const size_t Tpad = (size_t)(T + CHUNK - 1) / CHUNK * CHUNK;
@@ -905,9 +924,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   if ((e = cudaFuncSetAttribute(prefill_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = device_sm_count();
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
   if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
   a.side_norm = a.ft == 0 && a.norm == VATP_NORM_L1 && !lse_in;   // the side warp belongs to pass 1

@@ -40,6 +40,10 @@ __global__ void bounded_wait_kernel(unsigned long long limit_ns, int32_t* dev_st
 
 extern "C" int32_t vatp_selftest_overlap_policy(void* stream, const uint64_t* begin, const uint64_t* bytes, int32_t n,
                                                 double share) {
+  if (share < 0.0) {        // what any other call of the library on the stream does to the record
+    vatp::decode_history_forget(static_cast<cudaStream_t>(stream), true);
+    return 0;
+  }
   if (!begin || !bytes || n <= 0) return -1;
   return vatp::decode_overlap_policy_probe(stream, begin, bytes, n, share) ? 1 : 0;
 }

@@ -22,6 +22,7 @@ vatp_status check_params(const vatp_params* p, bool need_T) {
   if ((int64_t)p->n_sink + p->n_recent > p->budget) return VATP_ERR_INVALID_ARG;
   if (!(p->scale > 0.f)) return VATP_ERR_INVALID_ARG;
   if (p->stride_b < 0 || p->stride_h < 0 || p->stride_t < 0) return VATP_ERR_INVALID_ARG;
+  if (p->flags & ~(int32_t)VATP_FLAG_DECODE_OVERLAP) return VATP_ERR_INVALID_ARG;
   return VATP_OK;
 }
 
@@ -75,6 +76,7 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
     return VATP_ERR_WORKSPACE;
   float* ws = static_cast<float*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  decode_history_forget(st);
   cudaError_t e;
   if (p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available()) {
     e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st, lse_in);
@@ -135,6 +137,7 @@ vatp_status vatp_select(const vatp_params* p, const float* score, int32_t* kept_
   vatp_status s = check_params(p, true);
   if (s != VATP_OK) return s;
   if (!score || !kept_idx) return VATP_ERR_INVALID_ARG;
+  decode_history_forget(static_cast<cudaStream_t>(cuda_stream));
   cudaError_t e = launch_select(p->batch * p->heads, p->seq_len, p->budget, p->n_sink, p->n_recent, score, kept_idx,
                                 static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
@@ -153,6 +156,7 @@ vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, con
   Shape sh;
   s = make_shape(p, &sh);
   if (s != VATP_OK) return s;
+  decode_history_forget(static_cast<cudaStream_t>(cuda_stream));
   cudaError_t e = launch_compact(sh, p->dtype, p->budget, k, v, attn_acc, vnorm, win_rows, kept_idx, *cache,
                                  static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
@@ -175,7 +179,8 @@ vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, cons
   sh.window = windowed ? p->window_w : 0;
   sh.norm = p->norm_kind;
   cudaError_t e = launch_decode(sh, p->dtype, p->budget, p->n_sink, p->n_recent, *cache, q_new, k_new, v_new, out,
-                                evicted_pos, dev_status, static_cast<cudaStream_t>(cuda_stream));
+                                evicted_pos, dev_status, static_cast<cudaStream_t>(cuda_stream),
+                                (p->flags & VATP_FLAG_DECODE_OVERLAP) != 0);
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
 

@@ -40,8 +40,10 @@ __host__ __device__ inline int64_t unit_offset(const Shape& s, int u) {
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 
-// true once the tensor-core prefill kernel is usable on the current device (sm_100, driver entry points found)
+// true when the tensor-core kernels are usable on the current device (sm_100, driver entry points found)
 bool vatp_tc_available();
+// multiprocessors of the current device (looked up once per device)
+int device_sm_count();
 
 // 2-D tensor map over `rows` contiguous rows of 128 bf16: box = 64 columns x box_rows rows, 128-byte
 // swizzle, rows beyond the end read as zeros.  False when the driver entry point is missing.
@@ -80,11 +82,18 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
                            cudaStream_t st);
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
-                          const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st);
+                          const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
+                          bool may_overlap);
 
 // bf16, head_dim 128 only; cudaErrorNotSupported when the shape does not fit (take launch_decode's general kernel)
+// may_overlap: the caller opted in to launches that run beside earlier decode launches on the stream when they share
+// no buffer with them (VATP_FLAG_DECODE_OVERLAP)
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
-                              const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st);
+                              const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
+                              bool may_overlap);
+// other work of this library was enqueued on the stream: the next decode launch waits for all of it
+// (probe_only: `st` is only a key of the host-side self-test, not a stream the runtime may be asked about)
+void decode_history_forget(cudaStream_t st, bool probe_only = false);
 
 bool decode_overlap_policy_probe(void* stream, const uint64_t* begin, const uint64_t* bytes, int n, double share);
 

@@ -19,6 +19,7 @@ OK = 0
 BF16, F32 = 0, 1
 IND_H2O, IND_WINDOW = 0, 1
 NORM_KINDS = {"l1": 0, "l2": 1, "linf": 2}
+FLAG_DECODE_OVERLAP = 1
 STATIC_SCRATCH_BYTES = (4 << 20) + 256
 EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_from_lse", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
            "vatp_selftest_bounded_wait", "vatp_selftest_overlap_policy", "vatp_status_string"]
@@ -28,7 +29,7 @@ class Params(C.Structure):
     _fields_ = [("batch", C.c_int32), ("heads", C.c_int32), ("seq_len", C.c_int32), ("head_dim", C.c_int32),
                 ("dtype", C.c_int32), ("indicator", C.c_int32), ("window_w", C.c_int32), ("scale", C.c_float),
                 ("budget", C.c_int32), ("n_sink", C.c_int32), ("n_recent", C.c_int32), ("norm_kind", C.c_int32),
-                ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
+                ("flags", C.c_int32), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
 
 
 class CacheStruct(C.Structure):
@@ -83,11 +84,14 @@ def _stream(stream=None):
 
 
 def make_params(*, batch, heads, seq_len, head_dim, dtype, budget, n_sink=0, n_recent=0, scale=None,
-                indicator="h2o", window=0, strides=(0, 0, 0), norm="l1") -> Params:
-    """norm: the value norm of Eq. 4, "l1" (the method) or the Ablation Study's "l2" / "linf"."""
+                indicator="h2o", window=0, strides=(0, 0, 0), norm="l1", decode_overlap=False) -> Params:
+    """norm: the value norm of Eq. 4, "l1" (the method) or the Ablation Study's "l2" / "linf".
+    decode_overlap: sets VATP_FLAG_DECODE_OVERLAP (decode steps of independent caches may run side by side;
+    see vatp_decode_step in include/vatp.h for what the caller then guarantees)."""
     dt = {torch.bfloat16: BF16, torch.float32: F32, "bf16": BF16, "f32": F32}[dtype]
     return Params(batch, heads, seq_len, head_dim, dt, IND_WINDOW if indicator == "window" else IND_H2O, window,
-                  float(scale if scale is not None else head_dim ** -0.5), budget, n_sink, n_recent, NORM_KINDS[norm], *strides)
+                  float(scale if scale is not None else head_dim ** -0.5), budget, n_sink, n_recent, NORM_KINDS[norm],
+                  FLAG_DECODE_OVERLAP if decode_overlap else 0, *strides)
 
 
 def params_for(x: torch.Tensor, **kw) -> Params:

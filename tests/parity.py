@@ -39,7 +39,9 @@ def attention_forward_lse(q: torch.Tensor, k: torch.Tensor, scale: float) -> tor
 class GpuPrefill:
     """Device buffers and the three prefill-side calls for one layer of a workload."""
 
-    def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None, lse_given=False):
+    def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None, lse_given=False, decode_overlap=False):
+        """decode_overlap: decode steps through this object carry VATP_FLAG_DECODE_OVERLAP (steps of
+        caches that share no buffer may run side by side on the GPU)."""
         V = vatp()
         self.wl = wl
         self.lse_given = lse_given
@@ -48,7 +50,7 @@ class GpuPrefill:
         b, h, T = wl.batch, wl.heads, wl.seq_len
         self.q, self.k, self.v = q, k, v
         self.p = V.params_for(q, budget=wl.budget, n_sink=self.F, n_recent=wl.n_recent, scale=wl.scale,
-                              indicator=wl.indicator, window=wl.window, norm=wl.norm)
+                              indicator=wl.indicator, window=wl.window, norm=wl.norm, decode_overlap=decode_overlap)
         f32 = dict(dtype=torch.float32, device=dev)
         self.lse = torch.empty(b, h, T, **f32)
         self.attn_acc = torch.empty(b, h, T, **f32)

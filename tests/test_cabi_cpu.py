@@ -27,8 +27,8 @@ def test_exports_every_declared_symbol(V):
 
 
 def test_struct_layout_matches_header(V):
-    assert C.sizeof(V.Params) == 72       # 7 int32 + float + 3 int32 + pad + 3 int64
-    assert V.Params.stride_b.offset == 48
+    assert C.sizeof(V.Params) == 80       # 7 int32 + float + 5 int32 + pad + 3 int64
+    assert V.Params.norm_kind.offset == 44 and V.Params.flags.offset == 48 and V.Params.stride_b.offset == 56
     assert C.sizeof(V.CacheStruct) == 88
 
 
@@ -68,15 +68,20 @@ def test_host_side_validation(V):
     assert V.lib.vatp_prefill_scores(C.byref(sp), 16, 16, 16, 16, 16, 16, 16, null, null, 0, null, null) == 1
     # decode: null cache
     assert V.lib.vatp_decode_step(C.byref(p), null, 16, 16, 16, 16, null, null, null) == 1
-    # value norm kinds: l1 / l2 / linf are accepted, anything else is unsupported; the field fills what
-    # used to be padding before the 64-bit strides, so the struct keeps its size
-    assert C.sizeof(V.Params) == 72 and V.Params.norm_kind.offset == 44 and V.Params.stride_b.offset == 48
+    # value norm kinds: l1 / l2 / linf are accepted, anything else is unsupported
     for kind in ("l1", "l2", "linf"):
         assert V.vatp_workspace_bytes(V.make_params(**ok, norm=kind)) == 2048 + 256
     odd = V.make_params(**ok)
     odd.norm_kind = 3
     assert V.vatp_workspace_bytes(odd) == 0
     assert V.lib.vatp_select(C.byref(odd), 16, 16, null, 0, null, null) == 2
+    # flags: the decode-overlap bit is the only one defined
+    assert V.make_params(**ok, decode_overlap=True).flags == V.FLAG_DECODE_OVERLAP == 1
+    assert V.vatp_workspace_bytes(V.make_params(**ok, decode_overlap=True)) == 2048 + 256
+    odd = V.make_params(**ok)
+    odd.flags = 6
+    assert V.vatp_workspace_bytes(odd) == 0
+    assert V.lib.vatp_decode_step(C.byref(odd), null, 16, 16, 16, 16, null, null, null) == 1
 
 
 def _probe(V, stream, caches, share):
@@ -116,3 +121,9 @@ def test_decode_overlap_policy(V):
     # streams do not see each other's launches
     assert _probe(V, 0xA005, cache(0), 0.43) == 0 and _probe(V, 0xA005, cache(1), 0.43) == 1
     assert _probe(V, 0xA005, [], 0.5) == -1
+    # other work of the library on the stream (prefill, selection, compaction) ends the record: the next
+    # launch waits whatever it touches, the ones after it are judged against it alone
+    s = 0xA006
+    assert [_probe(V, s, cache(i), 0.43) for i in range(4)] == [0, 1, 1, 1]
+    assert _probe(V, s, cache(0), -1.0) == 0
+    assert [_probe(V, s, cache(i), 0.43) for i in (7, 8, 7)] == [0, 1, 0]

@@ -161,17 +161,18 @@ def test_config4_long_context_layer():
     _run_case(synth.CONFIGS[4], units=[(0, 5)], check_state_every=32, layer=31)
 
 
-def _interleaved_equals_alone(wls, steps):
+def _interleaved_equals_alone(wls, steps, overlap=True):
     """Steps the caches of `wls` (a) one after the other, each alone with a synchronisation after every
-    step, and (b) round robin with no synchronisation; outputs, evictions and final state must be equal
-    bit for bit.  Returns a function that prefills fresh caches and the decode inputs."""
+    step, and (b) round robin with no synchronisation (with `overlap`, carrying the flag that lets steps
+    of independent caches run side by side); outputs, evictions and final state must be equal bit for
+    bit.  Returns a function that prefills fresh caches and the decode inputs."""
     V = P.vatp()
 
-    def prefilled():
+    def prefilled(decode_overlap=False):
         gs = []
         for wl in wls:
             q, k, v = synth.prefill_inputs(wl, 0, "cuda")
-            gs.append(P.GpuPrefill(wl, q, k, v).run())
+            gs.append(P.GpuPrefill(wl, q, k, v, decode_overlap=decode_overlap).run())
         return gs
 
     ins = [synth.decode_inputs(wl, 0, device="cuda") for wl in wls]
@@ -182,7 +183,7 @@ def _interleaved_equals_alone(wls, steps):
         for s in range(steps):
             V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
             torch.cuda.synchronize()
-    inter = prefilled()
+    inter = prefilled(decode_overlap=overlap)
     outs_b = [torch.empty_like(o) for o in outs_a]
     evs_b = [torch.empty_like(e) for e in evs_a]
     for s in range(steps):
@@ -197,8 +198,9 @@ def _interleaved_equals_alone(wls, steps):
     return prefilled, ins
 
 
+@pytest.mark.parametrize("overlap", [True, False])
 @pytest.mark.parametrize("b,h", [(1, 3), (5, 32)])
-def test_interleaved_caches_match_separate_runs(b, h):
+def test_interleaved_caches_match_separate_runs(b, h, overlap):
     """Decode steps of three independent caches issued back to back on one stream (launches that share
     no buffer may overlap on the GPU) give bit for bit what each cache gives when stepped alone, and
     the result agrees with the oracle.  With 3 units per cache every launch could still be in flight
@@ -206,7 +208,7 @@ def test_interleaved_caches_match_separate_runs(b, h):
     fills half the machine and the steps of different caches run side by side."""
     steps = 12
     wls = [_small("bf16", 128, 900, 300, 2, 30, b=b, h=h, steps=steps, cid=70 + i) for i in range(3)]
-    prefilled, ins = _interleaved_equals_alone(wls, steps)
+    prefilled, ins = _interleaved_equals_alone(wls, steps, overlap)
     # (c) and the trajectory of some units of one cache against the oracle
     g = prefilled()[1]
     units = [(0, 0), (b - 1, h - 1), (b // 2, h // 2)]
@@ -333,52 +335,96 @@ def test_expired_device_wait_reports_timeout_and_context_survives():
     _run_case(_small("bf16", 128, 300, 100, 2, 10, steps=3, cid=63))  # the context is intact
 
 
-def test_config1_layers_interleaved_in_a_graph_match_stepping_alone():
-    """The launch configuration the benchmark times: several independently seeded config-1 layers, their
-    decode steps interleaved and replayed from a CUDA graph (consecutive launches overlap on the GPU).
-    Outputs, evictions and final state must equal, bit for bit, each layer stepped alone with a
-    synchronisation after every step."""
+def _graphs_equal_stepping_alone(wls, plan, *, overlap, eager_first=0, replays=1, oracle_unit=None, layers=None):
+    """Decode steps recorded into a CUDA graph against the same steps issued one by one with a
+    synchronisation after each.  plan: list of (cache index, step index) in issue order; the first
+    `eager_first` entries are issued directly (not captured), the rest are captured once and the graph is
+    replayed `replays` times back to back (every replay repeats the same steps on the advancing caches and
+    overwrites the same output rows, which the reference arm does too).  Outputs, evictions and the final state must be equal bit for bit.  With oracle_unit =
+    (cache, b, h) that unit's trajectory of the reference arm is also checked against the oracle."""
     V = P.vatp()
-    wl = synth.CONFIGS[1].with_(decode_steps=12)
-    L, steps = 3, wl.decode_steps
+    layers = layers or [0] * len(wls)
 
-    def prefilled():
+    def prefilled(decode_overlap):
         gs = []
-        for layer in range(L):
+        for wl, layer in zip(wls, layers):
             q, k, v = synth.prefill_inputs(wl, layer, "cuda")
-            gs.append(P.GpuPrefill(wl, q, k, v).run())
+            gs.append(P.GpuPrefill(wl, q, k, v, decode_overlap=decode_overlap).run())
         return gs
 
-    ins = [synth.decode_inputs(wl, layer, device="cuda") for layer in range(L)]
-    shape = (steps, wl.batch, wl.heads, wl.head_dim)
-    alone = prefilled()
-    outs_a = [torch.empty(shape, dtype=torch.bfloat16, device="cuda") for _ in range(L)]
-    evs_a = [torch.empty(shape[:3], dtype=torch.int32, device="cuda") for _ in range(L)]
-    for g, (dq, dk, dv), o, e in zip(alone, ins, outs_a, evs_a):
-        for s in range(steps):
-            V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
+    ins = [synth.decode_inputs(wl, layer, device="cuda") for wl, layer in zip(wls, layers)]
+    nsteps = max(s for _, s in plan) + 1
+    mk = lambda dt, tail: [torch.zeros((2, nsteps, wl.batch, wl.heads) + tail(wl), dtype=dt, device="cuda") for wl in wls]
+    outs_a, outs_b = mk(torch.bfloat16, lambda wl: (wl.head_dim,)), mk(torch.bfloat16, lambda wl: (wl.head_dim,))
+    evs_a, evs_b = mk(torch.int32, lambda wl: ()), mk(torch.int32, lambda wl: ())
+
+    def issue(gs, outs, evs, entries, rep):
+        for ci, s in entries:
+            g, (dq, dk, dv) = gs[ci], ins[ci]
+            V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], outs[ci][rep, s], evicted_pos=evs[ci][rep, s], dev_status=g.status)
+
+    # reference arm: one by one, no flag
+    alone = prefilled(False)
+    for rep, entries in enumerate([plan[:eager_first]] + [plan[eager_first:]] * replays):
+        for e in entries:
+            issue(alone, outs_a, evs_a, [e], min(rep, 1))
             torch.cuda.synchronize()
-    inter = prefilled()
-    outs_b = [torch.empty_like(o) for o in outs_a]
-    evs_b = [torch.empty_like(e) for e in evs_a]
-
-    def all_steps(first, last):
-        for s in range(first, last):
-            for g, (dq, dk, dv), o, e in zip(inter, ins, outs_b, evs_b):
-                V.vatp_decode_step(g.p, g.cache, dq[s], dk[s], dv[s], o[s], evicted_pos=e[s], dev_status=g.status)
-
-    all_steps(0, 2)                     # first calls outside the capture
-    torch.cuda.synchronize()
+    # graph arm
+    inter = prefilled(overlap)
+    issue(inter, outs_b, evs_b, plan[:eager_first], 0)
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        all_steps(2, steps)
-    graph.replay()
+        issue(inter, outs_b, evs_b, plan[eager_first:], 1)
+    for _ in range(replays):
+        graph.replay()
     torch.cuda.synchronize()
     for ga, gb, oa, ob, ea, eb in zip(alone, inter, outs_a, outs_b, evs_a, evs_b):
-        assert int(gb.status.item()) == 0
+        assert int(ga.status.item()) == 0 and int(gb.status.item()) == 0
         assert torch.equal(oa, ob) and torch.equal(ea, eb)
         for name in ("k_cache", "v_cache", "acc", "vnorm", "pos", "len", "free_slot", "next_pos"):
             assert torch.equal(getattr(ga.cache, name), getattr(gb.cache, name)), name
+    if oracle_unit is not None:
+        ci, b, h = oracle_unit
+        g = prefilled(False)[ci]
+        ref, kept, _ = P.check_prefill_unit(g, b, h, P.TOL["bf16"])
+        order = [s for c, s in plan[:eager_first] if c == ci] + [s for c, s in plan[eager_first:] if c == ci] * replays
+        dq, dk, dv = (x[order] for x in ins[ci])
+        P.run_decode_and_check(g, {(b, h): (ref, kept)}, dq, dk, dv, len(order), P.TOL["bf16"], check_state_every=4)
+
+
+@pytest.mark.parametrize("overlap", [True, False])
+@pytest.mark.parametrize("h", [3, 8])
+def test_same_cache_steps_in_a_graph_with_few_units(h, overlap):
+    """One small cache (3 or 8 units: grids of a few dozen CTAs, so that many launches fit on the machine
+    together) stepped 24 times from a graph: every step depends on the one before it, and a step may only
+    ever run ahead of ONE unfinished predecessor, whose appended row it re-reads."""
+    wl = _small("bf16", 128, 900, 300, 2, 30, b=1, h=h, steps=24, cid=71)
+    plan = [(0, s) for s in range(24)]
+    _graphs_equal_stepping_alone([wl], plan, overlap=overlap, eager_first=2, oracle_unit=(0, 0, h - 1))
+
+
+@pytest.mark.parametrize("eager_first", [0, 7])
+@pytest.mark.parametrize("ncaches", [2, 5])
+def test_graph_of_independent_caches_replayed_back_to_back(ncaches, eager_first):
+    """Graphs [A, B] and [A .. E] of steps of independent caches (overlap flag set), captured cold
+    (eager_first = 0) or after unrelated steps issued directly, replayed three times back to back.
+    Whatever preceded a replay - the previous replay's tail included - the result must be that of
+    stepping one by one."""
+    wls = [_small("bf16", 128, 900, 300, 2, 30, b=2, h=32, steps=8, cid=72 + i) for i in range(ncaches)]
+    pre = [(c, 0) for c in range(ncaches)] * 4
+    plan = pre[:eager_first] + [(c, 1) for c in range(ncaches)]
+    _graphs_equal_stepping_alone(wls, plan, overlap=True, eager_first=eager_first, replays=3, oracle_unit=(1, 1, 31))
+
+
+def test_config1_layers_interleaved_in_a_graph_match_stepping_alone():
+    """The launch configuration the benchmark times: eight independently seeded config-1 layers, their
+    decode steps interleaved with the overlap flag set and replayed from a CUDA graph (consecutive
+    launches run side by side on the GPU).  Outputs, evictions and final state must equal, bit for bit,
+    each layer stepped alone with a synchronisation after every step."""
+    wl = synth.CONFIGS[1].with_(decode_steps=6)
+    L = 8
+    plan = [(l, s) for s in range(wl.decode_steps) for l in range(L)]
+    _graphs_equal_stepping_alone([wl] * L, plan, overlap=True, eager_first=2 * L, layers=list(range(L)))
 
 
 @pytest.mark.parametrize("dtype,d", [("bf16", 128), ("f32", 64)])
