@@ -9,10 +9,11 @@
 //     accumulate): S^T = q K^T leaves the probabilities of 16 rows in exactly the registers the
 //     A operand of p V wants, so a 16-row group costs about 80 instructions.  p is split into two
 //     bf16 halves (rows 0-7 / 8-15 of the A tile carry hi / lo): the product keeps ~16 bits of p;
-//   * a unit is split over a thread-block cluster when units are few.  The CTAs PUSH what rank 0
-//     needs (every logit, and per CTA the running max, sum and partial output) into rank 0's shared
-//     memory, meet at ONE cluster barrier and retire; rank 0 alone normalises, updates the
-//     indicators and finds the arg-min.  No global scratch, one launch;
+//   * a unit is split over a thread-block cluster when units are few.  Every CTA PUSHES its running
+//     max and sum into the shared memory of all CTAs of the unit and its partial output into rank
+//     0's; after one cluster barrier each CTA knows the softmax normaliser, updates the indicators of
+//     its own slots and proposes its own eviction candidate to rank 0; after a second barrier rank 0
+//     picks the candidate of the whole unit.  No global scratch, one launch;
 //   * consecutive steps overlap (programmatic dependent launch).  By default a step requests its
 //     first K/V tiles early and reads everything else only after all earlier work in the stream has
 //     completed; its control warp releases the next launch once that wait is over, so at most one
@@ -122,10 +123,12 @@ __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" 
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 
-// what the CTAs of a unit push into rank 0
+// what the CTAs of a unit push into one another
 struct Exch {
-  float m[MAX_SPLIT], l[MAX_SPLIT];       // per rank: max of its logits (log2 domain), sum of exp2(s - m)
-  float o[MAX_SPLIT][HD];                 // partial outputs of every rank
+  float m[MAX_SPLIT], l[MAX_SPLIT];       // in every rank: per rank the max of its logits (log2 domain) and the sum of exp2(s - m)
+  float o[MAX_SPLIT][HD];                 // in rank 0: partial outputs of every rank
+  unsigned long long key[MAX_SPLIT];      // in rank 0: every rank's eviction candidate (NO_KEY: none) ...
+  int key_slot[MAX_SPLIT], key_pos[MAX_SPLIT];   // ... its slot in the unit and its position
 };
 
 static_assert(WT == HD, "one streaming thread per output channel");
@@ -152,23 +155,23 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
   extern __shared__ unsigned char dyn_raw[];
   unsigned char* dyn = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dyn_raw) + 1023) & ~uintptr_t(1023));
-  // [MW][nstage] stages | logits[tot] | acc[tot] | vnorm[tot] | pos[tot]; the per-slot arrays span the
-  // whole unit and are used by rank 0 only.  For large caches only the logits are held here, which keeps
-  // the CTA small enough for two launches to be resident together; acc, vnorm and pos are then copied
-  // into the stage memory once the streaming is over (state_in_smem == 2) or, if even that is too
-  // small, read from global memory in the tail (state_in_smem == 0).
-  const int tot = split * chunk;
+  // [MW][nstage] stages | logits[chunk] | acc[chunk] | vnorm[chunk] | pos[chunk]: the per-slot arrays of
+  // this CTA's own slots.  For large caches only the logits are held here, which keeps the CTA small
+  // enough for two launches to be resident together; acc, vnorm and pos are then copied into the stage
+  // memory once the streaming is over (state_in_smem == 2) or, if even that is too small, read from
+  // global memory in the tail (state_in_smem == 0).
   unsigned char* stage_base = dyn;
   float* logit_s = reinterpret_cast<float*>(dyn + (size_t)MW * nstage * STAGE_BYTES);
-  float* acc_s = state_in_smem == 2 ? reinterpret_cast<float*>(stage_base) : logit_s + tot;
-  float* vn_s = acc_s + (state_in_smem == 2 ? cap : tot);
-  int* pos_s = reinterpret_cast<int*>(vn_s + (state_in_smem == 2 ? cap : tot));
+  float* acc_s = state_in_smem == 2 ? reinterpret_cast<float*>(stage_base) : logit_s + chunk;
+  float* vn_s = acc_s + chunk;
+  int* pos_s = reinterpret_cast<int*>(vn_s + chunk);
 
   __shared__ __align__(8) uint64_t bars[MW * 4 + 1];
   __shared__ __align__(16) Exch ex;
   __shared__ __align__(16) float part_o[MW][HD];
   __shared__ float part_m[MW], part_l[MW];
   __shared__ unsigned long long warp_key[MW];
+  __shared__ int ctrl_evicting;
 
   cg::cluster_group cluster = cg::this_cluster();
   const int rank = split > 1 ? (int)cluster.block_rank() : 0;
@@ -183,6 +186,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   if (wid == MW) {
     // ---- control warp: release the next launch, then hold this CTA until the previous launch has completed
     // (it arrives at the unit's barrier at once, so that the streaming warps never wait for it)
+    // (its arrivals at the unit's two barriers come as early as the barrier's phases allow)
     if (split > 1) { cluster_wait_acquire(); cluster_arrive_release(); }
     if (lane == 0) {
       // An independent launch lets its successor start at once.  A launch that waits for its
@@ -193,7 +197,11 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       if (!independent) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     }
     __syncwarp();
-    if (split > 1) cluster_wait_acquire();
+    if (split > 1) {
+      cluster_wait_acquire();
+      // a second barrier follows when the step evicts (the streaming warps have published that by now)
+      if (*reinterpret_cast<volatile int*>(&ctrl_evicting)) { cluster_arrive_release(); cluster_wait_acquire(); }
+    }
     return;
   }
 
@@ -226,17 +234,17 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   // The next launch in the stream may start now; nothing below this line is read before the previous
   // launch has completed and its writes are visible.
   if (!independent) asm volatile("griddepcontrol.wait;" ::: "memory");
-  if (rank == 0 && tid == 32) {      // per-slot state of the whole unit
-    const int64_t o = (int64_t)u * cap;
+  if (tid == 32 && rows_alloc > 0) {      // per-slot state of this CTA's slots
+    const int64_t o = (int64_t)u * cap + s0;
     if (state_in_smem == 1) {
-      mbar_expect_tx(state_bar, 3u * cap * 4u);
-      bulk_g2s(acc_s, c.acc + o, cap * 4, state_bar);
-      bulk_g2s(vn_s, c.vnorm + o, cap * 4, state_bar);
-      bulk_g2s(pos_s, c.pos + o, cap * 4, state_bar);
+      mbar_expect_tx(state_bar, 3u * rows_alloc * 4u);
+      bulk_g2s(acc_s, c.acc + o, rows_alloc * 4, state_bar);
+      bulk_g2s(vn_s, c.vnorm + o, rows_alloc * 4, state_bar);
+      bulk_g2s(pos_s, c.pos + o, rows_alloc * 4, state_bar);
     } else if (state_in_smem == 0) {
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.acc + o), "r"(cap * 4) : "memory");
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.vnorm + o), "r"(cap * 4) : "memory");
-      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.pos + o), "r"(cap * 4) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.acc + o), "r"(rows_alloc * 4) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.vnorm + o), "r"(rows_alloc * 4) : "memory");
+      asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.pos + o), "r"(rows_alloc * 4) : "memory");
     }
   }
 
@@ -248,11 +256,12 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int cnt = max(min(hi - s0, rows_alloc), 0);
   const int fs_local = fs - s0;          // row of the incoming token inside this CTA's range (if owned)
   const bool owns_new = fs_local >= 0 && fs_local < cnt;
-  if (WINDOWED && rank == 0 && tid == 64) {
+  if (WINDOWED && tid == 64 && rows_alloc > 0) {
     // the tail reads the ring row that leaves the window and the exact sums: have them in L2 by then
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.ring + ((int64_t)u * w + (t % w)) * cap), "r"(cap * 4) : "memory");
-    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.acc_fixed + (int64_t)u * cap), "r"(cap * 8) : "memory");
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.ring + ((int64_t)u * w + (t % w)) * cap + s0), "r"(rows_alloc * 4) : "memory");
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(c.acc_fixed + (int64_t)u * cap + s0), "r"(rows_alloc * 8) : "memory");
   }
+  if (tid == 0) ctrl_evicting = hi > B ? 1 : 0;     // read by the control warp after the first barrier
   const int ls_local = ls - s0;          // row the previous step appended (its tile may predate that store)
   const bool owns_last = !independent && ls >= 0 && ls != fs && ls_local >= 0 && ls_local < cnt;
 
@@ -292,7 +301,6 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     }
   }
   if (split > 1) cluster_wait_acquire();
-  float* logit_r0 = split > 1 ? cluster.map_shared_rank(logit_s, 0) : logit_s;
 
   // ---- stream the groups: logits, online softmax, partial output ----
   float m_run = -INFINITY, l_run = 0.f;
@@ -355,7 +363,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       if (lane < 4) {
 #pragma unroll
         for (int i = 0; i < 4; ++i)
-          if (rows[i] < cnt) logit_r0[s0 + rows[i]] = s[i];
+          if (rows[i] < cnt) logit_s[rows[i]] = s[i];
       }
       float gmax = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
       gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
@@ -405,18 +413,18 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (lane == 0) { part_m[wid] = m_run; part_l[wid] = l_run; }
   }
   workers_sync();
-  if (state_in_smem == 2 && rank == 0 && tid == 32) {
-    // every stage of this CTA has been consumed: the per-slot state of the unit lands there while the
+  if (state_in_smem == 2 && tid == 32 && rows_alloc > 0) {
+    // every stage of this CTA has been consumed: the per-slot state of its slots lands there while the
     // cluster gathers (the stages were last written by bulk copies and read by ldmatrix; warps that
     // stored into them have fenced)
-    const int64_t o = (int64_t)u * cap;
-    mbar_expect_tx(state_bar, 3u * cap * 4u);
-    bulk_g2s(acc_s, c.acc + o, cap * 4, state_bar);
-    bulk_g2s(vn_s, c.vnorm + o, cap * 4, state_bar);
-    bulk_g2s(pos_s, c.pos + o, cap * 4, state_bar);
+    const int64_t o = (int64_t)u * cap + s0;
+    mbar_expect_tx(state_bar, 3u * rows_alloc * 4u);
+    bulk_g2s(acc_s, c.acc + o, rows_alloc * 4, state_bar);
+    bulk_g2s(vn_s, c.vnorm + o, rows_alloc * 4, state_bar);
+    bulk_g2s(pos_s, c.pos + o, rows_alloc * 4, state_bar);
   }
 
-  // ---- CTA partial, pushed into rank 0 ----
+  // ---- CTA partial: max and sum to every CTA of the unit, partial output to rank 0 ----
   {
     float m_c = -INFINITY;
 #pragma unroll
@@ -434,15 +442,15 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       for (int i = 0; i < MW; ++i) a = fmaf(part_o[i][tid], fw[i], a);
       e0->o[rank][tid] = a;
     }
-    if (tid == 0) {
-      e0->m[rank] = m_c;
-      e0->l[rank] = l_c;
+    if (tid < split) {
+      Exch* er = split > 1 ? cluster.map_shared_rank(&ex, tid) : &ex;
+      er->m[rank] = m_c;
+      er->l[rank] = l_c;
     }
   }
   if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync();
-  if (rank != 0) return;      // nothing of this CTA's shared memory is read by others
 
-  // ---- rank 0: combine the CTAs of the unit (all data is local now) ----
+  // ---- every CTA: the unit's softmax normaliser (all data is local now) ----
   float m_all = -INFINITY, L = 0.f;
   float fr[MAX_SPLIT];
 #pragma unroll
@@ -454,7 +462,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (r < split) L += ex.l[r] * fr[r];
   }
   const float invL = 1.f / L;
-  if (tid < HD) {
+  if (rank == 0 && tid < HD) {
     float a = 0.f;
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r)
@@ -462,72 +470,100 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     out[(int64_t)u * HD + tid] = __float2bfloat16(a * invL);
   }
 
-  // ---- indicator update (Eq. 2 / Eq. 3), importance (Eq. 4), arg-min ----
-  if (state_in_smem && !mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
+  // ---- indicator update (Eq. 2 / Eq. 3) and importance (Eq. 4) of this CTA's slots, its arg-min ----
+  if (state_in_smem && rows_alloc > 0 && !mbar_wait(state_bar, 0) && dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
   const bool evicting = hi > B;
   unsigned long long my_key = NO_KEY;
   int my_slot = -1, my_pos = -1;
+  {
+    // local copies: the stores into the state arrays below cannot alias what the loop reads
+    const float* __restrict__ lg = logit_s;
+    const float* __restrict__ as = acc_s;
+    const float* __restrict__ vs = vn_s;
+    const int* __restrict__ ps_s = pos_s;
+    float* __restrict__ acc_g = c.acc + (int64_t)u * cap + s0;
 #pragma unroll 4
-  for (int slot = tid; slot < hi; slot += WT) {
-    const int64_t o = (int64_t)u * cap + slot;
-    const float p = ex2(logit_s[slot] - m_all) * invL;
-    const bool is_new = slot == fs;
-    float S;
-    if (WINDOWED) {
-      float* ring_row = c.ring + ((int64_t)u * w + (t % w)) * cap;
-      long long fx;
-      if (is_new) {
-        fx = prob_to_fixed(p);     // (the recycled slot's ring column is cleared below)
+    for (int i = tid; i < cnt; i += WT) {
+      const int slot = s0 + i;
+      const float p = ex2(lg[i] - m_all) * invL;
+      const bool is_new = slot == fs;
+      float S;
+      if (WINDOWED) {
+        float* ring_row = c.ring + ((int64_t)u * w + (t % w)) * cap;
+        const int64_t o = (int64_t)u * cap + slot;
+        long long fx;
+        if (is_new) {
+          fx = prob_to_fixed(p);     // (the recycled slot's ring column is cleared below)
+        } else {
+          fx = c.acc_fixed[o] + prob_to_fixed(p) - prob_to_fixed(ring_row[slot]);
+        }
+        ring_row[slot] = p;
+        c.acc_fixed[o] = fx;
+        S = fixed_to_prob(fx);
       } else {
-        fx = c.acc_fixed[o] + prob_to_fixed(p) - prob_to_fixed(ring_row[slot]);
+        S = is_new ? p : (state_in_smem ? as[i] : acc_g[i]) + p;
       }
-      ring_row[slot] = p;
-      c.acc_fixed[o] = fx;
-      S = fixed_to_prob(fx);
-    } else {
-      S = is_new ? p : (state_in_smem ? acc_s[slot] : c.acc[o]) + p;
-    }
-    c.acc[o] = S;
-    if (evicting) {
-      const int ps = is_new ? t : (state_in_smem ? pos_s[slot] : c.pos[o]);
-      const float I = S * (is_new ? new_norm : (state_in_smem ? vn_s[slot] : c.vnorm[o]));
-      if (ps >= F && ps <= t - R) {
-        const unsigned long long key = evict_key(I, ps);
-        if (key < my_key) { my_key = key; my_slot = slot; my_pos = ps; }
+      acc_g[i] = S;
+      if (evicting) {
+        const int ps = is_new ? t : (state_in_smem ? ps_s[i] : c.pos[(int64_t)u * cap + slot]);
+        const float I = S * (is_new ? new_norm : (state_in_smem ? vs[i] : c.vnorm[(int64_t)u * cap + slot]));
+        if (ps >= F && ps <= t - R) {
+          const unsigned long long key = evict_key(I, ps);
+          if (key < my_key) { my_key = key; my_slot = slot; my_pos = ps; }
+        }
       }
     }
   }
   if (WINDOWED) {
-    // recycled slot: the other rows of its ring column belong to the previous occupant
-    for (int rr = tid; rr < w; rr += WT)
+    // recycled slot: the other rows of its ring column belong to the previous occupant (shared out over the unit's CTAs)
+    for (int rr = rank * WT + tid; rr < w; rr += split * WT)
       if (rr != t % w) c.ring[((int64_t)u * w + rr) * cap + fs] = 0.f;
   }
-  if (evicting) {
+  if (!evicting) {
+    if (rank == 0 && tid == 0) {
+      c.len[u] = hi;
+      c.free_slot[u] = hi;
+      c.next_pos[u] = t + 1;
+      c.last_slot[u] = fs;
+      if (evicted) evicted[u] = -1;
+    }
+    return;
+  }
+  // this CTA's candidate (positions are unique: exactly one thread holds the winning key), pushed to rank 0
+  {
     const unsigned long long wkey = warp_min_key(my_key);
     if (lane == 0) warp_key[wid] = wkey;
     workers_sync();
     const unsigned long long win = warp_min_key(lane < MW ? warp_key[lane] : NO_KEY);
-    if (win != NO_KEY && my_key == win) {      // positions are unique: exactly one thread matches
-      c.pos[(int64_t)u * cap + my_slot] = -1;
-      c.free_slot[u] = my_slot;
+    Exch* e0 = split > 1 ? cluster.map_shared_rank(&ex, 0) : &ex;
+    if (win == NO_KEY) {
+      if (tid == 0) e0->key[rank] = NO_KEY;
+    } else if (my_key == win) {
+      e0->key[rank] = win;
+      e0->key_slot[rank] = my_slot;
+      e0->key_pos[rank] = my_pos;
+    }
+  }
+  if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync();
+  if (rank != 0 || tid != 0) return;      // nothing of the other CTAs' shared memory is read by anyone
+  {
+    unsigned long long best = NO_KEY;
+    int br = -1;
+    for (int r = 0; r < split; ++r)
+      if (ex.key[r] < best) { best = ex.key[r]; br = r; }
+    if (br >= 0) {
+      const int slot = ex.key_slot[br];
+      c.pos[(int64_t)u * cap + slot] = -1;
+      c.free_slot[u] = slot;
       c.len[u] = hi - 1;
-      if (evicted) evicted[u] = my_pos;
+      if (evicted) evicted[u] = ex.key_pos[br];
+    } else {   // nothing eligible (cannot happen when F + R <= B): keep the state consistent
+      c.len[u] = hi;
+      c.free_slot[u] = min(hi, cap - 1);
+      if (evicted) evicted[u] = -1;
     }
-    if (tid == 0) {
-      if (win == NO_KEY) {   // nothing eligible (cannot happen when F + R <= B): keep the state consistent
-        c.len[u] = hi;
-        c.free_slot[u] = min(hi, cap - 1);
-        if (evicted) evicted[u] = -1;
-      }
-      c.next_pos[u] = t + 1;
-      c.last_slot[u] = fs;
-    }
-  } else if (tid == 0) {
-    c.len[u] = hi;
-    c.free_slot[u] = hi;
     c.next_pos[u] = t + 1;
     c.last_slot[u] = fs;
-    if (evicted) evicted[u] = -1;
   }
 }
 
@@ -657,7 +693,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   };
   const size_t half_sm = 104 * 1024, whole_sm = 215 * 1024;     // dynamic bytes, 1 KB of it alignment slack
   const size_t stage_set = (size_t)MW * STAGE_BYTES;
-  const size_t tot = (size_t)chunk * split;
+  const size_t tot = (size_t)chunk;      // slots whose logits and state one CTA holds
   auto make_plan = [&](bool alone) {
     Plan p{};
     size_t state_bytes = 4 * sizeof(float) * tot;
@@ -665,7 +701,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     const bool fits_half = !alone && state_bytes + 1024 + 2 * stage_set <= half_sm;
     if (!alone && !fits_half && sizeof(float) * tot + 1024 + 2 * stage_set <= half_sm) {
       state_bytes = sizeof(float) * tot;
-      p.state_in_smem = (size_t)cap * 12 <= 2 * stage_set ? 2 : 0;
+      p.state_in_smem = tot * 12 <= 2 * stage_set ? 2 : 0;
     }
     p.ok = state_bytes + stage_set + 1024 <= whole_sm;
     if (!p.ok) return p;
@@ -674,7 +710,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     p.nstage = p.nstage > 4 ? 4 : p.nstage;
     const int groups_per_warp = ((chunk / GROUP) + MW - 1) / MW;
     if (p.nstage > groups_per_warp) p.nstage = groups_per_warp > 0 ? groups_per_warp : 1;
-    if (p.state_in_smem == 2 && (size_t)cap * 12 > (size_t)MW * p.nstage * STAGE_BYTES) p.state_in_smem = 0;
+    if (p.state_in_smem == 2 && tot * 12 > (size_t)MW * p.nstage * STAGE_BYTES) p.state_in_smem = 0;
     p.dyn = (size_t)MW * p.nstage * STAGE_BYTES + state_bytes + 1024;
     return p;
   };
