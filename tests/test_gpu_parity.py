@@ -16,21 +16,43 @@ def _small(dtype, d, T, B, F, R, b=1, h=2, indicator="h2o", window=0, steps=0, c
     return synth.Workload(cid, f"case_T{T}", dtype, b, h, 1, d, T, B, F, R, indicator, window, steps)
 
 
-def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0, lse_given=False):
+# What the comparison is allowed to forgive, per oracle unit: kept indices that differ from the oracle's only
+# because their score lies within the tolerance of the boundary score, and decode steps where the GPU evicted the
+# oracle's runner-up because the two importances lie within twice the tolerance of each other (the oracle then
+# follows the GPU).  Both are counted, printed and bounded: a handful per unit is arithmetic, more would be a bug.
+MAX_BOUNDARY_PER_UNIT = 6
+
+
+def _max_adopted(steps, n_units):
+    return n_units * (2 + steps // 32)
+
+
+def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0, lse_given=False,
+              decode_units=None):
+    """units: the units the oracle checks at prefill (default: all); decode_units: those of them whose decode
+    trajectory it follows (default: all of `units`)."""
     q, k, v = synth.prefill_inputs(wl, layer, "cuda")
     g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink, lse_given=lse_given).run()
     P.gpu_invariants(g)
     tol = P.TOL[wl.dtype]
     units = units or [(b, h) for b in range(wl.batch) for h in range(wl.heads)]
+    decode_units = units if decode_units is None else decode_units
     refs, nb = {}, 0
     for (b, h) in units:
         ref, kept, n_boundary = P.check_prefill_unit(g, b, h, tol)
-        refs[(b, h)] = (ref, kept)
+        ref.pop("a")                     # the T x T matrix (8.6 GB at T = 32768) is not needed beyond this point
+        if (b, h) in decode_units:
+            refs[(b, h)] = (ref, kept)
+        assert n_boundary <= MAX_BOUNDARY_PER_UNIT, f"unit {(b, h)}: {n_boundary} kept indices differ from the oracle's"
         nb += n_boundary
+        del ref
     adopted = 0
-    if decode and wl.decode_steps:
+    if decode and wl.decode_steps and refs:
         dq, dk, dv = synth.decode_inputs(wl, layer, device="cuda")
         adopted = P.run_decode_and_check(g, refs, dq, dk, dv, wl.decode_steps, tol, check_state_every)
+        assert adopted <= _max_adopted(wl.decode_steps, len(refs)), f"{adopted} near-tie evictions adopted"
+    print(f"[parity] {wl.name} layer {layer}: {len(units)} oracle units, {nb} boundary indices tolerated, "
+          f"{len(refs)} decode units x {wl.decode_steps if decode else 0} steps, {adopted} near-tie evictions adopted")
     return g, nb, adopted
 
 
@@ -135,17 +157,31 @@ def test_config1_llama_layer():
     _run_case(wl, units=[(0, 0), (0, 13), (0, 31)], check_state_every=64)
 
 
-def test_config1_prefill_all_heads():
+@pytest.mark.parametrize("F", [0, 2, 20])
+def test_config1_prefill_all_heads(F):
+    """Config 1 at its full size, every head against the oracle, without kept leading tokens (the config as
+    written) and with F = 2 and F = 20 (the paper's value for LLaMA2-7B-chat)."""
     wl = synth.CONFIGS[1].with_(decode_steps=0)
-    _run_case(wl, decode=False)
+    g, _, _ = _run_case(wl, decode=False, n_sink=F)
+    assert torch.all(g.kept[..., :F].cpu() == torch.arange(F))
 
 
-@pytest.mark.parametrize("layer,units", [(0, [(0, 0), (7, 31)]), (31, [(3, 17), (5, 2)])])
+def test_config1_decode_with_sink_retention():
+    """Config 1 with the first 20 tokens kept: decode trajectories of sampled heads (the low-norm sink tokens
+    must never be released)."""
+    wl = synth.CONFIGS[1].with_(decode_steps=96)
+    g, _, _ = _run_case(wl, n_sink=20, units=[(0, 3), (0, 28)], check_state_every=32)
+    assert torch.all(g.cache.pos[0, :, :20].cpu() == torch.arange(20))
+
+
+@pytest.mark.parametrize("layer,units", [(0, [(0, 0), (7, 31), (4, 9)]), (15, [(1, 30), (6, 4), (2, 16)]),
+                                         (31, [(3, 17), (5, 2), (0, 22)])])
 def test_config2_stack_layer(layer, units):
     """Config 2 at its full per-layer size (batch 8, 32 heads, T 8192, budget 1638, recent 256; the
-    value-norm spread grows with the layer): first and last layer, oracle on sampled units, oracle-free
-    invariants on all 256 units of the layer, 128 decode steps."""
-    _run_case(synth.CONFIGS[2], units=units, check_state_every=64, layer=layer)
+    value-norm spread grows with the layer: sigma 0.5, 0.98 and 1.5 here): first, middle and last layer,
+    the oracle on nine sampled units in all (prefill; 128 decode steps on two of each layer's three),
+    oracle-free invariants on all 256 units of each layer."""
+    _run_case(synth.CONFIGS[2], units=units, decode_units=units[:2], check_state_every=64, layer=layer)
 
 
 def test_config3_windowed():
@@ -154,11 +190,22 @@ def test_config3_windowed():
     _run_case(synth.CONFIGS[3], units=[(0, 0), (9, 14), (15, 31)], check_state_every=128)
 
 
-def test_config4_long_context_layer():
+@pytest.mark.parametrize("layer,units", [(0, [(0, 0), (0, 19)]), (31, [(0, 5), (0, 30)])])
+def test_config4_long_context_layer(layer, units):
     """Config 4 at full size: T 32768, budget 3277, recent 512, 64 boosted-norm tokens per layer.  The
-    oracle materialises the 32768 x 32768 matrix, so it runs on one unit of the last layer; every other
-    unit of that layer is covered by the invariants."""
-    _run_case(synth.CONFIGS[4], units=[(0, 5)], check_state_every=32, layer=31)
+    oracle materialises the 32768 x 32768 matrix (8.6 GB in float64), one unit at a time: two units of
+    the first and two of the last layer (64 decode steps on one of each pair); every other unit of those
+    layers is covered by the invariants."""
+    _run_case(synth.CONFIGS[4], units=units, decode_units=units[:1], check_state_every=32, layer=layer)
+
+
+@pytest.mark.parametrize("cid,layer", [(4, 16), (2, 23)])
+def test_stack_middle_layers_invariants(cid, layer):
+    """Oracle-free checks on every unit of further layers of the 32-layer configs: indicators sum to the
+    number of query rows, kept counts, kept leading and recent tokens, ascending order."""
+    wl = synth.CONFIGS[cid]
+    q, k, v = synth.prefill_inputs(wl, layer, "cuda")
+    P.gpu_invariants(P.GpuPrefill(wl, q, k, v).run())
 
 
 def _interleaved_equals_alone(wls, steps, overlap=True):
