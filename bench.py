@@ -219,7 +219,8 @@ def run_cuda(args, wl):
 
     lse_given, fill_lse = [False], [True]   # the first call below fills every layer's lse; --lse-given then times pass 2 alone
 
-    def prefill_all(ev=None):
+    def prefill_all(ev=None, upto=3):
+        """upto: 1 = scoring only, 2 = + selection, 3 = + compaction (the whole prefill side)."""
         for i, ls in enumerate(layers):
             if ev: ev[i][0].record()
             if lse_given[0]:
@@ -230,8 +231,10 @@ def run_cuda(args, wl):
                                       attn_acc=ls.attn_acc, vnorm=ls.vnorm, score=ls.score, win_rows=ls.win_rows,
                                       workspace=ls.ws, dev_status=status)
             if ev: ev[i][1].record()
+            if upto < 2: continue
             V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
             if ev: ev[i][2].record()
+            if upto < 3: continue
             V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows,
                            dev_status=status)
             if ev: ev[i][3].record()
@@ -295,6 +298,24 @@ def run_cuda(args, wl):
     # per-kernel breakdown of the prefill side: a few extra steps with an event after every call
     brk = [one_step(True) for _ in range(max(2, min(args.steps, 5)))]
     barrier()
+
+    # The same breakdown without events between the calls.  Selection and compaction are programmatic dependents of
+    # the launch before them (they set up while it drains); an event between two calls breaks that and adds a full
+    # launch latency to each.  Here the chain is timed whole, with its last call(s) left out, and a call's cost is the
+    # difference: what it adds to the chain it runs in.
+    def chain_ms(upto):
+        flush.fill_(rank + 1)
+        a, b = E(), E()
+        a.record(); prefill_all(upto=upto); b.record()
+        return a, b
+
+    chain = {}
+    for upto in (1, 2, 3):
+        chain_ms(upto)
+        recs_c = [chain_ms(upto) for _ in range(max(3, min(args.steps, 6)))]
+        barrier()
+        chain[upto] = statistics.median(a.elapsed_time(b) for a, b in recs_c) / L       # ms per layer
+    prefill_all(); barrier()     # leave complete caches behind
 
     # the same decode steps with every launch waiting for all earlier work in the stream (no opt-in to
     # overlapping launches): what a chain of dependent steps costs - in a model, layer l + 1's q/k/v come
@@ -379,13 +400,17 @@ def run_cuda(args, wl):
     bytes_decode = units * (B + 1) * (2 * d * 2 + 16 + (8 if wl.indicator == "window" else 0))  # K,V rows once, acc r+w, vnorm, pos (+ ring row r+w)
     bytes_select = units * (4 * T + 4 * B)
     ms = statistics.mean
+    t_score_c, t_select_c, t_compact_c = chain[1], chain[2] - chain[1], chain[3] - chain[2]      # ms per layer, in the chain
     kernels = {
-        "prefill_scores": {"bound": "tensor", "achieved": flops_score / (ms(t_score) * 1e-3) / 1e12,
-                           "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "ms_per_launch_pair": ms(t_score)},
-        "select": {"bound": "hbm", "achieved": bytes_select / (ms(t_select) * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                   "unit": "GB/s", "us_per_launch": ms(t_select) * 1e3},
-        "compact": {"bound": "hbm", "achieved": bytes_compact / (ms(t_compact) * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "us_per_launch": ms(t_compact) * 1e3},
+        "prefill_scores": {"bound": "tensor", "achieved": flops_score / (t_score_c * 1e-3) / 1e12,
+                           "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "ms_per_launch_pair": t_score_c,
+                           "ms_isolated": ms(t_score), "achieved_isolated": flops_score / (ms(t_score) * 1e-3) / 1e12},
+        "select": {"bound": "hbm", "achieved": bytes_select / (t_select_c * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                   "unit": "GB/s", "us_per_launch": t_select_c * 1e3,
+                   "us_isolated": ms(t_select) * 1e3, "achieved_isolated": bytes_select / (ms(t_select) * 1e-3) / 1e9},
+        "compact": {"bound": "hbm", "achieved": bytes_compact / (t_compact_c * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "us_per_launch": t_compact_c * 1e3,
+                    "us_isolated": ms(t_compact) * 1e3, "achieved_isolated": bytes_compact / (ms(t_compact) * 1e-3) / 1e9},
         "decode_step": {"bound": "hbm", "achieved": bytes_decode / (dec_us * 1e-6) / 1e9, "peak": peaks["hbm_gbs"],
                         "unit": "GB/s", "us_per_launch": dec_us,
                         "launches": f"steps of {L} independent layer caches in rotation, overlap flag set: consecutive launches run side by side"},
@@ -395,8 +420,15 @@ def run_cuda(args, wl):
     }
     for kd in kernels.values():
         kd["frac"] = kd["achieved"] / kd["peak"]
+        if "achieved_isolated" in kd:
+            kd["frac_isolated"] = kd["achieved_isolated"] / kd["peak"]
         kd["peak_source"] = peaks["source"]
-    share = {"prefill_scores": ms(t_score) * L, "select": ms(t_select) * L, "compact": ms(t_compact) * L,
+    timing_note = ("prefill-side calls: CUDA events over a region of back-to-back calls, as in the timed steps (scoring: a "
+                   "chain of scoring calls over all layers, per layer; selection and compaction: what each adds to that "
+                   "chain, i.e. the chain timed whole minus the chain without the call - both are programmatic dependents "
+                   "of the launch before them and set up while it drains).  *_isolated: CUDA events around every single "
+                   "call instead; an event between two calls breaks that overlap and costs each call a full launch latency")
+    share = {"prefill_scores": t_score_c * L, "select": t_select_c * L, "compact": t_compact_c * L,
              "decode_step": dec_ms}          # (decode_step_dependent is an extra measurement, not part of the timed step)
     dominant = max(share, key=share.get)
     roof = dict(kernels[dominant])
@@ -421,7 +453,7 @@ def run_cuda(args, wl):
                    "decode_graph": graph is not None},
         "prefill_ms_per_layer": pre_ms / L, "decode_us_per_layer_step": dec_us,
         "decode_us_per_layer_step_dependent": dec_wait_us,
-        "roofline": roof, "roofline_all": kernels,
+        "roofline": roof, "roofline_all": kernels, "roofline_all_timing": timing_note,
         "e2e": None if host is None else
                {"value": replica_throughput(tokens, e2e_pre_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "decode_us_per_layer_step": e2e_dec_ms * 1e3 / (steps_dec * L)},

@@ -853,6 +853,17 @@ bool make_rows_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint32_
                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_row_gather_map(CUtensorMap* m, const void* base, uint32_t row_words, uint64_t rows, uint64_t row_stride_bytes) {
+  if (!encode_fn()) return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)row_words, (cuuint64_t)rows};
+  const cuuint64_t strides[1] = {(cuuint64_t)row_stride_bytes};
+  const cuuint32_t box[2] = {row_words, 1};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Per-device facts, looked up on first use with that device current (a process may drive several GPUs).
 namespace {
 constexpr int kMaxDevices = 64;

@@ -146,7 +146,6 @@ vatp_status vatp_select(const vatp_params* p, const float* score, int32_t* kept_
 vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, const float* attn_acc,
                          const float* vnorm, const float* win_rows, const int32_t* kept_idx, const vatp_cache* cache,
                          int32_t* dev_status, void* cuda_stream) {
-  (void)dev_status;
   vatp_status s = check_params(p, true);
   if (s != VATP_OK) return s;
   const bool windowed = p->indicator == VATP_IND_WINDOW;
@@ -158,7 +157,7 @@ vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, con
   if (s != VATP_OK) return s;
   decode_history_forget(static_cast<cudaStream_t>(cuda_stream));
   cudaError_t e = launch_compact(sh, p->dtype, p->budget, k, v, attn_acc, vnorm, win_rows, kept_idx, *cache,
-                                 static_cast<cudaStream_t>(cuda_stream));
+                                 dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
 

@@ -49,6 +49,10 @@ int device_sm_count();
 // swizzle, rows beyond the end read as zeros.  False when the driver entry point is missing.
 bool make_rows_map_bf16(CUtensorMap* m, const void* base, uint64_t rows, uint32_t box_rows);
 
+// 2-D tensor map over `rows` rows of row_words 32-bit words, row_stride_bytes apart (a multiple of 16); the box
+// is one row: for gathers of whole rows by row index.  False when the driver entry point is missing.
+bool make_row_gather_map(CUtensorMap* m, const void* base, uint32_t row_words, uint64_t rows, uint64_t row_stride_bytes);
+
 // Launch configuration of a kernel that may be scheduled before the previous launch in the stream has
 // drained (programmatic dependent launch).  Such a kernel executes griddepcontrol.wait before it reads
 // anything an earlier launch wrote.
@@ -80,7 +84,7 @@ size_t prefill_tc_workspace_bytes(int units, int T);  // padded log2-domain row 
 cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st);
 cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, const void* v, const float* attn_acc,
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
-                           cudaStream_t st);
+                           int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
                           const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
                           bool may_overlap);
