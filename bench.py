@@ -219,9 +219,14 @@ def run_cuda(args, wl):
 
     lse_given, fill_lse = [False], [True]   # the first call below fills every layer's lse; --lse-given then times pass 2 alone
 
-    def prefill_all(ev=None, upto=3):
-        """upto: 1 = scoring only, 2 = + selection, 3 = + compaction (the whole prefill side)."""
+    def prefill_all(ev=None, parts=(True, True, True)):
+        """parts: which of (scoring, selection, compaction) to issue for every layer."""
         for i, ls in enumerate(layers):
+            if not parts[0]:
+                if parts[1]: V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
+                if parts[2]: V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows,
+                                            dev_status=status)
+                continue
             if ev: ev[i][0].record()
             if lse_given[0]:
                 V.vatp_prefill_scores_from_lse(ls.p, ls.q, ls.k, ls.v, ls.lse, attn_acc=ls.attn_acc, vnorm=ls.vnorm,
@@ -231,10 +236,10 @@ def run_cuda(args, wl):
                                       attn_acc=ls.attn_acc, vnorm=ls.vnorm, score=ls.score, win_rows=ls.win_rows,
                                       workspace=ls.ws, dev_status=status)
             if ev: ev[i][1].record()
-            if upto < 2: continue
+            if not parts[1]: continue
             V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
             if ev: ev[i][2].record()
-            if upto < 3: continue
+            if not parts[2]: continue
             V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows,
                            dev_status=status)
             if ev: ev[i][3].record()
@@ -301,20 +306,20 @@ def run_cuda(args, wl):
 
     # The same breakdown without events between the calls.  Selection and compaction are programmatic dependents of
     # the launch before them (they set up while it drains); an event between two calls breaks that and adds a full
-    # launch latency to each.  Here the chain is timed whole, with its last call(s) left out, and a call's cost is the
-    # difference: what it adds to the chain it runs in.
-    def chain_ms(upto):
+    # launch latency to each.  Here CUDA events bracket a region of back-to-back calls over all layers: scoring calls
+    # only; selection calls only; selection + compaction.  Compaction's cost is the last minus the one before.
+    def chain_ms(parts):
         flush.fill_(rank + 1)
         a, b = E(), E()
-        a.record(); prefill_all(upto=upto); b.record()
+        a.record(); prefill_all(parts=parts); b.record()
         return a, b
 
     chain = {}
-    for upto in (1, 2, 3):
-        chain_ms(upto)
-        recs_c = [chain_ms(upto) for _ in range(max(3, min(args.steps, 6)))]
+    for key, parts in (("score", (True, False, False)), ("select", (False, True, False)), ("select+compact", (False, True, True))):
+        chain_ms(parts)
+        recs_c = [chain_ms(parts) for _ in range(max(3, min(args.steps, 6)))]
         barrier()
-        chain[upto] = statistics.median(a.elapsed_time(b) for a, b in recs_c) / L       # ms per layer
+        chain[key] = statistics.median(a.elapsed_time(b) for a, b in recs_c) / L       # ms per layer
     prefill_all(); barrier()     # leave complete caches behind
 
     # the same decode steps with every launch waiting for all earlier work in the stream (no opt-in to
@@ -400,7 +405,8 @@ def run_cuda(args, wl):
     bytes_decode = units * (B + 1) * (2 * d * 2 + 16 + (8 if wl.indicator == "window" else 0))  # K,V rows once, acc r+w, vnorm, pos (+ ring row r+w)
     bytes_select = units * (4 * T + 4 * B)
     ms = statistics.mean
-    t_score_c, t_select_c, t_compact_c = chain[1], chain[2] - chain[1], chain[3] - chain[2]      # ms per layer, in the chain
+    t_score_c, t_select_c = chain["score"], chain["select"]                       # ms per layer, back-to-back calls
+    t_compact_c = chain["select+compact"] - chain["select"]
     kernels = {
         "prefill_scores": {"bound": "tensor", "achieved": flops_score / (t_score_c * 1e-3) / 1e12,
                            "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "ms_per_launch_pair": t_score_c,
@@ -423,11 +429,11 @@ def run_cuda(args, wl):
         if "achieved_isolated" in kd:
             kd["frac_isolated"] = kd["achieved_isolated"] / kd["peak"]
         kd["peak_source"] = peaks["source"]
-    timing_note = ("prefill-side calls: CUDA events over a region of back-to-back calls, as in the timed steps (scoring: a "
-                   "chain of scoring calls over all layers, per layer; selection and compaction: what each adds to that "
-                   "chain, i.e. the chain timed whole minus the chain without the call - both are programmatic dependents "
-                   "of the launch before them and set up while it drains).  *_isolated: CUDA events around every single "
-                   "call instead; an event between two calls breaks that overlap and costs each call a full launch latency")
+    timing_note = ("prefill-side calls: CUDA events over a region of back-to-back calls over all layers, per layer "
+                   "(scoring calls only; selection calls only; compaction = the region of selection + compaction calls "
+                   "minus the region of selection calls: both are programmatic dependents of the launch before them and "
+                   "set up while it drains).  *_isolated: CUDA events around every single call of a whole prefill chain "
+                   "instead; an event between two calls breaks that overlap and costs each call a full launch latency")
     share = {"prefill_scores": t_score_c * L, "select": t_select_c * L, "compact": t_compact_c * L,
              "decode_step": dec_ms}          # (decode_step_dependent is an extra measurement, not part of the timed step)
     dominant = max(share, key=share.get)

@@ -3,6 +3,12 @@
 // the kept indices written in ascending order (first F, selected middle, last R).
 // One CTA per unit; the unit's scores are staged in shared memory once when they fit and read
 // from global memory (L2-resident) otherwise.  Pure integer work after the key transform.
+// Every warp counts into a histogram of its own and the 32 histograms are summed per bin.  The scores
+// of a head share a few exponents, so in the first passes nearly all keys of a warp fall into one bin:
+// the lanes that agree with the warp's first candidate are counted by one addition (a ballot), the
+// others by shared-memory atomics, which rarely collide once the digits spread.  (Grouping all equal
+// digits with match.any cost more than everything else in the kernel: it takes time in proportion to
+// the number of distinct values in the warp.)
 #include "vatp_internal.cuh"
 
 namespace vatp {
@@ -20,8 +26,9 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 template <bool STAGED>
 __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F, int R, const float* __restrict__ score,
                                                              int32_t* __restrict__ kept) {
-  extern __shared__ uint32_t keys_s[];  // STAGED: keys of the middle range
+  extern __shared__ __align__(16) uint32_t keys_s[];  // STAGED: keys of the middle range (from index `pad` on)
   __shared__ uint32_t hist[256];
+  __shared__ uint32_t hist_w[SEL_WARPS][256];      // per-warp counts of the current pass
   __shared__ uint32_t sh_prefix, sh_need;
   __shared__ uint32_t warp_keep[SEL_WARPS], warp_eq[SEL_WARPS];
 
@@ -44,20 +51,46 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
   for (int i = tid; i < R; i += SEL_THREADS) out[B - R + i] = T - R + i;
   if (ksel == 0) return;
 
+  // Staging: key i sits at keys_s[pad + i], pad chosen so that 16-byte loads from global memory pair with
+  // 16-byte stores to shared memory.  Several loads per thread are in flight at once: one CTA has to pull the
+  // whole unit through one SM, and with one 4-byte load per thread in flight that took longer than all the
+  // rest of the kernel.
+  int pad = 0;
   if (STAGED) {
-    for (int i = tid; i < n; i += SEL_THREADS) keys_s[i] = order_key(sc[F + i]);
+    const float* mid = sc + F;
+    const int a0 = min((int)(((16u - (uint32_t)(reinterpret_cast<uintptr_t>(mid) & 15u)) & 15u) >> 2), n);   // scalars before alignment
+    pad = (4 - a0) & 3;
+    const int nvec = (n - a0) >> 2;
+    const float4* src4 = reinterpret_cast<const float4*>(mid + a0);
+    uint4* dst4 = reinterpret_cast<uint4*>(keys_s + pad + a0);
+    for (int v0 = 0; v0 < nvec; v0 += 4 * SEL_THREADS) {
+      float4 x[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int v = v0 + j * SEL_THREADS + tid;
+        if (v < nvec) x[j] = __ldg(src4 + v);
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int v = v0 + j * SEL_THREADS + tid;
+        if (v < nvec) dst4[v] = make_uint4(order_key(x[j].x), order_key(x[j].y), order_key(x[j].z), order_key(x[j].w));
+      }
+    }
+    if (tid < a0) keys_s[pad + tid] = order_key(mid[tid]);
+    const int tail0 = a0 + 4 * nvec;
+    if (tid < n - tail0) keys_s[pad + tail0 + tid] = order_key(mid[tail0 + tid]);
     __syncthreads();
   }
-  auto key_at = [&](int i) -> uint32_t { return STAGED ? keys_s[i] : order_key(sc[F + i]); };
+  auto key_at = [&](int i) -> uint32_t { return STAGED ? keys_s[pad + i] : order_key(sc[F + i]); };
 
   // radix select, most significant byte first: find the key value tau of rank ksel (descending).
-  // Scores of one head share a few exponents, so most keys of a pass fall into a handful of bins:
-  // lanes with the same digit are counted by one of them (match + one atomic per distinct digit).
+  // Lanes that share the digit of the warp's first candidate are counted together; the rest add one each.
   uint32_t prefix = 0, mask = 0, need = (uint32_t)ksel;
   const int lane = tid & 31, wid = tid >> 5;
   for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int i = tid; i < 256; i += SEL_THREADS) hist[i] = 0;
-    __syncthreads();
+#pragma unroll
+    for (int i = lane; i < 256; i += 32) hist_w[wid][i] = 0;
+    __syncwarp();
     for (int base = 0; base < n; base += SEL_THREADS) {
       const int i = base + tid;
       uint32_t digit = 256u;                       // lanes without a candidate share a dummy digit
@@ -65,8 +98,21 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
         const uint32_t key = key_at(i);
         if ((key & mask) == prefix) digit = (key >> shift) & 255u;
       }
-      const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-      if (digit < 256u && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], (uint32_t)__popc(peers));
+      const uint32_t cand = __ballot_sync(0xffffffffu, digit < 256u);
+      if (cand) {
+        const int first = __ffs(cand) - 1;
+        const uint32_t d0 = __shfl_sync(0xffffffffu, digit, first);
+        const uint32_t same = __ballot_sync(0xffffffffu, digit == d0);
+        if (lane == first) atomicAdd(&hist_w[wid][d0], (uint32_t)__popc(same));
+        else if (digit < 256u && digit != d0) atomicAdd(&hist_w[wid][digit], 1u);
+      }
+    }
+    __syncthreads();
+    if (tid < 256) {
+      uint32_t tot = 0;
+#pragma unroll 8
+      for (int w = 0; w < SEL_WARPS; ++w) tot += hist_w[w][tid];
+      hist[tid] = tot;
     }
     __syncthreads();
     if (tid < 32) {
@@ -101,46 +147,42 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
   const uint32_t tau = prefix;     // the ksel-th largest key; `need` of the keys equal to tau survive
   const uint32_t need_eq = need;
 
-  // ordered compaction: keep key > tau, and the first need_eq (lowest index) keys equal to tau.
-  // Thread t owns the contiguous range [t * per, (t + 1) * per); one block-wide exclusive scan of
-  // (kept, equal) counts gives every thread its output offset and the rank of its first tie.
-  const int per = (n + SEL_THREADS - 1) / SEL_THREADS;
-  const int lo = min(tid * per, n), hi_i = min(lo + per, n);
-  uint32_t n_gt = 0, n_eq = 0;
-  for (int i = lo; i < hi_i; ++i) {
-    const uint32_t key = key_at(i);
-    n_gt += key > tau;
-    n_eq += key == tau;
+  // Ordered compaction: keep key > tau, and the first need_eq (lowest index) keys equal to tau.
+  // Warp w owns the contiguous range [w * per_w, (w + 1) * per_w) and walks it 32 consecutive keys at a time
+  // (consecutive shared-memory words: no bank conflicts; one key per lane and a ballot give the order inside a
+  // step).  First the warps count their kept and tied keys, one scan over the 32 warp totals gives every warp its
+  // output offset and the rank of its first tie, then the warps write.
+  const int per_w = ((n + SEL_WARPS - 1) / SEL_WARPS + 31) & ~31;
+  const int lo = min(wid * per_w, n), hi_i = min(lo + per_w, n);
+  const uint32_t lt_mask = (1u << lane) - 1u;
+  uint32_t n_gt = 0, n_eq = 0;                      // warp-uniform
+  for (int i0 = lo; i0 < hi_i; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t key = i < hi_i ? key_at(i) : 0u;
+    n_gt += __popc(__ballot_sync(0xffffffffu, i < hi_i && key > tau));
+    n_eq += __popc(__ballot_sync(0xffffffffu, i < hi_i && key == tau));
   }
-  // inclusive scan inside the warp, then over the warp totals
-  uint32_t s_gt = n_gt, s_eq = n_eq;
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const uint32_t a = __shfl_up_sync(0xffffffffu, s_gt, off), b = __shfl_up_sync(0xffffffffu, s_eq, off);
-    if (lane >= off) { s_gt += a; s_eq += b; }
-  }
-  if (lane == 31) { warp_keep[wid] = s_gt; warp_eq[wid] = s_eq; }
+  if (lane == 0) { warp_keep[wid] = n_gt; warp_eq[wid] = n_eq; }
   __syncthreads();
-  if (wid == 0) {
-    uint32_t a = warp_keep[lane], b = warp_eq[lane];
+  // exclusive prefix over the warps, computed by every warp for itself
+  uint32_t a = lane < wid ? warp_keep[lane] : 0u, b = lane < wid ? warp_eq[lane] : 0u;
 #pragma unroll
-    for (int off = 1; off < 32; off <<= 1) {
-      const uint32_t x = __shfl_up_sync(0xffffffffu, a, off), y = __shfl_up_sync(0xffffffffu, b, off);
-      if (lane >= off) { a += x; b += y; }
-    }
-    warp_keep[lane] = a;      // inclusive totals up to and including warp `lane`
-    warp_eq[lane] = b;
+  for (int off = 16; off; off >>= 1) {
+    a += __shfl_xor_sync(0xffffffffu, a, off);
+    b += __shfl_xor_sync(0xffffffffu, b, off);
   }
-  __syncthreads();
-  const uint32_t gt_before = s_gt - n_gt + (wid ? warp_keep[wid - 1] : 0u);
-  uint32_t eq_rank = s_eq - n_eq + (wid ? warp_eq[wid - 1] : 0u);
-  // ties before index i that survive = min(eq_rank, need_eq)
-  uint32_t o = gt_before + min(eq_rank, need_eq);
-  for (int i = lo; i < hi_i; ++i) {
-    const uint32_t key = key_at(i);
-    const bool keep = key > tau || (key == tau && eq_rank < need_eq);
-    eq_rank += key == tau;
-    if (keep) out[F + o++] = F + i;
+  uint32_t eq_rank = b;                             // ties before this warp's range
+  uint32_t o = a + min(eq_rank, need_eq);           // output offset of this warp's first kept key
+  for (int i0 = lo; i0 < hi_i; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t key = i < hi_i ? key_at(i) : 0u;
+    const bool is_eq = i < hi_i && key == tau;
+    const uint32_t eq_b = __ballot_sync(0xffffffffu, is_eq);
+    const bool keep = i < hi_i && (key > tau || (is_eq && eq_rank + __popc(eq_b & lt_mask) < need_eq));
+    const uint32_t keep_b = __ballot_sync(0xffffffffu, keep);
+    if (keep) out[F + o + __popc(keep_b & lt_mask)] = F + i;
+    o += __popc(keep_b);
+    eq_rank += __popc(eq_b);
   }
 }
 
@@ -148,8 +190,8 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
 
 cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st) {
   const int n = T > B ? T - R - F : 0;
-  const size_t bytes = (size_t)n * sizeof(uint32_t);
-  if (bytes <= 200 * 1024) {
+  const size_t bytes = (size_t)(n + 4) * sizeof(uint32_t);     // up to three words of alignment padding
+  if (bytes <= 160 * 1024) {      // beside the 33 KB of histograms
     cudaError_t e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
     if (e != cudaSuccess) return e;
     DependentLaunch dl(dim3(units), dim3(SEL_THREADS), bytes, st);
