@@ -175,7 +175,7 @@ def replica_throughput(units_per_rank: float, ms: float, world: int) -> float:
 
 
 class LayerState:
-    def __init__(self, V, wl, layer, dev):
+    def __init__(self, V, wl, layer, dev, win_rows=False):
         from paper_2406_12335_b200 import synth
         self.q, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
         self.p = V.params_for(self.q, budget=wl.budget, n_sink=wl.n_sink, n_recent=wl.n_recent, scale=wl.scale,
@@ -189,7 +189,9 @@ class LayerState:
         self.vnorm = torch.empty(b, h, T, **f32)
         self.score = torch.empty(b, h, T, **f32)
         self.lse = torch.empty(b, h, T, **f32)
-        self.win_rows = torch.empty(b, h, wl.window, T, **f32) if wl.indicator == "window" else None
+        # Eq. 3: by default the history of the kept tokens is rebuilt by vatp_compact_window; --win-rows times the
+        # variant in which the scoring call writes all w x T probabilities and vatp_compact gathers from them
+        self.win_rows = torch.empty(b, h, wl.window, T, **f32) if wl.indicator == "window" and win_rows else None
         self.kept = torch.empty(b, h, wl.budget, dtype=torch.int32, device=dev)
         self.ws = torch.empty(max(V.vatp_workspace_bytes(self.p), 256), dtype=torch.uint8, device=dev)
         self.cache = V.Cache(self.p, device=dev)
@@ -213,7 +215,14 @@ def run_cuda(args, wl):
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
     L, steps_dec = args.layers, wl.decode_steps
-    layers = [LayerState(V, wl, l, dev) for l in range(L)]
+    layers = [LayerState(V, wl, l, dev, win_rows=args.win_rows) for l in range(L)]
+    windowed = wl.indicator == "window"
+
+    def compact(ls):
+        if windowed and ls.win_rows is None:
+            V.vatp_compact_window(ls.p, ls.q, ls.k, ls.v, ls.lse, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, dev_status=status)
+        else:
+            V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows, dev_status=status)
     status = torch.zeros(1, dtype=torch.int32, device=dev)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
@@ -224,15 +233,14 @@ def run_cuda(args, wl):
         for i, ls in enumerate(layers):
             if not parts[0]:
                 if parts[1]: V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
-                if parts[2]: V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows,
-                                            dev_status=status)
+                if parts[2]: compact(ls)
                 continue
             if ev: ev[i][0].record()
             if lse_given[0]:
                 V.vatp_prefill_scores_from_lse(ls.p, ls.q, ls.k, ls.v, ls.lse, attn_acc=ls.attn_acc, vnorm=ls.vnorm,
                                                score=ls.score, win_rows=ls.win_rows, workspace=ls.ws, dev_status=status)
             else:
-                V.vatp_prefill_scores(ls.p, ls.q, ls.k, ls.v, lse_out=ls.lse if fill_lse[0] else None,
+                V.vatp_prefill_scores(ls.p, ls.q, ls.k, ls.v, lse_out=ls.lse if (fill_lse[0] or windowed) else None,
                                       attn_acc=ls.attn_acc, vnorm=ls.vnorm, score=ls.score, win_rows=ls.win_rows,
                                       workspace=ls.ws, dev_status=status)
             if ev: ev[i][1].record()
@@ -240,8 +248,7 @@ def run_cuda(args, wl):
             V.vatp_select(ls.p, ls.score, ls.kept, dev_status=status)
             if ev: ev[i][2].record()
             if not parts[2]: continue
-            V.vatp_compact(ls.p, ls.k, ls.v, ls.attn_acc, ls.vnorm, ls.kept, ls.cache, win_rows=ls.win_rows,
-                           dev_status=status)
+            compact(ls)
             if ev: ev[i][3].record()
 
     def decode_all(overlap=True):
@@ -401,7 +408,8 @@ def run_cuda(args, wl):
     flops_score = passes * (2.0 * d) * pairs * units           # each pass recomputes the causal part of QK^T
     bytes_compact = units * (2 * 2 * B * d * 2 + 12 * B)       # K,V rows read + written, 12 B of state per slot
     if wl.indicator == "window":
-        bytes_compact += units * 2 * 4 * B * min(wl.window, T)  # kept columns of the last-w rows read, ring written
+        # history ring written; with --win-rows the kept columns of the last-w rows are read too
+        bytes_compact += units * (2 if args.win_rows else 1) * 4 * B * min(wl.window, T)
     bytes_decode = units * (B + 1) * (2 * d * 2 + 16 + (8 if wl.indicator == "window" else 0))  # K,V rows once, acc r+w, vnorm, pos (+ ring row r+w)
     bytes_select = units * (4 * T + 4 * B)
     ms = statistics.mean
@@ -487,6 +495,9 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-graph", action="store_true", help="launch decode steps directly instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--win-rows", action="store_true",
+                    help="history-window workloads: let the scoring call write all w x T probabilities and gather the "
+                         "kept columns from them (vatp_compact) instead of rebuilding them (vatp_compact_window)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--layers", type=int, default=LAYERS, help="independently seeded layers held on the device")
     ap.add_argument("--config", type=int, default=1, choices=sorted([0, 1, 2, 3, 4, 5]),

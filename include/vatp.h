@@ -109,8 +109,10 @@ size_t vatp_workspace_bytes(const vatp_params* params);
  * q, k, v: inputs as described above (read only).
  * lse_out:  [batch, heads, T] fp32 output (natural log), nullable.
  * attn_acc, vnorm, score: [batch, heads, T] fp32 outputs.
- * win_rows: VATP_IND_WINDOW only: [batch, heads, w, T] fp32 output, row r = probabilities of
- *           query T - w + r (zero where masked or where T - w + r < 0); NULL for H2O.
+ * win_rows: VATP_IND_WINDOW only, nullable: [batch, heads, w, T] fp32 output, row r = probabilities
+ *           of query T - w + r (zero where masked or where T - w + r < 0), for vatp_compact.  NULL
+ *           (always for H2O): nothing is written per (query, key) pair; the decode state of the
+ *           history window is then built by vatp_compact_window, which recomputes the kept columns.
  * workspace: >= vatp_workspace_bytes(params) bytes of device scratch, 256-byte aligned; holds the
  *           row normalisers between the two passes and two work-item counters.
  * bf16 with head_dim 128 runs on the tensor cores; other combinations use an fp32 FMA kernel.
@@ -188,11 +190,31 @@ vatp_status vatp_select(const vatp_params* params, const float* score, int32_t* 
  * pos <- kept index, len <- min(T, B), free_slot <- len, next_pos <- T, last_slot <- -1; unused slots
  * get pos -1.
  * VATP_IND_WINDOW also gathers win_rows columns into `ring` (row (T - w + r) mod w) and sets
- * acc_fixed to the fixed-point window sums.
+ * acc_fixed to the fixed-point window sums; win_rows is then required (see vatp_compact_window for
+ * the variant that needs none).
  */
 vatp_status vatp_compact(const vatp_params* params, const void* k, const void* v, const float* attn_acc,
                          const float* vnorm, const float* win_rows, const int32_t* kept_idx,
                          const vatp_cache* cache, int32_t* dev_status, void* cuda_stream);
+
+/*
+ * Compaction for the history-window indicator (Eq. 3) without the [w, T] probability rows.  The
+ * Limitations section notes that this indicator only needs the attention of the last w queries;
+ * of those w x T probabilities the decode state keeps the B kept columns.  This call gathers K/V and
+ * initialises the state as vatp_compact does, and recomputes the kept block itself:
+ *   ring[(j mod w)][slot] = exp(scale * <q_j, k_slot> - lse[j]) for T - w <= j < T, pos[slot] <= j
+ *   acc_fixed[slot] = sum over those j of the 2^52 fixed-point image, acc[slot] = that sum as float
+ * (a w x B x d contraction per unit), so vatp_prefill_scores may be called with win_rows = NULL.
+ * q: the prompt's queries (as given to vatp_prefill_scores); lse: [batch, heads, T] fp32 natural-log
+ * row normalisers (lse_out of vatp_prefill_scores, or an attention forward's), of which rows
+ * j >= T - w are read.  Other arguments and errors as vatp_compact; params->indicator must be
+ * VATP_IND_WINDOW.  The recomputed probabilities equal those of the scoring pass to fp32 rounding,
+ * not bit for bit (another kernel sums the dot products in another order).
+ */
+vatp_status vatp_compact_window(const vatp_params* params, const void* q, const void* k, const void* v,
+                                const float* lse, const float* attn_acc, const float* vnorm,
+                                const int32_t* kept_idx, const vatp_cache* cache, int32_t* dev_status,
+                                void* cuda_stream);
 
 /*
  * One generation step on the budgeted cache (Eq. 1-4 at step t = next_pos):

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libvatp.so")
-SOURCES = ["vatp_api.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_static.cu", "select.cu", "compact.cu", "decode.cu", "decode_mma.cu", "selftest.cu"]
+SOURCES = ["vatp_api.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_static.cu", "select.cu", "compact.cu", "window_ring.cu", "decode.cu", "decode_mma.cu", "selftest.cu"]
 
 
 def _nvcc() -> str:

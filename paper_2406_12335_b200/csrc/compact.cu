@@ -231,7 +231,7 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
   e = cudaLaunchKernelEx(&dl.cfg, compact_kernel, tm_k, tm_v, rs, s, eb, B, cap, (const char*)k, (const char*)v, attn_acc,
                          vnorm, kept, c, rows_pb, nbuf, dev_status);
   if (e != cudaSuccess) return e;
-  if (s.window > 0) {
+  if (s.window > 0 && win_rows) {
     ring_kernel<<<dim3((cap + 127) / 128, s.units), 128, 0, st>>>(s.units, s.T, s.window, B, cap, win_rows, kept, c);
     e = cudaGetLastError();
   }

@@ -116,6 +116,13 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, u
       : "memory");
 }
 
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(s32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(s32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
 // untiled global -> shared bulk copy; both addresses and the size are multiples of 16 bytes
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
@@ -811,6 +818,139 @@ __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a, const float* __res
   }
 }
 
+
+// ---- history-window state from Q and the compacted keys (Eq. 3) ------------------------------------------
+// For the kept tokens of a unit, their probabilities under the last w prompt queries, written in the layout the
+// decode step keeps (ring[u][j mod w][slot]) together with the exact fixed-point sum per slot:
+//   p[j][slot] = exp2(scale_log2 * <q_j, k_slot> - lse2_j)   for pos[slot] <= j (causal), else 0
+// One CTA takes 128 slots of a unit (TMEM lanes = keys, as in pass 2) against the window's queries in chunks
+// of 256 (accumulator columns): S^T = K_kept Q_win^T is one 128 x 256 x 128 block of MMAs per chunk.  Sixteen
+// warps read it back: warp (quarter, group) takes 32 slots (one per thread) and 64 of the chunk's queries, so
+// a slot's window sum is a running sum in four threads' registers (added up at the end; integers, so the order
+// is immaterial), and for each query the 32 lanes of a warp store 32 consecutive slots of one ring row.
+constexpr int RG_THREADS = 512;
+struct RingSmem {
+  alignas(1024) unsigned char keys[TILE_BYTES];     // 128 cached keys: two K halves of [128 rows][128 bytes]
+  alignas(1024) unsigned char qrows[CHUNK_BYTES];   // 256 window queries: [K half][256 rows][128 bytes]
+  float nlse[CHUNK];                                // their negated log2 normalisers (-inf: no such query)
+  long long part[3][TILE];                          // window sums of column groups 1-3
+  alignas(8) uint64_t bar_ld, bar_mma;
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+__global__ void __launch_bounds__(RG_THREADS, 2)
+window_ring_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_kc, int heads, int T,
+                      int w, int B, int cap, float scale_log2, const float* __restrict__ lse, vatp_cache c,
+                      int32_t* dev_status) {
+  extern __shared__ unsigned char smem_raw[];
+  RingSmem& sm = *reinterpret_cast<RingSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int u = blockIdx.y, slot0 = blockIdx.x * TILE;
+  const int b = u / heads, h = u - b * heads;
+  volatile int* abort_flag = &sm.abort_flag;
+  if (tid == 0) {
+    mbar_init(&sm.bar_ld, 1);
+    mbar_init(&sm.bar_mma, 1);
+    sm.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (wid == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)), "r"(CHUNK) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+
+  const int quarter = wid & 3, grp = wid >> 2;      // TMEM lanes this warp may touch; which 64 columns of a chunk it takes
+  const int row = quarter * 32 + lane;
+  const int slot = slot0 + row;                     // this thread's slot = its TMEM lane
+  const int len = min(T, B);
+  const int ps = slot < len ? c.pos[(int64_t)u * cap + slot] : -1;      // position of the cached token, -1: empty slot
+  float* ring_s = c.ring + (int64_t)u * w * cap + slot;     // this slot's column of the unit's ring
+  long long fx = 0;
+  bool ok = true;
+  uint32_t it = 0;
+  for (int c0 = 0; c0 < w && ok; c0 += CHUNK, ++it) {
+    // the previous chunk's accumulator and normalisers have been consumed by every warp
+    tc_fence_before();
+    __syncthreads();
+    for (int i = tid; i < CHUNK; i += RG_THREADS) {
+      const int r = c0 + i, j = T - w + r;
+      sm.nlse[i] = (r < w && j >= 0) ? -__ldg(lse + (int64_t)u * T + j) * 1.4426950408889634f : -INFINITY;
+    }
+    if (tid == 0) {
+      mbar_expect_tx(&sm.bar_ld, CHUNK_BYTES + (it == 0 ? TILE_BYTES : 0));
+      if (it == 0) {
+        tma_load_2d(sm.keys, &tm_kc, &sm.bar_ld, 0, u * cap + slot0);
+        tma_load_2d(sm.keys + SLAB_BYTES, &tm_kc, &sm.bar_ld, 64, u * cap + slot0);
+      }
+      // rows before the prompt (negative coordinate) and beyond it arrive as zeros
+#pragma unroll
+      for (int kh = 0; kh < 2; ++kh)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh)
+          tma_load_4d(sm.qrows + kh * (2 * SLAB_BYTES) + hh * SLAB_BYTES, &tm_q, &sm.bar_ld, 64 * kh, T - w + c0 + hh * TILE, h, b);
+      if (mbar_wait(&sm.bar_ld, it & 1, abort_flag, dev_status)) {
+        tc_fence_after();
+        umma_tile<0, 256>(tmem, umma_desc(s32(sm.keys)), umma_desc(s32(sm.qrows)));
+        umma_commit(&sm.bar_mma);
+      }
+    }
+    __syncthreads();                                 // normalisers written (thread 0 has issued the MMAs or given up)
+    const bool got = mbar_wait(&sm.bar_mma, it & 1, abort_flag, dev_status);
+    if (!__syncthreads_and(got ? 1 : 0)) { ok = false; break; }     // the same verdict for every warp of the CTA
+    tc_fence_after();
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const int n_cols = min(CHUNK, w - c0);
+    for (int cs = 64 * grp; cs < min(n_cols, 64 * grp + 64); cs += 32) {
+      float x[32];
+      tmem_ld32(lane_addr + cs, x);
+      tmem_ld_wait();
+      // window row r = c0 + cs + i is query j = T - w + r and ring row j mod w; both advance by one per column
+      // (the ring row wraps at w; -w < j < 0 when the prompt is shorter than the window)
+      const int j0 = T - w + c0 + cs;
+      int rr = j0 >= 0 ? j0 % w : j0 + w;
+      uint32_t off = (uint32_t)rr * (uint32_t)cap;          // element offset of the ring row (w * cap < 2^31: checked on the host)
+      const int live = min(32, n_cols - cs);
+      const uint32_t lp = s32(&sm.nlse[cs]);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        if (i < live) {
+          float nl;
+          asm("ld.shared.f32 %0, [%1];" : "=f"(nl) : "r"(lp + 4 * i));
+          float pr = 0.f;
+          if (ps >= 0 && ps <= j0 + i) pr = ex2(fmaf(x[i], scale_log2, nl));
+          fx += prob_to_fixed(pr);
+          if (slot < cap) ring_s[off] = pr;
+          off += cap;
+          if (++rr == w) { rr = 0; off = 0; }
+        }
+      }
+    }
+  }
+  if (grp > 0) sm.part[grp - 1][row] = fx;
+  __syncthreads();
+  if (ok && grp == 0 && slot < cap) {
+    fx += sm.part[0][row] + sm.part[1][row] + sm.part[2][row];
+    c.acc_fixed[(int64_t)u * cap + slot] = fx;
+    c.acc[(int64_t)u * cap + slot] = fixed_to_prob(fx);
+  }
+  // ---- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (sm.abort_flag) {
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);   // copies that may still be in flight
+    __syncthreads();
+  }
+  if (wid == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(CHUNK) : "memory");
+  }
+}
+
 // ---- host side -------------------------------------------------------------------------------
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -957,8 +1097,24 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return win ? cudaLaunchKernelEx(&cfg, prefill_tc_kernel<2, true>, tm_q, tm_k, a)
-             : cudaLaunchKernelEx(&cfg, prefill_tc_kernel<2, false>, tm_q, tm_k, a);
+  // the probabilities of the window's rows are written only when the caller wants them
+  return win && win_rows ? cudaLaunchKernelEx(&cfg, prefill_tc_kernel<2, true>, tm_q, tm_k, a)
+                         : cudaLaunchKernelEx(&cfg, prefill_tc_kernel<2, false>, tm_q, tm_k, a);
+}
+
+// Window history from Q and the compacted keys on the tensor cores (bf16, head_dim 128); see window_ring_tc_kernel.
+cudaError_t launch_window_ring_tc(const Shape& s, int B, const void* q, const float* lse, const vatp_cache& c,
+                                  int32_t* dev_status, cudaStream_t st) {
+  const int cap = cache_capacity(B);
+  CUtensorMap tm_q, tm_kc;
+  if (!make_map(&tm_q, q, s) || !make_rows_map_bf16(&tm_kc, c.k_cache, (uint64_t)s.units * cap, TILE)) return cudaErrorInvalidValue;
+  if ((int64_t)s.window * cap >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
+  const size_t smem = sizeof(RingSmem) + 1024;
+  cudaError_t e = cudaFuncSetAttribute(window_ring_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  window_ring_tc_kernel<<<dim3((cap + TILE - 1) / TILE, s.units), RG_THREADS, smem, st>>>(
+      tm_q, tm_kc, s.heads, s.T, s.window, B, cap, s.scale * 1.4426950408889634f, lse, c, dev_status);
+  return cudaGetLastError();
 }
 
 }  // namespace vatp

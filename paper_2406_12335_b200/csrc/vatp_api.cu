@@ -67,8 +67,6 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
   if (s != VATP_OK) return s;
   if (!q || !k || !v || !attn_acc || !vnorm || !score) return VATP_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
-  const bool windowed = p->indicator == VATP_IND_WINDOW;
-  if (windowed && !win_rows) return VATP_ERR_INVALID_ARG;
   Shape sh;
   s = make_shape(p, &sh);
   if (s != VATP_OK) return s;
@@ -158,6 +156,24 @@ vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, con
   decode_history_forget(static_cast<cudaStream_t>(cuda_stream));
   cudaError_t e = launch_compact(sh, p->dtype, p->budget, k, v, attn_acc, vnorm, win_rows, kept_idx, *cache,
                                  dev_status, static_cast<cudaStream_t>(cuda_stream));
+  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+}
+
+vatp_status vatp_compact_window(const vatp_params* p, const void* q, const void* k, const void* v, const float* lse,
+                                const float* attn_acc, const float* vnorm, const int32_t* kept_idx,
+                                const vatp_cache* cache, int32_t* dev_status, void* cuda_stream) {
+  vatp_status s = check_params(p, true);
+  if (s != VATP_OK) return s;
+  if (p->indicator != VATP_IND_WINDOW) return VATP_ERR_INVALID_ARG;
+  if (!q || !k || !v || !lse || !attn_acc || !vnorm || !kept_idx || !cache_ok(cache, true)) return VATP_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
+  Shape sh;
+  s = make_shape(p, &sh);
+  if (s != VATP_OK) return s;
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  decode_history_forget(st);
+  cudaError_t e = launch_compact(sh, p->dtype, p->budget, k, v, attn_acc, vnorm, nullptr, kept_idx, *cache, dev_status, st);
+  if (e == cudaSuccess) e = launch_window_ring(sh, p->dtype, p->budget, q, lse, *cache, dev_status, st);
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
 

@@ -4,6 +4,7 @@
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include "vatp.h"
 
@@ -85,6 +86,11 @@ cudaError_t launch_select(int units, int T, int B, int F, int R, const float* sc
 cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, const void* v, const float* attn_acc,
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
                            int32_t* dev_status, cudaStream_t st);
+// windowed decode state from Q, the compacted keys and the row normalisers (natural log): ring, acc_fixed, acc
+cudaError_t launch_window_ring(const Shape& s, int dtype, int B, const void* q, const float* lse, const vatp_cache& c,
+                               int32_t* dev_status, cudaStream_t st);
+cudaError_t launch_window_ring_tc(const Shape& s, int B, const void* q, const float* lse, const vatp_cache& c,
+                                  int32_t* dev_status, cudaStream_t st);   // bf16, head_dim 128, tensor cores
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
                           const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
                           bool may_overlap);
@@ -101,8 +107,24 @@ void decode_history_forget(cudaStream_t st, bool probe_only = false);
 
 bool decode_overlap_policy_probe(void* stream, const uint64_t* begin, const uint64_t* bytes, int n, double share);
 
-// fixed-point image of a probability for the exact window sums (Eq. 3): p in [0, 1] -> p * 2^52
-__host__ __device__ inline long long prob_to_fixed(float p) { return (long long)((double)p * 4503599627370496.0); }
+// Fixed-point image of a probability for the exact window sums (Eq. 3): p in [0, 1] -> trunc(p * 2^52), taken from
+// the bits of the float: its 24-bit significand shifted by (biased exponent - 98).  Exact, like the product in
+// double precision it replaces, without the conversions (which run at a fraction of the integer rate).
+__host__ __device__ inline long long prob_to_fixed(float p) {
+#ifdef __CUDA_ARCH__
+  // on the device the same value in two instructions: the product with 2^52 is exact in fp32 (a power of two), and
+  // the conversion truncates towards zero (negative or NaN inputs do not occur: p is a probability)
+  return __float2ll_rz(p * 4503599627370496.0f);
+#else
+  uint32_t b;
+  memcpy(&b, &p, sizeof(b));
+  const int e = (int)((b >> 23) & 0xffu);
+  if (e == 0 || (b >> 31)) return 0;                   // zero, subnormal (below 2^-52 in any case) or negative
+  const long long m = (long long)((b & 0x7fffffu) | 0x800000u);
+  const int s = e - 98;                                // p = m * 2^(e - 150); times 2^52
+  return s >= 0 ? (s < 39 ? m << s : 0x7fffffffffffffffll) : (s > -24 ? m >> -s : 0);
+#endif
+}
 __host__ __device__ inline float fixed_to_prob(long long x) { return (float)((double)x * (1.0 / 4503599627370496.0)); }
 
 }  // namespace vatp

@@ -21,7 +21,7 @@ IND_H2O, IND_WINDOW = 0, 1
 NORM_KINDS = {"l1": 0, "l2": 1, "linf": 2}
 FLAG_DECODE_OVERLAP = 1
 STATIC_SCRATCH_BYTES = (4 << 20) + 256
-EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_from_lse", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_decode_step",
+EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_from_lse", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_compact_window", "vatp_decode_step",
            "vatp_selftest_bounded_wait", "vatp_selftest_overlap_policy", "vatp_status_string"]
 
 
@@ -53,6 +53,8 @@ lib.vatp_select.restype = C.c_int
 lib.vatp_select.argtypes = [C.POINTER(Params), _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.vatp_compact.restype = C.c_int
 lib.vatp_compact.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(CacheStruct), _vp, _vp]
+lib.vatp_compact_window.restype = C.c_int
+lib.vatp_compact_window.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(CacheStruct), _vp, _vp]
 lib.vatp_decode_step.restype = C.c_int
 lib.vatp_decode_step.argtypes = [C.POINTER(Params), C.POINTER(CacheStruct), _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.vatp_selftest_bounded_wait.restype = C.c_int
@@ -173,6 +175,14 @@ def vatp_compact(p: Params, k, v, attn_acc, vnorm, kept_idx, cache: Cache, *, wi
                  stream=None):
     _check(lib.vatp_compact(C.byref(p), _ptr(k), _ptr(v), _ptr(attn_acc), _ptr(vnorm), _ptr(win_rows), _ptr(kept_idx),
                             C.byref(cache.struct), _ptr(dev_status), _stream(stream)), "vatp_compact")
+
+
+def vatp_compact_window(p: Params, q, k, v, lse, attn_acc, vnorm, kept_idx, cache: Cache, *, dev_status=None, stream=None):
+    """vatp_compact for the history-window indicator without win_rows: the kept block of the last-w
+    probability rows is recomputed from q, the compacted keys and the row normalisers `lse` (natural log)."""
+    _check(lib.vatp_compact_window(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse), _ptr(attn_acc), _ptr(vnorm),
+                                   _ptr(kept_idx), C.byref(cache.struct), _ptr(dev_status), _stream(stream)),
+           "vatp_compact_window")
 
 
 def vatp_decode_step(p: Params, cache: Cache, q_new, k_new, v_new, out, *, evicted_pos=None, dev_status=None,

@@ -39,9 +39,11 @@ def attention_forward_lse(q: torch.Tensor, k: torch.Tensor, scale: float) -> tor
 class GpuPrefill:
     """Device buffers and the three prefill-side calls for one layer of a workload."""
 
-    def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None, lse_given=False, decode_overlap=False):
+    def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None, lse_given=False, decode_overlap=False,
+                 recompute_window=False):
         """decode_overlap: decode steps through this object carry VATP_FLAG_DECODE_OVERLAP (steps of
-        caches that share no buffer may run side by side on the GPU)."""
+        caches that share no buffer may run side by side on the GPU).  recompute_window (Eq. 3 only): the
+        scoring call writes no win_rows and vatp_compact_window rebuilds the kept block of the history."""
         V = vatp()
         self.wl = wl
         self.lse_given = lse_given
@@ -56,7 +58,8 @@ class GpuPrefill:
         self.attn_acc = torch.empty(b, h, T, **f32)
         self.vnorm = torch.empty(b, h, T, **f32)
         self.score = torch.empty(b, h, T, **f32)
-        self.win_rows = torch.empty(b, h, wl.window, T, **f32) if wl.indicator == "window" else None
+        self.recompute_window = recompute_window and wl.indicator == "window"
+        self.win_rows = torch.empty(b, h, wl.window, T, **f32) if wl.indicator == "window" and not self.recompute_window else None
         self.ws = torch.empty(max(V.vatp_workspace_bytes(self.p), 256), dtype=torch.uint8, device=dev)
         self.status = torch.zeros(1, dtype=torch.int32, device=dev)
         self.kept = torch.empty(b, h, wl.budget, dtype=torch.int32, device=dev)
@@ -75,8 +78,12 @@ class GpuPrefill:
                                   vnorm=self.vnorm, score=self.score, win_rows=self.win_rows, workspace=self.ws,
                                   dev_status=self.status)
         V.vatp_select(self.p, self.score, self.kept, workspace=self.ws, dev_status=self.status)
-        V.vatp_compact(self.p, self.k, self.v, self.attn_acc, self.vnorm, self.kept, self.cache,
-                       win_rows=self.win_rows, dev_status=self.status)
+        if self.recompute_window:
+            V.vatp_compact_window(self.p, self.q, self.k, self.v, self.lse, self.attn_acc, self.vnorm, self.kept,
+                                  self.cache, dev_status=self.status)
+        else:
+            V.vatp_compact(self.p, self.k, self.v, self.attn_acc, self.vnorm, self.kept, self.cache,
+                           win_rows=self.win_rows, dev_status=self.status)
         torch.cuda.synchronize()
         assert int(self.status.item()) == 0, "device status word set"
         return self
@@ -102,7 +109,7 @@ def check_prefill_unit(g: GpuPrefill, b: int, h: int, tol: float):
         got = to_np64(getattr(g, name)[b, h])
         e = rel_err(got, ref[key])
         assert e <= tol, f"{name} rel err {e:.3g} > {tol} (unit {b},{h})"
-    if window:
+    if window and g.win_rows is not None:
         rows = to_np64(g.win_rows[b, h])
         want = np.zeros_like(rows)
         n = ref["window_rows"].shape[0]
@@ -137,6 +144,20 @@ def check_prefill_unit(g: GpuPrefill, b: int, h: int, tol: float):
     assert torch.equal(cache.vnorm[b, h, :n_live], g.vnorm[b, h][idx])
     if not window:
         assert torch.equal(cache.acc[b, h, :n_live], g.attn_acc[b, h][idx])
+    else:
+        # history ring: row (j mod w) holds the probabilities of query j on the kept tokens; exact window sums
+        w = wl.window
+        ring = to_np64(cache.ring[b, h])                      # [w, cap]
+        want = np.zeros((w, n_live))
+        rows_ref = ref["window_rows"]                         # rows of queries max(T - w, 0) .. T - 1
+        j0 = T - rows_ref.shape[0]
+        for r in range(rows_ref.shape[0]):
+            want[(j0 + r) % w] = rows_ref[r][kept_gpu]
+        assert np.max(np.abs(ring[:, :n_live] - want) - tol * np.abs(want)) <= 1e-30, "history ring"
+        assert np.all(ring[:, n_live:] == 0)
+        fixed = cache.acc_fixed[b, h, :n_live].cpu().numpy().astype(np.float64) / 2.0 ** 52
+        assert rel_err(fixed, ref["S"][kept_gpu]) <= tol, "fixed-point window sums"
+        assert rel_err(to_np64(cache.acc[b, h, :n_live]), ref["S"][kept_gpu]) <= tol
     assert int(cache.len[b, h]) == n_live and int(cache.next_pos[b, h]) == T and int(cache.free_slot[b, h]) == n_live
     if sg == sr:
         assert cache.k_cache[b, h, :n_live].cpu().view(torch.uint8).numpy().tobytes() == \

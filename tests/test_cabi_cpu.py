@@ -62,7 +62,14 @@ def test_host_side_validation(V):
     wp = V.make_params(**{**ok, "indicator": "window", "window": 0})
     assert V.lib.vatp_select(C.byref(wp), 16, 16, null, 0, null, null) == 1
     wp = V.make_params(**{**ok, "indicator": "window", "window": 8})
-    assert V.lib.vatp_prefill_scores(C.byref(wp), 16, 16, 16, 16, 16, 16, 16, null, null, 0, null, null) == 1  # win_rows
+    # the [w, T] probability rows are optional (vatp_compact_window needs none): the call gets as far as the workspace check
+    assert V.lib.vatp_prefill_scores(C.byref(wp), 16, 16, 16, 16, 16, 16, 16, null, null, 0, null, null) == 3
+    # vatp_compact needs them with a history window; vatp_compact_window needs the window, q and the row normalisers
+    cs = V.CacheStruct(*([16] * 11))
+    assert V.lib.vatp_compact(C.byref(wp), 16, 16, 16, 16, null, 16, C.byref(cs), null, null) == 1
+    assert V.lib.vatp_compact_window(C.byref(p), 16, 16, 16, 16, 16, 16, 16, C.byref(cs), null, null) == 1     # H2O parameters
+    assert V.lib.vatp_compact_window(C.byref(wp), 16, 16, 16, null, 16, 16, 16, C.byref(cs), null, null) == 1   # no lse
+    assert V.lib.vatp_compact_window(C.byref(wp), null, 16, 16, 16, 16, 16, 16, C.byref(cs), null, null) == 1   # no q
     # strides that are not multiples of 16 bytes
     sp = V.make_params(**{**ok, "strides": (0, 0, 65)})
     assert V.lib.vatp_prefill_scores(C.byref(sp), 16, 16, 16, 16, 16, 16, 16, null, null, 0, null, null) == 1

@@ -28,11 +28,11 @@ def _max_adopted(steps, n_units):
 
 
 def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0, lse_given=False,
-              decode_units=None):
+              decode_units=None, recompute_window=False):
     """units: the units the oracle checks at prefill (default: all); decode_units: those of them whose decode
     trajectory it follows (default: all of `units`)."""
     q, k, v = synth.prefill_inputs(wl, layer, "cuda")
-    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink, lse_given=lse_given).run()
+    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink, lse_given=lse_given, recompute_window=recompute_window).run()
     P.gpu_invariants(g)
     tol = P.TOL[wl.dtype]
     units = units or [(b, h) for b in range(wl.batch) for h in range(wl.heads)]
@@ -184,10 +184,12 @@ def test_config2_stack_layer(layer, units):
     _run_case(synth.CONFIGS[2], units=units, decode_units=units[:2], check_state_every=64, layer=layer)
 
 
-def test_config3_windowed():
+@pytest.mark.parametrize("recompute", [True, False])
+def test_config3_windowed(recompute):
     """Config 3 at full size: last-256-queries indicator (Eq. 3), batch 16, 32 heads, T 2048, budget
-    1024, 512 decode steps with the cache held at budget; oracle on sampled units."""
-    _run_case(synth.CONFIGS[3], units=[(0, 0), (9, 14), (15, 31)], check_state_every=128)
+    1024, 512 decode steps with the cache held at budget; oracle on sampled units.  Once with the history
+    rebuilt from Q and the kept keys (no win_rows), once through win_rows."""
+    _run_case(synth.CONFIGS[3], units=[(0, 0), (9, 14), (15, 31)], check_state_every=128, recompute_window=recompute)
 
 
 @pytest.mark.parametrize("layer,units", [(0, [(0, 0), (0, 19)]), (31, [(0, 5), (0, 30)])])
@@ -270,14 +272,37 @@ def test_interleaved_caches_match_separate_runs(b, h, overlap):
     (513, 1, 200, 0, 0),         # a window of one query
     (640, 640, 256, 2, 16),      # window = whole prompt
 ])
-def test_windowed_indicator_shapes(T, w, B, F, R):
+@pytest.mark.parametrize("recompute", [True, False])
+def test_windowed_indicator_shapes(T, w, B, F, R, recompute):
     """Eq. 3 on the tensor-core path (bf16, d 128) for windows that start anywhere, with decode steps that
-    roll the history ring."""
-    _run_case(_small("bf16", 128, T, B, F, R, b=1, h=2, indicator="window", window=w, steps=8, cid=60))
+    roll the history ring; the history either gathered from win_rows or rebuilt by vatp_compact_window."""
+    _run_case(_small("bf16", 128, T, B, F, R, b=1, h=2, indicator="window", window=w, steps=8, cid=60),
+              recompute_window=recompute)
 
 
-def test_windowed_indicator_fp32_path():
-    _run_case(_small("f32", 64, 300, 120, 2, 10, b=1, h=2, indicator="window", window=77, steps=6, cid=61))
+@pytest.mark.parametrize("recompute", [True, False])
+@pytest.mark.parametrize("dtype,d", [("f32", 64), ("bf16", 64), ("f32", 128)])
+def test_windowed_indicator_general_kernels(dtype, d, recompute):
+    _run_case(_small(dtype, d, 300, 120, 2, 10, b=1, h=2, indicator="window", window=77, steps=6, cid=61),
+              recompute_window=recompute)
+
+
+def test_window_history_rebuilt_equals_gathered():
+    """The two ways to the windowed decode state on the same inputs: probabilities gathered from win_rows and
+    probabilities recomputed from Q and the kept keys agree to the accuracy of the scoring pass's exponential
+    (one pair in eight takes a polynomial with 7.5e-5 relative error there; the rebuild uses ex2 throughout),
+    ring entries and exact window sums alike, and everything else in the state is identical."""
+    wl = _small("bf16", 128, 1500, 600, 4, 10, b=2, h=5, indicator="window", window=400, steps=0, cid=69)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    a = P.GpuPrefill(wl, q, k, v).run()
+    b = P.GpuPrefill(wl, q, k, v, recompute_window=True).run()
+    assert torch.equal(a.score, b.score) and torch.equal(a.kept, b.kept)
+    for name in ("k_cache", "v_cache", "vnorm", "pos", "len", "free_slot", "next_pos"):
+        assert torch.equal(getattr(a.cache, name), getattr(b.cache, name)), name
+    ra, rb = a.cache.ring.double(), b.cache.ring.double()
+    assert torch.all((ra - rb).abs() <= 1e-4 * ra.abs() + 1e-30), "ring entries"
+    fa, fb = a.cache.acc_fixed.double(), b.cache.acc_fixed.double()
+    assert torch.all((fa - fb).abs() <= 1e-4 * fa.abs() + 1.0), "fixed-point sums"
 
 
 @pytest.mark.parametrize("norm", ["l2", "linf"])
@@ -323,7 +348,7 @@ def test_config5_throughput_table_shape():
     w = 400, F = 20) at the 50% budget, full per-layer size: oracle on sampled units with decode steps,
     oracle-free invariants on all 384 units."""
     wl = synth.CONFIGS[5].with_(decode_steps=24)
-    _run_case(wl, units=[(0, 0), (11, 31)], check_state_every=12)
+    _run_case(wl, units=[(0, 0), (11, 31)], check_state_every=12, recompute_window=True)
 
 
 @pytest.mark.parametrize("dtype,d,T,B,indicator,window,norm", [
