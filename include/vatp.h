@@ -24,6 +24,10 @@
  *     *dev_status (device int32, 0 = fine; caller zeroes it and reads it after sync); the
  *     kernels never trap.
  *   - Inputs are assumed finite.
+ *   - A second build of the library (compiled with -DVATP_DEBUG_BOUNDS) range-checks every row, slot,
+ *     window-row and scratch index its kernels compute before the access; an index outside its array is
+ *     not dereferenced, VATP_ERR_BOUNDS goes to *dev_status, and the kernel carries on.  It stands in
+ *     for a memory checker where none can be run; results are those of the ordinary build.
  */
 #ifndef VATP_H_
 #define VATP_H_
@@ -42,7 +46,8 @@ typedef enum {
   VATP_ERR_WORKSPACE = 3,
   VATP_ERR_CUDA = 4,
   VATP_ERR_TIMEOUT = 5,
-  VATP_ERR_STATIC_SCRATCH = 6  /* problem needs more scratch than the built-in array holds */
+  VATP_ERR_STATIC_SCRATCH = 6, /* problem needs more scratch than the built-in array holds */
+  VATP_ERR_BOUNDS = 7          /* bounds-checking build only: a kernel computed an index outside its array */
 } vatp_status;
 
 typedef enum { VATP_BF16 = 0, VATP_F32 = 1 } vatp_dtype;

@@ -91,7 +91,16 @@ compact_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(cb_s32(bar)), "r"(2 * live * row_bytes) : "memory");
       __syncwarp();
       unsigned char* half = my_buf + (size_t)slot * buf_bytes + (lane < 16 ? 0 : rows_pb * row_bytes);
-      if (gather_rs > 0 && live == rows_pb) {
+      bool gather = gather_rs > 0 && live == rows_pb;
+#ifdef VATP_DEBUG_BOUNDS
+      // the kept indices come from another kernel: a row outside the prompt, or a buffer offset outside the ring,
+      // is not fetched (the batch's wait then runs out and is reported as well)
+      if (src >= 0 && !VATP_INB(src, sh.T, dev_status)) src = -1;
+      if (!VATP_INB((size_t)slot * buf_bytes + (lane < 16 ? 0 : rows_pb * row_bytes) + (l16 + 1) * row_bytes - 1,
+                    (size_t)nbuf * buf_bytes, dev_status)) src = -1;
+      gather = gather && __all_sync(0xffffffffu, src >= 0 || l16 >= rows_pb);
+#endif
+      if (gather) {
         // row index in the table of all rows; lanes 0-3 (K) and 16-19 (V) each gather four rows of the batch
         const int g = src >= 0 ? (int)((unit_offset(sh, u) + (int64_t)src * sh.st) / gather_rs) : 0;
         const int base_lane = (lane & 16) + 4 * (lane & 3);
@@ -110,7 +119,7 @@ compact_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
       }
     }
     // per-slot decode state, and the unit's scalars with its first slot
-    if (lane < rows_pb && s < cap) {
+    if (lane < rows_pb && s < cap && VATP_INB((int64_t)u * cap + s, (int64_t)sh.units * cap, dev_status)) {
       const int64_t o = (int64_t)u * cap + s;
       c.pos[o] = src;
       c.acc[o] = src >= 0 ? __ldg(attn_acc + (int64_t)u * sh.T + src) : 0.f;
@@ -176,12 +185,13 @@ compact_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__
 // Windowed indicator state: ring[u][(T - w + r) mod w][slot] = win_rows[u][r][kept[slot]] and the
 // exact fixed-point window sum of every slot (Eq. 3).
 __global__ void ring_kernel(int units, int T, int w, int B, int cap, const float* __restrict__ win_rows,
-                            const int32_t* __restrict__ kept, vatp_cache c) {
+                            const int32_t* __restrict__ kept, vatp_cache c, int32_t* dev_status) {
   const int u = blockIdx.y;
   const int slot = blockIdx.x * blockDim.x + threadIdx.x;
   if (slot >= cap) return;
   const int len = min(T, B);
-  const int src = slot < len ? kept[(int64_t)u * B + slot] : -1;
+  int src = slot < len ? kept[(int64_t)u * B + slot] : -1;
+  if (src >= 0 && !VATP_INB(src, T, dev_status)) src = -1;
   long long fx = 0;
   for (int r = 0; r < w; ++r) {
     const int j = T - w + r;                 // query position of this window row (may be < 0)
@@ -232,7 +242,7 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                          vnorm, kept, c, rows_pb, nbuf, dev_status);
   if (e != cudaSuccess) return e;
   if (s.window > 0 && win_rows) {
-    ring_kernel<<<dim3((cap + 127) / 128, s.units), 128, 0, st>>>(s.units, s.T, s.window, B, cap, win_rows, kept, c);
+    ring_kernel<<<dim3((cap + 127) / 128, s.units), 128, 0, st>>>(s.units, s.T, s.window, B, cap, win_rows, kept, c, dev_status);
     e = cudaGetLastError();
   }
   return e;

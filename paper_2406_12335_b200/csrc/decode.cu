@@ -168,6 +168,9 @@ decode_kernel(int split, int chunk, int B, int cap, int F, int R, int w, int nor
   const int len = c.len[u];
   const int fs = c.free_slot[u];
   const int t = c.next_pos[u];
+  // (bounds-checking build: state words out of range are reported; every access below is clamped to the CTA's rows)
+  (void)VATP_INB(len, cap, dev_status);
+  (void)VATP_INB(fs, cap, dev_status);
   const int hi = len + 1;                // slots [0, hi) are live once the new token is in
   const int cnt = max(min(hi - s0, rows_alloc), 0);
 

@@ -252,6 +252,17 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int fs = c.free_slot[u];
   const int t = c.next_pos[u];
   const int ls = c.last_slot[u];
+#ifdef VATP_DEBUG_BOUNDS
+  // the state words come from memory: out of range, nothing of this unit is touched
+  if (!VATP_INB(len, cap, dev_status) || !VATP_INB(fs, cap, dev_status) || !VATP_INB(ls + 1, cap + 1, dev_status)) {
+    if (tid == 0) ctrl_evicting = 0;
+    if (split > 1) {      // the unit's first barrier is still reached by every thread (all its CTAs read the same words)
+      cluster_wait_acquire();
+      cluster_arrive_release(); cluster_wait_acquire();
+    }
+    return;
+  }
+#endif
   const int hi = len + 1;                // slots [0, hi) are live once the new token is in
   const int cnt = max(min(hi - s0, rows_alloc), 0);
   const int fs_local = fs - s0;          // row of the incoming token inside this CTA's range (if owned)
@@ -503,7 +514,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       } else {
         S = is_new ? p : (state_in_smem ? as[i] : acc_g[i]) + p;
       }
-      acc_g[i] = S;
+      if (VATP_INB((int64_t)u * cap + slot, (int64_t)gridDim.x / split * cap, dev_status)) acc_g[i] = S;
       if (evicting) {
         const int ps = is_new ? t : (state_in_smem ? ps_s[i] : c.pos[(int64_t)u * cap + slot]);
         const float I = S * (is_new ? new_norm : (state_in_smem ? vs[i] : c.vnorm[(int64_t)u * cap + slot]));
@@ -517,7 +528,8 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   if (WINDOWED) {
     // recycled slot: the other rows of its ring column belong to the previous occupant (shared out over the unit's CTAs)
     for (int rr = rank * WT + tid; rr < w; rr += split * WT)
-      if (rr != t % w) c.ring[((int64_t)u * w + rr) * cap + fs] = 0.f;
+      if (rr != t % w && VATP_INB(((int64_t)u * w + rr) * cap + fs, (int64_t)gridDim.x / split * w * cap, dev_status))
+        c.ring[((int64_t)u * w + rr) * cap + fs] = 0.f;
   }
   if (!evicting) {
     if (rank == 0 && tid == 0) {
@@ -553,7 +565,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       if (ex.key[r] < best) { best = ex.key[r]; br = r; }
     if (br >= 0) {
       const int slot = ex.key_slot[br];
-      c.pos[(int64_t)u * cap + slot] = -1;
+      if (VATP_INB(slot, cap, dev_status)) c.pos[(int64_t)u * cap + slot] = -1;
       c.free_slot[u] = slot;
       c.len[u] = hi - 1;
       if (evicted) evicted[u] = ex.key_pos[br];

@@ -459,7 +459,8 @@ __device__ __forceinline__ void side_value_norms(const TcArgs& a, int lane) {
 #pragma unroll
         for (int o = 8; o; o >>= 1) acc = norm_merge(KIND, acc, __shfl_xor_sync(0xffffffffu, acc, o));
         const int tok = it.tile * TILE + r0 + 2 * j + sub;
-        if (part == 0 && tok < a.T) a.vnorm[(int64_t)it.u * a.T + tok] = norm_finish(KIND, acc);
+        if (part == 0 && tok < a.T && VATP_INB((int64_t)it.u * a.T + tok, (int64_t)a.units * a.T, a.dev_status))
+          a.vnorm[(int64_t)it.u * a.T + tok] = norm_finish(KIND, acc);
       }
     }
   }
@@ -571,7 +572,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             // has handed back accumulator n - 4 and is past the normalisers of chunk n - 5 and of all before it.
             // They are pass 1's output: nothing of it is read before that launch has completed.
             if (!waited_for_pass1) { asm volatile("griddepcontrol.wait;" ::: "memory"); waited_for_pass1 = true; }
-            bulk_load(sm.nlse[n % NLSE], a.lse2 + (int64_t)it.u * a.Tpad + tok0, CHUNK * 4, &sm.full[stg]);
+            if (VATP_INB((int64_t)it.u * a.Tpad + tok0 + CHUNK - 1, (int64_t)a.units * a.Tpad, a.dev_status))
+              bulk_load(sm.nlse[n % NLSE], a.lse2 + (int64_t)it.u * a.Tpad + tok0, CHUNK * 4, &sm.full[stg]);
           }
         }
       }
@@ -586,6 +588,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       for (uint32_t itl = 0; ok; ++itl) {
         const Item it = next_item(itl, false);
         if (it.u < 0) break;
+        if (!VATP_INB(it.u, a.units, a.dev_status) || !VATP_INB(it.tile, a.nt, a.dev_status) ||
+            !VATP_INB(it.c_first + it.c_count - 1, a.nch, a.dev_status)) break;
         const int fb = itl & 1;
         ok = mbar_wait(&sm.fixed_full[fb], (itl >> 1) & 1, abort_flag, a.dev_status);
         if (!ok) break;
@@ -652,6 +656,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           wo.base = reinterpret_cast<char*>(a.win_rows + (int64_t)u * a.window * a.T);
           wo.off = wo.full ? ((uint32_t)(q0 - a.wrow0) * (uint32_t)a.T + (uint32_t)tok) * 4u : 0u;
           wo.row4 = (uint32_t)a.T * 4u;
+#ifdef VATP_DEBUG_BOUNDS
+          // the first and the last window entry this slice may write
+          const int64_t lim = (int64_t)a.units * a.window * a.T;
+          if (wo.hi > wo.lo && (!VATP_INB((wo.p - a.win_rows) + (int64_t)wo.lo * a.T, lim, a.dev_status) ||
+                                !VATP_INB((wo.p - a.win_rows) + (int64_t)(wo.hi - 1) * a.T, lim, a.dev_status))) {
+            wo.lo = wo.hi = 0;
+            wo.full = false;
+          }
+#endif
         }
         return wo;
       };
@@ -676,6 +689,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         // pass 2: the chunk's negated normalisers arrived with its tiles (the accumulator being complete
         // implies that those copies are); indexed by the column inside this warp's tile
         const float* lse_t = sm.nlse[(n0 + c) % NLSE] + half * TILE;
+        if (!VATP_INB(it.u, a.units, a.dev_status) || !VATP_INB(tok - row, (int64_t)a.nt * TILE, a.dev_status)) { ok = false; break; }
         tmem_ld32(t_addr, x);
         tmem_ld_wait();
         if (stile == it.tile) consume32<PASS, true, WIN>(x, cbase, row, a.scale_log2, m_run, l_run, cs, lse_t, wout(stile, cbase));
@@ -713,14 +727,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           const float lse2 = m + log2f(l);
           // queries outside the prompt or before the history window contribute nothing to pass 2
           // (stored negated: pass 2 adds it to the scaled dot product)
-          a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? -lse2 : -INFINITY;
+          if (VATP_INB((int64_t)u * a.Tpad + tok, (int64_t)a.units * a.Tpad, a.dev_status))
+            a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? -lse2 : -INFINITY;
           // an odd tile count leaves half a chunk of padding that pass 2 reads as "no query"
-          if ((a.nt & 1) && it.tile == a.nt - 1) a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
-          if (a.lse_out && tok < a.T) a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
+          if ((a.nt & 1) && it.tile == a.nt - 1 && VATP_INB((int64_t)u * a.Tpad + tok + TILE, (int64_t)a.units * a.Tpad, a.dev_status))
+            a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
+          if (a.lse_out && tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status))
+            a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
         } else {
           const float tot = hsum2(add2(cs[0], cs[1])) + (sm.part_a[pi][0][row] + sm.part_a[pi][1][row]) + sm.part_a[pi][2][row];
           mbar_arrive(&sm.comb_empty[pi]);
-          if (tok < a.T) {
+          if (tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status)) {
             const int64_t o = (int64_t)u * a.T + tok;
             a.attn_acc[o] = tot;
             a.score[o] = tot * n1;
@@ -924,7 +941,7 @@ window_ring_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
           float pr = 0.f;
           if (ps >= 0 && ps <= j0 + i) pr = ex2(fmaf(x[i], scale_log2, nl));
           fx += prob_to_fixed(pr);
-          if (slot < cap) ring_s[off] = pr;
+          if (slot < cap && VATP_INB(off, (int64_t)w * cap, dev_status)) ring_s[off] = pr;
           off += cap;
           if (++rr == w) { rr = 0; off = 0; }
         }

@@ -25,7 +25,7 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 
 template <bool STAGED>
 __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F, int R, const float* __restrict__ score,
-                                                             int32_t* __restrict__ kept) {
+                                                             int32_t* __restrict__ kept, int32_t* dev_status) {
   extern __shared__ __align__(16) uint32_t keys_s[];  // STAGED: keys of the middle range (from index `pad` on)
   __shared__ uint32_t hist[256];
   __shared__ uint32_t hist_w[SEL_WARPS][256];      // per-warp counts of the current pass
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int v = v0 + j * SEL_THREADS + tid;
-        if (v < nvec) dst4[v] = make_uint4(order_key(x[j].x), order_key(x[j].y), order_key(x[j].z), order_key(x[j].w));
+        if (v < nvec && VATP_INB(pad + a0 + 4 * v + 3, n + 4, dev_status)) dst4[v] = make_uint4(order_key(x[j].x), order_key(x[j].y), order_key(x[j].z), order_key(x[j].w));
       }
     }
     if (tid < a0) keys_s[pad + tid] = order_key(mid[tid]);
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
     const uint32_t eq_b = __ballot_sync(0xffffffffu, is_eq);
     const bool keep = i < hi_i && (key > tau || (is_eq && eq_rank + __popc(eq_b & lt_mask) < need_eq));
     const uint32_t keep_b = __ballot_sync(0xffffffffu, keep);
-    if (keep) out[F + o + __popc(keep_b & lt_mask)] = F + i;
+    if (keep && VATP_INB(F + o + __popc(keep_b & lt_mask), B - R, dev_status)) out[F + o + __popc(keep_b & lt_mask)] = F + i;
     o += __popc(keep_b);
     eq_rank += __popc(eq_b);
   }
@@ -188,17 +188,18 @@ __global__ void __launch_bounds__(SEL_THREADS) select_kernel(int T, int B, int F
 
 }  // namespace
 
-cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st) {
+cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, int32_t* dev_status,
+                          cudaStream_t st) {
   const int n = T > B ? T - R - F : 0;
   const size_t bytes = (size_t)(n + 4) * sizeof(uint32_t);     // up to three words of alignment padding
   if (bytes <= 160 * 1024) {      // beside the 33 KB of histograms
     cudaError_t e = cudaFuncSetAttribute(select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
     if (e != cudaSuccess) return e;
     DependentLaunch dl(dim3(units), dim3(SEL_THREADS), bytes, st);
-    return cudaLaunchKernelEx(&dl.cfg, select_kernel<true>, T, B, F, R, score, kept);
+    return cudaLaunchKernelEx(&dl.cfg, select_kernel<true>, T, B, F, R, score, kept, dev_status);
   }
   DependentLaunch dl(dim3(units), dim3(SEL_THREADS), 0, st);
-  return cudaLaunchKernelEx(&dl.cfg, select_kernel<false>, T, B, F, R, score, kept);
+  return cudaLaunchKernelEx(&dl.cfg, select_kernel<false>, T, B, F, R, score, kept, dev_status);
 }
 
 }  // namespace vatp

@@ -102,6 +102,7 @@ const char* vatp_status_string(vatp_status s) {
     case VATP_ERR_CUDA: return "CUDA error";
     case VATP_ERR_TIMEOUT: return "device-side wait ran out";
     case VATP_ERR_STATIC_SCRATCH: return "problem exceeds the library's built-in scratch array";
+    case VATP_ERR_BOUNDS: return "a kernel computed an index outside its array (bounds-checking build)";
   }
   return "unknown status";
 }
@@ -131,13 +132,13 @@ vatp_status vatp_prefill_scores_from_lse(const vatp_params* p, const void* q, co
 
 vatp_status vatp_select(const vatp_params* p, const float* score, int32_t* kept_idx, void* workspace,
                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
-  (void)workspace; (void)workspace_bytes; (void)dev_status;
+  (void)workspace; (void)workspace_bytes;
   vatp_status s = check_params(p, true);
   if (s != VATP_OK) return s;
   if (!score || !kept_idx) return VATP_ERR_INVALID_ARG;
   decode_history_forget(static_cast<cudaStream_t>(cuda_stream));
   cudaError_t e = launch_select(p->batch * p->heads, p->seq_len, p->budget, p->n_sink, p->n_recent, score, kept_idx,
-                                static_cast<cudaStream_t>(cuda_stream));
+                                dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
 

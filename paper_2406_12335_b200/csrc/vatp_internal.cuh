@@ -29,6 +29,20 @@ __device__ __forceinline__ float norm_fold(int kind, float part, float x) {
 __device__ __forceinline__ float norm_merge(int kind, float a, float b) { return kind == VATP_NORM_LINF ? fmaxf(a, b) : a + b; }
 __device__ __forceinline__ float norm_finish(int kind, float part) { return kind == VATP_NORM_L2 ? sqrtf(part) : part; }
 
+// Bounds-checking build (-DVATP_DEBUG_BOUNDS): VATP_INB(i, n, status) is false, and records VATP_ERR_BOUNDS in the
+// status word, when index i lies outside [0, n); the caller then skips the access.  In the ordinary build it is the
+// constant true and costs nothing.
+#ifdef VATP_DEBUG_BOUNDS
+__device__ __forceinline__ bool vatp_in_bounds(long long i, long long n, int32_t* status) {
+  if (i >= 0 && i < n) return true;
+  if (status) atomicExch(status, (int)VATP_ERR_BOUNDS);
+  return false;
+}
+#define VATP_INB(i, n, status) vatp::vatp_in_bounds((long long)(i), (long long)(n), (status))
+#else
+#define VATP_INB(i, n, status) true
+#endif
+
 // slots per unit in the decode state: budget + 1, rounded up to a multiple of 8 so that every
 // per-slot array of a unit starts on a 32-byte boundary (bulk copies need 16)
 __host__ __device__ inline int cache_capacity(int budget) { return (budget + 1 + 7) & ~7; }
@@ -82,7 +96,8 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
                               int32_t* dev_status, cudaStream_t st, const float* lse_in = nullptr);
 size_t prefill_tc_workspace_bytes(int units, int T);  // padded log2-domain row normalisers
-cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, cudaStream_t st);
+cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, int32_t* dev_status,
+                          cudaStream_t st);
 cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, const void* v, const float* attn_acc,
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
                            int32_t* dev_status, cudaStream_t st);

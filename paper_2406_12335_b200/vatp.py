@@ -10,7 +10,8 @@ import os
 
 import torch
 
-_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libvatp.so")
+# VATP_LIBRARY selects another build of the library (the bounds-checking build libvatp_dbg.so)
+_LIB_PATH = os.environ.get("VATP_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libvatp.so")
 if not os.path.exists(_LIB_PATH):
     raise ImportError(f"{_LIB_PATH} is missing: build it with `python -m paper_2406_12335_b200.build`")
 lib = C.CDLL(_LIB_PATH)

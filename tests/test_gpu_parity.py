@@ -523,3 +523,26 @@ def test_optional_outputs_may_be_null(dtype, d):
         torch.cuda.synchronize()
         assert torch.equal(o1, o2)
     assert torch.equal(full.cache.pos, bare.cache.pos) and torch.equal(full.cache.acc, bare.cache.acc)
+
+
+def test_bounds_checking_build_reports_no_violation():
+    """The library built with -DVATP_DEBUG_BOUNDS range-checks every row, slot, window-row and scratch index its
+    kernels compute (an index outside its array is skipped and reported as VATP_ERR_BOUNDS in the status word,
+    which every test here asserts to be zero).  Ragged, windowed, large-cache and graph cases run once more on
+    that build, in a process of their own; it stands in for a memory checker, which cannot be run here."""
+    import os
+    import subprocess
+    import sys
+    from paper_2406_12335_b200 import build
+    lib = build.build(debug_bounds=True)
+    env = dict(os.environ, VATP_LIBRARY=lib)
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    sel = ("ragged or degenerate or windowed_indicator_shapes or general_kernels or large_cache or few_units "
+           "or exact_ties or unstaged or strided or static_scratch_matches or rebuilt")
+    r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "tests/test_zz_no_alloc.py", "-x", "-q",
+                        "-m", "gpu", "-k", sel, "-p", "no:cacheprovider"], cwd=root, env=env, capture_output=True, text=True)
+    tail = (r.stdout + r.stderr)[-2000:]
+    assert r.returncode == 0, tail
+    assert " passed" in tail and "libvatp_dbg" in subprocess.run(
+        [sys.executable, "-c", "from paper_2406_12335_b200 import vatp; print(vatp._LIB_PATH)"], cwd=root, env=env,
+        capture_output=True, text=True).stdout
