@@ -518,3 +518,81 @@ def test_workload5_is_the_scissorhands_split_at_half_budget():
     assert (wl.batch, wl.heads, wl.head_dim, wl.seq_len, wl.decode_steps) == (12, 32, 128, 4096, 128)
     p = presets.appendix_a("scissorhands", wl.seq_len, 0.5)
     assert (p["budget"], p["n_sink"], p["n_recent"], p["window"]) == (wl.budget, wl.n_sink, wl.n_recent, wl.window)
+
+
+# ------------------------------------------------------------------ grouped-query attention (Limitations)
+def _loop_group_indicator(qg, k, scale):
+    """Mean over the group's heads of the accumulated attention, by explicit loops with math.exp."""
+    G, T, d = qg.shape
+    S = [0.0] * T
+    for g in range(G):
+        for j in range(T):
+            logits = [scale * sum(float(qg[g, j, c]) * float(k[i, c]) for c in range(d)) for i in range(j + 1)]
+            m = max(logits)
+            e = [math.exp(x - m) for x in logits]
+            z = math.fsum(e)
+            for i in range(j + 1):
+                S[i] += e[i] / z / G
+    return np.array(S)
+
+
+def test_gqa_prefill_matches_loops_and_reductions():
+    rng = np.random.default_rng(11)
+    G, T, d = 3, 7, 4
+    qg, k, v = rng.normal(size=(G, T, d)), rng.normal(size=(T, d)), rng.normal(size=(T, d))
+    r = O.prefill_gqa(qg, k, v, 0.5)
+    assert np.allclose(r["S"], _loop_group_indicator(qg, k, 0.5), rtol=1e-12, atol=1e-14)
+    assert np.allclose(r["I"], r["S"] * np.abs(v).sum(1), rtol=1e-14)
+    assert abs(r["S"].sum() - T) < 1e-12                       # a mean of G indicators that each sum to T
+    # one head per group is plain multi-head attention
+    one = O.prefill_gqa(qg[:1], k, v, 0.5)
+    mha = O.prefill(qg[0], k, v, 0.5)
+    assert np.array_equal(one["S"], mha["S"]) and np.array_equal(one["I"], mha["I"]) and np.array_equal(one["lse"][0], mha["lse"])
+    # identical query heads change nothing either
+    same = O.prefill_gqa(np.stack([qg[0]] * 4), k, v, 0.5)
+    assert np.allclose(same["S"], mha["S"], rtol=1e-13)
+    # the group mean really mixes the heads: it differs from every single head's indicator and is their average
+    assert all(not np.allclose(r["S"], r["S_heads"][g]) for g in range(G))
+    assert np.allclose(r["S"], r["S_heads"].mean(axis=0), rtol=1e-14)
+    # a head that puts all its mass on key 0 lifts S_0 by exactly T / G over the other heads' share
+    hot = qg.copy(); kk = k.copy()
+    kk[0] = 0; kk[0, 0] = 200.0
+    hot[1] = 0; hot[1, :, 0] = 1.0                             # head 1: logit 100 on key 0, 0 elsewhere
+    rh = O.prefill_gqa(hot, kk, v, 0.5)
+    assert abs(rh["S_heads"][1][0] - T) < 1e-9 and np.all(rh["S_heads"][1][1:] < 1e-9)
+    # windowed indicator (Eq. 3) under the same group mean; w >= T is the accumulated one
+    rw = O.prefill_gqa(qg, k, v, 0.5, window=3)
+    assert abs(rw["S"].sum() - 3) < 1e-12
+    assert np.allclose(O.prefill_gqa(qg, k, v, 0.5, window=T)["S"], r["S"], rtol=1e-14)
+
+
+def test_gqa_decode_step_matches_prefill_on_the_longer_prompt():
+    """Prefill on T tokens + one grouped decode step with nothing evicted = prefill on T + 1 tokens: the
+    indicator (group mean) and every head's output row."""
+    rng = np.random.default_rng(12)
+    G, T, d = 4, 9, 6
+    qg, k, v = rng.normal(size=(G, T + 1, d)), rng.normal(size=(T + 1, d)), rng.normal(size=(T + 1, d))
+    scale = 0.4
+    short = O.prefill_gqa(qg[:, :T], k[:T], v[:T], scale)
+    full = O.prefill_gqa(qg, k, v, scale)
+    st = O.DecodeState(k[:T], v[:T], short["S"], short["n1"], np.arange(T), T)
+    res = O.decode_step(st, qg[:, T], k[T], v[T], scale, B=T + 5, F=0, R=0)
+    assert res["evicted"] == -1 and res["out"].shape == (G, d)
+    assert np.allclose(st.indicator(), full["S"], rtol=1e-12)
+    for g in range(G):
+        a = O.attention_probs(qg[g], k, scale)
+        assert np.allclose(res["out"][g], a[T] @ v, rtol=1e-12)
+    # one head per group is the ordinary step
+    st1 = O.DecodeState(k[:T], v[:T], short["S"], short["n1"], np.arange(T), T)
+    st2 = O.DecodeState(k[:T], v[:T], short["S"], short["n1"], np.arange(T), T)
+    r1 = O.decode_step(st1, qg[:1, T], k[T], v[T], scale, B=4, F=1, R=2)
+    r2 = O.decode_step(st2, qg[0, T], k[T], v[T], scale, B=4, F=1, R=2)
+    assert r1["evicted"] == r2["evicted"] and np.allclose(r1["out"][0], r2["out"]) and np.allclose(st1.S, st2.S)
+    # the step evicts on the group-mean indicator: with equal norms the victim is the arg-min of the mean
+    st3 = O.DecodeState(k[:T], np.ones((T, d)), short["S"], np.full(T, float(d)), np.arange(T), T)
+    r3 = O.decode_step(st3, qg[:, T], k[T], np.ones(d), scale, B=T, F=0, R=1)
+    mean_after = short["S"] + r3["p"][:T]
+    assert r3["evicted"] == int(np.argmin(mean_after))
+    with pytest.raises(ValueError):
+        stw = O.DecodeState(k[:T], v[:T], short["S"], short["n1"], np.arange(T), T, window=4, window_rows=np.zeros((4, T)))
+        O.decode_step(stw, qg[:, T], k[T], v[T], scale, B=T + 5, F=0, R=0)
