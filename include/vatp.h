@@ -23,6 +23,17 @@
  *     VATP_ERR_CUDA.  Device-side conditions (a bounded wait that ran out) are written to
  *     *dev_status (device int32, 0 = fine; caller zeroes it and reads it after sync); the
  *     kernels never trap.
+ *   - Grouped-query attention (the Limitations section's "Compatibility with grouped-query
+ *     attention", left there to future work with a pointer to a group-wise score): with
+ *     params->kv_heads < heads, q (and q_new, out, lse_out) keep `heads` heads while k, v, every
+ *     per-token output (attn_acc, vnorm, score, kept_idx) and the decode state have kv_heads heads:
+ *     a unit is a (batch, KV head) pair, the G = heads / kv_heads query heads h = g * G .. g * G + G - 1
+ *     share KV head g, and the indicator of a cached token is the MEAN over those query heads of its
+ *     Eq. 2 / Eq. 3 indicator (prefill), advanced per step by the mean of the heads' probabilities
+ *     (decode; accumulated indicator only).  Layouts must be contiguous (stride fields 0); the
+ *     history-window decode state, vatp_prefill_scores_from_lse and win_rows are not available with it
+ *     (VATP_ERR_UNSUPPORTED), and the workspace grows by G partial indicators.  The decode step runs a
+ *     plain general kernel, not the tuned one.
  *   - Inputs are assumed finite.
  *   - A second build of the library (compiled with -DVATP_DEBUG_BOUNDS) range-checks every row, slot,
  *     window-row and scratch index its kernels compute before the access; an index outside its array is
@@ -73,6 +84,8 @@ typedef struct {
   int32_t n_recent;          /* R: most recent tokens always kept; F + R <= B                  */
   int32_t norm_kind;         /* vatp_norm_kind of the value norm in Eq. 4; 0 = the paper's l1   */
   int32_t flags;             /* OR of vatp_flags; 0 = none                                     */
+  int32_t kv_heads;          /* grouped-query attention: KV heads (a divisor of heads); 0 or
+                                == heads = multi-head attention.  See "Grouped-query attention" */
   int64_t stride_b, stride_h, stride_t; /* element strides of q, k, v; 0 = contiguous          */
 } vatp_params;
 

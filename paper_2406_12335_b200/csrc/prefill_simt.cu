@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(NTHREADS) rowstats_kernel(Shape sh, const T* _
   const int u = blockIdx.y;
   const int q0 = first_row + blockIdx.x * TILE;
   if (q0 >= sh.T) return;
-  const T* qu = q + unit_offset(sh, u);
+  const T* qu = q + unit_offset_q(sh, u);
   const T* ku = k + unit_offset(sh, u);
   const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
 
@@ -111,7 +111,7 @@ __global__ void __launch_bounds__(NTHREADS) rowstats_kernel(Shape sh, const T* _
       }
     }
     const int row = q0 + ty + 16 * i;
-    if (tx == 0 && row < sh.T) lse[(int64_t)u * sh.T + row] = m[i] + logf(l[i]);
+    if (tx == 0 && row < sh.T) lse[unit_offset_lse(sh, u) + row] = m[i] + logf(l[i]);
   }
 }
 
@@ -129,7 +129,7 @@ colsum_kernel(Shape sh, const T* __restrict__ q, const T* __restrict__ k, const 
   float* red = lse_s + TILE;            // [16][TILE]
   const int u = blockIdx.y;
   const int k0 = blockIdx.x * TILE;
-  const T* qu = q + unit_offset(sh, u);
+  const T* qu = q + unit_offset_q(sh, u);
   const T* ku = k + unit_offset(sh, u);
   const T* vu = v + unit_offset(sh, u);
   const int ty = threadIdx.x / 16, tx = threadIdx.x % 16;
@@ -157,7 +157,7 @@ colsum_kernel(Shape sh, const T* __restrict__ q, const T* __restrict__ k, const 
     __syncthreads();
     const int rows_valid = min(TILE, sh.T - q0);
     load_tile(Qs, ld, qu, sh.st, q0, rows_valid, sh.d);
-    if (threadIdx.x < TILE) lse_s[threadIdx.x] = threadIdx.x < rows_valid ? lse[(int64_t)u * sh.T + q0 + threadIdx.x] : 0.f;
+    if (threadIdx.x < TILE) lse_s[threadIdx.x] = threadIdx.x < rows_valid ? lse[unit_offset_lse(sh, u) + q0 + threadIdx.x] : 0.f;
     __syncthreads();
     float s[4][4];
     micro_gemm(Qs, Ks, ld, sh.d, ty, tx, s);

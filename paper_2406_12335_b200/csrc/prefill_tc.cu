@@ -377,7 +377,8 @@ struct TcArgs {
   const __nv_bfloat16* v;
   int64_t sb, sh, st;       // element strides of v
   float* lse2;              // [units][Tpad] NEGATED log2-domain row normalisers (-inf where no query counts)
-  float* lse_out;           // [units][T] natural-log copy, nullable
+  float* lse_out;           // natural-log copy, nullable: unit (b, h)'s T values start at b * lse_sb + h * lse_sh
+  int64_t lse_sb, lse_sh;
   float* attn_acc;
   float* vnorm;
   float* score;
@@ -732,8 +733,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           // an odd tile count leaves half a chunk of padding that pass 2 reads as "no query"
           if ((a.nt & 1) && it.tile == a.nt - 1 && VATP_INB((int64_t)u * a.Tpad + tok + TILE, (int64_t)a.units * a.Tpad, a.dev_status))
             a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
-          if (a.lse_out && tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status))
-            a.lse_out[(int64_t)u * a.T + tok] = lse2 * 0.69314718055994531f;
+          if (a.lse_out && tok < a.T)
+            a.lse_out[(int64_t)(u / a.heads) * a.lse_sb + (int64_t)(u % a.heads) * a.lse_sh + tok] = lse2 * 0.69314718055994531f;
         } else {
           const float tot = hsum2(add2(cs[0], cs[1])) + (sm.part_a[pi][0][row] + sm.part_a[pi][1][row]) + sm.part_a[pi][2][row];
           mbar_arrive(&sm.comb_empty[pi]);
@@ -987,9 +988,9 @@ EncodeTiledFn encode_fn() {
 }
 
 // [batch, heads, T, 128] bf16 with element strides (sb, sh, st, 1); box = 64 x 128 rows, 128-byte swizzle
-bool make_map(CUtensorMap* m, const void* base, const Shape& s) {
+bool make_map(CUtensorMap* m, const void* base, const Shape& s, bool of_q = false) {
   const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)s.T, (cuuint64_t)s.heads, (cuuint64_t)(s.units / s.heads)};
-  const cuuint64_t strides[3] = {(cuuint64_t)s.st * 2, (cuuint64_t)s.sh * 2, (cuuint64_t)s.sb * 2};
+  const cuuint64_t strides[3] = {(cuuint64_t)s.st * 2, (cuuint64_t)(of_q ? s.qsh : s.sh) * 2, (cuuint64_t)(of_q ? s.qsb : s.sb) * 2};
   const cuuint32_t box[4] = {64, TILE, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return encode_fn()(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
@@ -1058,7 +1059,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
                               int32_t* dev_status, cudaStream_t st, const float* lse_in) {
   CUtensorMap tm_q, tm_k;
-  if (!make_map(&tm_q, q, s) || !make_map(&tm_k, k, s)) return cudaErrorInvalidValue;
+  if (!make_map(&tm_q, q, s, true) || !make_map(&tm_k, k, s)) return cudaErrorInvalidValue;
   TcArgs a;
   a.units = s.units; a.heads = s.heads; a.T = s.T;
   a.nt = (s.T + TILE - 1) / TILE;
@@ -1067,6 +1068,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.scale_log2 = s.scale * 1.4426950408889634f;
   a.v = static_cast<const __nv_bfloat16*>(v);
   a.sb = s.sb; a.sh = s.sh; a.st = s.st;
+  a.lse_sb = s.lse_sb; a.lse_sh = s.lse_sh;
   a.lse2 = lse_ws; a.lse_out = lse_out; a.attn_acc = attn_acc; a.vnorm = vnorm; a.score = score;
   a.dev_status = dev_status;
   a.norm = s.norm;
@@ -1124,7 +1126,7 @@ cudaError_t launch_window_ring_tc(const Shape& s, int B, const void* q, const fl
                                   int32_t* dev_status, cudaStream_t st) {
   const int cap = cache_capacity(B);
   CUtensorMap tm_q, tm_kc;
-  if (!make_map(&tm_q, q, s) || !make_rows_map_bf16(&tm_kc, c.k_cache, (uint64_t)s.units * cap, TILE)) return cudaErrorInvalidValue;
+  if (!make_map(&tm_q, q, s, true) || !make_rows_map_bf16(&tm_kc, c.k_cache, (uint64_t)s.units * cap, TILE)) return cudaErrorInvalidValue;
   if ((int64_t)s.window * cap >= ((int64_t)1 << 31)) return cudaErrorInvalidValue;
   const size_t smem = sizeof(RingSmem) + 1024;
   cudaError_t e = cudaFuncSetAttribute(window_ring_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -23,17 +23,31 @@ vatp_status check_params(const vatp_params* p, bool need_T) {
   if (!(p->scale > 0.f)) return VATP_ERR_INVALID_ARG;
   if (p->stride_b < 0 || p->stride_h < 0 || p->stride_t < 0) return VATP_ERR_INVALID_ARG;
   if (p->flags & ~(int32_t)VATP_FLAG_DECODE_OVERLAP) return VATP_ERR_INVALID_ARG;
+  if (p->kv_heads < 0 || p->kv_heads > p->heads || (p->kv_heads && p->heads % p->kv_heads)) return VATP_ERR_INVALID_ARG;
+  if (p->kv_heads && p->kv_heads < p->heads && (p->stride_b || p->stride_h || p->stride_t)) return VATP_ERR_INVALID_ARG;
   return VATP_OK;
 }
 
+// query heads per KV head (1: multi-head attention) and the number of KV heads
+inline int group_of(const vatp_params* p) { return p->kv_heads > 0 ? p->heads / p->kv_heads : 1; }
+inline int kv_heads_of(const vatp_params* p) { return p->kv_heads > 0 ? p->kv_heads : p->heads; }
+
+// The units are the (batch, KV head) pairs.  With grouped queries (contiguous layouts only) q has G times as many
+// heads: a launch takes one query head of every group, i.e. q as a view with head stride G * T * d (the caller
+// offsets the q pointer by g * T * d and the row-normaliser pointer by g * T).
 vatp_status make_shape(const vatp_params* p, Shape* s) {
-  s->units = p->batch * p->heads;
-  s->heads = p->heads;
+  const int kvh = kv_heads_of(p), G = group_of(p);
+  s->units = p->batch * kvh;
+  s->heads = kvh;
   s->T = p->seq_len;
   s->d = p->head_dim;
   s->st = p->stride_t ? p->stride_t : p->head_dim;
   s->sh = p->stride_h ? p->stride_h : (int64_t)p->seq_len * s->st;
-  s->sb = p->stride_b ? p->stride_b : (int64_t)p->heads * s->sh;
+  s->sb = p->stride_b ? p->stride_b : (int64_t)kvh * s->sh;
+  s->qsh = (int64_t)G * s->sh;
+  s->qsb = G > 1 ? (int64_t)p->heads * s->sh : s->sb;
+  s->lse_sh = (int64_t)G * p->seq_len;
+  s->lse_sb = (int64_t)p->heads * p->seq_len;
   s->scale = p->scale;
   s->window = p->indicator == VATP_IND_WINDOW ? p->window_w : 0;
   s->norm = p->norm_kind;
@@ -43,10 +57,17 @@ vatp_status make_shape(const vatp_params* p, Shape* s) {
   return VATP_OK;
 }
 
-// row normalisers of pass 1, padded to whole 128-row tiles per unit
+// row normalisers of pass 1, padded to whole 128-row tiles per unit; with grouped queries, then the G partial
+// indicators [G][units][T] that the group mean is taken of
 inline size_t lse_bytes(const vatp_params* p) {
-  size_t n = prefill_tc_workspace_bytes(p->batch * p->heads, p->seq_len);
+  size_t n = prefill_tc_workspace_bytes(p->batch * kv_heads_of(p), p->seq_len);
   return (n + 255) / 256 * 256;
+}
+inline size_t workspace_need(const vatp_params* p) {
+  const int G = group_of(p);
+  size_t n = lse_bytes(p);
+  if (G > 1) n += ((size_t)G * p->batch * kv_heads_of(p) * p->seq_len * sizeof(float) + 255) / 256 * 256;
+  return n;
 }
 
 bool cache_ok(const vatp_cache* c, bool windowed) {
@@ -70,12 +91,39 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
   Shape sh;
   s = make_shape(p, &sh);
   if (s != VATP_OK) return s;
-  if (!workspace || workspace_bytes < lse_bytes(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
+  const int G = group_of(p);
+  if (G > 1 && (lse_in || win_rows)) return VATP_ERR_UNSUPPORTED;
+  if (!workspace || workspace_bytes < workspace_need(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return VATP_ERR_WORKSPACE;
   float* ws = static_cast<float*>(workspace);
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   decode_history_forget(st);
   cudaError_t e;
+  if (G > 1) {
+    // One query head of every KV group per round: the multi-head kernels on strided views of q, each round's
+    // indicator into its own slice of the workspace, then the mean over the rounds (fixed order) and Eq. 4.
+    const size_t n = (size_t)sh.units * sh.T;
+    float* part = reinterpret_cast<float*>(static_cast<char*>(workspace) + lse_bytes(p));
+    const int eb = p->dtype == VATP_F32 ? 4 : 2;
+    const bool tc = p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available();
+    // the general kernel keeps its (natural-log) normalisers in the caller's layout: lse_out, or a scratch copy of
+    // that layout at the head of the workspace when the caller wants none (it fits: G * units * T floats <= `part`)
+    e = cudaSuccess;
+    for (int g = 0; g < G && e == cudaSuccess; ++g) {
+      const char* qg = static_cast<const char*>(q) + (size_t)g * sh.sh * eb;
+      float* lse_g = lse_out ? lse_out + (size_t)g * sh.T : nullptr;
+      if (tc) {
+        e = launch_prefill_tc(sh, qg, k, v, ws, lse_g, part + g * n, vnorm, score, nullptr, dev_status, st, nullptr);
+      } else {
+        Shape sg = sh;
+        float* lse_buf = lse_g;
+        if (!lse_buf) { lse_buf = ws; sg.lse_sb = (int64_t)sh.heads * sh.T; sg.lse_sh = sh.T; }   // plain [units][T] scratch
+        e = launch_prefill_simt(sg, p->dtype, qg, k, v, lse_buf, part + g * n, vnorm, score, nullptr, st);
+      }
+    }
+    if (e == cudaSuccess) e = launch_group_mean(G, (int64_t)n, part, vnorm, attn_acc, score, st);
+    return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+  }
   if (p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available()) {
     e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st, lse_in);
   } else if (lse_in) {
@@ -111,7 +159,7 @@ int32_t vatp_cache_capacity(int32_t budget) { return budget > 0 ? cache_capacity
 
 size_t vatp_workspace_bytes(const vatp_params* p) {
   if (check_params(p, true) != VATP_OK) return 0;
-  return lse_bytes(p);
+  return workspace_need(p);
 }
 
 vatp_status vatp_prefill_scores(const vatp_params* p, const void* q, const void* k, const void* v, float* lse_out,
@@ -137,7 +185,7 @@ vatp_status vatp_select(const vatp_params* p, const float* score, int32_t* kept_
   if (s != VATP_OK) return s;
   if (!score || !kept_idx) return VATP_ERR_INVALID_ARG;
   decode_history_forget(static_cast<cudaStream_t>(cuda_stream));
-  cudaError_t e = launch_select(p->batch * p->heads, p->seq_len, p->budget, p->n_sink, p->n_recent, score, kept_idx,
+  cudaError_t e = launch_select(p->batch * kv_heads_of(p), p->seq_len, p->budget, p->n_sink, p->n_recent, score, kept_idx,
                                 dev_status, static_cast<cudaStream_t>(cuda_stream));
   return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
 }
@@ -150,6 +198,7 @@ vatp_status vatp_compact(const vatp_params* p, const void* k, const void* v, con
   const bool windowed = p->indicator == VATP_IND_WINDOW;
   if (!k || !v || !attn_acc || !vnorm || !kept_idx || !cache_ok(cache, windowed)) return VATP_ERR_INVALID_ARG;
   if (windowed && !win_rows) return VATP_ERR_INVALID_ARG;
+  if (windowed && group_of(p) > 1) return VATP_ERR_UNSUPPORTED;
   if (!aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
   Shape sh;
   s = make_shape(p, &sh);
@@ -166,6 +215,7 @@ vatp_status vatp_compact_window(const vatp_params* p, const void* q, const void*
   vatp_status s = check_params(p, true);
   if (s != VATP_OK) return s;
   if (p->indicator != VATP_IND_WINDOW) return VATP_ERR_INVALID_ARG;
+  if (group_of(p) > 1) return VATP_ERR_UNSUPPORTED;
   if (!q || !k || !v || !lse || !attn_acc || !vnorm || !kept_idx || !cache_ok(cache, true)) return VATP_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
   Shape sh;
@@ -186,6 +236,15 @@ vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, cons
   const bool windowed = p->indicator == VATP_IND_WINDOW;
   if (!q_new || !k_new || !v_new || !out || !cache_ok(cache, windowed)) return VATP_ERR_INVALID_ARG;
   if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return VATP_ERR_INVALID_ARG;
+  if (group_of(p) > 1) {
+    if (windowed) return VATP_ERR_UNSUPPORTED;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    decode_history_forget(st);
+    const cudaError_t e = launch_decode_gqa(p->batch * kv_heads_of(p), group_of(p), p->head_dim, p->dtype, p->budget, p->n_sink,
+                                            p->n_recent, p->norm_kind, p->scale, *cache, q_new, k_new, v_new, out, evicted_pos,
+                                            dev_status, st);
+    return e == cudaSuccess ? VATP_OK : (e == cudaErrorNotSupported ? VATP_ERR_UNSUPPORTED : VATP_ERR_CUDA);
+  }
   Shape sh;
   std::memset(&sh, 0, sizeof(sh));
   sh.units = p->batch * p->heads;

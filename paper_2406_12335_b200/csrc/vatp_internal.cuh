@@ -14,7 +14,10 @@ struct Shape {
   int units;           // batch * heads
   int heads;
   int T, d;
-  int64_t sb, sh, st;  // element strides of q/k/v
+  int64_t sb, sh, st;  // element strides of k and v (and of q, unless qsb / qsh say otherwise)
+  int64_t qsb, qsh;    // batch and head strides of q (grouped-query attention runs one query head of every KV
+                       // group per launch: the units are then the KV heads and q is a strided view)
+  int64_t lse_sb, lse_sh;  // where unit (b, h)'s row normalisers start in the caller's [.., T] array: b * lse_sb + h * lse_sh
   float scale;
   int window;          // 0 = accumulate over all queries (Eq. 2); >0 = last `window` queries (Eq. 3)
   int norm;            // vatp_norm_kind of the value norm in Eq. 4
@@ -47,9 +50,15 @@ __device__ __forceinline__ bool vatp_in_bounds(long long i, long long n, int32_t
 // per-slot array of a unit starts on a 32-byte boundary (bulk copies need 16)
 __host__ __device__ inline int cache_capacity(int budget) { return (budget + 1 + 7) & ~7; }
 
-// offset (in elements) of unit u's first row
+// offset (in elements) of unit u's first row in k and v, in q, and in the caller's row-normaliser array
 __host__ __device__ inline int64_t unit_offset(const Shape& s, int u) {
   return (int64_t)(u / s.heads) * s.sb + (int64_t)(u % s.heads) * s.sh;
+}
+__host__ __device__ inline int64_t unit_offset_q(const Shape& s, int u) {
+  return (int64_t)(u / s.heads) * s.qsb + (int64_t)(u % s.heads) * s.qsh;
+}
+__host__ __device__ inline int64_t unit_offset_lse(const Shape& s, int u) {
+  return (int64_t)(u / s.heads) * s.lse_sb + (int64_t)(u % s.heads) * s.lse_sh;
 }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }
@@ -106,6 +115,12 @@ cudaError_t launch_window_ring(const Shape& s, int dtype, int B, const void* q, 
                                int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_window_ring_tc(const Shape& s, int B, const void* q, const float* lse, const vatp_cache& c,
                                   int32_t* dev_status, cudaStream_t st);   // bf16, head_dim 128, tensor cores
+// grouped-query attention: mean over the group's G partial indicators [G][n] and Eq. 4; the decode step of a KV group
+cudaError_t launch_group_mean(int G, int64_t n, const float* part, const float* vnorm, float* attn_acc, float* score,
+                              cudaStream_t st);
+cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, int R, int norm, float scale,
+                              const vatp_cache& c, const void* q, const void* k, const void* v, void* out, int32_t* evicted,
+                              int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,
                           const void* k, const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
                           bool may_overlap);

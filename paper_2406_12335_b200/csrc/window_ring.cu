@@ -59,10 +59,10 @@ cudaError_t launch_window_ring(const Shape& s, int dtype, int B, const void* q, 
   if (dtype == VATP_BF16 && s.d == 128 && vatp_tc_available()) return launch_window_ring_tc(s, B, q, lse, c, dev_status, st);
   if (dtype == VATP_F32) {
     window_ring_general_kernel<float><<<dim3((cap + 127) / 128, s.units), 128, s.d * sizeof(float), st>>>(
-        s.heads, s.T, s.d, s.window, B, cap, s.scale, static_cast<const float*>(q), s.sb, s.sh, s.st, lse, c);
+        s.heads, s.T, s.d, s.window, B, cap, s.scale, static_cast<const float*>(q), s.qsb, s.qsh, s.st, lse, c);
   } else {
     window_ring_general_kernel<__nv_bfloat16><<<dim3((cap + 127) / 128, s.units), 128, s.d * sizeof(float), st>>>(
-        s.heads, s.T, s.d, s.window, B, cap, s.scale, static_cast<const __nv_bfloat16*>(q), s.sb, s.sh, s.st, lse, c);
+        s.heads, s.T, s.d, s.window, B, cap, s.scale, static_cast<const __nv_bfloat16*>(q), s.qsb, s.qsh, s.st, lse, c);
   }
   return cudaGetLastError();
 }

@@ -30,7 +30,7 @@ class Params(C.Structure):
     _fields_ = [("batch", C.c_int32), ("heads", C.c_int32), ("seq_len", C.c_int32), ("head_dim", C.c_int32),
                 ("dtype", C.c_int32), ("indicator", C.c_int32), ("window_w", C.c_int32), ("scale", C.c_float),
                 ("budget", C.c_int32), ("n_sink", C.c_int32), ("n_recent", C.c_int32), ("norm_kind", C.c_int32),
-                ("flags", C.c_int32), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
+                ("flags", C.c_int32), ("kv_heads", C.c_int32), ("stride_b", C.c_int64), ("stride_h", C.c_int64), ("stride_t", C.c_int64)]
 
 
 class CacheStruct(C.Structure):
@@ -87,14 +87,14 @@ def _stream(stream=None):
 
 
 def make_params(*, batch, heads, seq_len, head_dim, dtype, budget, n_sink=0, n_recent=0, scale=None,
-                indicator="h2o", window=0, strides=(0, 0, 0), norm="l1", decode_overlap=False) -> Params:
+                indicator="h2o", window=0, strides=(0, 0, 0), norm="l1", decode_overlap=False, kv_heads=0) -> Params:
     """norm: the value norm of Eq. 4, "l1" (the method) or the Ablation Study's "l2" / "linf".
     decode_overlap: sets VATP_FLAG_DECODE_OVERLAP (decode steps of independent caches may run side by side;
     see vatp_decode_step in include/vatp.h for what the caller then guarantees)."""
     dt = {torch.bfloat16: BF16, torch.float32: F32, "bf16": BF16, "f32": F32}[dtype]
     return Params(batch, heads, seq_len, head_dim, dt, IND_WINDOW if indicator == "window" else IND_H2O, window,
                   float(scale if scale is not None else head_dim ** -0.5), budget, n_sink, n_recent, NORM_KINDS[norm],
-                  FLAG_DECODE_OVERLAP if decode_overlap else 0, *strides)
+                  FLAG_DECODE_OVERLAP if decode_overlap else 0, kv_heads, *strides)
 
 
 def params_for(x: torch.Tensor, **kw) -> Params:
@@ -113,7 +113,7 @@ class Cache:
     """Device arrays of the decode state (allocated with torch, owned by this object)."""
 
     def __init__(self, p: Params, device="cuda"):
-        b, h, d, cap = p.batch, p.heads, p.head_dim, int(lib.vatp_cache_capacity(p.budget))
+        b, h, d, cap = p.batch, (p.kv_heads or p.heads), p.head_dim, int(lib.vatp_cache_capacity(p.budget))
         dt = torch.float32 if p.dtype == F32 else torch.bfloat16
         self.cap = cap
         self.k_cache = torch.zeros(b, h, cap, d, dtype=dt, device=device)

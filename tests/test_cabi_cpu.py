@@ -27,8 +27,9 @@ def test_exports_every_declared_symbol(V):
 
 
 def test_struct_layout_matches_header(V):
-    assert C.sizeof(V.Params) == 80       # 7 int32 + float + 5 int32 + pad + 3 int64
-    assert V.Params.norm_kind.offset == 44 and V.Params.flags.offset == 48 and V.Params.stride_b.offset == 56
+    assert C.sizeof(V.Params) == 80       # 7 int32 + float + 6 int32 + 3 int64
+    assert V.Params.norm_kind.offset == 44 and V.Params.flags.offset == 48 and V.Params.kv_heads.offset == 52
+    assert V.Params.stride_b.offset == 56
     assert C.sizeof(V.CacheStruct) == 88
 
 
@@ -82,6 +83,16 @@ def test_host_side_validation(V):
     odd.norm_kind = 3
     assert V.vatp_workspace_bytes(odd) == 0
     assert V.lib.vatp_select(C.byref(odd), 16, 16, null, 0, null, null) == 2
+    # grouped-query attention: kv_heads divides heads, contiguous layouts only; the workspace also holds the G partial indicators
+    gq = dict(ok, heads=4)
+    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=4)) == V.vatp_workspace_bytes(V.make_params(**gq))
+    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=2)) == (2 * 256 * 4 + 256) + 2 * 2 * 64 * 4
+    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=3)) == 0
+    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=8)) == 0
+    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=2, strides=(0, 0, 128))) == 0
+    gw = V.make_params(**gq, kv_heads=2, indicator="window", window=8)
+    assert V.lib.vatp_prefill_scores(C.byref(gw), 16, 16, 16, 16, 16, 16, 16, 16, 256, 1 << 20, null, null) == 2   # no win_rows with grouped queries
+    assert V.lib.vatp_decode_step(C.byref(gw), C.byref(cs), 16, 16, 16, 16, null, null, null) == 2
     # flags: the decode-overlap bit is the only one defined
     assert V.make_params(**ok, decode_overlap=True).flags == V.FLAG_DECODE_OVERLAP == 1
     assert V.vatp_workspace_bytes(V.make_params(**ok, decode_overlap=True)) == 2048 + 256

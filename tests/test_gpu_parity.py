@@ -546,3 +546,80 @@ def test_bounds_checking_build_reports_no_violation():
     assert " passed" in tail and "libvatp_dbg" in subprocess.run(
         [sys.executable, "-c", "from paper_2406_12335_b200 import vatp; print(vatp._LIB_PATH)"], cwd=root, env=env,
         capture_output=True, text=True).stdout
+
+
+@pytest.mark.parametrize("dtype,d,heads,kv_heads,T,B,F,R", [
+    ("bf16", 128, 8, 2, 700, 250, 2, 20),      # tensor-core scoring, four query heads per KV head
+    ("bf16", 128, 6, 3, 1000, 1100, 0, 8),     # budget beyond the prompt: the cache grows before evictions start
+    ("f32", 64, 4, 2, 333, 100, 3, 17),        # general kernels
+    ("bf16", 64, 8, 1, 257, 128, 2, 16),       # multi-query attention: one KV head
+])
+def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R):
+    """Grouped-query attention (the Limitations section's open case, read as a group-mean indicator): the G query
+    heads of a KV group share one kept set and one cache.  Scoring, selection, compaction and decode steps of
+    every KV unit against the oracle; the row normalisers of every query head as well."""
+    from oracle import vatp_oracle as O
+    V = P.vatp()
+    b, G, steps = 2, heads // kv_heads, 10
+    tol = P.TOL[dtype]
+    wl_kv = _small(dtype, d, T, B, F, R, b=b, h=kv_heads, steps=steps, cid=77)
+    _, k, v = synth.prefill_inputs(wl_kv, 0, "cuda")
+    # queries of all heads: Gaussian plus the sink direction of their KV head (the keys of tokens 0 and 1 carry it)
+    u = synth.sink_direction(wl_kv, 0, "cuda").repeat_interleave(G, dim=1)
+    gq = torch.Generator(device="cuda").manual_seed(4077)
+    q = (torch.randn(b, heads, T, d, generator=gq, device="cuda") + synth.sink_alpha(wl_kv) * u).to(k.dtype)
+    dq = (torch.randn(steps, b, heads, d, generator=gq, device="cuda") + synth.sink_alpha(wl_kv) * u.squeeze(2)).to(k.dtype)
+    _, dk, dv = synth.decode_inputs(wl_kv, 0, device="cuda")
+
+    p = V.make_params(batch=b, heads=heads, kv_heads=kv_heads, seq_len=T, head_dim=d, dtype=dtype, budget=B, n_sink=F,
+                      n_recent=R, scale=wl_kv.scale)
+    f32 = dict(dtype=torch.float32, device="cuda")
+    lse = torch.empty(b, heads, T, **f32)
+    attn_acc, vnorm, score = (torch.empty(b, kv_heads, T, **f32) for _ in range(3))
+    ws = torch.empty(V.vatp_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kept = torch.empty(b, kv_heads, B, dtype=torch.int32, device="cuda")
+    cache = V.Cache(p)
+    V.vatp_prefill_scores(p, q, k, v, lse_out=lse, attn_acc=attn_acc, vnorm=vnorm, score=score, workspace=ws, dev_status=status)
+    V.vatp_select(p, score, kept, dev_status=status)
+    V.vatp_compact(p, k, v, attn_acc, vnorm, kept, cache, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.all((attn_acc.double().sum(-1) - T).abs() <= 2e-3 * T)
+
+    n_live = min(T, B)
+    states = {}
+    for bi in range(b):
+        for g in range(kv_heads):
+            ref = O.prefill_gqa(P.to_np64(q[bi, g * G:(g + 1) * G]), P.to_np64(k[bi, g]), P.to_np64(v[bi, g]), wl_kv.scale)
+            assert np.max(np.abs(P.to_np64(lse[bi, g * G:(g + 1) * G]) - ref["lse"])) <= 10 * tol
+            for name, key in (("attn_acc", "S"), ("vnorm", "n1"), ("score", "I")):
+                e = P.rel_err(P.to_np64(locals()[name][bi, g]), ref[key])
+                assert e <= tol, f"{name} rel err {e:.3g} (unit {bi},{g})"
+            want = O.select_keep(ref["I"], B, F, R)
+            got = kept[bi, g, :n_live].cpu().numpy().astype(np.int64)
+            assert np.array_equal(got, want), "kept set"
+            assert torch.equal(cache.k_cache[bi, g, :n_live], k[bi, g][torch.from_numpy(got).cuda()])
+            states[(bi, g)] = O.DecodeState(P.to_np64(k[bi, g]), P.to_np64(v[bi, g]), ref["S"], ref["n1"], got, T)
+
+    out = torch.empty(b, heads, d, dtype=k.dtype, device="cuda")
+    evicted = torch.empty(b, kv_heads, dtype=torch.int32, device="cuda")
+    out_eps = 2.0 ** -8 if dtype == "bf16" else 0.0
+    for s in range(steps):
+        V.vatp_decode_step(p, cache, dq[s], dk[s], dv[s], out, evicted_pos=evicted, dev_status=status)
+        torch.cuda.synchronize()
+        for (bi, g), st in states.items():
+            ev = int(evicted[bi, g])
+            res = O.decode_step(st, P.to_np64(dq[s, bi, g * G:(g + 1) * G]), P.to_np64(dk[s, bi, g]), P.to_np64(dv[s, bi, g]),
+                                wl_kv.scale, B, F, R, force_evict=None if ev < 0 else ev, tie_tol=2 * tol, tie_abs=1e-30)
+            assert res["evicted"] == ev and not res["adopted"]
+            ref_out = res["out"]
+            bound = tol * np.max(np.abs(ref_out)) + out_eps * np.abs(ref_out) + 1e-30
+            assert np.all(np.abs(P.to_np64(out[bi, g * G:(g + 1) * G]) - ref_out) <= bound), f"step {s} unit {(bi, g)}: out"
+    assert int(status.item()) == 0
+    for (bi, g), st in states.items():
+        pos = cache.pos[bi, g].cpu().numpy()
+        live = pos >= 0
+        order = np.argsort(pos[live])
+        assert pos[live][order].tolist() == st.pos and int(cache.len[bi, g]) == len(st.pos)
+        assert P.rel_err(P.to_np64(cache.acc[bi, g])[live][order], st.indicator()) <= 2 * tol
