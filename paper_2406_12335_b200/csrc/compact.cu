@@ -12,7 +12,7 @@
 namespace vatp {
 namespace {
 
-constexpr int CB_WARPS = 8;
+constexpr int CB_WARPS = 12;           // (with two batches in flight each: more warps with shallower rings beat 8 x 3 and 6 x 4)
 constexpr int CB_THREADS = CB_WARPS * 32;
 constexpr int CB_ROWS = 16;            // destination slots per batch at most (8 when the rows are 512 bytes)
 constexpr int CB_MAXBUF = 4;           // batches in flight per warp (fewer when the rows are long)
@@ -220,7 +220,7 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
   const size_t per_buf = (size_t)CB_WARPS * 2 * rows_pb * row_bytes;     // one ring slot of every warp
   int nbuf = (int)(CB_SMEM / per_buf);
   nbuf = nbuf > CB_MAXBUF ? CB_MAXBUF : nbuf;
-  if (nbuf < 2) return cudaErrorInvalidValue;                            // (head_dim <= 128 gives at least 3)
+  if (nbuf < 2) return cudaErrorInvalidValue;                            // (head_dim <= 128 gives at least 2)
   const size_t smem = per_buf * nbuf;
   // Row gathers need the inputs as ONE table of equally spaced rows: the largest spacing that divides all three
   // strides (the row length itself for contiguous tensors and for [batch, T, heads, d] storage alike).
