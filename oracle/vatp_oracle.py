@@ -29,6 +29,7 @@ import numpy as np
 
 __all__ = [
     "attention_probs",
+    "attention_output",
     "indicator_h2o",
     "indicator_window",
     "value_l1_norm",
@@ -77,6 +78,13 @@ def row_logsumexp(q, k, scale: float) -> np.ndarray:
     s = np.where(causal, s, -np.inf)
     m = s.max(axis=1)
     return m + np.log(np.exp(s - m[:, None]).sum(axis=1))
+
+
+def attention_output(a: np.ndarray, v) -> np.ndarray:
+    """The attention layer's output rows o_j = sum_{i<=j} a_i^j v_i (Section 3.1: the
+    output is the probability-weighted sum of the value vectors, which is why
+    Eq. 4 looks at their norms).  a: [T, T] from attention_probs, v: [T, d]."""
+    return a @ _f64(v)
 
 
 def indicator_h2o(a: np.ndarray) -> np.ndarray:
@@ -185,7 +193,7 @@ def compact_rows(x: np.ndarray, kept: np.ndarray) -> np.ndarray:
 
 
 def prefill(q, k, v, scale: float, *, window: int | None = None, inclusive_extra: int = 0, norm: str = "l1"):
-    """One unit's prefill quantities: dict with a, lse, S, n1, I (and the
+    """One unit's prefill quantities: dict with a, out, lse, S, n1, I (and the
     window rows a[T-w:, :] when the indicator is Eq. 3).  norm: which value
     norm Eq. 4 multiplies by ("l1" is the method; "l2" / "linf" are the
     ablation's variants); the key stays "n1" for all kinds."""
@@ -200,6 +208,7 @@ def prefill(q, k, v, scale: float, *, window: int | None = None, inclusive_extra
     n1 = value_l1_norm(v) if norm == "l1" else value_norm(v, norm)
     return {
         "a": a,
+        "out": attention_output(a, v),
         "lse": row_logsumexp(q, k, scale),
         "S": S,
         "n1": n1,

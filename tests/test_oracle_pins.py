@@ -596,3 +596,42 @@ def test_gqa_decode_step_matches_prefill_on_the_longer_prompt():
     with pytest.raises(ValueError):
         stw = O.DecodeState(k[:T], v[:T], short["S"], short["n1"], np.arange(T), T, window=4, window_rows=np.zeros((4, T)))
         O.decode_step(stw, qg[:, T], k[T], v[T], scale, B=T + 5, F=0, R=0)
+
+
+# ----------------------------------------------------------------- attention output (Section 3.1)
+def test_attention_output_matches_loops_and_closed_forms():
+    rng = np.random.default_rng(5)
+    T, d = 9, 4
+    q, k, v = rng.standard_normal((T, d)), rng.standard_normal((T, d)), rng.standard_normal((T, d))
+    scale = 0.5
+    a = brute_attention(q.tolist(), k.tolist(), scale)
+    out = O.attention_output(O.attention_probs(q, k, scale), v)
+    for j in range(T):
+        for c in range(d):
+            acc = 0.0
+            for i in range(j + 1):
+                acc += a[j][i] * float(v[i][c])
+            assert abs(out[j, c] - acc) < 1e-12
+    # a transposed probability matrix would put future values into early rows
+    assert np.abs(O.attention_probs(q, k, scale).T @ v - out).max() > 1e-3
+    # the first query sees only the first token
+    np.testing.assert_allclose(out[0], v[0], rtol=0, atol=1e-15)
+    # constant values come back unchanged (rows of a sum to one)
+    ones = np.full((T, d), 3.25)
+    np.testing.assert_allclose(O.attention_output(O.attention_probs(q, k, scale), ones), ones, rtol=0, atol=1e-13)
+    # uniform attention (all keys equal): row j is the mean of the first j + 1 values
+    ku = np.tile(k[:1], (T, 1))
+    outu = O.prefill(q, ku, v, scale)["out"]
+    for j in range(T):
+        np.testing.assert_allclose(outu[j], v[: j + 1].mean(axis=0), rtol=0, atol=1e-13)
+
+
+def test_attention_output_last_row_is_the_decode_steps_output():
+    """Row T of the prompt's output equals what the decode step returns for token T (no eviction yet)."""
+    rng = np.random.default_rng(6)
+    T, d = 12, 8
+    q, k, v = rng.standard_normal((T + 1, d)), rng.standard_normal((T + 1, d)), rng.standard_normal((T + 1, d))
+    scale = d ** -0.5
+    st, _ = _state(q[:T], k[:T], v[:T], scale, B=T + 4, F=1, R=2)
+    res = O.decode_step(st, q[T], k[T], v[T], scale, T + 4, 1, 2)
+    np.testing.assert_allclose(res["out"], O.prefill(q, k, v, scale)["out"][T], rtol=0, atol=1e-12)
