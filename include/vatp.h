@@ -162,6 +162,28 @@ vatp_status vatp_prefill_scores_from_lse(const vatp_params* params, const void* 
                                          int32_t* dev_status, void* cuda_stream);
 
 /*
+ * Attention forward fused with prefill scoring: the layer's output rows (Section 3.1, Eq. 1)
+ *   attn_out[j] = sum_{i<=j} a_i^j v_i
+ * and the row normalisers come out of ONE streaming sweep over K and V (never materialising the
+ * T x T matrix), and the indicator then costs one recomputation of QK^T (pass 2 of
+ * vatp_prefill_scores).  A caller that needs the attention output anyway - every prefill does -
+ * pays three contraction sweeps for output, indicator and importance together instead of the
+ * forward's two plus the scoring call's two: the remedy for the cost the Limitations section names
+ * ("FlashAttention Support for H2O"), built in.
+ * attn_out: [batch, heads, T, head_dim] contiguous device array of the params dtype, 16-byte
+ *           aligned, output; required (NULL is VATP_ERR_INVALID_ARG).  bf16 carries the rounding
+ *           of the probabilities to bf16 before they meet V (as fused attention kernels do):
+ *           |error| <= 2^-8 * max|v| per element, typically far less.
+ * All other arguments, outputs, the workspace requirement and the error behaviour are those of
+ * vatp_prefill_scores; both indicators (Eq. 2, Eq. 3) are supported, grouped-query attention is not
+ * (VATP_ERR_UNSUPPORTED), nor is head_dim > 256 outside the tensor-core shape.
+ */
+vatp_status vatp_prefill_attention_scores(const vatp_params* params, const void* q, const void* k, const void* v,
+                                          void* attn_out, float* lse_out, float* attn_acc, float* vnorm, float* score,
+                                          float* win_rows, void* workspace, size_t workspace_bytes,
+                                          int32_t* dev_status, void* cuda_stream);
+
+/*
  * vatp_prefill_scores for callers that cannot allocate device memory.  (The paper has no
  * counterpart; this is a packaging variant of the call above and computes exactly the same thing.)
  *

@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libvatp.so")
 LIB_DEBUG = os.path.join(HERE, "libvatp_dbg.so")      # the bounds-checking build (-DVATP_DEBUG_BOUNDS)
-SOURCES = ["vatp_api.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_static.cu", "select.cu", "compact.cu", "window_ring.cu", "decode.cu", "decode_mma.cu", "decode_gqa.cu", "selftest.cu"]
+SOURCES = ["vatp_api.cu", "prefill_simt.cu", "prefill_tc.cu", "prefill_static.cu", "attn_fwd.cu", "select.cu", "compact.cu", "window_ring.cu", "decode.cu", "decode_mma.cu", "decode_gqa.cu", "selftest.cu"]
 
 
 def _nvcc() -> str:

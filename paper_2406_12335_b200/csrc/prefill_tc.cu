@@ -785,6 +785,378 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   }
 }
 
+// ---------------------------------------------------------------------------------------------------
+// Fused attention forward (Section 3.1, Eq. 1): out[j] = sum_{i<=j} a_i^j v_i and the row normalisers in
+// ONE streaming sweep, so that a caller who needs the layer's output anyway pays a single further
+// recomputation of QK^T (pass 2 above) for the indicator - the cost the Limitations section ("FlashAttention
+// Support for H2O") asks to remove.  It stands in for pass 1: same normalisers, same workspace layout.
+//
+//   per work item (unit, tile of 128 queries), streamed key / value chunks of 128 tokens 0 .. diagonal:
+//     S   = Q K^T            tcgen05, both operands K-major, fp32 in TMEM (two buffers)
+//     P   = exp2(S - m)      one thread per query row, written to shared memory as bf16 (the A operand's layout)
+//     O  += P V              tcgen05, V straight from its [token, d] rows as an MN-major B operand, O in TMEM
+//     out = O / l, lse = m + log2 l
+//   m is a per-row reference that follows the running maximum lazily: O and l are rescaled only when the
+//   maximum has grown by more than 2^8 since the reference was set (probabilities stay below 2^8, far
+//   inside bf16 and fp32 range; once the first chunks - which hold the attention sinks - are past, almost
+//   no chunk rescales).  A rescale is a TMEM load / multiply / store of the thread's own row, done after
+//   the previous P V product has completed and before this chunk's product is released.
+// Warp roles (224 threads): warp 0 TMA producer and work-item FIFO, warp 1 MMA issuer, warps 2-5 softmax
+// (row = TMEM lane), warp 6 value norms (Eq. 4).  MMA order: S(c+1) is issued before O += P(c) V(c), so the
+// tensor pipe recomputes the next logits while the softmax warps are still on chunk c.
+constexpr int FW_THREADS = 7 * 32;
+constexpr int FW_ST = 2;               // stages of K, of V and of P
+constexpr int FW_O_COL = 2 * TILE;     // TMEM columns: S buffers at 0 and 128, O at 256
+constexpr float FW_LAZY = 8.f;         // log2 of the growth of a row maximum that forces a rescale
+
+struct FwdSmem {
+  alignas(1024) unsigned char q[TILE_BYTES];
+  alignas(1024) unsigned char k[FW_ST][TILE_BYTES];    // [d half][128 tokens][128 bytes]
+  alignas(1024) unsigned char v[FW_ST][TILE_BYTES];    // [d half][128 tokens][128 bytes]
+  alignas(1024) unsigned char p[FW_ST][TILE_BYTES];    // [key half][128 queries][128 bytes]
+  alignas(8) uint64_t q_full, q_empty;
+  uint64_t k_full[FW_ST], k_empty[FW_ST], v_full[FW_ST], v_empty[FW_ST];
+  uint64_t s_full[2], s_empty[2], p_full[FW_ST], p_empty[FW_ST];
+  uint64_t o_full, o_empty;
+  uint64_t item_full[4], item_empty[4];
+  int item_ring[4][2];                  // u, tile (u < 0: no more items)
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+// Shared-memory matrix descriptor of a V chunk as the B operand of O += P V: N (= d) is the contiguous
+// dimension.  128-byte swizzle; a row of 64 d-values per token, 8 tokens per 1024-byte group (stride
+// offset), the second 64 d-values one slab further on (leading offset).
+__device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr >> 4) & 0x3FFFu) | ((uint64_t)(SLAB_BYTES >> 4) << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+constexpr uint32_t IDESC_PV = idesc<128>() | (1u << 16);   // B operand MN-major
+
+__device__ __forceinline__ void umma_bf16_rt(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t id, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "l"(da), "l"(db), "r"(id), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t addr, const float (&v)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+      ::"r"(addr), "r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+        "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+        "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+        "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+        "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+        "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+        "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+        "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31]))
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+  const __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);     // .x = lo is the lower address
+  return *reinterpret_cast<const uint32_t*>(&t);
+}
+
+__global__ void __launch_bounds__(FW_THREADS, 1)
+attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                        const __grid_constant__ CUtensorMap tm_v, TcArgs a, __nv_bfloat16* __restrict__ out) {
+  extern __shared__ unsigned char smem_raw[];
+  FwdSmem& sm = *reinterpret_cast<FwdSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  volatile int* abort_flag = &sm.abort_flag;
+  const int items = a.units * a.nt;
+
+  if (tid == 0) {
+    mbar_init(&sm.q_full, 1); mbar_init(&sm.q_empty, 1);
+    for (int i = 0; i < FW_ST; ++i) {
+      mbar_init(&sm.k_full[i], 1); mbar_init(&sm.k_empty[i], 1);
+      mbar_init(&sm.v_full[i], 1); mbar_init(&sm.v_empty[i], 1);
+      mbar_init(&sm.p_full[i], 4); mbar_init(&sm.p_empty[i], 1);
+    }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.s_empty[i], 4); }
+    mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, 4);
+    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 5); }   // MMA warp + 4 softmax warps
+    sm.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (wid == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&sm.tmem_base)), "r"(512)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    tc_fence_before();
+  }
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = sm.tmem_base;
+  // pass 2, a programmatic dependent, may set up while this kernel runs
+  if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+  // the itl-th item of this CTA: (u, tile), u < 0 ends the kernel (also when the CTA is aborting)
+  auto next_item = [&](uint32_t itl, bool whole_warp, int& u, int& tile) {
+    const int slot = itl & 3;
+    bool got = mbar_wait(&sm.item_full[slot], (itl >> 2) & 1, abort_flag, a.dev_status);
+    if (whole_warp) got = __all_sync(0xffffffffu, got);
+    u = -1; tile = 0;
+    if (got) {
+      const volatile int* f = &sm.item_ring[slot][0];
+      u = f[0]; tile = f[1];
+    }
+    if (whole_warp) __syncwarp();
+    if (got && (!whole_warp || lane == 0)) mbar_arrive(&sm.item_empty[slot]);
+  };
+
+  if (wid == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t n = 0;
+      int next = (int)atomicAdd(&a.counters[0], 1u);
+      for (uint32_t itl = 0; ok; ++itl) {
+        const int id = next;
+        const int slot = itl & 3;
+        int u = -1, tile = 0;
+        if (id < items) {
+          // units in groups whose K, V and Q stay in L2 together; inside a group, longest items first
+          const int grp = id / (a.gu * a.nt);
+          const int rem = id - grp * (a.gu * a.nt);
+          const int u0 = grp * a.gu;
+          const int nu = min(a.gu, a.units - u0);
+          const int r = rem / nu;
+          u = u0 + (rem - r * nu);
+          tile = a.nt - 1 - r;
+        }
+        ok = mbar_wait<20>(&sm.item_empty[slot], ((itl >> 2) & 1) ^ 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        {
+          volatile int* f = &sm.item_ring[slot][0];
+          f[0] = u; f[1] = tile;
+        }
+        mbar_arrive(&sm.item_full[slot]);
+        if (id >= items) break;
+        next = (int)atomicAdd(&a.counters[0], 1u);
+        const int b = u / a.heads, h = u - b * a.heads;
+        ok = mbar_wait<20>(&sm.q_empty, (itl & 1) ^ 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        mbar_expect_tx(&sm.q_full, TILE_BYTES);
+        tma_load_4d(sm.q, &tm_q, &sm.q_full, 0, tile * TILE, h, b);
+        tma_load_4d(sm.q + SLAB_BYTES, &tm_q, &sm.q_full, 64, tile * TILE, h, b);
+        for (int c = 0; c <= tile; ++c, ++n) {
+          const int stg = n % FW_ST;
+          const uint32_t par = ((n / FW_ST) & 1) ^ 1;
+          ok = mbar_wait<20>(&sm.k_empty[stg], par, abort_flag, a.dev_status);
+          if (!ok) break;
+          mbar_expect_tx(&sm.k_full[stg], TILE_BYTES);     // tokens beyond T arrive as zeros
+          tma_load_4d(sm.k[stg], &tm_k, &sm.k_full[stg], 0, c * TILE, h, b);
+          tma_load_4d(sm.k[stg] + SLAB_BYTES, &tm_k, &sm.k_full[stg], 64, c * TILE, h, b);
+          ok = mbar_wait<20>(&sm.v_empty[stg], par, abort_flag, a.dev_status);
+          if (!ok) break;
+          mbar_expect_tx(&sm.v_full[stg], TILE_BYTES);
+          tma_load_4d(sm.v[stg], &tm_v, &sm.v_full[stg], 0, c * TILE, h, b);
+          tma_load_4d(sm.v[stg] + SLAB_BYTES, &tm_v, &sm.v_full[stg], 64, c * TILE, h, b);
+        }
+      }
+    }
+  } else if (wid == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t n = 0;
+      const uint64_t q_desc = umma_desc(s32(sm.q));
+      const uint64_t k_desc0 = umma_desc(s32(sm.k[0])), p_desc0 = umma_desc(s32(sm.p[0]));
+      const uint64_t v_desc0 = umma_desc_mn(s32(sm.v[0]));
+      // S(g) = Q K(g)^T into S buffer g % 2
+      auto issue_qk = [&](uint32_t g) -> bool {
+        const int stg = g % FW_ST, sb = g & 1;
+        if (!mbar_wait(&sm.k_full[stg], (g / FW_ST) & 1, abort_flag, a.dev_status) ||
+            !mbar_wait(&sm.s_empty[sb], ((g >> 1) & 1) ^ 1, abort_flag, a.dev_status))
+          return false;
+        tc_fence_after();
+        const uint64_t kd = k_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
+#pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk)
+          umma_bf16_rt(tmem + sb * TILE, q_desc + k_off_fixed(kk), kd + k_off_fixed(kk), idesc<128>(), kk > 0);
+        umma_commit(&sm.k_empty[stg]);
+        umma_commit(&sm.s_full[sb]);
+        return true;
+      };
+      for (uint32_t itl = 0; ok; ++itl) {
+        int u, tile;
+        next_item(itl, false, u, tile);
+        if (u < 0) break;
+        if (!VATP_INB(u, a.units, a.dev_status) || !VATP_INB(tile, a.nt, a.dev_status)) break;
+        ok = mbar_wait(&sm.q_full, itl & 1, abort_flag, a.dev_status);
+        if (!ok) break;
+        const int nc = tile + 1;
+        ok = issue_qk(n);
+        for (int c = 0; c < nc && ok; ++c) {
+          const uint32_t g = n + c;
+          if (c + 1 < nc) { ok = issue_qk(g + 1); if (!ok) break; }
+          else umma_commit(&sm.q_empty);            // the item's last S has been issued: the query tile may be replaced
+          const int stg = g % FW_ST;
+          ok = mbar_wait(&sm.p_full[stg], (g / FW_ST) & 1, abort_flag, a.dev_status) &&
+               mbar_wait(&sm.v_full[stg], (g / FW_ST) & 1, abort_flag, a.dev_status) &&
+               (c > 0 || mbar_wait(&sm.o_empty, (itl & 1) ^ 1, abort_flag, a.dev_status));
+          if (!ok) break;
+          tc_fence_after();
+          const uint64_t pd = p_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
+          const uint64_t vd = v_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
+#pragma unroll
+          for (int kk = 0; kk < TILE / 16; ++kk)      // 16 keys per step: 2048 bytes further on in V
+            umma_bf16_rt(tmem + FW_O_COL, pd + k_off_fixed(kk), vd + (uint64_t)(kk * 128), IDESC_PV, (c > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(&sm.v_empty[stg]);
+          umma_commit(&sm.p_empty[stg]);
+          if (c == nc - 1) umma_commit(&sm.o_full);
+        }
+        n += nc;
+      }
+    }
+  } else if (wid < 6) {
+    // ------------------------------------------------------------------ softmax: one thread per query row
+    const int quarter = wid & 3;                  // TMEM lanes this warp may touch
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const float sc = a.scale_log2;
+    bool ok = true;
+    uint32_t n = 0;
+    for (uint32_t itl = 0; ok; ++itl) {
+      int u, tile;
+      next_item(itl, true, u, tile);
+      if (u < 0) break;
+      if (!VATP_INB(u, a.units, a.dev_status) || !VATP_INB(tile, a.nt, a.dev_status)) break;
+      const int tok = tile * TILE + row;
+      const int nc = tile + 1;
+      float m_ref = -INFINITY, l_run = 0.f;
+      for (int c = 0; c < nc; ++c) {
+        const uint32_t g = n + c;
+        const int sb = g & 1, stg = g % FW_ST;
+        bool w = mbar_wait(&sm.s_full[sb], (g >> 1) & 1, abort_flag, a.dev_status);
+        w = __all_sync(0xffffffffu, w);
+        if (!w) { ok = false; break; }
+        tc_fence_after();
+        float x[4][32];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(lane_addr + sb * TILE + q4 * 32, x[q4]);
+        tmem_ld_wait();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.s_empty[sb]);
+        if (c == tile) {
+#pragma unroll
+          for (int q4 = 0; q4 < 4; ++q4) mask_after_diagonal(x[q4], q4 * 32, row);
+        }
+        // scaled maximum of the row's 128 logits (scale > 0)
+        const float mx = fmaxf(fmaxf(slice_max(x[0]), slice_max(x[1])), fmaxf(slice_max(x[2]), slice_max(x[3]))) * sc;
+        const float m_new = fmaxf(m_ref, mx);
+        if (c == 0) {
+          m_ref = m_new;              // finite: column 0 is never masked
+        } else {
+          const bool need = m_new > m_ref + FW_LAZY;
+          if (__any_sync(0xffffffffu, need)) {
+            // O += P(g-1) V(g-1) must have completed before this thread's row of O is rewritten
+            bool w2 = mbar_wait(&sm.p_empty[(g - 1) % FW_ST], ((g - 1) / FW_ST) & 1, abort_flag, a.dev_status);
+            w2 = __all_sync(0xffffffffu, w2);
+            if (!w2) { ok = false; break; }
+            tc_fence_after();
+            const float f = need ? ex2(m_ref - m_new) : 1.f;
+#pragma unroll
+            for (int q4 = 0; q4 < 4; ++q4) {
+              float y[32];
+              tmem_ld32(lane_addr + FW_O_COL + q4 * 32, y);
+              tmem_ld_wait();
+#pragma unroll
+              for (int i = 0; i < 32; ++i) y[i] *= f;
+              tmem_st32(lane_addr + FW_O_COL + q4 * 32, y);
+            }
+            tmem_st_wait();
+            l_run *= f;
+            if (need) m_ref = m_new;
+          }
+        }
+        // the P buffer is free once the product that read it two chunks ago has completed
+        bool w3 = mbar_wait(&sm.p_empty[stg], ((g / FW_ST) & 1) ^ 1, abort_flag, a.dev_status);
+        w3 = __all_sync(0xffffffffu, w3);
+        if (!w3) { ok = false; break; }
+        unsigned char* prow = sm.p[stg] + row * 128;
+        const f32x2 c2 = pk2(sc, sc), nm2 = pk2(-m_ref, -m_ref);
+        f32x2 la = pk2(0.f, 0.f), lb = la;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {            // 16-byte pieces of the row: 8 probabilities each
+          const float* xs = &x[j >> 2][(j & 3) * 8];
+          float p[8];
+#pragma unroll
+          for (int i = 0; i < 8; i += 2) {
+            const f32x2 e = ex2_sfu2(fma2(pk2(xs[i], xs[i + 1]), c2, nm2));
+            if (i & 2) lb = add2(lb, e); else la = add2(la, e);
+            upk2(e, p[i], p[i + 1]);
+          }
+          const uint4 pk = make_uint4(pack2_bf16(p[0], p[1]), pack2_bf16(p[2], p[3]), pack2_bf16(p[4], p[5]), pack2_bf16(p[6], p[7]));
+          *reinterpret_cast<uint4*>(prow + (j >> 3) * SLAB_BYTES + (((j & 7) ^ (row & 7)) << 4)) = pk;
+        }
+        l_run += hsum2(add2(la, lb));
+        // P (generic-proxy stores) and any rescaled O (TMEM stores) are complete before the MMA warp is told
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.p_full[stg]);
+      }
+      if (!ok) break;
+      n += nc;
+      // ---- end of item: out = O / l, lse = m + log2 l
+      bool w4 = mbar_wait(&sm.o_full, itl & 1, abort_flag, a.dev_status);
+      w4 = __all_sync(0xffffffffu, w4);
+      if (!w4) { ok = false; break; }
+      tc_fence_after();
+      const float inv = 1.f / l_run;
+      __nv_bfloat16* orow = out + ((int64_t)u * a.T + tok) * HD;
+      const bool live = tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status);
+#pragma unroll
+      for (int q4 = 0; q4 < 4; ++q4) {
+        float y[32];
+        tmem_ld32(lane_addr + FW_O_COL + q4 * 32, y);
+        tmem_ld_wait();
+        if (live) {
+#pragma unroll
+          for (int j = 0; j < 4; ++j)
+            reinterpret_cast<uint4*>(orow + q4 * 32)[j] =
+                make_uint4(pack2_bf16(y[8 * j] * inv, y[8 * j + 1] * inv), pack2_bf16(y[8 * j + 2] * inv, y[8 * j + 3] * inv),
+                           pack2_bf16(y[8 * j + 4] * inv, y[8 * j + 5] * inv), pack2_bf16(y[8 * j + 6] * inv, y[8 * j + 7] * inv));
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.o_empty);
+      const float lse2 = m_ref + log2f(l_run);
+      // the layout pass 2 reads: negated, -inf where a query contributes nothing (beyond the prompt, before the
+      // history window), half a chunk of padding after an odd tile count
+      if (VATP_INB((int64_t)u * a.Tpad + tok, (int64_t)a.units * a.Tpad, a.dev_status))
+        a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? -lse2 : -INFINITY;
+      if ((a.nt & 1) && tile == a.nt - 1 && VATP_INB((int64_t)u * a.Tpad + tok + TILE, (int64_t)a.units * a.Tpad, a.dev_status))
+        a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
+      if (a.lse_out && tok < a.T)
+        a.lse_out[(int64_t)(u / a.heads) * a.lse_sb + (int64_t)(u % a.heads) * a.lse_sh + tok] = lse2 * 0.69314718055994531f;
+    }
+  } else if (a.side_norm) {
+    // ------------------------------------------------------------------ value norms (Eq. 4)
+    side_value_norms<VATP_NORM_L1>(a, lane);
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (sm.abort_flag) {
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (wid == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+  }
+}
+
 // Value norms as a kernel of their own (Eq. 4): used with a history window, where pass 1 covers only
 // the window's query tiles and is too short to hide one warp per SM walking all of V, and for the
 // l2 / l-infinity variants.  Sixteen lanes
@@ -1057,9 +1429,10 @@ size_t prefill_tc_workspace_bytes(int units, int T) {
 
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
-                              int32_t* dev_status, cudaStream_t st, const float* lse_in) {
-  CUtensorMap tm_q, tm_k;
+                              int32_t* dev_status, cudaStream_t st, const float* lse_in, void* attn_out) {
+  CUtensorMap tm_q, tm_k, tm_v;
   if (!make_map(&tm_q, q, s, true) || !make_map(&tm_k, k, s)) return cudaErrorInvalidValue;
+  if (attn_out && (lse_in || !make_map(&tm_v, v, s))) return cudaErrorInvalidValue;
   TcArgs a;
   a.units = s.units; a.heads = s.heads; a.T = s.T;
   a.nt = (s.T + TILE - 1) / TILE;
@@ -1097,14 +1470,29 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   const int sms = device_sm_count();
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
   if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
-  a.side_norm = a.ft == 0 && a.norm == VATP_NORM_L1 && !lse_in;   // the side warp belongs to pass 1
+  // the side warp belongs to pass 1 (too short under a history window) or to the fused forward (always all tiles)
+  a.side_norm = (a.ft == 0 || attn_out) && a.norm == VATP_NORM_L1 && !lse_in;
   if (!a.side_norm) {
     const dim3 grid(a.units, (s.T + 127) / 128);
     if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a, lse_in);
     else if (a.norm == VATP_NORM_L2) vnorm_kernel<VATP_NORM_L2><<<grid, 256, 0, st>>>(a, lse_in);
     else vnorm_kernel<VATP_NORM_LINF><<<grid, 256, 0, st>>>(a, lse_in);
   }
-  if (!lse_in) prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  if (attn_out) {
+    // the forward sweep stands in for pass 1; it streams K and V, so a group's units share the L2 three ways
+    const size_t fsmem = sizeof(FwdSmem) + 1024;
+    if ((e = cudaFuncSetAttribute(attention_fwd_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsmem)) != cudaSuccess) return e;
+    TcArgs af = a;
+    const size_t unit_bytes = (size_t)3 * s.T * HD * 2;
+    if ((size_t)s.units * unit_bytes > ((size_t)96 << 20)) {
+      const size_t g = ((size_t)48 << 20) / unit_bytes;
+      af.gu = g < 1 ? 1 : (g > (size_t)s.units ? s.units : (int)g);
+    }
+    attention_fwd_tc_kernel<<<items2 < sms ? items2 : sms, FW_THREADS, fsmem, st>>>(tm_q, tm_k, tm_v, af,
+                                                                                    static_cast<__nv_bfloat16*>(attn_out));
+  } else if (!lse_in) {
+    prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
+  }
   if ((e = cudaGetLastError()) != cudaSuccess) return e;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(items2 < sms ? items2 : sms);

@@ -80,10 +80,11 @@ bool cache_ok(const vatp_cache* c, bool windowed) {
   return true;
 }
 
-// Both prefill entry points: lse_in == nullptr runs pass 1, otherwise the caller's normalisers replace it.
+// The prefill entry points: lse_in == nullptr runs pass 1, otherwise the caller's normalisers replace it;
+// attn_out != nullptr runs the attention forward in pass 1's place (it yields the same normalisers).
 vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, const void* v, const float* lse_in,
                          float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows, void* workspace,
-                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+                         size_t workspace_bytes, int32_t* dev_status, void* cuda_stream, void* attn_out = nullptr) {
   vatp_status s = check_params(p, true);
   if (s != VATP_OK) return s;
   if (!q || !k || !v || !attn_acc || !vnorm || !score) return VATP_ERR_INVALID_ARG;
@@ -92,7 +93,8 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
   s = make_shape(p, &sh);
   if (s != VATP_OK) return s;
   const int G = group_of(p);
-  if (G > 1 && (lse_in || win_rows)) return VATP_ERR_UNSUPPORTED;
+  if (G > 1 && (lse_in || win_rows || attn_out)) return VATP_ERR_UNSUPPORTED;
+  if (attn_out && (lse_in || !aligned16(attn_out))) return VATP_ERR_INVALID_ARG;
   if (!workspace || workspace_bytes < workspace_need(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return VATP_ERR_WORKSPACE;
   float* ws = static_cast<float*>(workspace);
@@ -125,7 +127,14 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
     return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
   }
   if (p->dtype == VATP_BF16 && p->head_dim == 128 && vatp_tc_available()) {
-    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st, lse_in);
+    e = launch_prefill_tc(sh, q, k, v, ws, lse_out, attn_acc, vnorm, score, win_rows, dev_status, st, lse_in, attn_out);
+  } else if (attn_out) {
+    // general path: the forward leaves natural-log normalisers where pass 2 reads them (the caller's array, or
+    // the workspace in the same layout)
+    float* lse_buf = lse_out ? lse_out : ws;
+    e = launch_attention_fwd_general(sh, p->dtype, q, k, v, attn_out, lse_buf, st);
+    if (e == cudaErrorNotSupported) return VATP_ERR_UNSUPPORTED;
+    if (e == cudaSuccess) e = launch_prefill_simt(sh, p->dtype, q, k, v, lse_buf, attn_acc, vnorm, score, win_rows, st, true);
   } else if (lse_in) {
     // pass 2 of the general kernel reads natural-log normalisers [units][T] directly
     e = launch_prefill_simt(sh, p->dtype, q, k, v, const_cast<float*>(lse_in), attn_acc, vnorm, score, win_rows, st, true);
@@ -167,6 +176,14 @@ vatp_status vatp_prefill_scores(const vatp_params* p, const void* q, const void*
                                 size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
   return prefill_impl(p, q, k, v, nullptr, lse_out, attn_acc, vnorm, score, win_rows, workspace, workspace_bytes,
                       dev_status, cuda_stream);
+}
+
+vatp_status vatp_prefill_attention_scores(const vatp_params* p, const void* q, const void* k, const void* v, void* attn_out,
+                                          float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
+                                          void* workspace, size_t workspace_bytes, int32_t* dev_status, void* cuda_stream) {
+  if (!attn_out) return VATP_ERR_INVALID_ARG;
+  return prefill_impl(p, q, k, v, nullptr, lse_out, attn_acc, vnorm, score, win_rows, workspace, workspace_bytes, dev_status,
+                      cuda_stream, attn_out);
 }
 
 vatp_status vatp_prefill_scores_from_lse(const vatp_params* p, const void* q, const void* k, const void* v,

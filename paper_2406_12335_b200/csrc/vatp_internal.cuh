@@ -101,9 +101,13 @@ cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const 
                                 float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st,
                                 bool lse_given = false);
 // lse_in: row normalisers [units][T] (natural log) from the caller; non-null skips pass 1
+// attn_out: non-null replaces pass 1 by the fused attention forward, which also writes out [units, T, 128] (bf16)
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
-                              int32_t* dev_status, cudaStream_t st, const float* lse_in = nullptr);
+                              int32_t* dev_status, cudaStream_t st, const float* lse_in = nullptr, void* attn_out = nullptr);
+// attention forward of the general path: out [units, T, d] and natural-log normalisers
+cudaError_t launch_attention_fwd_general(const Shape& s, int dtype, const void* q, const void* k, const void* v, void* out,
+                                         float* lse, cudaStream_t st);
 size_t prefill_tc_workspace_bytes(int units, int T);  // padded log2-domain row normalisers
 cudaError_t launch_select(int units, int T, int B, int F, int R, const float* score, int32_t* kept, int32_t* dev_status,
                           cudaStream_t st);

@@ -22,7 +22,7 @@ IND_H2O, IND_WINDOW = 0, 1
 NORM_KINDS = {"l1": 0, "l2": 1, "linf": 2}
 FLAG_DECODE_OVERLAP = 1
 STATIC_SCRATCH_BYTES = (4 << 20) + 256
-EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_from_lse", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_compact_window", "vatp_decode_step",
+EXPORTS = ["vatp_cache_capacity", "vatp_workspace_bytes", "vatp_prefill_scores", "vatp_prefill_scores_from_lse", "vatp_prefill_attention_scores", "vatp_prefill_scores_static", "vatp_select", "vatp_compact", "vatp_compact_window", "vatp_decode_step",
            "vatp_selftest_bounded_wait", "vatp_selftest_overlap_policy", "vatp_status_string"]
 
 
@@ -48,6 +48,8 @@ lib.vatp_prefill_scores.restype = C.c_int
 lib.vatp_prefill_scores.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.vatp_prefill_scores_from_lse.restype = C.c_int
 lib.vatp_prefill_scores_from_lse.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
+lib.vatp_prefill_attention_scores.restype = C.c_int
+lib.vatp_prefill_attention_scores.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, C.c_size_t, _vp, _vp]
 lib.vatp_prefill_scores_static.restype = C.c_int
 lib.vatp_prefill_scores_static.argtypes = [C.POINTER(Params), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.vatp_select.restype = C.c_int
@@ -153,6 +155,16 @@ def vatp_prefill_scores_from_lse(p: Params, q, k, v, lse_in, *, lse_out=None, at
     _check(lib.vatp_prefill_scores_from_lse(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(lse_in), _ptr(lse_out),
                                             _ptr(attn_acc), _ptr(vnorm), _ptr(score), _ptr(win_rows), _ptr(workspace),
                                             ws_bytes, _ptr(dev_status), _stream(stream)), "vatp_prefill_scores_from_lse")
+
+
+def vatp_prefill_attention_scores(p: Params, q, k, v, attn_out, *, lse_out=None, attn_acc, vnorm, score, win_rows=None,
+                                  workspace=None, dev_status=None, stream=None):
+    """Attention forward fused with prefill scoring: also writes the layer's output rows attn_out
+    [batch, heads, T, head_dim] (Eq. 1); the indicator then costs one recomputation of QK^T."""
+    ws_bytes = 0 if workspace is None else workspace.numel() * workspace.element_size()
+    _check(lib.vatp_prefill_attention_scores(C.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(attn_out), _ptr(lse_out),
+                                             _ptr(attn_acc), _ptr(vnorm), _ptr(score), _ptr(win_rows), _ptr(workspace),
+                                             ws_bytes, _ptr(dev_status), _stream(stream)), "vatp_prefill_attention_scores")
 
 
 def vatp_prefill_scores_static(p: Params, q, k, v, *, lse_out=None, attn_acc, vnorm, score, win_rows=None,

@@ -40,13 +40,16 @@ class GpuPrefill:
     """Device buffers and the three prefill-side calls for one layer of a workload."""
 
     def __init__(self, wl: synth.Workload, q, k, v, *, n_sink=None, lse_given=False, decode_overlap=False,
-                 recompute_window=False):
+                 recompute_window=False, fused_forward=False):
         """decode_overlap: decode steps through this object carry VATP_FLAG_DECODE_OVERLAP (steps of
         caches that share no buffer may run side by side on the GPU).  recompute_window (Eq. 3 only): the
-        scoring call writes no win_rows and vatp_compact_window rebuilds the kept block of the history."""
+        scoring call writes no win_rows and vatp_compact_window rebuilds the kept block of the history.
+        fused_forward: scoring through vatp_prefill_attention_scores, which also writes the attention output."""
         V = vatp()
         self.wl = wl
         self.lse_given = lse_given
+        self.fused_forward = fused_forward
+        self.attn_out = torch.empty_like(q) if fused_forward else None
         self.F = wl.n_sink if n_sink is None else n_sink
         dev = q.device
         b, h, T = wl.batch, wl.heads, wl.seq_len
@@ -67,7 +70,11 @@ class GpuPrefill:
 
     def run(self):
         V = vatp()
-        if self.lse_given:
+        if self.fused_forward:
+            V.vatp_prefill_attention_scores(self.p, self.q, self.k, self.v, self.attn_out, lse_out=self.lse,
+                                            attn_acc=self.attn_acc, vnorm=self.vnorm, score=self.score,
+                                            win_rows=self.win_rows, workspace=self.ws, dev_status=self.status)
+        elif self.lse_given:
             # the row normalisers arrive from outside, as from an attention forward that ran before
             self.lse_in = attention_forward_lse(self.q, self.k, self.wl.scale)
             V.vatp_prefill_scores_from_lse(self.p, self.q, self.k, self.v, self.lse_in, lse_out=self.lse,
@@ -93,6 +100,20 @@ def rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     return float(np.max(np.abs(got - ref) / np.maximum(np.abs(ref), ABS_FLOOR))) if ref.size else 0.0
 
 
+def check_attention_output(got: np.ndarray, ref: np.ndarray, v: np.ndarray, dtype: str):
+    """Rows of the attention output against the oracle's (Eq. 1).  fp32: 1e-5 of the largest value.  bf16: the
+    probabilities are rounded to bf16 (relative 2^-9) before they meet V and the result is rounded to bf16
+    again, so every element is within 2^-9 * sum_i a_i |v_i| + 2^-9 * |out| <= 2^-8 * max|v|; the typical error
+    is an order of magnitude below that (independent roundings), and the mean error is held to a tenth of the bound."""
+    vmax = float(np.abs(v).max())
+    err = np.abs(got - ref)
+    if dtype == "f32":
+        assert err.max() <= 1e-5 * vmax, f"attention output: max err {err.max():.3g}"
+    else:
+        assert err.max() <= 2.0 ** -8 * vmax, f"attention output: max err {err.max():.3g} vs bound {2.0 ** -8 * vmax:.3g}"
+        assert err.mean() <= 0.1 * 2.0 ** -8 * vmax, f"attention output: mean err {err.mean():.3g}"
+
+
 def check_prefill_unit(g: GpuPrefill, b: int, h: int, tol: float):
     """Scores, kept set and compacted cache of one unit against the oracle.  Returns the oracle's
     prefill dict and the (validated) kept indices the GPU chose."""
@@ -104,6 +125,9 @@ def check_prefill_unit(g: GpuPrefill, b: int, h: int, tol: float):
 
     first = max(T - wl.window, 0) if window else 0
     lse = to_np64(g.lse[b, h])
+    if g.fused_forward:
+        first = 0                       # the forward normalises every row, inside the history window or not
+        check_attention_output(to_np64(g.attn_out[b, h]), ref["out"], vn, wl.dtype)
     assert np.max(np.abs(lse[first:] - ref["lse"][first:])) <= tol * 10, "lse"
     for name, key in (("attn_acc", "S"), ("vnorm", "n1"), ("score", "I")):
         got = to_np64(getattr(g, name)[b, h])

@@ -28,11 +28,12 @@ def _max_adopted(steps, n_units):
 
 
 def _run_case(wl, n_sink=None, decode=True, units=None, check_state_every=4, layer=0, lse_given=False,
-              decode_units=None, recompute_window=False):
+              decode_units=None, recompute_window=False, fused_forward=False):
     """units: the units the oracle checks at prefill (default: all); decode_units: those of them whose decode
     trajectory it follows (default: all of `units`)."""
     q, k, v = synth.prefill_inputs(wl, layer, "cuda")
-    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink, lse_given=lse_given, recompute_window=recompute_window).run()
+    g = P.GpuPrefill(wl, q, k, v, n_sink=n_sink, lse_given=lse_given, recompute_window=recompute_window,
+                     fused_forward=fused_forward).run()
     P.gpu_invariants(g)
     tol = P.TOL[wl.dtype]
     units = units or [(b, h) for b in range(wl.batch) for h in range(wl.heads)]
@@ -378,6 +379,50 @@ def test_prefill_from_given_row_normalisers_config1():
     """Config 1's shape (32 heads, prompt 4096) with given normalisers: oracle on sampled heads."""
     wl = synth.CONFIGS[1].with_(decode_steps=0)
     _run_case(wl, decode=False, units=[(0, 0), (0, 17)], lse_given=True)
+
+
+@pytest.mark.parametrize("dtype,d,T,B,indicator,window", [
+    ("bf16", 128, 1000, 300, "h2o", 0),       # tensor-core forward: 8 query tiles, ragged last tile
+    ("bf16", 128, 130, 65, "h2o", 0),         # two tiles, the second almost empty
+    ("bf16", 128, 100, 40, "h2o", 0),         # shorter than one tile
+    ("bf16", 128, 700, 200, "window", 150),   # Eq. 3: normalisers of every row, indicator over the last w
+    ("f32", 64, 333, 100, "h2o", 0),          # general forward
+    ("f32", 64, 200, 64, "window", 50),
+    ("bf16", 64, 257, 128, "h2o", 0),
+])
+def test_fused_attention_forward(dtype, d, T, B, indicator, window):
+    """vatp_prefill_attention_scores: the attention output rows (Eq. 1) against the oracle, and everything the
+    two-pass call produces - normalisers, indicator, norms, scores, kept sets, compaction, decode steps - checked
+    the same way; its scores agree with the two-pass call's within the score tolerance."""
+    wl = _small(dtype, d, T, B, 2, 10, b=2, h=3, indicator=indicator, window=window, steps=4, cid=75)
+    g, _, _ = _run_case(wl, fused_forward=True)
+    two = P.GpuPrefill(wl, g.q, g.k, g.v).run()
+    tol = P.TOL[dtype]
+    for name in ("attn_acc", "vnorm", "score"):
+        a, b_ = getattr(g, name).double(), getattr(two, name).double()
+        assert torch.all((a - b_).abs() <= 2 * tol * b_.abs() + 1e-30), name
+
+
+def test_fused_attention_forward_config1():
+    """Config 1's shape through the fused forward: oracle on two sampled heads (output rows, scores, kept set)."""
+    wl = synth.CONFIGS[1].with_(decode_steps=0)
+    _run_case(wl, decode=False, units=[(0, 3), (0, 30)], fused_forward=True)
+
+
+def test_fused_attention_forward_rescales_when_the_maximum_grows():
+    """Keys whose logits keep growing along the prompt force the forward to move its reference maximum (and
+    rescale the running output) in every chunk; keys whose logits fall never do.  Both against the oracle."""
+    wl = _small("bf16", 128, 640, 200, 2, 10, b=1, h=2, steps=0, cid=76)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    ramp = torch.linspace(0.0, 6.0, wl.seq_len, device="cuda")
+    for sign in (1.0, -1.0):
+        # every query has a positive component along one direction; the keys' component along it ramps up or down
+        q2, k2 = q.clone(), k.clone()
+        q2[..., 0] = 8.0
+        k2[..., 0] = (sign * ramp * 8.0).to(k.dtype)[None, None, :]
+        g = P.GpuPrefill(wl, q2, k2, v, fused_forward=True).run()
+        for h in range(wl.heads):
+            P.check_prefill_unit(g, 0, h, P.TOL["bf16"])
 
 
 def test_decode_large_cache_state_paths():
