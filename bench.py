@@ -227,6 +227,9 @@ def run_cuda(args, wl):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
     lse_given, fill_lse = [False], [True]   # the first call below fills every layer's lse; --lse-given then times pass 2 alone
+    # the fused call (attention output + scoring) is timed in a region of its own; one output buffer serves every layer
+    fused = [False]
+    attn_out = torch.empty_like(layers[0].q)
 
     def prefill_all(ev=None, parts=(True, True, True)):
         """parts: which of (scoring, selection, compaction) to issue for every layer."""
@@ -236,7 +239,11 @@ def run_cuda(args, wl):
                 if parts[2]: compact(ls)
                 continue
             if ev: ev[i][0].record()
-            if lse_given[0]:
+            if fused[0]:
+                V.vatp_prefill_attention_scores(ls.p, ls.q, ls.k, ls.v, attn_out, lse_out=ls.lse if windowed else None,
+                                                attn_acc=ls.attn_acc, vnorm=ls.vnorm, score=ls.score, win_rows=ls.win_rows,
+                                                workspace=ls.ws, dev_status=status)
+            elif lse_given[0]:
                 V.vatp_prefill_scores_from_lse(ls.p, ls.q, ls.k, ls.v, ls.lse, attn_acc=ls.attn_acc, vnorm=ls.vnorm,
                                                score=ls.score, win_rows=ls.win_rows, workspace=ls.ws, dev_status=status)
             else:
@@ -327,6 +334,13 @@ def run_cuda(args, wl):
         recs_c = [chain_ms(parts) for _ in range(max(3, min(args.steps, 6)))]
         barrier()
         chain[key] = statistics.median(a.elapsed_time(b) for a, b in recs_c) / L       # ms per layer
+    # the fused call in the scoring call's place: attention output rows, normalisers, indicator, norms, scores
+    fused[0] = True
+    chain_ms((True, False, False)); barrier()
+    recs_c = [chain_ms((True, False, False)) for _ in range(max(3, min(args.steps, 6)))]
+    barrier()
+    chain["score_fused"] = statistics.median(a.elapsed_time(b) for a, b in recs_c) / L
+    fused[0] = False
     prefill_all(); barrier()     # leave complete caches behind
 
     # the same decode steps with every launch waiting for all earlier work in the stream (no opt-in to
@@ -406,6 +420,8 @@ def run_cuda(args, wl):
         pairs = T * (T + 1) / 2
     passes = 1 if args.lse_given else 2
     flops_score = passes * (2.0 * d) * pairs * units           # each pass recomputes the causal part of QK^T
+    # fused call: the forward's two contractions over every causal pair, then pass 2's one
+    flops_fused = (2 * (2.0 * d) * (T * (T + 1) / 2) + (2.0 * d) * pairs) * units
     bytes_compact = units * (2 * 2 * B * d * 2 + 12 * B)       # K,V rows read + written, 12 B of state per slot
     if wl.indicator == "window":
         # history ring written; with --win-rows the kept columns of the last-w rows are read too
@@ -419,6 +435,9 @@ def run_cuda(args, wl):
         "prefill_scores": {"bound": "tensor", "achieved": flops_score / (t_score_c * 1e-3) / 1e12,
                            "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "ms_per_launch_pair": t_score_c,
                            "ms_isolated": ms(t_score), "achieved_isolated": flops_score / (ms(t_score) * 1e-3) / 1e12},
+        # vatp_prefill_attention_scores in the scoring call's place (not part of the timed step): three contraction sweeps
+        "attention_forward_scores": {"bound": "tensor", "achieved": flops_fused / (chain["score_fused"] * 1e-3) / 1e12,
+                                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "ms_per_call": chain["score_fused"]},
         "select": {"bound": "hbm", "achieved": bytes_select / (t_select_c * 1e-3) / 1e9, "peak": peaks["hbm_gbs"],
                    "unit": "GB/s", "us_per_launch": t_select_c * 1e3,
                    "us_isolated": ms(t_select) * 1e3, "achieved_isolated": bytes_select / (ms(t_select) * 1e-3) / 1e9},

@@ -793,7 +793,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 //
 //   per work item (unit, tile of 128 queries), streamed key / value chunks of 128 tokens 0 .. diagonal:
 //     S   = Q K^T            tcgen05, both operands K-major, fp32 in TMEM (two buffers)
-//     P   = exp2(S - m)      one thread per query row, written to shared memory as bf16 (the A operand's layout)
+//     P   = exp2(S - m)      two threads per query row, written back to TMEM as bf16 pairs (the A operand of the
+//                            next product is read from there: P never touches shared memory, whose bandwidth
+//                            the two products' operand reads and the incoming K and V tiles already use up)
 //     O  += P V              tcgen05, V straight from its [token, d] rows as an MN-major B operand, O in TMEM
 //     out = O / l, lse = m + log2 l
 //   m is a per-row reference that follows the running maximum lazily: O and l are rescaled only when the
@@ -801,28 +803,38 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 //   inside bf16 and fp32 range; once the first chunks - which hold the attention sinks - are past, almost
 //   no chunk rescales).  A rescale is a TMEM load / multiply / store of the thread's own row, done after
 //   the previous P V product has completed and before this chunk's product is released.
-// Warp roles (224 threads): warp 0 TMA producer and work-item FIFO, warp 1 MMA issuer, warps 2-5 softmax
-// (row = TMEM lane), warp 6 value norms (Eq. 4).  MMA order: S(c+1) is issued before O += P(c) V(c), so the
+// Warp roles (352 threads): warp 0 TMA producer and work-item FIFO, warp 1 MMA issuer, warps 2-9 softmax (row = TMEM
+// lane; two threads per row, 64 keys each, so that every scheduler has two warps to alternate between; a share of
+// the exponentials runs as a polynomial on the FMA pipe, as in pass 1), warp 10 value norms (Eq. 4).  MMA order: S(c+1) is issued before O += P(c) V(c), so the
 // tensor pipe recomputes the next logits while the softmax warps are still on chunk c.
-constexpr int FW_THREADS = 7 * 32;
-constexpr int FW_ST = 2;               // stages of K, of V and of P
-constexpr int FW_O_COL = 2 * TILE;     // TMEM columns: S buffers at 0 and 128, O at 256
+constexpr int FW_NSW = 8;               // softmax warps: two per quarter of the rows
+constexpr int FW_THREADS = (2 + FW_NSW + 1) * 32;
+#ifndef FW_POLY_MASK
+#define FW_POLY_MASK 0x0            // of the four pairs of an 8-probability piece, those whose exponential runs on the FMA pipe
+#endif
+constexpr int FW_ST = 3;               // stages of K and of V in shared memory
+constexpr int FW_PB = 2;               // P buffers in TMEM
+constexpr int FW_O_COL = 2 * TILE;     // TMEM columns: S buffers at 0 and 128, O at 256,
+constexpr int FW_P_COL = 3 * TILE;     // P buffers (bf16 pairs, 64 columns each) at 384 and 448
 constexpr float FW_LAZY = 8.f;         // log2 of the growth of a row maximum that forces a rescale
 
 struct FwdSmem {
   alignas(1024) unsigned char q[TILE_BYTES];
   alignas(1024) unsigned char k[FW_ST][TILE_BYTES];    // [d half][128 tokens][128 bytes]
   alignas(1024) unsigned char v[FW_ST][TILE_BYTES];    // [d half][128 tokens][128 bytes]
-  alignas(1024) unsigned char p[FW_ST][TILE_BYTES];    // [key half][128 queries][128 bytes]
   alignas(8) uint64_t q_full, q_empty;
   uint64_t k_full[FW_ST], k_empty[FW_ST], v_full[FW_ST], v_empty[FW_ST];
-  uint64_t s_full[2], s_empty[2], p_full[FW_ST], p_empty[FW_ST];
+  uint64_t s_full[2], s_empty[2], p_full[FW_PB], p_empty[FW_PB];
   uint64_t o_full, o_empty;
   uint64_t item_full[4], item_empty[4];
+  uint64_t pair_bar[4];                 // softmax warps q and q + 4 (same rows, other keys)
   int item_ring[4][2];                  // u, tile (u < 0: no more items)
+  float lsum[2][TILE];                  // per key half: the row sums, exchanged at the end of an item
   uint32_t tmem_base;
   int abort_flag;
 };
+
+static_assert(sizeof(FwdSmem) + 1024 <= 227 * 1024, "the forward kernel's shared memory (with alignment slack) must fit one CTA");
 
 // Shared-memory matrix descriptor of a V chunk as the B operand of O += P V: N (= d) is the contiguous
 // dimension.  128-byte swizzle; a row of 64 d-values per token, 8 tokens per 1024-byte group (stride
@@ -838,6 +850,15 @@ __device__ __forceinline__ void umma_bf16_rt(uint32_t tmem_d, uint64_t da, uint6
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(tmem_d), "l"(da), "l"(db), "r"(id), "r"(acc)
+      : "memory");
+}
+// the same with the A operand in TMEM: lane = row, 16-bit elements packed two to a column (K = 16 is 8 columns)
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t db, uint32_t id, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+      ::"r"(tmem_d), "r"(tmem_a), "l"(db), "r"(id), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void tmem_st32(uint32_t addr, const float (&v)[32]) {
@@ -875,11 +896,12 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     for (int i = 0; i < FW_ST; ++i) {
       mbar_init(&sm.k_full[i], 1); mbar_init(&sm.k_empty[i], 1);
       mbar_init(&sm.v_full[i], 1); mbar_init(&sm.v_empty[i], 1);
-      mbar_init(&sm.p_full[i], 4); mbar_init(&sm.p_empty[i], 1);
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.s_empty[i], 4); }
-    mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, 4);
-    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 5); }   // MMA warp + 4 softmax warps
+    for (int i = 0; i < FW_PB; ++i) { mbar_init(&sm.p_full[i], FW_NSW); mbar_init(&sm.p_empty[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.s_empty[i], FW_NSW); }
+    mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, FW_NSW);
+    for (int i = 0; i < 4; ++i) mbar_init(&sm.pair_bar[i], 2);
+    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 1 + FW_NSW); }   // MMA warp + softmax warps
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -966,7 +988,7 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       bool ok = true;
       uint32_t n = 0;
       const uint64_t q_desc = umma_desc(s32(sm.q));
-      const uint64_t k_desc0 = umma_desc(s32(sm.k[0])), p_desc0 = umma_desc(s32(sm.p[0]));
+      const uint64_t k_desc0 = umma_desc(s32(sm.k[0]));
       const uint64_t v_desc0 = umma_desc_mn(s32(sm.v[0]));
       // S(g) = Q K(g)^T into S buffer g % 2
       auto issue_qk = [&](uint32_t g) -> bool {
@@ -996,32 +1018,43 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           const uint32_t g = n + c;
           if (c + 1 < nc) { ok = issue_qk(g + 1); if (!ok) break; }
           else umma_commit(&sm.q_empty);            // the item's last S has been issued: the query tile may be replaced
-          const int stg = g % FW_ST;
-          ok = mbar_wait(&sm.p_full[stg], (g / FW_ST) & 1, abort_flag, a.dev_status) &&
+          const int stg = g % FW_ST, pb = g % FW_PB;
+          ok = mbar_wait(&sm.p_full[pb], (g / FW_PB) & 1, abort_flag, a.dev_status) &&
                mbar_wait(&sm.v_full[stg], (g / FW_ST) & 1, abort_flag, a.dev_status) &&
                (c > 0 || mbar_wait(&sm.o_empty, (itl & 1) ^ 1, abort_flag, a.dev_status));
           if (!ok) break;
           tc_fence_after();
-          const uint64_t pd = p_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
           const uint64_t vd = v_desc0 + (uint64_t)stg * (TILE_BYTES >> 4);
 #pragma unroll
-          for (int kk = 0; kk < TILE / 16; ++kk)      // 16 keys per step: 2048 bytes further on in V
-            umma_bf16_rt(tmem + FW_O_COL, pd + k_off_fixed(kk), vd + (uint64_t)(kk * 128), IDESC_PV, (c > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < TILE / 16; ++kk)      // 16 keys per step: 8 columns further on in P, 2048 bytes in V
+            umma_bf16_ts(tmem + FW_O_COL, tmem + FW_P_COL + pb * 64 + kk * 8, vd + (uint64_t)(kk * 128), IDESC_PV,
+                         (c > 0 || kk > 0) ? 1u : 0u);
           umma_commit(&sm.v_empty[stg]);
-          umma_commit(&sm.p_empty[stg]);
+          umma_commit(&sm.p_empty[pb]);
           if (c == nc - 1) umma_commit(&sm.o_full);
         }
         n += nc;
       }
     }
-  } else if (wid < 6) {
-    // ------------------------------------------------------------------ softmax: one thread per query row
+  } else if (wid < 2 + FW_NSW) {
+    // ------------------------------------------------------------------ softmax: two threads per query row
     const int quarter = wid & 3;                  // TMEM lanes this warp may touch
+    const int half = (wid - 2) >> 2;              // which 64 of a chunk's 128 keys (and of O's 128 columns) are this thread's
     const int row = quarter * 32 + lane;
-    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)(quarter * 32) << 16) + half * 64;
     const float sc = a.scale_log2;
     bool ok = true;
     uint32_t n = 0;
+    // the two warps that share a quarter of the rows meet at an mbarrier of their own (a bounded wait like all
+    // others: one arrival per warp, after which the partner's shared-memory stores are visible)
+    uint32_t pair_phase = 0;
+    auto pair_sync = [&]() -> bool {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sm.pair_bar[quarter]);
+      bool got = mbar_wait(&sm.pair_bar[quarter], pair_phase & 1, abort_flag, a.dev_status);
+      ++pair_phase;
+      return __all_sync(0xffffffffu, got);
+    };
     for (uint32_t itl = 0; ok; ++itl) {
       int u, tile;
       next_item(itl, true, u, tile);
@@ -1029,47 +1062,58 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       if (!VATP_INB(u, a.units, a.dev_status) || !VATP_INB(tile, a.nt, a.dev_status)) break;
       const int tok = tile * TILE + row;
       const int nc = tile + 1;
-      float m_ref = -INFINITY, l_run = 0.f;
+      float m_ref = -INFINITY, l_run = 0.f;       // l_run: this thread's 64 columns only
       for (int c = 0; c < nc; ++c) {
         const uint32_t g = n + c;
-        const int sb = g & 1, stg = g % FW_ST;
+        const int sb = g & 1, pb = g % FW_PB;
         bool w = mbar_wait(&sm.s_full[sb], (g >> 1) & 1, abort_flag, a.dev_status);
         w = __all_sync(0xffffffffu, w);
         if (!w) { ok = false; break; }
         tc_fence_after();
-        float x[4][32];
-#pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) tmem_ld32(lane_addr + sb * TILE + q4 * 32, x[q4]);
-        tmem_ld_wait();
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.s_empty[sb]);
-        if (c == tile) {
-#pragma unroll
-          for (int q4 = 0; q4 < 4; ++q4) mask_after_diagonal(x[q4], q4 * 32, row);
+        // own 64 columns (kept), then the partner's 64 for the row maximum only: reading them from TMEM
+        // again costs less than an exchange through shared memory and a rendezvous in every chunk
+        float x[2][32];
+        float mx;
+        {
+          float y[2][32];
+          const uint32_t other = lane_addr + sb * TILE + (half ? -64 : 64);
+          tmem_ld32(lane_addr + sb * TILE, x[0]);
+          tmem_ld32(lane_addr + sb * TILE + 32, x[1]);
+          tmem_ld32(other, y[0]);
+          tmem_ld32(other + 32, y[1]);
+          tmem_ld_wait();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.s_empty[sb]);
+          if (c == tile) {
+            mask_after_diagonal(x[0], half * 64, row);
+            mask_after_diagonal(x[1], half * 64 + 32, row);
+            mask_after_diagonal(y[0], (half ^ 1) * 64, row);
+            mask_after_diagonal(y[1], (half ^ 1) * 64 + 32, row);
+          }
+          // scaled maximum of the row's 128 logits (scale > 0)
+          mx = fmaxf(fmaxf(slice_max(x[0]), slice_max(x[1])), fmaxf(slice_max(y[0]), slice_max(y[1]))) * sc;
         }
-        // scaled maximum of the row's 128 logits (scale > 0)
-        const float mx = fmaxf(fmaxf(slice_max(x[0]), slice_max(x[1])), fmaxf(slice_max(x[2]), slice_max(x[3]))) * sc;
         const float m_new = fmaxf(m_ref, mx);
         if (c == 0) {
           m_ref = m_new;              // finite: column 0 is never masked
         } else {
           const bool need = m_new > m_ref + FW_LAZY;
           if (__any_sync(0xffffffffu, need)) {
-            // O += P(g-1) V(g-1) must have completed before this thread's row of O is rewritten
-            bool w2 = mbar_wait(&sm.p_empty[(g - 1) % FW_ST], ((g - 1) / FW_ST) & 1, abort_flag, a.dev_status);
+            // O += P(g-1) V(g-1) must have completed before this thread's part of its row of O is rewritten
+            bool w2 = mbar_wait(&sm.p_empty[(g - 1) % FW_PB], ((g - 1) / FW_PB) & 1, abort_flag, a.dev_status);
             w2 = __all_sync(0xffffffffu, w2);
             if (!w2) { ok = false; break; }
             tc_fence_after();
             const float f = need ? ex2(m_ref - m_new) : 1.f;
 #pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
+            for (int q2 = 0; q2 < 2; ++q2) {
               float y[32];
-              tmem_ld32(lane_addr + FW_O_COL + q4 * 32, y);
+              tmem_ld32(lane_addr + FW_O_COL + q2 * 32, y);
               tmem_ld_wait();
 #pragma unroll
               for (int i = 0; i < 32; ++i) y[i] *= f;
-              tmem_st32(lane_addr + FW_O_COL + q4 * 32, y);
+              tmem_st32(lane_addr + FW_O_COL + q2 * 32, y);
             }
             tmem_st_wait();
             l_run *= f;
@@ -1077,51 +1121,57 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           }
         }
         // the P buffer is free once the product that read it two chunks ago has completed
-        bool w3 = mbar_wait(&sm.p_empty[stg], ((g / FW_ST) & 1) ^ 1, abort_flag, a.dev_status);
+        bool w3 = mbar_wait(&sm.p_empty[pb], ((g / FW_PB) & 1) ^ 1, abort_flag, a.dev_status);
         w3 = __all_sync(0xffffffffu, w3);
         if (!w3) { ok = false; break; }
-        unsigned char* prow = sm.p[stg] + row * 128;
+        tc_fence_after();
         const f32x2 c2 = pk2(sc, sc), nm2 = pk2(-m_ref, -m_ref);
         f32x2 la = pk2(0.f, 0.f), lb = la;
+        float pk[32];                              // 64 probabilities as bf16 pairs: this thread's columns of the P buffer
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {            // 16-byte pieces of the row: 8 probabilities each
+        for (int j = 0; j < 8; ++j) {
           const float* xs = &x[j >> 2][(j & 3) * 8];
-          float p[8];
 #pragma unroll
           for (int i = 0; i < 8; i += 2) {
-            const f32x2 e = ex2_sfu2(fma2(pk2(xs[i], xs[i + 1]), c2, nm2));
+            const f32x2 t = fma2(pk2(xs[i], xs[i + 1]), c2, nm2);
+            const f32x2 e = ((FW_POLY_MASK >> (i >> 1)) & 1) ? ex2_fma2(t) : ex2_sfu2(t);
             if (i & 2) lb = add2(lb, e); else la = add2(la, e);
-            upk2(e, p[i], p[i + 1]);
+            float p0, p1;
+            upk2(e, p0, p1);
+            pk[j * 4 + (i >> 1)] = __uint_as_float(pack2_bf16(p0, p1));
           }
-          const uint4 pk = make_uint4(pack2_bf16(p[0], p[1]), pack2_bf16(p[2], p[3]), pack2_bf16(p[4], p[5]), pack2_bf16(p[6], p[7]));
-          *reinterpret_cast<uint4*>(prow + (j >> 3) * SLAB_BYTES + (((j & 7) ^ (row & 7)) << 4)) = pk;
         }
+        tmem_st32(tmem + ((uint32_t)(quarter * 32) << 16) + FW_P_COL + pb * 64 + half * 32, pk);
         l_run += hsum2(add2(la, lb));
-        // P (generic-proxy stores) and any rescaled O (TMEM stores) are complete before the MMA warp is told
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        // P and any rescaled O (TMEM stores) are complete before the MMA warp is told
+        tmem_st_wait();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&sm.p_full[stg]);
+        if (lane == 0) mbar_arrive(&sm.p_full[pb]);
       }
       if (!ok) break;
       n += nc;
-      // ---- end of item: out = O / l, lse = m + log2 l
+      // ---- end of item: out = O / l, lse = m + log2 l (l: both halves of the row)
+      sm.lsum[half][row] = l_run;
+      if (!pair_sync()) { ok = false; break; }
+      const float l_row = sm.lsum[0][row] + sm.lsum[1][row];
+      if (!pair_sync()) { ok = false; break; }      // both have read: the next item may overwrite
       bool w4 = mbar_wait(&sm.o_full, itl & 1, abort_flag, a.dev_status);
       w4 = __all_sync(0xffffffffu, w4);
       if (!w4) { ok = false; break; }
       tc_fence_after();
-      const float inv = 1.f / l_run;
-      __nv_bfloat16* orow = out + ((int64_t)u * a.T + tok) * HD;
+      const float inv = 1.f / l_row;
+      __nv_bfloat16* orow = out + ((int64_t)u * a.T + tok) * HD + half * 64;
       const bool live = tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status);
 #pragma unroll
-      for (int q4 = 0; q4 < 4; ++q4) {
+      for (int q2 = 0; q2 < 2; ++q2) {
         float y[32];
-        tmem_ld32(lane_addr + FW_O_COL + q4 * 32, y);
+        tmem_ld32(lane_addr + FW_O_COL + q2 * 32, y);
         tmem_ld_wait();
         if (live) {
 #pragma unroll
           for (int j = 0; j < 4; ++j)
-            reinterpret_cast<uint4*>(orow + q4 * 32)[j] =
+            reinterpret_cast<uint4*>(orow + q2 * 32)[j] =
                 make_uint4(pack2_bf16(y[8 * j] * inv, y[8 * j + 1] * inv), pack2_bf16(y[8 * j + 2] * inv, y[8 * j + 3] * inv),
                            pack2_bf16(y[8 * j + 4] * inv, y[8 * j + 5] * inv), pack2_bf16(y[8 * j + 6] * inv, y[8 * j + 7] * inv));
         }
@@ -1129,15 +1179,17 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sm.o_empty);
-      const float lse2 = m_ref + log2f(l_run);
-      // the layout pass 2 reads: negated, -inf where a query contributes nothing (beyond the prompt, before the
-      // history window), half a chunk of padding after an odd tile count
-      if (VATP_INB((int64_t)u * a.Tpad + tok, (int64_t)a.units * a.Tpad, a.dev_status))
-        a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? -lse2 : -INFINITY;
-      if ((a.nt & 1) && tile == a.nt - 1 && VATP_INB((int64_t)u * a.Tpad + tok + TILE, (int64_t)a.units * a.Tpad, a.dev_status))
-        a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
-      if (a.lse_out && tok < a.T)
-        a.lse_out[(int64_t)(u / a.heads) * a.lse_sb + (int64_t)(u % a.heads) * a.lse_sh + tok] = lse2 * 0.69314718055994531f;
+      if (half == 0) {
+        const float lse2 = m_ref + log2f(l_row);
+        // the layout pass 2 reads: negated, -inf where a query contributes nothing (beyond the prompt, before the
+        // history window), half a chunk of padding after an odd tile count
+        if (VATP_INB((int64_t)u * a.Tpad + tok, (int64_t)a.units * a.Tpad, a.dev_status))
+          a.lse2[(int64_t)u * a.Tpad + tok] = (tok < a.T && tok >= a.first_row) ? -lse2 : -INFINITY;
+        if ((a.nt & 1) && tile == a.nt - 1 && VATP_INB((int64_t)u * a.Tpad + tok + TILE, (int64_t)a.units * a.Tpad, a.dev_status))
+          a.lse2[(int64_t)u * a.Tpad + tok + TILE] = -INFINITY;
+        if (a.lse_out && tok < a.T)
+          a.lse_out[(int64_t)(u / a.heads) * a.lse_sb + (int64_t)(u % a.heads) * a.lse_sh + tok] = lse2 * 0.69314718055994531f;
+      }
     }
   } else if (a.side_norm) {
     // ------------------------------------------------------------------ value norms (Eq. 4)
