@@ -25,7 +25,8 @@
 //     flight (another layer's or another sequence's cache) never waits: its control warp releases
 //     the next launch at once and only holds the CTA until the previous launch has completed, so
 //     launches still complete in order and the number in flight is bounded by what fits on the
-//     machine (two CTAs fit on an SM).
+//     machine (two CTAs fit on an SM).  A launch that does wait has its SMs to itself and runs the
+//     eight-warp variant of the kernel (same arithmetic, see MW below).
 #include <cooperative_groups.h>
 
 #include <mutex>
@@ -37,9 +38,18 @@ namespace cg = cooperative_groups;
 namespace vatp {
 namespace {
 
-constexpr int MW = 4;                 // streaming warps per CTA
-constexpr int WT = MW * 32;           // their threads
-constexpr int MT = WT + 32;           // plus one control warp
+// Streaming warps per CTA (template parameter MW of the kernel; their threads WT = 32 MW, plus one control warp):
+// four when launches of different caches run side by side (two CTAs per SM), eight for a launch that waits for its
+// predecessor and has the SM to itself - one warp per scheduler cannot hide the latency of its own
+// ldmatrix / mma.sync / softmax chain, so such a launch streams faster with two.
+// The arithmetic does not depend on MW: a CTA's 16-row groups are always dealt to NSTREAM = 8 online-softmax streams -
+// the groups below the midpoint H (a multiple of four) to streams 0-3 by g mod 4, those from H on to streams 4-7 -
+// each stream is folded in ascending group order, and the eight partials are merged in stream order.  A warp of the
+// eight-warp kernel folds one stream; warp w of the four-warp kernel walks groups w, w + 4, ... in one sweep,
+// files its partial under stream w where it crosses H and starts afresh for stream w + 4.  Results are
+// bit-identical whichever kernel a launch gets.
+constexpr int MW_BESIDE = 4, MW_ALONE = 8;
+constexpr int NSTREAM = 8;
 constexpr int HD = 128;
 constexpr int GROUP = 16;             // rows per MMA group = rows of K (and of V) per stage
 constexpr int ROW_BYTES = HD * 2;
@@ -119,6 +129,7 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // barrier over the streaming warps only (the control warp does not take part)
+template <int WT>
 __device__ __forceinline__ void workers_sync() { asm volatile("bar.sync 1, %0;" ::"n"(WT) : "memory"); }
 __device__ __forceinline__ void cluster_arrive_release() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
 __device__ __forceinline__ void cluster_wait_acquire() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
@@ -131,7 +142,6 @@ struct Exch {
   int key_slot[MAX_SPLIT], key_pos[MAX_SPLIT];   // ... its slot in the unit and its position
 };
 
-static_assert(WT == HD, "one streaming thread per output channel");
 
 // eviction order as one integer: lower importance first, among equals the higher position first
 __device__ __forceinline__ unsigned long long evict_key(float I, int pos) {
@@ -145,14 +155,16 @@ __device__ __forceinline__ unsigned long long warp_min_key(unsigned long long ke
   return ((unsigned long long)mh << 32) | ml;
 }
 
-template <bool WINDOWED>
-__global__ void __launch_bounds__(MT, 2)
+template <bool WINDOWED, int MW>
+__global__ void __launch_bounds__(MW * 32 + 32, MW == MW_BESIDE ? 2 : 1)
 decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int independent,
                   int state_in_smem, int split, int chunk, int nstage, int B, int cap, int F, int R, int w, int norm, float scale_log2,
                   vatp_cache c,
                   const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
                   const __nv_bfloat16* __restrict__ v_new, __nv_bfloat16* __restrict__ out,
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
+  constexpr int WT = MW * 32;           // streaming threads (at least HD: one per output channel where outputs are formed)
+  static_assert(WT >= HD, "one streaming thread per output channel");
   extern __shared__ unsigned char dyn_raw[];
   unsigned char* dyn = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dyn_raw) + 1023) & ~uintptr_t(1023));
   // [MW][nstage] stages | logits[chunk] | acc[chunk] | vnorm[chunk] | pos[chunk]: the per-slot arrays of
@@ -168,8 +180,10 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 
   __shared__ __align__(8) uint64_t bars[MW * 4 + 1];
   __shared__ __align__(16) Exch ex;
-  __shared__ __align__(16) float part_o[MW][HD];
-  __shared__ float part_m[MW], part_l[MW];
+  constexpr int SPW = NSTREAM / MW;     // streams per warp
+  static_assert(SPW == 1 || SPW == 2, "a warp folds one or two streams");
+  __shared__ __align__(16) float part_o[NSTREAM][HD];
+  __shared__ float part_m[NSTREAM], part_l[NSTREAM];
   __shared__ unsigned long long warp_key[MW];
   __shared__ int ctrl_evicting;
 
@@ -229,8 +243,12 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     __syncwarp();
     if (lane < 4) tma_load_2d(dst + lane * TILE_BYTES, lane < 2 ? &tm_k : &tm_v, bar, (lane & 1) * 64, row_base + g * GROUP);
   };
+  // This warp's groups: g_first, g_first + 4, ... below g_end.  H: where streams 4-7 begin.
+  const int H = ((ngroups + 7) >> 3) << 2;
+  const int g_first = SPW == 2 ? wid : (wid < 4 ? wid : H + wid - 4);
+  const int g_end = (SPW == 2 || wid >= 4) ? ngroups : min(H, ngroups);
   for (int s = 0; s < nstage; ++s)
-    if (wid + s * MW < ngroups) issue(wid + s * MW, s);
+    if (g_first + s * 4 < g_end) issue(g_first + s * 4, s);
   // The next launch in the stream may start now; nothing below this line is read before the previous
   // launch has completed and its writes are visible.
   if (!independent) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -326,104 +344,133 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const int lm_i = lane >> 3, lm_r = lane & 7;
   const uint32_t k_row_off = (uint32_t)(((lm_i >> 1) * 8 + lm_r) * 128), k_x = (uint32_t)((lm_i & 1) ^ lm_r);
   const uint32_t v_row_off = (uint32_t)(((lm_i & 1) * 8 + lm_r) * 128), v_x = (uint32_t)((lm_i >> 1) ^ lm_r);
-  int it = 0;
-  for (int g = wid; g < ngroups; g += MW, ++it) {
-    if (it >= nstage && g * GROUP >= cnt) break;     // never requested (see the end of the loop body)
-    const int stage = it % nstage;
-    const uint32_t parity = (it / nstage) & 1;
-    if (ok && !mbar_wait(&my_bars[stage], parity)) ok = false;
-    ok = __all_sync(0xffffffffu, ok);
-    unsigned char* ks = my_stages + stage * STAGE_BYTES;
-    unsigned char* vs = ks + 2 * TILE_BYTES;
-    const int r0 = g * GROUP;
-    bool wrote = false;
-    if (ok && r0 < cnt) {
-      // the incoming token's row is not in the cache yet: patch it in; rows beyond the live range
-      // must not reach the p V product (their probability is 0, but 0 * garbage need not be 0)
-      if (owns_new && fs_local >= r0 && fs_local < r0 + GROUP) {
-        const int rr = fs_local - r0, ch = lane & 15;
-        *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = new_raw;
-        wrote = true;
-      }
-      if (owns_last && ls_local >= r0 && ls_local < r0 + GROUP) {
-        const int rr = ls_local - r0, ch = lane & 15;
-        *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = last_raw;
-        wrote = true;
-      }
-      if (cnt < r0 + GROUP) {
-        for (int rr = cnt - r0 + (lane >> 4); rr < GROUP; rr += 2)
-          *reinterpret_cast<uint4*>(vs + ((lane >> 3) & 1) * TILE_BYTES + rr * 128 + ((lane & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-        wrote = true;
-      }
-      __syncwarp();
-      // S^T = q K^T: two n-tiles of 8 rows; c[0], c[1] = logits of rows 2 j4, 2 j4 + 1 of the tile
-      float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
-      const uint32_t kaddr = smem_u32(ks) + k_row_off;
+  // the running partial goes to its stream's slot (every lane with the same j4 holds the same values; rows 0-7
+  // are the hi part, 8-15 the lo part)
+  auto flush = [&](int stream) {
+    float l = l_run;
+    l += __shfl_xor_sync(0xffffffffu, l, 1);
+    l += __shfl_xor_sync(0xffffffffu, l, 2);
+    if (lane < 4) {
 #pragma unroll
-      for (int kk = 0; kk < HD / 16; ++kk) {
-        uint32_t bf[4];
-        ldsm_x4(kaddr + (kk >> 2) * TILE_BYTES + ((k_x ^ ((2 * kk) & 7)) << 4), bf);
-        mma_bf16(sa, qa[kk][0], 0u, qa[kk][1], 0u, bf[0], bf[1]);
-        mma_bf16(sb, qa[kk][0], 0u, qa[kk][1], 0u, bf[2], bf[3]);
-      }
-      float s[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
-      const int rows[4] = {r0 + 2 * j4, r0 + 2 * j4 + 1, r0 + 8 + 2 * j4, r0 + 9 + 2 * j4};
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (rows[i] >= cnt) s[i] = -INFINITY;
-      if (lane < 4) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i)
-          if (rows[i] < cnt) logit_s[rows[i]] = s[i];
-      }
-      float gmax = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
-      gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
-      gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
-      if (gmax > m_run) {          // warp-uniform (r0 < cnt guarantees a live row, so gmax is finite)
-        const float f = ex2(m_run - gmax);   // 0 on the first group
-        l_run *= f;
-#pragma unroll
-        for (int i = 0; i < HD / 8; ++i) { o_acc[i][0] *= f; o_acc[i][1] *= f; o_acc[i][2] *= f; o_acc[i][3] *= f; }
-        m_run = gmax;
-      }
-      float p[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) { p[i] = ex2(s[i] - m_run); l_run += p[i]; }
-      // A operand of p V: rows 0-7 carry the high bf16 half of p, rows 8-15 the remainder
-      const uint32_t hi0 = pack_bf16(p[0], p[1]), hi1 = pack_bf16(p[2], p[3]);
-      const uint32_t lo0 = pack_bf16(p[0] - __uint_as_float(hi0 << 16), p[1] - __uint_as_float(hi0 & 0xffff0000u));
-      const uint32_t lo1 = pack_bf16(p[2] - __uint_as_float(hi1 << 16), p[3] - __uint_as_float(hi1 & 0xffff0000u));
-      const uint32_t vaddr = smem_u32(vs) + v_row_off;
-#pragma unroll
-      for (int nn = 0; nn < HD / 16; ++nn) {
-        uint32_t bf[4];
-        ldsm_x4_t(vaddr + (nn >> 2) * TILE_BYTES + ((v_x ^ ((2 * nn) & 7)) << 4), bf);
-        mma_bf16(o_acc[2 * nn], hi0, lo0, hi1, lo1, bf[0], bf[1]);
-        mma_bf16(o_acc[2 * nn + 1], hi0, lo0, hi1, lo1, bf[2], bf[3]);
-      }
+      for (int i = 0; i < HD / 8; ++i)
+        *reinterpret_cast<float2*>(&part_o[stream][i * 8 + 2 * j4]) = make_float2(o_acc[i][0] + o_acc[i][2], o_acc[i][1] + o_acc[i][3]);
+      if (lane == 0) { part_m[stream] = m_run; part_l[stream] = l; }
     }
-    // generic-proxy stores into a stage must be ordered before the next bulk copy into it
-    if (wrote) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    __syncwarp();
-    const int next = g + nstage * MW;
-    // later requests know the live range: groups beyond it are not fetched
-    if (ok && next < ngroups && next * GROUP < cnt) issue(next, stage);
+  };
+  if (SPW == 2) {      // the second stream may stay empty
+    *reinterpret_cast<float4*>(&part_o[wid + MW][lane * 4]) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (lane == 0) { part_m[wid + MW] = -INFINITY; part_l[wid + MW] = 0.f; }
+  }
+  int it = 0, g = g_first;
+  bool past_live = false, second = false;
+  // folds this warp's groups below g_stop into the running partial
+  auto fold_groups = [&](int g_stop) {
+    for (; g < g_stop; g += 4, ++it) {
+      if (it >= nstage && g * GROUP >= cnt) { past_live = true; break; }     // never requested (see the end of the loop body)
+      const int stage = it % nstage;
+      const uint32_t parity = (it / nstage) & 1;
+      if (ok && !mbar_wait(&my_bars[stage], parity)) ok = false;
+      ok = __all_sync(0xffffffffu, ok);
+      unsigned char* ks = my_stages + stage * STAGE_BYTES;
+      unsigned char* vs = ks + 2 * TILE_BYTES;
+      const int r0 = g * GROUP;
+      bool wrote = false;
+      if (ok && r0 < cnt) {
+        // the incoming token's row is not in the cache yet: patch it in; rows beyond the live range
+        // must not reach the p V product (their probability is 0, but 0 * garbage need not be 0)
+        if (owns_new && fs_local >= r0 && fs_local < r0 + GROUP) {
+          const int rr = fs_local - r0, ch = lane & 15;
+          *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = new_raw;
+          wrote = true;
+        }
+        if (owns_last && ls_local >= r0 && ls_local < r0 + GROUP) {
+          const int rr = ls_local - r0, ch = lane & 15;
+          *reinterpret_cast<uint4*>((lane < 16 ? ks : vs) + (ch >> 3) * TILE_BYTES + rr * 128 + (((ch & 7) ^ (rr & 7)) << 4)) = last_raw;
+          wrote = true;
+        }
+        if (cnt < r0 + GROUP) {
+          for (int rr = cnt - r0 + (lane >> 4); rr < GROUP; rr += 2)
+            *reinterpret_cast<uint4*>(vs + ((lane >> 3) & 1) * TILE_BYTES + rr * 128 + ((lane & 7) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          wrote = true;
+        }
+        __syncwarp();
+        // S^T = q K^T: two n-tiles of 8 rows; c[0], c[1] = logits of rows 2 j4, 2 j4 + 1 of the tile
+        float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t kaddr = smem_u32(ks) + k_row_off;
+  #pragma unroll
+        for (int kk = 0; kk < HD / 16; ++kk) {
+          uint32_t bf[4];
+          ldsm_x4(kaddr + (kk >> 2) * TILE_BYTES + ((k_x ^ ((2 * kk) & 7)) << 4), bf);
+          mma_bf16(sa, qa[kk][0], 0u, qa[kk][1], 0u, bf[0], bf[1]);
+          mma_bf16(sb, qa[kk][0], 0u, qa[kk][1], 0u, bf[2], bf[3]);
+        }
+        float s[4] = {sa[0] * scale_log2, sa[1] * scale_log2, sb[0] * scale_log2, sb[1] * scale_log2};
+        const int rows[4] = {r0 + 2 * j4, r0 + 2 * j4 + 1, r0 + 8 + 2 * j4, r0 + 9 + 2 * j4};
+  #pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (rows[i] >= cnt) s[i] = -INFINITY;
+        if (lane < 4) {
+  #pragma unroll
+          for (int i = 0; i < 4; ++i)
+            if (rows[i] < cnt) logit_s[rows[i]] = s[i];
+        }
+        float gmax = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
+        gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
+        if (gmax > m_run) {          // warp-uniform (r0 < cnt guarantees a live row, so gmax is finite)
+          const float f = ex2(m_run - gmax);   // 0 on the first group
+          l_run *= f;
+  #pragma unroll
+          for (int i = 0; i < HD / 8; ++i) { o_acc[i][0] *= f; o_acc[i][1] *= f; o_acc[i][2] *= f; o_acc[i][3] *= f; }
+          m_run = gmax;
+        }
+        float p[4];
+  #pragma unroll
+        for (int i = 0; i < 4; ++i) { p[i] = ex2(s[i] - m_run); l_run += p[i]; }
+        // A operand of p V: rows 0-7 carry the high bf16 half of p, rows 8-15 the remainder
+        const uint32_t hi0 = pack_bf16(p[0], p[1]), hi1 = pack_bf16(p[2], p[3]);
+        const uint32_t lo0 = pack_bf16(p[0] - __uint_as_float(hi0 << 16), p[1] - __uint_as_float(hi0 & 0xffff0000u));
+        const uint32_t lo1 = pack_bf16(p[2] - __uint_as_float(hi1 << 16), p[3] - __uint_as_float(hi1 & 0xffff0000u));
+        const uint32_t vaddr = smem_u32(vs) + v_row_off;
+  #pragma unroll
+        for (int nn = 0; nn < HD / 16; ++nn) {
+          uint32_t bf[4];
+          ldsm_x4_t(vaddr + (nn >> 2) * TILE_BYTES + ((v_x ^ ((2 * nn) & 7)) << 4), bf);
+          mma_bf16(o_acc[2 * nn], hi0, lo0, hi1, lo1, bf[0], bf[1]);
+          mma_bf16(o_acc[2 * nn + 1], hi0, lo0, hi1, lo1, bf[2], bf[3]);
+        }
+      }
+      // generic-proxy stores into a stage must be ordered before the next bulk copy into it
+      if (wrote) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      const int next = g + nstage * 4;
+      // later requests know the live range: groups beyond it are not fetched
+      if (ok && next < g_end && next * GROUP < cnt) issue(next, stage);
+    }
+  };
+  if (SPW == 2) {
+    // the four-warp kernel: stream wid up to the midpoint, filed, then stream wid + 4 from a fresh partial
+    fold_groups(min(H, g_end));
+    if (!past_live && g < g_end) {
+      flush(wid);
+      second = true;
+      m_run = -INFINITY;
+      l_run = 0.f;
+#pragma unroll
+      for (int i = 0; i < HD / 8; ++i) { o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f; }
+      fold_groups(g_end);
+    }
+  } else {
+    fold_groups(g_end);
   }
   if (!ok && lane == 0) {
     // a copy never completed: flag it and give what is still in flight one more bounded wait
     if (dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
     for (int s = 0; s < nstage; ++s) mbar_wait(&my_bars[s], 0);
   }
-  // warp partial: every lane with the same j4 holds the same values; rows 0-7 are the hi part, 8-15 the lo part
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 1);
-  l_run += __shfl_xor_sync(0xffffffffu, l_run, 2);
-  if (lane < 4) {
-#pragma unroll
-    for (int i = 0; i < HD / 8; ++i)
-      *reinterpret_cast<float2*>(&part_o[wid][i * 8 + 2 * j4]) = make_float2(o_acc[i][0] + o_acc[i][2], o_acc[i][1] + o_acc[i][3]);
-    if (lane == 0) { part_m[wid] = m_run; part_l[wid] = l_run; }
-  }
-  workers_sync();
+  // (a four-warp kernel that never reached the midpoint files everything under stream wid: its stream wid + 4 is empty)
+  flush(second ? wid + MW : wid);
+  workers_sync<WT>();
   if (state_in_smem == 2 && tid == 32 && rows_alloc > 0) {
     // every stage of this CTA has been consumed: the per-slot state of its slots lands there while the
     // cluster gathers (the stages were last written by bulk copies and read by ldmatrix; warps that
@@ -439,10 +486,10 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   {
     float m_c = -INFINITY;
 #pragma unroll
-    for (int i = 0; i < MW; ++i) m_c = fmaxf(m_c, part_m[i]);
-    float fw[MW], l_c = 0.f;
+    for (int i = 0; i < NSTREAM; ++i) m_c = fmaxf(m_c, part_m[i]);
+    float fw[NSTREAM], l_c = 0.f;
 #pragma unroll
-    for (int i = 0; i < MW; ++i) {
+    for (int i = 0; i < NSTREAM; ++i) {
       fw[i] = part_m[i] > -INFINITY ? ex2(part_m[i] - m_c) : 0.f;
       l_c += part_l[i] * fw[i];
     }
@@ -450,7 +497,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (tid < HD) {
       float a = 0.f;
 #pragma unroll
-      for (int i = 0; i < MW; ++i) a = fmaf(part_o[i][tid], fw[i], a);
+      for (int i = 0; i < NSTREAM; ++i) a = fmaf(part_o[i][tid], fw[i], a);
       e0->o[rank][tid] = a;
     }
     if (tid < split) {
@@ -459,7 +506,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       er->l[rank] = l_c;
     }
   }
-  if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync();
+  if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync<WT>();
 
   // ---- every CTA: the unit's softmax normaliser (all data is local now) ----
   float m_all = -INFINITY, L = 0.f;
@@ -545,7 +592,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   {
     const unsigned long long wkey = warp_min_key(my_key);
     if (lane == 0) warp_key[wid] = wkey;
-    workers_sync();
+    workers_sync<WT>();
     const unsigned long long win = warp_min_key(lane < MW ? warp_key[lane] : NO_KEY);
     Exch* e0 = split > 1 ? cluster.map_shared_rank(&ex, 0) : &ex;
     if (win == NO_KEY) {
@@ -556,7 +603,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       e0->key_pos[rank] = my_pos;
     }
   }
-  if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync();
+  if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync<WT>();
   if (rank != 0 || tid != 0) return;      // nothing of the other CTAs' shared memory is read by anyone
   {
     unsigned long long best = NO_KEY;
@@ -704,10 +751,11 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     bool ok;
   };
   const size_t half_sm = 104 * 1024, whole_sm = 215 * 1024;     // dynamic bytes, 1 KB of it alignment slack
-  const size_t stage_set = (size_t)MW * STAGE_BYTES;
   const size_t tot = (size_t)chunk;      // slots whose logits and state one CTA holds
   auto make_plan = [&](bool alone) {
     Plan p{};
+    const int MW = alone ? MW_ALONE : MW_BESIDE;
+    const size_t stage_set = (size_t)MW * STAGE_BYTES;
     size_t state_bytes = 4 * sizeof(float) * tot;
     p.state_in_smem = 1;
     const bool fits_half = !alone && state_bytes + 1024 + 2 * stage_set <= half_sm;
@@ -742,23 +790,28 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
                        {win ? (const char*)c.ring : nullptr, win ? slots * s.window * 4 : 0},
                        {win ? (const char*)c.acc_fixed : nullptr, win ? slots * 8 : 0},
                        {(const char*)q, units * ROW_BYTES}, {(const char*)k, units * ROW_BYTES}, {(const char*)v, units * ROW_BYTES}};
-  auto kern = win ? decode_mma_kernel<true> : decode_mma_kernel<false>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
+  auto kern_beside = win ? decode_mma_kernel<true, MW_BESIDE> : decode_mma_kernel<false, MW_BESIDE>;
+  auto kern_alone = win ? decode_mma_kernel<true, MW_ALONE> : decode_mma_kernel<false, MW_ALONE>;
+  cudaError_t e = cudaFuncSetAttribute(kern_beside, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(kern_alone, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
   if (e != cudaSuccess) return e;
   // share of the machine this launch holds while resident (every CTA waits for the previous launch before it retires)
-  auto share_of = [&](const Plan& p) {
+  auto share_of = [&](const Plan& p, bool alone) {
     int occ = 0;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, kern, MT, p.dyn) != cudaSuccess || occ < 1) occ = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, alone ? kern_alone : kern_beside,
+                                                      (alone ? MW_ALONE : MW_BESIDE) * 32 + 32, p.dyn) != cudaSuccess || occ < 1)
+      occ = 1;
     return (double)(s.units * split) / ((double)occ * sms);
   };
-  const int independent =
-      independent_of_in_flight(st, capture_of(st), may_overlap, written, 16, written, share_of(beside), share_of(lone)) ? 1 : 0;
+  const int independent = independent_of_in_flight(st, capture_of(st), may_overlap, written, 16, written, share_of(beside, false),
+                                                   share_of(lone, true)) ? 1 : 0;
   const Plan& pl = independent ? beside : lone;
+  auto kern = independent ? kern_beside : kern_alone;
   const int nstage = pl.nstage, state_in_smem = pl.state_in_smem;
   const size_t dyn = pl.dyn;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(s.units * split);
-  cfg.blockDim = dim3(MT);
+  cfg.blockDim = dim3((independent ? MW_BESIDE : MW_ALONE) * 32 + 32);
   cfg.dynamicSmemBytes = dyn;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
