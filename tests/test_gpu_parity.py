@@ -409,6 +409,31 @@ def test_fused_attention_forward_config1():
     _run_case(wl, decode=False, units=[(0, 3), (0, 30)], fused_forward=True)
 
 
+def test_fused_attention_forward_strided_inputs_and_determinism():
+    """[b, T, h, d] storage viewed as [b, h, T, d]: same bits as the contiguous call (the output is always
+    contiguous); and two runs over enough work items that the CTAs draw them in a different order give the same bits."""
+    wl = _small("bf16", 128, 300, 100, 2, 10, b=2, h=3, cid=78)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    qs, ks, vs = (x.transpose(1, 2).contiguous().transpose(1, 2) for x in (q, k, v))
+    g1 = P.GpuPrefill(wl, q, k, v, fused_forward=True).run()
+    g2 = P.GpuPrefill(wl, qs, ks, vs, fused_forward=True)
+    g2.attn_out = torch.empty_like(q)
+    g2.run()
+    assert torch.equal(g1.attn_out, g2.attn_out) and torch.equal(g1.score, g2.score) and torch.equal(g1.lse, g2.lse)
+    wl = _small("bf16", 128, 700, 200, 2, 20, b=2, h=100, cid=79)
+    q, k, v = synth.prefill_inputs(wl, 0, "cuda")
+    a = P.GpuPrefill(wl, q, k, v, fused_forward=True).run()
+    b = P.GpuPrefill(wl, q, k, v, fused_forward=True).run()
+    assert torch.equal(a.attn_out, b.attn_out) and torch.equal(a.score, b.score) and torch.equal(a.kept, b.kept)
+
+
+def test_fused_attention_forward_config2_shape():
+    """Config 2's per-layer shape (256 units, prompt 8192, the L2-grouped item order) through the fused call: oracle on
+    two units of a late layer (wide logits), invariants on all."""
+    wl = synth.CONFIGS[2].with_(decode_steps=0)
+    _run_case(wl, decode=False, units=[(0, 5), (7, 31)], layer=31, fused_forward=True)
+
+
 def test_fused_attention_forward_rescales_when_the_maximum_grows():
     """Keys whose logits keep growing along the prompt force the forward to move its reference maximum (and
     rescale the running output) in every chunk; keys whose logits fall never do.  Both against the oracle."""
