@@ -357,10 +357,6 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
       if (lane == 0) { part_m[stream] = m_run; part_l[stream] = l; }
     }
   };
-  if (SPW == 2) {      // the second stream may stay empty
-    *reinterpret_cast<float4*>(&part_o[wid + MW][lane * 4]) = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (lane == 0) { part_m[wid + MW] = -INFINITY; part_l[wid + MW] = 0.f; }
-  }
   int it = 0, g = g_first;
   bool past_live = false, second = false;
   // folds this warp's groups below g_stop into the running partial
@@ -468,8 +464,11 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (dev_status) atomicExch(dev_status, (int)VATP_ERR_TIMEOUT);
     for (int s = 0; s < nstage; ++s) mbar_wait(&my_bars[s], 0);
   }
-  // (a four-warp kernel that never reached the midpoint files everything under stream wid: its stream wid + 4 is empty)
   flush(second ? wid + MW : wid);
+  if (SPW == 2 && !second) {      // the four-warp kernel never reached the midpoint: its stream wid + 4 is empty
+    *reinterpret_cast<float4*>(&part_o[wid + MW][lane * 4]) = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (lane == 0) { part_m[wid + MW] = -INFINITY; part_l[wid + MW] = 0.f; }
+  }
   workers_sync<WT>();
   if (state_in_smem == 2 && tid == 32 && rows_alloc > 0) {
     // every stage of this CTA has been consumed: the per-slot state of its slots lands there while the
