@@ -468,7 +468,7 @@ def run_cuda(args, wl):
     roof["kernel"] = dominant
     # dram__bytes_read.sum + dram__bytes_write.sum per launch from the committed ncu capture of this kernel at
     # this shape (profiles/); other kernels / shapes: not captured
-    roof["traffic"] = 34.52e6 if (dominant == "decode_step" and wl.cid == 1) else None
+    roof["traffic"] = 34.54e6 if (dominant == "decode_step" and wl.cid == 1) else None
     roof["traffic_source"] = ("ncu capture of this kernel at this shape, summarised in profiles/decode_mma_config1.md "
                               "(not measured in this run)") if roof["traffic"] else None
     roof["algorithmic_bytes_per_launch"] = bytes_decode if dominant == "decode_step" else None
