@@ -30,6 +30,7 @@ import numpy as np
 __all__ = [
     "attention_probs",
     "attention_output",
+    "attention_row",
     "indicator_h2o",
     "indicator_window",
     "value_l1_norm",
@@ -85,6 +86,18 @@ def attention_output(a: np.ndarray, v) -> np.ndarray:
     output is the probability-weighted sum of the value vectors, which is why
     Eq. 4 looks at their norms).  a: [T, T] from attention_probs, v: [T, d]."""
     return a @ _f64(v)
+
+
+def attention_row(q_j, k, v, scale: float):
+    """One query row of Eq. 1 on its own: query j = len(k) - 1 against the keys 0..j it may see.
+    Returns (o_j, lse_j).  For prompts whose T x T matrix is too large to materialise; the same arithmetic
+    as attention_probs / attention_output / row_logsumexp restricted to one row."""
+    q_j, k, v = _f64(q_j), _f64(k), _f64(v)
+    s = scale * (k @ q_j)
+    m = s.max()
+    e = np.exp(s - m)
+    den = e.sum()
+    return (e / den) @ v, m + np.log(den)
 
 
 def indicator_h2o(a: np.ndarray) -> np.ndarray:

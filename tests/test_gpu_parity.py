@@ -434,6 +434,30 @@ def test_fused_attention_forward_config2_shape():
     _run_case(wl, decode=False, units=[(0, 5), (7, 31)], layer=31, fused_forward=True)
 
 
+def test_fused_attention_forward_config4_sampled_rows():
+    """Config 4's per-layer shape (prompt 32768: the T x T matrix of a head is 8.6 GB) through the fused call: output rows and
+    normalisers of sampled (head, query) pairs, each computed on its own by the oracle; scores of every head satisfy the
+    oracle-free invariants, and equal the two-pass call's within the score tolerance."""
+    from oracle import vatp_oracle as O
+    wl = synth.CONFIGS[4].with_(decode_steps=0)
+    q, k, v = synth.prefill_inputs(wl, 31, "cuda")
+    g = P.GpuPrefill(wl, q, k, v, fused_forward=True).run()
+    P.gpu_invariants(g)
+    rng = np.random.default_rng(4)
+    rows = [0, 1, 127, 128, 255, 256, 16383, 16384, 32639, 32640, 32767] + rng.integers(0, wl.seq_len, 13).tolist()
+    for h in (0, 9, 31):
+        kn, vn = P.to_np64(k[0, h]), P.to_np64(v[0, h])
+        for j in rows:
+            o, lse = O.attention_row(P.to_np64(q[0, h, j]), kn[: j + 1], vn[: j + 1], wl.scale)
+            P.check_attention_output(P.to_np64(g.attn_out[0, h, j])[None], o[None], vn[: j + 1], "bf16")
+            assert abs(float(g.lse[0, h, j]) - lse) <= 1e-2, (h, j)
+    two = P.GpuPrefill(wl, q, k, v).run()
+    for name in ("attn_acc", "vnorm", "score"):
+        a, b_ = getattr(g, name).double(), getattr(two, name).double()
+        assert torch.all((a - b_).abs() <= 2e-3 * b_.abs() + 1e-30), name
+    assert torch.equal(g.kept, two.kept) or (g.kept != two.kept).sum().item() <= 2 * MAX_BOUNDARY_PER_UNIT * wl.heads
+
+
 def test_fused_attention_forward_rescales_when_the_maximum_grows():
     """Keys whose logits keep growing along the prompt force the forward to move its reference maximum (and
     rescale the running output) in every chunk; keys whose logits fall never do.  Both against the oracle."""

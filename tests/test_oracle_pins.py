@@ -635,3 +635,18 @@ def test_attention_output_last_row_is_the_decode_steps_output():
     st, _ = _state(q[:T], k[:T], v[:T], scale, B=T + 4, F=1, R=2)
     res = O.decode_step(st, q[T], k[T], v[T], scale, T + 4, 1, 2)
     np.testing.assert_allclose(res["out"], O.prefill(q, k, v, scale)["out"][T], rtol=0, atol=1e-12)
+
+
+def test_attention_row_is_a_row_of_the_matrix_form():
+    rng = np.random.default_rng(8)
+    T, d = 11, 5
+    q, k, v = rng.standard_normal((T, d)), rng.standard_normal((T, d)), rng.standard_normal((T, d))
+    full = O.prefill(q, k, v, 0.4)
+    a = brute_attention(q.tolist(), k.tolist(), 0.4)
+    for j in (0, 3, T - 1):
+        o, lse = O.attention_row(q[j], k[: j + 1], v[: j + 1], 0.4)
+        np.testing.assert_allclose(o, full["out"][j], rtol=0, atol=1e-14)
+        assert abs(lse - full["lse"][j]) < 1e-13
+        # against the loops: probabilities of row j times the values
+        want = [sum(a[j][i] * float(v[i][c]) for i in range(j + 1)) for c in range(d)]
+        np.testing.assert_allclose(o, want, rtol=0, atol=1e-13)
