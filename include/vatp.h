@@ -175,8 +175,9 @@ vatp_status vatp_prefill_scores_from_lse(const vatp_params* params, const void* 
  *           of the probabilities to bf16 before they meet V (as fused attention kernels do):
  *           |error| <= 2^-8 * max|v| per element, typically far less.
  * All other arguments, outputs, the workspace requirement and the error behaviour are those of
- * vatp_prefill_scores; both indicators (Eq. 2, Eq. 3) are supported, grouped-query attention is not
- * (VATP_ERR_UNSUPPORTED), nor is head_dim > 256 outside the tensor-core shape.
+ * vatp_prefill_scores; both indicators (Eq. 2, Eq. 3) and grouped-query attention (one forward per
+ * query head of the KV groups, attn_out covering all `heads` query heads) are supported; head_dim > 256
+ * outside the tensor-core shape is not (VATP_ERR_UNSUPPORTED).
  */
 vatp_status vatp_prefill_attention_scores(const vatp_params* params, const void* q, const void* k, const void* v,
                                           void* attn_out, float* lse_out, float* attn_acc, float* vnorm, float* score,

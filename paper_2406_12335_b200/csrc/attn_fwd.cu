@@ -15,7 +15,7 @@ template <typename T>
 __global__ void __launch_bounds__(FG_WARPS * 32)
 attention_fwd_general_kernel(int heads, int T_len, int d, float scale, const T* __restrict__ q, const T* __restrict__ k,
                              const T* __restrict__ v, int64_t sb, int64_t sh, int64_t st, int64_t qsb, int64_t qsh,
-                             T* __restrict__ out, float* __restrict__ lse, int64_t lse_sb, int64_t lse_sh) {
+                             T* __restrict__ out, int64_t osb, int64_t osh, float* __restrict__ lse, int64_t lse_sb, int64_t lse_sh) {
   const int u = blockIdx.y, lane = threadIdx.x & 31;
   const int j = blockIdx.x * FG_WARPS + (threadIdx.x >> 5);
   if (j >= T_len) return;
@@ -59,7 +59,7 @@ attention_fwd_general_kernel(int heads, int T_len, int d, float scale, const T* 
     }
   }
   const float inv = 1.f / l;
-  T* orow = out + ((int64_t)u * T_len + j) * d;
+  T* orow = out + (int64_t)b * osb + (int64_t)h * osh + (int64_t)j * d;
 #pragma unroll
   for (int c = 0; c < FG_MAXC; ++c) {
     const int ch = lane + 32 * c;
@@ -73,7 +73,7 @@ attention_fwd_general_kernel(int heads, int T_len, int d, float scale, const T* 
 
 }  // namespace
 
-// out: [units, T, d] contiguous, the inputs' dtype; lse: natural log, unit (b, h) at b * lse_sb + h * lse_sh.
+// out: the inputs' dtype, unit (b, h)'s rows at b * osb + h * osh; lse: natural log, unit (b, h) at b * lse_sb + h * lse_sh.
 cudaError_t launch_attention_fwd_general(const Shape& s, int dtype, const void* q, const void* k, const void* v, void* out,
                                          float* lse, cudaStream_t st) {
   if (s.d > 32 * FG_MAXC) return cudaErrorNotSupported;
@@ -81,12 +81,12 @@ cudaError_t launch_attention_fwd_general(const Shape& s, int dtype, const void* 
   if (dtype == VATP_F32)
     attention_fwd_general_kernel<float><<<grid, FG_WARPS * 32, 0, st>>>(
         s.heads, s.T, s.d, s.scale, static_cast<const float*>(q), static_cast<const float*>(k), static_cast<const float*>(v),
-        s.sb, s.sh, s.st, s.qsb, s.qsh, static_cast<float*>(out), lse, s.lse_sb, s.lse_sh);
+        s.sb, s.sh, s.st, s.qsb, s.qsh, static_cast<float*>(out), s.osb, s.osh, lse, s.lse_sb, s.lse_sh);
   else
     attention_fwd_general_kernel<__nv_bfloat16><<<grid, FG_WARPS * 32, 0, st>>>(
         s.heads, s.T, s.d, s.scale, static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k),
-        static_cast<const __nv_bfloat16*>(v), s.sb, s.sh, s.st, s.qsb, s.qsh, static_cast<__nv_bfloat16*>(out), lse, s.lse_sb,
-        s.lse_sh);
+        static_cast<const __nv_bfloat16*>(v), s.sb, s.sh, s.st, s.qsb, s.qsh, static_cast<__nv_bfloat16*>(out), s.osb, s.osh, lse,
+        s.lse_sb, s.lse_sh);
   return cudaGetLastError();
 }
 

@@ -379,6 +379,7 @@ struct TcArgs {
   float* lse2;              // [units][Tpad] NEGATED log2-domain row normalisers (-inf where no query counts)
   float* lse_out;           // natural-log copy, nullable: unit (b, h)'s T values start at b * lse_sb + h * lse_sh
   int64_t lse_sb, lse_sh;
+  int64_t out_sb, out_sh;   // fused forward: unit (b, h)'s output rows start at b * out_sb + h * out_sh (elements)
   float* attn_acc;
   float* vnorm;
   float* score;
@@ -1161,8 +1162,9 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       if (!w4) { ok = false; break; }
       tc_fence_after();
       const float inv = 1.f / l_row;
-      __nv_bfloat16* orow = out + ((int64_t)u * a.T + tok) * HD + half * 64;
-      const bool live = tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status);
+      const int64_t o_off = (int64_t)(u / a.heads) * a.out_sb + (int64_t)(u % a.heads) * a.out_sh + (int64_t)tok * HD;
+      __nv_bfloat16* orow = out + o_off + half * 64;
+      const bool live = tok < a.T && VATP_INB(o_off, (int64_t)(a.units / a.heads) * a.out_sb, a.dev_status);
 #pragma unroll
       for (int q2 = 0; q2 < 2; ++q2) {
         float y[32];
@@ -1494,6 +1496,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   a.v = static_cast<const __nv_bfloat16*>(v);
   a.sb = s.sb; a.sh = s.sh; a.st = s.st;
   a.lse_sb = s.lse_sb; a.lse_sh = s.lse_sh;
+  a.out_sb = s.osb; a.out_sh = s.osh;
   a.lse2 = lse_ws; a.lse_out = lse_out; a.attn_acc = attn_acc; a.vnorm = vnorm; a.score = score;
   a.dev_status = dev_status;
   a.norm = s.norm;

@@ -48,6 +48,8 @@ vatp_status make_shape(const vatp_params* p, Shape* s) {
   s->qsb = G > 1 ? (int64_t)p->heads * s->sh : s->sb;
   s->lse_sh = (int64_t)G * p->seq_len;
   s->lse_sb = (int64_t)p->heads * p->seq_len;
+  s->osh = (int64_t)G * p->seq_len * p->head_dim;
+  s->osb = (int64_t)p->heads * p->seq_len * p->head_dim;
   s->scale = p->scale;
   s->window = p->indicator == VATP_IND_WINDOW ? p->window_w : 0;
   s->norm = p->norm_kind;
@@ -93,7 +95,7 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
   s = make_shape(p, &sh);
   if (s != VATP_OK) return s;
   const int G = group_of(p);
-  if (G > 1 && (lse_in || win_rows || attn_out)) return VATP_ERR_UNSUPPORTED;
+  if (G > 1 && (lse_in || win_rows)) return VATP_ERR_UNSUPPORTED;
   if (attn_out && (lse_in || !aligned16(attn_out))) return VATP_ERR_INVALID_ARG;
   if (!workspace || workspace_bytes < workspace_need(p) || (reinterpret_cast<uintptr_t>(workspace) & 255u))
     return VATP_ERR_WORKSPACE;
@@ -114,13 +116,21 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
     for (int g = 0; g < G && e == cudaSuccess; ++g) {
       const char* qg = static_cast<const char*>(q) + (size_t)g * sh.sh * eb;
       float* lse_g = lse_out ? lse_out + (size_t)g * sh.T : nullptr;
+      // the fused call: this round's query heads' rows of the attention output (head kvh * G + g of every KV group)
+      void* out_g = attn_out ? static_cast<char*>(attn_out) + (size_t)g * sh.T * sh.d * eb : nullptr;
       if (tc) {
-        e = launch_prefill_tc(sh, qg, k, v, ws, lse_g, part + g * n, vnorm, score, nullptr, dev_status, st, nullptr);
+        e = launch_prefill_tc(sh, qg, k, v, ws, lse_g, part + g * n, vnorm, score, nullptr, dev_status, st, nullptr, out_g);
       } else {
         Shape sg = sh;
         float* lse_buf = lse_g;
         if (!lse_buf) { lse_buf = ws; sg.lse_sb = (int64_t)sh.heads * sh.T; sg.lse_sh = sh.T; }   // plain [units][T] scratch
-        e = launch_prefill_simt(sg, p->dtype, qg, k, v, lse_buf, part + g * n, vnorm, score, nullptr, st);
+        if (out_g) {
+          e = launch_attention_fwd_general(sg, p->dtype, qg, k, v, out_g, lse_buf, st);
+          if (e == cudaErrorNotSupported) return VATP_ERR_UNSUPPORTED;
+          if (e == cudaSuccess) e = launch_prefill_simt(sg, p->dtype, qg, k, v, lse_buf, part + g * n, vnorm, score, nullptr, st, true);
+        } else {
+          e = launch_prefill_simt(sg, p->dtype, qg, k, v, lse_buf, part + g * n, vnorm, score, nullptr, st);
+        }
       }
     }
     if (e == cudaSuccess) e = launch_group_mean(G, (int64_t)n, part, vnorm, attn_acc, score, st);

@@ -18,6 +18,7 @@ struct Shape {
   int64_t qsb, qsh;    // batch and head strides of q (grouped-query attention runs one query head of every KV
                        // group per launch: the units are then the KV heads and q is a strided view)
   int64_t lse_sb, lse_sh;  // where unit (b, h)'s row normalisers start in the caller's [.., T] array: b * lse_sb + h * lse_sh
+  int64_t osb, osh;        // likewise for the rows of the attention output [.., T, d] (elements): b * osb + h * osh
   float scale;
   int window;          // 0 = accumulate over all queries (Eq. 2); >0 = last `window` queries (Eq. 3)
   int norm;            // vatp_norm_kind of the value norm in Eq. 4
@@ -101,11 +102,12 @@ cudaError_t launch_prefill_simt(const Shape& s, int dtype, const void* q, const 
                                 float* attn_acc, float* vnorm, float* score, float* win_rows, cudaStream_t st,
                                 bool lse_given = false);
 // lse_in: row normalisers [units][T] (natural log) from the caller; non-null skips pass 1
-// attn_out: non-null replaces pass 1 by the fused attention forward, which also writes out [units, T, 128] (bf16)
+// attn_out: non-null replaces pass 1 by the fused attention forward, which also writes the output rows (bf16; unit
+// (b, h) at b * osb + h * osh, rows of 128 elements)
 cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, const void* v, float* lse_ws,
                               float* lse_out, float* attn_acc, float* vnorm, float* score, float* win_rows,
                               int32_t* dev_status, cudaStream_t st, const float* lse_in = nullptr, void* attn_out = nullptr);
-// attention forward of the general path: out [units, T, d] and natural-log normalisers
+// attention forward of the general path: out (unit (b, h) at b * osb + h * osh, rows of d elements) and natural-log normalisers
 cudaError_t launch_attention_fwd_general(const Shape& s, int dtype, const void* q, const void* k, const void* v, void* out,
                                          float* lse, cudaStream_t st);
 size_t prefill_tc_workspace_bytes(int units, int T);  // padded log2-domain row normalisers

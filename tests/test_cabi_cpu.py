@@ -93,13 +93,12 @@ def test_host_side_validation(V):
     gw = V.make_params(**gq, kv_heads=2, indicator="window", window=8)
     assert V.lib.vatp_prefill_scores(C.byref(gw), 16, 16, 16, 16, 16, 16, 16, 16, 256, 1 << 20, null, null) == 2   # no win_rows with grouped queries
     assert V.lib.vatp_decode_step(C.byref(gw), C.byref(cs), 16, 16, 16, 16, null, null, null) == 2
-    # attention forward fused with the scoring: the output array is required and 16-byte aligned, the usual checks follow,
-    # grouped queries are not supported
+    # attention forward fused with the scoring: the output array is required and 16-byte aligned, the usual checks follow
     fa = V.lib.vatp_prefill_attention_scores
     assert fa(C.byref(p), 16, 16, 16, null, null, 16, 16, 16, null, 256, 4096, null, null) == 1
     assert fa(C.byref(p), 16, 16, 16, 8, null, 16, 16, 16, null, 256, 4096, null, null) == 1
     assert fa(C.byref(p), 16, 16, 16, 16, null, 16, 16, 16, null, null, 0, null, null) == 3
-    assert fa(C.byref(V.make_params(**gq, kv_heads=2)), 16, 16, 16, 16, null, 16, 16, 16, null, 256, 1 << 20, null, null) == 2
+    assert fa(C.byref(V.make_params(**gq, kv_heads=2)), 16, 16, 16, 16, null, 16, 16, 16, null, null, 0, null, null) == 3   # grouped queries: as far as the workspace check
     # flags: the decode-overlap bit is the only one defined
     assert V.make_params(**ok, decode_overlap=True).flags == V.FLAG_DECODE_OVERLAP == 1
     assert V.vatp_workspace_bytes(V.make_params(**ok, decode_overlap=True)) == 2048 + 256

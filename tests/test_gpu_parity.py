@@ -648,10 +648,12 @@ def test_bounds_checking_build_reports_no_violation():
     ("f32", 64, 4, 2, 333, 100, 3, 17),        # general kernels
     ("bf16", 64, 8, 1, 257, 128, 2, 16),       # multi-query attention: one KV head
 ])
-def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R):
+@pytest.mark.parametrize("fused", [False, True])
+def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R, fused):
     """Grouped-query attention (the Limitations section's open case, read as a group-mean indicator): the G query
     heads of a KV group share one kept set and one cache.  Scoring, selection, compaction and decode steps of
-    every KV unit against the oracle; the row normalisers of every query head as well."""
+    every KV unit against the oracle; the row normalisers of every query head as well.  fused: through
+    vatp_prefill_attention_scores, the attention output rows of every query head too."""
     from oracle import vatp_oracle as O
     V = P.vatp()
     b, G, steps = 2, heads // kv_heads, 10
@@ -674,7 +676,12 @@ def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R):
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     kept = torch.empty(b, kv_heads, B, dtype=torch.int32, device="cuda")
     cache = V.Cache(p)
-    V.vatp_prefill_scores(p, q, k, v, lse_out=lse, attn_acc=attn_acc, vnorm=vnorm, score=score, workspace=ws, dev_status=status)
+    attn_out = torch.full_like(q, float("nan")) if fused else None
+    if fused:
+        V.vatp_prefill_attention_scores(p, q, k, v, attn_out, lse_out=lse, attn_acc=attn_acc, vnorm=vnorm, score=score,
+                                        workspace=ws, dev_status=status)
+    else:
+        V.vatp_prefill_scores(p, q, k, v, lse_out=lse, attn_acc=attn_acc, vnorm=vnorm, score=score, workspace=ws, dev_status=status)
     V.vatp_select(p, score, kept, dev_status=status)
     V.vatp_compact(p, k, v, attn_acc, vnorm, kept, cache, dev_status=status)
     torch.cuda.synchronize()
@@ -687,6 +694,11 @@ def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R):
         for g in range(kv_heads):
             ref = O.prefill_gqa(P.to_np64(q[bi, g * G:(g + 1) * G]), P.to_np64(k[bi, g]), P.to_np64(v[bi, g]), wl_kv.scale)
             assert np.max(np.abs(P.to_np64(lse[bi, g * G:(g + 1) * G]) - ref["lse"])) <= 10 * tol
+            if fused:
+                for hq in range(g * G, (g + 1) * G):
+                    want_out = O.attention_output(O.attention_probs(P.to_np64(q[bi, hq]), P.to_np64(k[bi, g]), wl_kv.scale),
+                                                  P.to_np64(v[bi, g]))
+                    P.check_attention_output(P.to_np64(attn_out[bi, hq]), want_out, P.to_np64(v[bi, g]), dtype)
             for name, key in (("attn_acc", "S"), ("vnorm", "n1"), ("score", "I")):
                 e = P.rel_err(P.to_np64(locals()[name][bi, g]), ref[key])
                 assert e <= tol, f"{name} rel err {e:.3g} (unit {bi},{g})"
