@@ -236,21 +236,28 @@ def prefill_gqa(q_group, k, v, scale: float, *, window: int | None = None, norm:
     grouped-query attention") leaves this to future work and points at a group-wise score:
     reading: the indicator of a cached token is the MEAN over the group's query heads of its Eq. 2 (or Eq. 3)
     indicator, S_k = (1/G) sum_g S_k^(g); Eq. 4 multiplies it by the norm of the shared value row.  With G = 1
-    this is `prefill`.  Returns dict with lse [G, T], S, n1, I, S_heads [G, T] (and no attention matrices)."""
+    this is `prefill`.  Returns dict with lse [G, T], S, n1, I, S_heads [G, T], and with a history window the
+    group mean of the heads' last-w probability rows (window_rows: what the decode state keeps); no attention
+    matrices."""
     q_group = _f64(q_group)
     if q_group.ndim != 3:
         raise ValueError("q_group must be [G, T, d]")
     per_head = []
     lse = []
+    rows = None
     for g in range(q_group.shape[0]):
         a = attention_probs(q_group[g], k, scale)
         per_head.append(indicator_h2o(a) if window is None else indicator_window(a, window))
         lse.append(row_logsumexp(q_group[g], k, scale))
+        if window is not None:
+            r = a[max(a.shape[0] - window, 0):, :]
+            rows = r.copy() if rows is None else rows + r
         del a
     S_heads = np.stack(per_head)
     S = S_heads.sum(axis=0) / q_group.shape[0]
     n1 = value_l1_norm(v) if norm == "l1" else value_norm(v, norm)
-    return {"lse": np.stack(lse), "S": S, "n1": n1, "I": importance(S, n1), "S_heads": S_heads, "window_rows": None}
+    return {"lse": np.stack(lse), "S": S, "n1": n1, "I": importance(S, n1), "S_heads": S_heads,
+            "window_rows": None if rows is None else rows / q_group.shape[0]}
 
 
 class DecodeState:
@@ -318,7 +325,7 @@ def decode_step(state: DecodeState, q, k, v, scale: float, B: int, F: int, R: in
 
     Grouped-query attention (see prefill_gqa): q may be [G, d], the new token's query under each head of the
     KV group.  Every head attends over the shared cache, out is [G, d], p is [G, entries], and the indicator
-    advances by the mean of the heads' probabilities (accumulated indicator only).
+    advances by the mean of the heads' probabilities (Eq. 2), or that mean row enters the history (Eq. 3).
 
     Returns dict(out, p, evicted (position or -1), runner_up, I_evicted,
     I_runner_up, adopted (a forced near-tie was taken), I (importances before eviction), pos (positions before
@@ -337,8 +344,6 @@ def decode_step(state: DecodeState, q, k, v, scale: float, B: int, F: int, R: in
     Vmat = np.stack(state.V)
     qv = _f64(q)
     if qv.ndim == 2:                         # grouped-query attention: one softmax per query head of the group
-        if state.window is not None:
-            raise ValueError("grouped queries: accumulated indicator only")
         s = scale * (qv @ Kmat.T)
         e = np.exp(s - s.max(axis=1, keepdims=True))
         p_heads = e / e.sum(axis=1, keepdims=True)

@@ -593,9 +593,23 @@ def test_gqa_decode_step_matches_prefill_on_the_longer_prompt():
     r3 = O.decode_step(st3, qg[:, T], k[T], np.ones(d), scale, B=T, F=0, R=1)
     mean_after = short["S"] + r3["p"][:T]
     assert r3["evicted"] == int(np.argmin(mean_after))
-    with pytest.raises(ValueError):
-        stw = O.DecodeState(k[:T], v[:T], short["S"], short["n1"], np.arange(T), T, window=4, window_rows=np.zeros((4, T)))
-        O.decode_step(stw, qg[:, T], k[T], v[T], scale, B=T + 5, F=0, R=0)
+    # history window (Eq. 3) with grouped queries: the group-mean row enters the history; prefill + steps = longer prefill
+    for w in (4, 1, 50):
+        shortw = O.prefill_gqa(qg[:, :T - 2], k[:T - 2], v[:T - 2], scale, window=w)
+        # the window rows are the mean over heads of each head's last rows, written out with loops
+        for r in range(shortw["window_rows"].shape[0]):
+            j = (T - 2) - shortw["window_rows"].shape[0] + r
+            for i in range(T - 2):
+                want = sum(O.attention_probs(qg[g, :T - 2], k[:T - 2], scale)[j, i] for g in range(G)) / G
+                assert abs(shortw["window_rows"][r, i] - want) < 1e-14
+        stw = O.DecodeState(k[:T - 2], v[:T - 2], shortw["S"], shortw["n1"], np.arange(T - 2), T - 2, window=w,
+                            window_rows=shortw["window_rows"])
+        for step in range(3):
+            tt = T - 2 + step
+            O.decode_step(stw, qg[:, tt], k[tt], v[tt], scale, B=T + 5, F=0, R=0)
+            fullw = O.prefill_gqa(qg[:, :tt + 1], k[:tt + 1], v[:tt + 1], scale, window=w)
+            assert np.allclose(stw.indicator(), fullw["S"], rtol=1e-12, atol=1e-15)
+            assert abs(stw.indicator().sum() - min(w, tt + 1)) < 1e-12
 
 
 # ----------------------------------------------------------------- attention output (Section 3.1)
