@@ -30,10 +30,12 @@
  *     a unit is a (batch, KV head) pair, the G = heads / kv_heads query heads h = g * G .. g * G + G - 1
  *     share KV head g, and the indicator of a cached token is the MEAN over those query heads of its
  *     Eq. 2 / Eq. 3 indicator (prefill), advanced per step by the mean of the heads' probabilities
- *     (decode; accumulated indicator only).  Layouts must be contiguous (stride fields 0); the
- *     history-window decode state, vatp_prefill_scores_from_lse and win_rows are not available with it
- *     (VATP_ERR_UNSUPPORTED), and the workspace grows by G partial indicators.  The decode step runs a
- *     plain general kernel, not the tuned one.
+ *     (decode; with a history window that mean row enters the ring, built after the prefill by
+ *     vatp_compact_window, which then needs lse for all `heads` query heads).  Layouts must be
+ *     contiguous (stride fields 0); vatp_prefill_scores_from_lse and win_rows (hence vatp_compact
+ *     with a history window) are not available with it (VATP_ERR_UNSUPPORTED), and the workspace
+ *     grows by G partial indicators.  The decode step and the history rebuild run plain general
+ *     kernels, not the tuned ones.
  *   - Inputs are assumed finite.
  *   - A second build of the library (compiled with -DVATP_DEBUG_BOUNDS) range-checks every row, slot,
  *     window-row and scratch index its kernels compute before the access; an index outside its array is

@@ -1,7 +1,8 @@
 // Decode step for grouped-query attention: the G query heads of a KV group attend over ONE shared, budgeted
 // cache.  The paper leaves this case to future work ("Compatibility with grouped-query attention") and points
 // at a group-wise score; here the indicator of a cached token advances by the MEAN of the probabilities the
-// group's heads give it (Eq. 2 under that mean), Eq. 4 multiplies by the norm of the shared value row, and
+// group's heads give it (Eq. 2 under that mean; with a history window, Eq. 3: that mean row enters the ring
+// and the exact fixed-point window sum moves by it), Eq. 4 multiplies by the norm of the shared value row, and
 // the lowest importance is released as in the multi-head step.
 //
 // A plain kernel, not a tuned one: one CTA per KV unit, any dtype and head_dim, the logits of all heads
@@ -37,7 +38,7 @@ __device__ __forceinline__ float block_sum(float x, float* red) {
 
 template <typename T>
 __global__ void __launch_bounds__(GQ_THREADS)
-decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int norm, float scale, vatp_cache c, const T* __restrict__ q_new,
+decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int w, int norm, float scale, vatp_cache c, const T* __restrict__ q_new,
                   const T* __restrict__ k_new, const T* __restrict__ v_new, T* __restrict__ out, int32_t* __restrict__ evicted,
                   int32_t* dev_status) {
   extern __shared__ float gq_smem[];            // p[G][cap] (logits, then probabilities) | q[G][d]
@@ -119,7 +120,17 @@ decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int norm, float sc
     pm *= invG;
     const int64_t o = (int64_t)u * cap + s;
     const bool is_new = s == fs;
-    const float S = is_new ? pm : c.acc[o] + pm;
+    float S;
+    if (w > 0) {
+      // Eq. 3: row t mod w of the ring is replaced; the window sum is kept as an exact integer
+      float* ring_row = c.ring + ((int64_t)u * w + (t % w)) * cap;
+      const long long fx = is_new ? prob_to_fixed(pm) : c.acc_fixed[o] + prob_to_fixed(pm) - prob_to_fixed(ring_row[s]);
+      ring_row[s] = pm;
+      c.acc_fixed[o] = fx;
+      S = fixed_to_prob(fx);
+    } else {
+      S = is_new ? pm : c.acc[o] + pm;
+    }
     c.acc[o] = S;
     if (is_new) { c.vnorm[o] = nn; c.pos[o] = t; }
     if (evicting) {
@@ -131,6 +142,9 @@ decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int norm, float sc
       }
     }
   }
+  // recycled slot: the other rows of its ring column belong to the previous occupant
+  for (int rr = tid; rr < w; rr += GQ_THREADS)
+    if (rr != t % w) c.ring[((int64_t)u * w + rr) * cap + fs] = 0.f;
   if (!evicting) {
     if (tid == 0) {
       c.len[u] = hi; c.free_slot[u] = hi; c.next_pos[u] = t + 1; c.last_slot[u] = fs;
@@ -188,7 +202,7 @@ cudaError_t launch_group_mean(int G, int64_t n, const float* part, const float* 
 }
 
 // units: batch * kv_heads.  cudaErrorNotSupported when the logits of a unit's heads do not fit in shared memory.
-cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, int R, int norm, float scale,
+cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, int R, int window, int norm, float scale,
                               const vatp_cache& c, const void* q, const void* k, const void* v, void* out, int32_t* evicted,
                               int32_t* dev_status, cudaStream_t st) {
   const int cap = cache_capacity(B);
@@ -198,12 +212,12 @@ cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, 
   if (dtype == VATP_F32) {
     e = cudaFuncSetAttribute(decode_gqa_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    decode_gqa_kernel<float><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, norm, scale, c, (const float*)q, (const float*)k,
+    decode_gqa_kernel<float><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, window, norm, scale, c, (const float*)q, (const float*)k,
                                                                (const float*)v, (float*)out, evicted, dev_status);
   } else {
     e = cudaFuncSetAttribute(decode_gqa_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    decode_gqa_kernel<__nv_bfloat16><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, norm, scale, c, (const __nv_bfloat16*)q,
+    decode_gqa_kernel<__nv_bfloat16><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, window, norm, scale, c, (const __nv_bfloat16*)q,
                                                                         (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                                                                         (__nv_bfloat16*)out, evicted, dev_status);
   }

@@ -242,7 +242,6 @@ vatp_status vatp_compact_window(const vatp_params* p, const void* q, const void*
   vatp_status s = check_params(p, true);
   if (s != VATP_OK) return s;
   if (p->indicator != VATP_IND_WINDOW) return VATP_ERR_INVALID_ARG;
-  if (group_of(p) > 1) return VATP_ERR_UNSUPPORTED;
   if (!q || !k || !v || !lse || !attn_acc || !vnorm || !kept_idx || !cache_ok(cache, true)) return VATP_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v)) return VATP_ERR_INVALID_ARG;
   Shape sh;
@@ -251,8 +250,10 @@ vatp_status vatp_compact_window(const vatp_params* p, const void* q, const void*
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   decode_history_forget(st);
   cudaError_t e = launch_compact(sh, p->dtype, p->budget, k, v, attn_acc, vnorm, nullptr, kept_idx, *cache, dev_status, st);
-  if (e == cudaSuccess) e = launch_window_ring(sh, p->dtype, p->budget, q, lse, *cache, dev_status, st);
-  return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+  if (e == cudaSuccess)
+    e = group_of(p) > 1 ? launch_window_ring_grouped(sh, group_of(p), p->dtype, p->budget, q, lse, *cache, st)
+                        : launch_window_ring(sh, p->dtype, p->budget, q, lse, *cache, dev_status, st);
+  return e == cudaSuccess ? VATP_OK : (e == cudaErrorNotSupported ? VATP_ERR_UNSUPPORTED : VATP_ERR_CUDA);
 }
 
 vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, const void* q_new, const void* k_new,
@@ -264,12 +265,11 @@ vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, cons
   if (!q_new || !k_new || !v_new || !out || !cache_ok(cache, windowed)) return VATP_ERR_INVALID_ARG;
   if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return VATP_ERR_INVALID_ARG;
   if (group_of(p) > 1) {
-    if (windowed) return VATP_ERR_UNSUPPORTED;
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     decode_history_forget(st);
     const cudaError_t e = launch_decode_gqa(p->batch * kv_heads_of(p), group_of(p), p->head_dim, p->dtype, p->budget, p->n_sink,
-                                            p->n_recent, p->norm_kind, p->scale, *cache, q_new, k_new, v_new, out, evicted_pos,
-                                            dev_status, st);
+                                            p->n_recent, windowed ? p->window_w : 0, p->norm_kind, p->scale, *cache, q_new, k_new,
+                                            v_new, out, evicted_pos, dev_status, st);
     return e == cudaSuccess ? VATP_OK : (e == cudaErrorNotSupported ? VATP_ERR_UNSUPPORTED : VATP_ERR_CUDA);
   }
   Shape sh;

@@ -117,6 +117,8 @@ cudaError_t launch_compact(const Shape& s, int dtype, int B, const void* k, cons
                            const float* vnorm, const float* win_rows, const int32_t* kept, const vatp_cache& c,
                            int32_t* dev_status, cudaStream_t st);
 // windowed decode state from Q, the compacted keys and the row normalisers (natural log): ring, acc_fixed, acc
+cudaError_t launch_window_ring_grouped(const Shape& s, int G, int dtype, int B, const void* q, const float* lse, const vatp_cache& c,
+                                       cudaStream_t st);
 cudaError_t launch_window_ring(const Shape& s, int dtype, int B, const void* q, const float* lse, const vatp_cache& c,
                                int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_window_ring_tc(const Shape& s, int B, const void* q, const float* lse, const vatp_cache& c,
@@ -124,7 +126,7 @@ cudaError_t launch_window_ring_tc(const Shape& s, int B, const void* q, const fl
 // grouped-query attention: mean over the group's G partial indicators [G][n] and Eq. 4; the decode step of a KV group
 cudaError_t launch_group_mean(int G, int64_t n, const float* part, const float* vnorm, float* attn_acc, float* score,
                               cudaStream_t st);
-cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, int R, int norm, float scale,
+cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, int R, int window, int norm, float scale,
                               const vatp_cache& c, const void* q, const void* k, const void* v, void* out, int32_t* evicted,
                               int32_t* dev_status, cudaStream_t st);
 cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const vatp_cache& c, const void* q,

@@ -51,7 +51,71 @@ window_ring_general_kernel(int heads, int T_len, int d, int w, int B, int cap, f
   }
 }
 
+// Grouped-query attention: the history holds the MEAN over the KV group's G query heads of their probabilities
+// (the group-mean indicator's rows).  A plain kernel like the one above: one thread per slot, the G query rows of
+// the current position in shared memory, heads summed in ascending order.
+template <typename T>
+__global__ void __launch_bounds__(128)
+window_ring_grouped_kernel(int G, int kv_heads, int T_len, int d, int w, int B, int cap, float scale, const T* __restrict__ q,
+                           int64_t qsb, int64_t qsh, int64_t q_head, int64_t st, const float* __restrict__ lse, int64_t lse_sb,
+                           int64_t lse_sh, vatp_cache c) {
+  extern __shared__ float q_rows[];      // [G][d], fp32
+  const int u = blockIdx.y;
+  const int slot = blockIdx.x * blockDim.x + threadIdx.x;
+  const int len = min(T_len, B);
+  const int b = u / kv_heads, h = u - b * kv_heads;
+  const T* qu = q + (int64_t)b * qsb + (int64_t)h * qsh;
+  const float* lu = lse + (int64_t)b * lse_sb + (int64_t)h * lse_sh;
+  const T* krow = static_cast<const T*>(c.k_cache) + ((int64_t)u * cap + slot) * d;
+  const int ps = slot < len ? c.pos[(int64_t)u * cap + slot] : -1;
+  const float invG = 1.f / (float)G;
+  long long fx = 0;
+  for (int r = 0; r < w; ++r) {
+    const int j = T_len - w + r;
+    const int rr = ((j % w) + w) % w;
+    __syncthreads();
+    if (j >= 0)
+      for (int i = threadIdx.x; i < G * d; i += blockDim.x)
+        q_rows[i] = to_f32(qu[(int64_t)(i / d) * q_head + (int64_t)j * st + (i % d)]);
+    __syncthreads();
+    float p = 0.f;
+    if (slot < cap && j >= 0 && ps >= 0 && ps <= j) {
+      for (int g = 0; g < G; ++g) {
+        float dot = 0.f;
+        for (int i = 0; i < d; ++i) dot = fmaf(q_rows[g * d + i], to_f32(krow[i]), dot);
+        p += __expf(dot * scale - __ldg(lu + (int64_t)g * T_len + j));
+      }
+      p *= invG;
+    }
+    if (slot < cap) {
+      c.ring[((int64_t)u * w + rr) * cap + slot] = p;
+      fx += prob_to_fixed(p);
+    }
+  }
+  if (slot < cap) {
+    c.acc_fixed[(int64_t)u * cap + slot] = fx;
+    c.acc[(int64_t)u * cap + slot] = fixed_to_prob(fx);
+  }
+}
+
 }  // namespace
+
+// lse: [batch, heads, T] contiguous (every query head's normalisers); s describes the KV units (see make_shape)
+cudaError_t launch_window_ring_grouped(const Shape& s, int G, int dtype, int B, const void* q, const float* lse, const vatp_cache& c,
+                                       cudaStream_t st) {
+  const int cap = cache_capacity(B);
+  const size_t smem = (size_t)G * s.d * sizeof(float);
+  if (smem > 48 * 1024) return cudaErrorNotSupported;
+  const dim3 grid((cap + 127) / 128, s.units);
+  if (dtype == VATP_F32)
+    window_ring_grouped_kernel<float><<<grid, 128, smem, st>>>(G, s.heads, s.T, s.d, s.window, B, cap, s.scale, static_cast<const float*>(q),
+                                                                s.qsb, s.qsh, s.sh, s.st, lse, s.lse_sb, s.lse_sh, c);
+  else
+    window_ring_grouped_kernel<__nv_bfloat16><<<grid, 128, smem, st>>>(G, s.heads, s.T, s.d, s.window, B, cap, s.scale,
+                                                                        static_cast<const __nv_bfloat16*>(q), s.qsb, s.qsh, s.sh, s.st,
+                                                                        lse, s.lse_sb, s.lse_sh, c);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_window_ring(const Shape& s, int dtype, int B, const void* q, const float* lse, const vatp_cache& c,
                                int32_t* dev_status, cudaStream_t st) {

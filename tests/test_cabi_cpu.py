@@ -92,7 +92,7 @@ def test_host_side_validation(V):
     assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=2, strides=(0, 0, 128))) == 0
     gw = V.make_params(**gq, kv_heads=2, indicator="window", window=8)
     assert V.lib.vatp_prefill_scores(C.byref(gw), 16, 16, 16, 16, 16, 16, 16, 16, 256, 1 << 20, null, null) == 2   # no win_rows with grouped queries
-    assert V.lib.vatp_decode_step(C.byref(gw), C.byref(cs), 16, 16, 16, 16, null, null, null) == 2
+    assert V.lib.vatp_compact(C.byref(gw), 16, 16, 16, 16, 16, 16, C.byref(cs), null, null) == 2                   # nor the gather from them
     # attention forward fused with the scoring: the output array is required and 16-byte aligned, the usual checks follow
     fa = V.lib.vatp_prefill_attention_scores
     assert fa(C.byref(p), 16, 16, 16, null, null, 16, 16, 16, null, 256, 4096, null, null) == 1

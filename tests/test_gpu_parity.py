@@ -729,3 +729,93 @@ def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R, fused):
         order = np.argsort(pos[live])
         assert pos[live][order].tolist() == st.pos and int(cache.len[bi, g]) == len(st.pos)
         assert P.rel_err(P.to_np64(cache.acc[bi, g])[live][order], st.indicator()) <= 2 * tol
+
+
+@pytest.mark.parametrize("dtype,d,heads,kv_heads,T,B,F,R,w", [
+    ("bf16", 128, 8, 2, 700, 250, 2, 10, 150),     # tensor-core scoring per query head, window starts inside a tile
+    ("f32", 64, 4, 2, 333, 100, 3, 10, 50),        # general kernels
+    ("bf16", 128, 4, 1, 300, 120, 0, 8, 400),      # window longer than the prompt, one KV head
+])
+def test_grouped_query_attention_with_history_window(dtype, d, heads, kv_heads, T, B, F, R, w):
+    """Grouped queries with the windowed indicator (Eq. 3 under the group-mean reading): the indicator over the last w
+    queries, the history ring rebuilt by vatp_compact_window as the mean of the heads' probabilities, and decode steps
+    through evictions and through the window sliding, every KV unit against the oracle."""
+    from oracle import vatp_oracle as O
+    V = P.vatp()
+    b, G, steps = 2, heads // kv_heads, 12
+    tol = P.TOL[dtype]
+    wl_kv = _small(dtype, d, T, B, F, R, b=b, h=kv_heads, indicator="window", window=w, steps=steps, cid=81)
+    _, k, v = synth.prefill_inputs(wl_kv, 0, "cuda")
+    u = synth.sink_direction(wl_kv, 0, "cuda").repeat_interleave(G, dim=1)
+    gq = torch.Generator(device="cuda").manual_seed(4081)
+    q = (torch.randn(b, heads, T, d, generator=gq, device="cuda") + synth.sink_alpha(wl_kv) * u).to(k.dtype)
+    dq = (torch.randn(steps, b, heads, d, generator=gq, device="cuda") + synth.sink_alpha(wl_kv) * u.squeeze(2)).to(k.dtype)
+    _, dk, dv = synth.decode_inputs(wl_kv, 0, device="cuda")
+
+    p = V.make_params(batch=b, heads=heads, kv_heads=kv_heads, seq_len=T, head_dim=d, dtype=dtype, budget=B, n_sink=F,
+                      n_recent=R, scale=wl_kv.scale, indicator="window", window=w)
+    f32 = dict(dtype=torch.float32, device="cuda")
+    lse = torch.empty(b, heads, T, **f32)
+    attn_acc, vnorm, score = (torch.empty(b, kv_heads, T, **f32) for _ in range(3))
+    ws = torch.empty(V.vatp_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    kept = torch.empty(b, kv_heads, B, dtype=torch.int32, device="cuda")
+    cache = V.Cache(p)
+    V.vatp_prefill_scores(p, q, k, v, lse_out=lse, attn_acc=attn_acc, vnorm=vnorm, score=score, workspace=ws, dev_status=status)
+    V.vatp_select(p, score, kept, dev_status=status)
+    V.vatp_compact_window(p, q, k, v, lse, attn_acc, vnorm, kept, cache, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.all((attn_acc.double().sum(-1) - min(w, T)).abs() <= 2e-3 * min(w, T))
+
+    n_live = min(T, B)
+    states = {}
+    for bi in range(b):
+        for g in range(kv_heads):
+            ref = O.prefill_gqa(P.to_np64(q[bi, g * G:(g + 1) * G]), P.to_np64(k[bi, g]), P.to_np64(v[bi, g]), wl_kv.scale, window=w)
+            first = max(T - w, 0)
+            assert np.max(np.abs(P.to_np64(lse[bi, g * G:(g + 1) * G, first:]) - ref["lse"][:, first:])) <= 10 * tol
+            for name, key in (("attn_acc", "S"), ("vnorm", "n1"), ("score", "I")):
+                e = P.rel_err(P.to_np64(locals()[name][bi, g]), ref[key])
+                assert e <= tol, f"{name} rel err {e:.3g} (unit {bi},{g})"
+            got = kept[bi, g, :n_live].cpu().numpy().astype(np.int64)
+            want = O.select_keep(ref["I"], B, F, R)
+            if not np.array_equal(got, want):        # only indices whose score ties the boundary within the tolerance may differ
+                mid = [i for i in want if F <= i < T - R]
+                tau = ref["I"][mid].min()
+                for i in set(got.tolist()) ^ set(want.tolist()):
+                    assert abs(ref["I"][i] - tau) <= tol * tau
+            # the ring: row (j mod w) = group-mean probabilities of query j on the kept tokens; exact window sums
+            ring = P.to_np64(cache.ring[bi, g])
+            rows_ref = ref["window_rows"]
+            j0 = T - rows_ref.shape[0]
+            want_ring = np.zeros((w, n_live))
+            for r in range(rows_ref.shape[0]):
+                want_ring[(j0 + r) % w] = rows_ref[r][got]
+            assert np.max(np.abs(ring[:, :n_live] - want_ring) - tol * np.abs(want_ring)) <= 1e-30, "history ring"
+            fixed = cache.acc_fixed[bi, g, :n_live].cpu().numpy().astype(np.float64) / 2.0 ** 52
+            assert P.rel_err(fixed, ref["S"][got]) <= tol
+            states[(bi, g)] = O.DecodeState(P.to_np64(k[bi, g]), P.to_np64(v[bi, g]), ref["S"], ref["n1"], got, T, window=w,
+                                            window_rows=ref["window_rows"])
+
+    out = torch.empty(b, heads, d, dtype=k.dtype, device="cuda")
+    evicted = torch.empty(b, kv_heads, dtype=torch.int32, device="cuda")
+    out_eps = 2.0 ** -8 if dtype == "bf16" else 0.0
+    for s_ in range(steps):
+        V.vatp_decode_step(p, cache, dq[s_], dk[s_], dv[s_], out, evicted_pos=evicted, dev_status=status)
+        torch.cuda.synchronize()
+        for (bi, g), st in states.items():
+            ev = int(evicted[bi, g])
+            res = O.decode_step(st, P.to_np64(dq[s_, bi, g * G:(g + 1) * G]), P.to_np64(dk[s_, bi, g]), P.to_np64(dv[s_, bi, g]),
+                                wl_kv.scale, B, F, R, force_evict=None if ev < 0 else ev, tie_tol=2 * tol, tie_abs=1e-30)
+            assert res["evicted"] == ev
+            ref_out = res["out"]
+            bound = tol * np.max(np.abs(ref_out)) + out_eps * np.abs(ref_out) + 1e-30
+            assert np.all(np.abs(P.to_np64(out[bi, g * G:(g + 1) * G]) - ref_out) <= bound), f"step {s_} unit {(bi, g)}: out"
+    assert int(status.item()) == 0
+    for (bi, g), st in states.items():
+        pos = cache.pos[bi, g].cpu().numpy()
+        live = pos >= 0
+        order = np.argsort(pos[live])
+        assert pos[live][order].tolist() == st.pos and int(cache.len[bi, g]) == len(st.pos)
+        assert P.rel_err(P.to_np64(cache.acc[bi, g])[live][order], st.indicator()) <= 2 * tol
