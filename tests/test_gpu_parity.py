@@ -390,11 +390,12 @@ def test_prefill_from_given_row_normalisers_config1():
     ("f32", 64, 200, 64, "window", 50),
     ("bf16", 64, 257, 128, "h2o", 0),
 ])
-def test_fused_attention_forward(dtype, d, T, B, indicator, window):
+@pytest.mark.parametrize("norm", ["l1", "linf"])
+def test_fused_attention_forward(dtype, d, T, B, indicator, window, norm):
     """vatp_prefill_attention_scores: the attention output rows (Eq. 1) against the oracle, and everything the
     two-pass call produces - normalisers, indicator, norms, scores, kept sets, compaction, decode steps - checked
     the same way; its scores agree with the two-pass call's within the score tolerance."""
-    wl = _small(dtype, d, T, B, 2, 10, b=2, h=3, indicator=indicator, window=window, steps=4, cid=75)
+    wl = _small(dtype, d, T, B, 2, 10, b=2, h=3, indicator=indicator, window=window, steps=4, cid=75).with_(norm=norm)
     g, _, _ = _run_case(wl, fused_forward=True)
     two = P.GpuPrefill(wl, g.q, g.k, g.v).run()
     tol = P.TOL[dtype]
