@@ -804,12 +804,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 //   inside bf16 and fp32 range; once the first chunks - which hold the attention sinks - are past, almost
 //   no chunk rescales).  A rescale is a TMEM load / multiply / store of the thread's own row, done after
 //   the previous P V product has completed and before this chunk's product is released.
-// Warp roles (352 threads): warp 0 TMA producer and work-item FIFO, warp 1 MMA issuer, warps 2-9 softmax (row = TMEM
-// lane; two threads per row, 64 keys each, so that every scheduler has two warps to alternate between; a share of
-// the exponentials runs as a polynomial on the FMA pipe, as in pass 1), warp 10 value norms (Eq. 4).  MMA order: S(c+1) is issued before O += P(c) V(c), so the
-// tensor pipe recomputes the next logits while the softmax warps are still on chunk c.
+// Warp roles (384 threads): warp 0 TMA producer and work-item FIFO, warp 1 issues S = Q K^T, warps 2-9 softmax (row =
+// TMEM lane; two threads per row, 64 keys each, so that every scheduler has two warps to alternate between), warp 10
+// value norms (Eq. 4), warp 11 issues O += P V.  The two products have an issuing thread each: they share no
+// accumulator, every hand-over between them goes through the softmax warps' barriers, and one thread issuing both
+// spent most of a chunk's time inside its sixteen MMA instructions and the waits between them (the logits of chunk
+// c + 1 are then ready long before the softmax warps have finished chunk c).
 constexpr int FW_NSW = 8;               // softmax warps: two per quarter of the rows
-constexpr int FW_THREADS = (2 + FW_NSW + 1) * 32;
+constexpr int FW_THREADS = (2 + FW_NSW + 2) * 32;
 #ifndef FW_POLY_MASK
 #define FW_POLY_MASK 0x0            // of the four pairs of an 8-probability piece, those whose exponential runs on the FMA pipe
 #endif
@@ -902,7 +904,7 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     for (int i = 0; i < 2; ++i) { mbar_init(&sm.s_full[i], 1); mbar_init(&sm.s_empty[i], FW_NSW); }
     mbar_init(&sm.o_full, 1); mbar_init(&sm.o_empty, FW_NSW);
     for (int i = 0; i < 4; ++i) mbar_init(&sm.pair_bar[i], 2);
-    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 1 + FW_NSW); }   // MMA warp + softmax warps
+    for (int i = 0; i < 4; ++i) { mbar_init(&sm.item_full[i], 1); mbar_init(&sm.item_empty[i], 2 + FW_NSW); }   // two MMA warps + softmax warps
     sm.abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -984,13 +986,12 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
       }
     }
   } else if (wid == 1) {
-    // ------------------------------------------------------------------ MMA issuer
+    // ------------------------------------------------------------------ MMA issuer: S = Q K^T
     if (lane == 0) {
       bool ok = true;
       uint32_t n = 0;
       const uint64_t q_desc = umma_desc(s32(sm.q));
       const uint64_t k_desc0 = umma_desc(s32(sm.k[0]));
-      const uint64_t v_desc0 = umma_desc_mn(s32(sm.v[0]));
       // S(g) = Q K(g)^T into S buffer g % 2
       auto issue_qk = [&](uint32_t g) -> bool {
         const int stg = g % FW_ST, sb = g & 1;
@@ -1014,11 +1015,25 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
         ok = mbar_wait(&sm.q_full, itl & 1, abort_flag, a.dev_status);
         if (!ok) break;
         const int nc = tile + 1;
-        ok = issue_qk(n);
+        for (int c = 0; c < nc && ok; ++c) ok = issue_qk(n + c);
+        if (ok) umma_commit(&sm.q_empty);            // the item's last S has been issued: the query tile may be replaced
+        n += nc;
+      }
+    }
+  } else if (wid == 3 + FW_NSW) {
+    // ------------------------------------------------------------------ second MMA issuer: O += P V
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t n = 0;
+      const uint64_t v_desc0 = umma_desc_mn(s32(sm.v[0]));
+      for (uint32_t itl = 0; ok; ++itl) {
+        int u, tile;
+        next_item(itl, false, u, tile);
+        if (u < 0) break;
+        if (!VATP_INB(u, a.units, a.dev_status) || !VATP_INB(tile, a.nt, a.dev_status)) break;
+        const int nc = tile + 1;
         for (int c = 0; c < nc && ok; ++c) {
           const uint32_t g = n + c;
-          if (c + 1 < nc) { ok = issue_qk(g + 1); if (!ok) break; }
-          else umma_commit(&sm.q_empty);            // the item's last S has been issued: the query tile may be replaced
           const int stg = g % FW_ST, pb = g % FW_PB;
           ok = mbar_wait(&sm.p_full[pb], (g / FW_PB) & 1, abort_flag, a.dev_status) &&
                mbar_wait(&sm.v_full[stg], (g / FW_ST) & 1, abort_flag, a.dev_status) &&
