@@ -1375,17 +1375,38 @@ window_ring_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_con
       uint32_t off = (uint32_t)rr * (uint32_t)cap;          // element offset of the ring row (w * cap < 2^31: checked on the host)
       const int live = min(32, n_cols - cs);
       const uint32_t lp = s32(&sm.nlse[cs]);
+      if (live == 32 && rr + 32 <= w) {
+        // the common case - a whole wave inside the window, no wrap of the ring row inside it: no per-column
+        // bookkeeping.  Column i is visible to this slot's token iff ps <= j0 + i, i.e. i >= first (-1 < first: ps >= 0).
+        const int first = ps >= 0 ? max(ps - j0, 0) : 32;
+        const bool st_ok = slot < cap;
+        float* out_p = ring_s + off;
 #pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        if (i < live) {
-          float nl;
-          asm("ld.shared.f32 %0, [%1];" : "=f"(nl) : "r"(lp + 4 * i));
-          float pr = 0.f;
-          if (ps >= 0 && ps <= j0 + i) pr = ex2(fmaf(x[i], scale_log2, nl));
-          fx += prob_to_fixed(pr);
-          if (slot < cap && VATP_INB(off, (int64_t)w * cap, dev_status)) ring_s[off] = pr;
-          off += cap;
-          if (++rr == w) { rr = 0; off = 0; }
+        for (int i4 = 0; i4 < 32; i4 += 4) {
+          float4 nl;
+          asm("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(nl.x), "=f"(nl.y), "=f"(nl.z), "=f"(nl.w) : "r"(lp + 4 * i4));
+          const float nls[4] = {nl.x, nl.y, nl.z, nl.w};
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int i = i4 + k;
+            const float pr = i >= first ? ex2(fmaf(x[i], scale_log2, nls[k])) : 0.f;
+            fx += prob_to_fixed(pr);
+            if (st_ok && VATP_INB(off + (uint32_t)i * (uint32_t)cap, (int64_t)w * cap, dev_status)) out_p[(size_t)i * cap] = pr;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          if (i < live) {
+            float nl;
+            asm("ld.shared.f32 %0, [%1];" : "=f"(nl) : "r"(lp + 4 * i));
+            float pr = 0.f;
+            if (ps >= 0 && ps <= j0 + i) pr = ex2(fmaf(x[i], scale_log2, nl));
+            fx += prob_to_fixed(pr);
+            if (slot < cap && VATP_INB(off, (int64_t)w * cap, dev_status)) ring_s[off] = pr;
+            off += cap;
+            if (++rr == w) { rr = 0; off = 0; }
+          }
         }
       }
     }
