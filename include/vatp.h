@@ -205,8 +205,9 @@ vatp_status vatp_prefill_attention_scores(const vatp_params* params, const void*
  * First call on a device: looks up the array's device address (once per device, with the current
  * device) - make that first call outside any stream capture.
  * Sharing: all calls on a device use the same array.  Calls on one stream are ordered and safe
- * (each call starts with a fully serialising memset of its counters, so it cannot begin before the
- * previous call on the stream has finished with the array);
+ * (each call starts by zeroing its counters - a memset, or a kernel that first waits for all
+ * earlier work in the stream - and touches nothing else before that, so it cannot begin before
+ * the previous call on the stream has finished with the array);
  * calls that may overlap on the GPU (different streams, different host threads) race on it and
  * give wrong scores - serialise them, or use vatp_prefill_scores with separate workspaces.  The
  * array keeps the previous call's contents; nothing in it needs clearing, because pass 1 writes

@@ -52,9 +52,10 @@ extern "C" vatp_status vatp_prefill_scores_static(const vatp_params* params, con
   if (need > 0 && scratch_address(&scratch) != cudaSuccess) return VATP_ERR_CUDA;
   // Nothing in the scratch has to start at zero: pass 1 writes every normaliser that pass 2 reads.
   // Two calls on one stream do not race on the array although pass 2 lets the work after it start early:
-  // every call begins with an ordinary (fully serialising) cudaMemsetAsync of its work-item counters, which
-  // waits for the previous call's pass 2 to finish.  A change that makes a call's first operation a
-  // programmatic dependent launch would have to restore that ordering some other way.
+  // every call begins by zeroing its work-item counters, either with an ordinary (fully serialising)
+  // cudaMemsetAsync or with a one-warp kernel that executes griddepcontrol.wait first, and the kernel after it
+  // (pass 1, resident early as that kernel's programmatic dependent) also waits before it touches global memory:
+  // both waits return only when everything earlier in the stream, the previous call's pass 2 included, has completed.
   // With invalid parameters (need == 0) the call below reports the precise reason.
   return vatp_prefill_scores(params, q, k, v, lse_out, attn_acc, vnorm, score, win_rows, scratch,
                              VATP_STATIC_SCRATCH_BYTES, dev_status, cuda_stream);

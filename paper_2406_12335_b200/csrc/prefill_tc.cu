@@ -391,6 +391,8 @@ struct TcArgs {
   int norm;                 // vatp_norm_kind of the value norm
   int side_norm;            // pass 1 reduces the value norms in its side warp (else vnorm_kernel has, before it)
   unsigned* counters;       // [2] next work item of pass 1 / pass 2 (zeroed before pass 1 is launched)
+  int wait_first;           // pass 1 was launched as a programmatic dependent (of the kernel that zeroes the counters):
+                            // nothing in global memory is touched before griddepcontrol.wait
   float* win_rows;
 };
 
@@ -498,6 +500,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
+  if (PASS == 1 && a.wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // Consumer side of the item FIFO: the itl-th item of this CTA (u < 0 ends the pass, also when the CTA
   // is aborting).  The producer has worked out what the item covers, once for the whole CTA (the index
@@ -917,6 +920,7 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = sm.tmem_base;
+  if (a.wait_first) asm volatile("griddepcontrol.wait;" ::: "memory");     // see reset_counters_kernel
   // pass 2, a programmatic dependent, may set up while this kernel runs
   if (tid == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
@@ -1224,6 +1228,15 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
   }
+}
+
+// Zeroes the two work-item counters.  Launched as a programmatic dependent, with pass 1 as its own dependent: both
+// are resident early and the launch latencies of a scoring call that follows other work on the stream are hidden;
+// nothing is written before everything earlier in the stream has completed.
+__global__ void reset_counters_kernel(unsigned* counters) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  if (threadIdx.x < 2) counters[threadIdx.x] = 0u;
 }
 
 // Value norms as a kernel of their own (Eq. 4): used with a history window, where pass 1 covers only
@@ -1560,9 +1573,17 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   if ((e = cudaFuncSetAttribute(prefill_tc_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
   const int sms = device_sm_count();
   const int items1 = a.units * (a.nt - a.ft), items2 = a.units * a.nt;
-  if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) return e;
   // the side warp belongs to pass 1 (too short under a history window) or to the fused forward (always all tiles)
   a.side_norm = (a.ft == 0 || attn_out) && a.norm == VATP_NORM_L1 && !lse_in;
+  // The counters are zeroed first.  When pass 1 follows at once, a one-warp kernel does it and pass 1 is its
+  // programmatic dependent (see reset_counters_kernel); otherwise a memset node.
+  a.wait_first = (a.side_norm && !lse_in) ? 1 : 0;
+  if (a.wait_first) {
+    DependentLaunch dr(dim3(1), dim3(32), 0, st);
+    if ((e = cudaLaunchKernelEx(&dr.cfg, reset_counters_kernel, a.counters)) != cudaSuccess) return e;
+  } else if ((e = cudaMemsetAsync(a.counters, 0, 2 * sizeof(unsigned), st)) != cudaSuccess) {
+    return e;
+  }
   if (!a.side_norm) {
     const dim3 grid(a.units, (s.T + 127) / 128);
     if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a, lse_in);
@@ -1579,8 +1600,18 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
       const size_t g = ((size_t)48 << 20) / unit_bytes;
       af.gu = g < 1 ? 1 : (g > (size_t)s.units ? s.units : (int)g);
     }
-    attention_fwd_tc_kernel<<<items2 < sms ? items2 : sms, FW_THREADS, fsmem, st>>>(tm_q, tm_k, tm_v, af,
-                                                                                    static_cast<__nv_bfloat16*>(attn_out));
+    if (a.wait_first) {
+      DependentLaunch df(dim3(items2 < sms ? items2 : sms), dim3(FW_THREADS), fsmem, st);
+      if ((e = cudaLaunchKernelEx(&df.cfg, attention_fwd_tc_kernel, tm_q, tm_k, tm_v, af, static_cast<__nv_bfloat16*>(attn_out))) !=
+          cudaSuccess)
+        return e;
+    } else {
+      attention_fwd_tc_kernel<<<items2 < sms ? items2 : sms, FW_THREADS, fsmem, st>>>(tm_q, tm_k, tm_v, af,
+                                                                                      static_cast<__nv_bfloat16*>(attn_out));
+    }
+  } else if (a.wait_first && !lse_in) {
+    DependentLaunch d1(dim3(items1 < sms ? items1 : sms), dim3(TC_THREADS), smem, st);
+    if ((e = cudaLaunchKernelEx(&d1.cfg, prefill_tc_kernel<1, false>, tm_q, tm_k, a)) != cudaSuccess) return e;
   } else if (!lse_in) {
     prefill_tc_kernel<1, false><<<items1 < sms ? items1 : sms, TC_THREADS, smem, st>>>(tm_q, tm_k, a);
   }
