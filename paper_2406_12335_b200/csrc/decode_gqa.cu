@@ -5,15 +5,25 @@
 // and the exact fixed-point window sum moves by it), Eq. 4 multiplies by the norm of the shared value row, and
 // the lowest importance is released as in the multi-head step.
 //
-// A plain kernel, not a tuned one: one CTA per KV unit, any dtype and head_dim, the logits of all heads
-// in shared memory.  Steps: append (k, v); per head logits, max, sum; per head output; indicator update and
-// arg-min over the slots.
+// A general kernel (any dtype and head_dim, one CTA of 512 threads per KV unit, the probabilities of all heads
+// in shared memory), laid out so that every K and V row is read ONCE for all heads of the group:
+//   logits   the 16-byte pieces of a row go to neighbouring threads (a coalesced read), a warp takes 32 / (pieces
+//            per row) rows at a time; a thread forms its piece's share of all G heads' dot products (its pieces of
+//            the queries in registers), shuffles add the shares up;
+//   softmax  per head over the slots (block reductions);
+//   output   the same thread-to-row layout over V: a thread accumulates, for every head, the outputs of its
+//            piece's channels; shuffles merge a warp's rows, shared memory the sixteen warps;
+//   indicator update and arg-min over the slots as in the multi-head step.
+// (The first version walked K once per head from one thread per slot and V once per head and channel, serially:
+// 1.8 ms per step for 64 units of 2049 slots; this one takes a few tens of microseconds.)
 #include "vatp_internal.cuh"
 
 namespace vatp {
 namespace {
 
-constexpr int GQ_THREADS = 256;
+constexpr int GQ_THREADS = 512;
+constexpr int GQ_WARPS = GQ_THREADS / 32;
+constexpr int GQ_FLY = 8;              // row steps a thread requests before it uses the first
 
 __device__ __forceinline__ float block_max(float x, float* red) {
 #pragma unroll
@@ -22,7 +32,7 @@ __device__ __forceinline__ float block_max(float x, float* red) {
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
   __syncthreads();
   float y = red[0];
-  for (int i = 1; i < GQ_THREADS / 32; ++i) y = fmaxf(y, red[i]);
+  for (int i = 1; i < GQ_WARPS; ++i) y = fmaxf(y, red[i]);
   return y;
 }
 __device__ __forceinline__ float block_sum(float x, float* red) {
@@ -32,21 +42,47 @@ __device__ __forceinline__ float block_sum(float x, float* red) {
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = x;
   __syncthreads();
   float y = 0.f;
-  for (int i = 0; i < GQ_THREADS / 32; ++i) y += red[i];      // fixed order
+  for (int i = 0; i < GQ_WARPS; ++i) y += red[i];      // fixed order
   return y;
 }
 
+// the 16-byte piece of a row starting at element e: EP = 8 bf16 or 4 fp32 values, as fp32
 template <typename T>
+struct Piece;
+template <>
+struct Piece<__nv_bfloat16> {
+  static constexpr int EP = 8;
+  __device__ static void load(const __nv_bfloat16* row, int e, float (&x)[8]) {
+    const uint4 r = *reinterpret_cast<const uint4*>(row + e);
+    const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { x[2 * i] = __uint_as_float(w[i] << 16); x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u); }
+  }
+};
+template <>
+struct Piece<float> {
+  static constexpr int EP = 4;
+  __device__ static void load(const float* row, int e, float (&x)[4]) {
+    const float4 r = *reinterpret_cast<const float4*>(row + e);
+    x[0] = r.x; x[1] = r.y; x[2] = r.z; x[3] = r.w;
+  }
+};
+
+// GT: compile-time bound on the heads per group (G <= GT): the per-head accumulators stay in registers.
+// TPR: threads per row = 16-byte pieces per row when known at compile time (8, 16, 32), 0: taken from d at run time.
+template <typename T, int GT, int TPR>
 __global__ void __launch_bounds__(GQ_THREADS)
 decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int w, int norm, float scale, vatp_cache c, const T* __restrict__ q_new,
                   const T* __restrict__ k_new, const T* __restrict__ v_new, T* __restrict__ out, int32_t* __restrict__ evicted,
                   int32_t* dev_status) {
-  extern __shared__ float gq_smem[];            // p[G][cap] (logits, then probabilities) | q[G][d]
-  __shared__ float red[GQ_THREADS / 32];
-  __shared__ unsigned long long key_red[GQ_THREADS / 32];
-  __shared__ int slot_red[GQ_THREADS / 32], pos_red[GQ_THREADS / 32];
+  extern __shared__ __align__(16) float gq_smem[];   // p[G][cap] (logits, then probabilities) | q[G][d] | part[warps][G][d]
+  __shared__ float red[GQ_WARPS];
+  __shared__ unsigned long long key_red[GQ_WARPS];
+  __shared__ int slot_red[GQ_WARPS], pos_red[GQ_WARPS];
+  constexpr int EP = Piece<T>::EP;
   float* p_s = gq_smem;
   float* q_s = gq_smem + (size_t)G * cap;
+  float* part_s = q_s + (size_t)G * d;
   const int u = blockIdx.x, tid = threadIdx.x;
   const int len = c.len[u], fs = c.free_slot[u], t = c.next_pos[u];
   if (!VATP_INB(len, cap, dev_status) || !VATP_INB(fs, cap, dev_status)) return;
@@ -71,22 +107,62 @@ decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int w, int norm, f
     if ((tid & 31) == 0) red[tid >> 5] = nn;
     __syncthreads();
     nn = red[0];
-    for (int i = 1; i < GQ_THREADS / 32; ++i) nn = norm_merge(norm, nn, red[i]);
+    for (int i = 1; i < GQ_WARPS; ++i) nn = norm_merge(norm, nn, red[i]);
     nn = norm_finish(norm, nn);
   }
   __syncthreads();                              // the appended rows and the queries are visible to the CTA
 
-  // ---- logits of every head over the live slots
-  for (int s = tid; s < hi; s += GQ_THREADS) {
-    const T* kr = kc + (int64_t)s * d;
-    for (int g = 0; g < G; ++g) {
-      float dot = 0.f;
-      for (int i = 0; i < d; ++i) dot = fmaf(q_s[g * d + i], to_f32(kr[i]), dot);
-      p_s[(size_t)g * cap + s] = dot * scale;
+  // ---- logits of every head over the live slots: one row read serves all heads.  tpr = d / EP threads share a
+  // row (its 16-byte pieces side by side: a coalesced read), a warp takes 32 / tpr rows at a time; every thread
+  // forms the partial dot products of its piece with all G heads, the tpr partials are summed by shuffles.
+  const int tpr = TPR ? TPR : d / EP;             // a power of two <= 32 (checked on the host)
+  const int rows_w = 32 / tpr;                   // rows per warp and step
+  const int lane = tid & 31, wid = tid >> 5;
+  const int sub = lane / tpr, piece = lane - sub * tpr;
+  {
+    float qreg[GT][EP];                          // this thread's piece of every head's query
+#pragma unroll
+    for (int g = 0; g < GT; ++g)
+#pragma unroll
+      for (int i = 0; i < EP; ++i) qreg[g][i] = g < G ? q_s[g * d + piece * EP + i] : 0.f;
+    // GQ_FLY row steps per thread are requested before any is used: one CTA has to pull the whole unit through one
+    // SM, and with one 16-byte load per thread in flight that took ten times longer than the arithmetic
+    const int stride = GQ_WARPS * rows_w;
+    for (int s0 = wid * rows_w; s0 < hi; s0 += GQ_FLY * stride) {
+      float x[GQ_FLY][EP];
+#pragma unroll
+      for (int j = 0; j < GQ_FLY; ++j) {
+        const int s = s0 + j * stride + sub;
+#pragma unroll
+        for (int i = 0; i < EP; ++i) x[j][i] = 0.f;
+        if (s < hi) Piece<T>::load(kc + (int64_t)s * d, piece * EP, x[j]);
+      }
+#pragma unroll
+      for (int j = 0; j < GQ_FLY; ++j) {
+        const int s = s0 + j * stride + sub;
+        if (s0 + j * stride >= hi) break;          // warp-uniform
+        float dot[GT];
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+          dot[g] = 0.f;
+          if (g < G) {
+#pragma unroll
+            for (int i = 0; i < EP; ++i) dot[g] = fmaf(qreg[g][i], x[j][i], dot[g]);
+#pragma unroll
+            for (int o = 16; o; o >>= 1)
+              if (o < tpr) dot[g] += __shfl_xor_sync(0xffffffffu, dot[g], o);
+          }
+        }
+        if (piece == 0 && s < hi) {
+#pragma unroll
+          for (int g = 0; g < GT; ++g)
+            if (g < G) p_s[(size_t)g * cap + s] = dot[g] * scale;
+        }
+      }
     }
   }
   __syncthreads();
-  // ---- per head: softmax over the slots, then the output row (Eq. 1)
+  // ---- per head: softmax over the slots (Eq. 1)
   for (int g = 0; g < G; ++g) {
     float m = -INFINITY;
     for (int s = tid; s < hi; s += GQ_THREADS) m = fmaxf(m, p_s[(size_t)g * cap + s]);
@@ -100,15 +176,61 @@ decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int w, int norm, f
     l = block_sum(l, red);
     const float inv = 1.f / l;
     for (int s = tid; s < hi; s += GQ_THREADS) p_s[(size_t)g * cap + s] *= inv;
-    __syncthreads();
-    for (int i = tid; i < d; i += GQ_THREADS) {
-      float a = 0.f;
-      for (int s = 0; s < hi; ++s) a = fmaf(p_s[(size_t)g * cap + s], to_f32(vc[(int64_t)s * d + i]), a);
-      if constexpr (sizeof(T) == 2) out[((int64_t)u * G + g) * d + i] = __float2bfloat16(a);
-      else out[((int64_t)u * G + g) * d + i] = a;
-    }
   }
   __syncthreads();
+  // ---- outputs of all heads in one walk over the value rows: the same thread-to-row layout; a thread holds, for
+  // every head, the outputs of its piece's EP channels; rows of one warp are merged by shuffles, the sixteen warps
+  // through shared memory.
+  {
+    float acc[GT][EP];
+#pragma unroll
+    for (int g = 0; g < GT; ++g)
+#pragma unroll
+      for (int i = 0; i < EP; ++i) acc[g][i] = 0.f;
+    const int stride = GQ_WARPS * rows_w;
+    for (int s0 = wid * rows_w; s0 < hi; s0 += GQ_FLY * stride) {      // GQ_FLY rows in flight per thread
+      float x[GQ_FLY][EP];
+#pragma unroll
+      for (int j = 0; j < GQ_FLY; ++j) {
+        const int s = s0 + j * stride + sub;
+#pragma unroll
+        for (int i = 0; i < EP; ++i) x[j][i] = 0.f;
+        if (s < hi) Piece<T>::load(vc + (int64_t)s * d, piece * EP, x[j]);
+      }
+#pragma unroll
+      for (int j = 0; j < GQ_FLY; ++j) {
+        const int s = s0 + j * stride + sub;
+#pragma unroll
+        for (int g = 0; g < GT; ++g) {
+          if (g < G) {
+            const float pj = s < hi ? p_s[(size_t)g * cap + s] : 0.f;
+#pragma unroll
+            for (int i = 0; i < EP; ++i) acc[g][i] = fmaf(pj, x[j][i], acc[g][i]);
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < GT; ++g) {
+      if (g < G) {
+#pragma unroll
+        for (int i = 0; i < EP; ++i) {
+          float a = acc[g][i];
+#pragma unroll
+          for (int o = 16; o; o >>= 1)
+            if (o >= tpr) a += __shfl_xor_sync(0xffffffffu, a, o);      // the warp's rows
+          if (sub == 0) part_s[((size_t)wid * G + g) * d + piece * EP + i] = a;
+        }
+      }
+    }
+    __syncthreads();
+    for (int i = tid; i < G * d; i += GQ_THREADS) {
+      float a = 0.f;
+      for (int pp = 0; pp < GQ_WARPS; ++pp) a += part_s[(size_t)pp * G * d + i];     // fixed order
+      if constexpr (sizeof(T) == 2) out[(int64_t)u * G * d + i] = __float2bfloat16(a);
+      else out[(int64_t)u * G * d + i] = a;
+    }
+  }
   // ---- indicator += mean of the heads' probabilities; importance; arg-min among the unprotected slots
   const bool evicting = hi > B;
   unsigned long long my_key = ~0ull;
@@ -152,7 +274,7 @@ decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int w, int norm, f
     }
     return;
   }
-  // lowest key of the CTA: warps first, then warp 0 over the warps' candidates
+  // lowest key of the CTA: warps first, then thread 0 over the warps' candidates
 #pragma unroll
   for (int o = 16; o; o >>= 1) {
     const unsigned long long k2 = __shfl_xor_sync(0xffffffffu, my_key, o);
@@ -164,7 +286,7 @@ decode_gqa_kernel(int G, int d, int B, int cap, int F, int R, int w, int norm, f
   if (tid == 0) {
     unsigned long long best = ~0ull;
     int bs = -1, bp = -1;
-    for (int i = 0; i < GQ_THREADS / 32; ++i)
+    for (int i = 0; i < GQ_WARPS; ++i)
       if (key_red[i] < best) { best = key_red[i]; bs = slot_red[i]; bp = pos_red[i]; }
     if (bs >= 0) {
       c.pos[(int64_t)u * cap + bs] = -1;
@@ -193,6 +315,29 @@ __global__ void group_mean_kernel(int G, int64_t n, const float* __restrict__ pa
   score[i] = s * vnorm[i];
 }
 
+template <typename T, int GT, int TPR>
+cudaError_t launch_gqa_t(int units, int G, int d, size_t smem, int B, int cap, int F, int R, int window, int norm, float scale,
+                       const vatp_cache& c, const void* q, const void* k, const void* v, void* out, int32_t* evicted,
+                       int32_t* dev_status, cudaStream_t st) {
+  cudaError_t e = cudaFuncSetAttribute(decode_gqa_kernel<T, GT, TPR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  decode_gqa_kernel<T, GT, TPR><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, window, norm, scale, c, static_cast<const T*>(q),
+                                                           static_cast<const T*>(k), static_cast<const T*>(v), static_cast<T*>(out),
+                                                           evicted, dev_status);
+  return cudaGetLastError();
+}
+
+// the common row lengths get kernels with the piece count known at compile time
+template <typename T, int GT>
+cudaError_t launch_gqa(int units, int G, int d, size_t smem, int B, int cap, int F, int R, int window, int norm, float scale,
+                       const vatp_cache& c, const void* q, const void* k, const void* v, void* out, int32_t* evicted,
+                       int32_t* dev_status, cudaStream_t st) {
+  const int tpr = d / Piece<T>::EP;
+  if (tpr == 16) return launch_gqa_t<T, GT, 16>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+  if (tpr == 8) return launch_gqa_t<T, GT, 8>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+  return launch_gqa_t<T, GT, 0>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+}
+
 }  // namespace
 
 cudaError_t launch_group_mean(int G, int64_t n, const float* part, const float* vnorm, float* attn_acc, float* score,
@@ -201,27 +346,24 @@ cudaError_t launch_group_mean(int G, int64_t n, const float* part, const float* 
   return cudaGetLastError();
 }
 
-// units: batch * kv_heads.  cudaErrorNotSupported when the logits of a unit's heads do not fit in shared memory.
+// units: batch * kv_heads.  cudaErrorNotSupported when the probabilities of a unit's heads do not fit in shared memory,
+// for more than 16 heads per group, or for a head_dim whose rows are not a power of two (at most 32) of 16-byte pieces.
 cudaError_t launch_decode_gqa(int units, int G, int d, int dtype, int B, int F, int R, int window, int norm, float scale,
                               const vatp_cache& c, const void* q, const void* k, const void* v, void* out, int32_t* evicted,
                               int32_t* dev_status, cudaStream_t st) {
   const int cap = cache_capacity(B);
-  const size_t smem = sizeof(float) * ((size_t)G * cap + (size_t)G * d);
+  const int tpr = d / (dtype == VATP_F32 ? 4 : 8);       // threads that share a row: its 16-byte pieces
+  if (G > 16 || d % 8 || tpr < 1 || tpr > 32 || (tpr & (tpr - 1))) return cudaErrorNotSupported;
+  const size_t smem = sizeof(float) * ((size_t)G * cap + (size_t)G * d + (size_t)GQ_WARPS * G * d);
   if (smem > 200 * 1024) return cudaErrorNotSupported;
-  cudaError_t e;
   if (dtype == VATP_F32) {
-    e = cudaFuncSetAttribute(decode_gqa_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    decode_gqa_kernel<float><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, window, norm, scale, c, (const float*)q, (const float*)k,
-                                                               (const float*)v, (float*)out, evicted, dev_status);
-  } else {
-    e = cudaFuncSetAttribute(decode_gqa_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
-    decode_gqa_kernel<__nv_bfloat16><<<units, GQ_THREADS, smem, st>>>(G, d, B, cap, F, R, window, norm, scale, c, (const __nv_bfloat16*)q,
-                                                                        (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
-                                                                        (__nv_bfloat16*)out, evicted, dev_status);
+    if (G <= 4) return launch_gqa<float, 4>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+    if (G <= 8) return launch_gqa<float, 8>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+    return launch_gqa<float, 16>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
   }
-  return cudaGetLastError();
+  if (G <= 4) return launch_gqa<__nv_bfloat16, 4>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+  if (G <= 8) return launch_gqa<__nv_bfloat16, 8>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
+  return launch_gqa<__nv_bfloat16, 16>(units, G, d, smem, B, cap, F, R, window, norm, scale, c, q, k, v, out, evicted, dev_status, st);
 }
 
 }  // namespace vatp
