@@ -648,6 +648,7 @@ def test_bounds_checking_build_reports_no_violation():
     ("bf16", 128, 6, 3, 1000, 1100, 0, 8),     # budget beyond the prompt: the cache grows before evictions start
     ("f32", 64, 4, 2, 333, 100, 3, 17),        # general kernels
     ("bf16", 64, 8, 1, 257, 128, 2, 16),       # multi-query attention: one KV head
+    ("f32", 128, 16, 1, 200, 80, 1, 8),        # sixteen heads per group, 32 pieces per row
 ])
 @pytest.mark.parametrize("fused", [False, True])
 def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R, fused):
