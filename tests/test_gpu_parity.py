@@ -96,19 +96,25 @@ def test_degenerate_budgets(dtype, d):
     _run_case(_small(dtype, d, 150, 50, 0, 0, steps=4))
 
 
-def test_exact_ties_prefer_lower_index():
+@pytest.mark.parametrize("T,B,heads", [
+    (5000, 1200, 3),        # one CTA per unit
+    (20000, 5000, 3),       # long prompt, 6 units: the range of a unit split over a cluster of four CTAs
+    (9000, 4000, 25),       # 50 units: clusters of two
+    (8300, 8250, 3),        # all but a handful survive
+])
+def test_exact_ties_prefer_lower_index(T, B, heads):
     """select on hand-made scores with many exact ties (integer work: bit-exact)."""
     V = P.vatp()
-    T, B, F, R = 5000, 1200, 3, 100
+    F, R = 3, 100
     rng = np.random.default_rng(0)
-    score = torch.from_numpy(rng.integers(0, 7, size=(2, 3, T)).astype(np.float32)).cuda()
-    p = V.make_params(batch=2, heads=3, seq_len=T, head_dim=64, dtype="f32", budget=B, n_sink=F, n_recent=R)
-    kept = torch.empty(2, 3, B, dtype=torch.int32, device="cuda")
+    score = torch.from_numpy(rng.integers(0, 7, size=(2, heads, T)).astype(np.float32)).cuda()
+    p = V.make_params(batch=2, heads=heads, seq_len=T, head_dim=64, dtype="f32", budget=B, n_sink=F, n_recent=R)
+    kept = torch.empty(2, heads, B, dtype=torch.int32, device="cuda")
     V.vatp_select(p, score, kept)
     torch.cuda.synchronize()
     from oracle import vatp_oracle as O
     for b in range(2):
-        for h in range(3):
+        for h in (0, 1, heads - 1):
             want = O.select_keep(score[b, h].cpu().numpy(), B, F, R)
             assert kept[b, h].cpu().numpy().tolist() == want.tolist()
 
@@ -118,16 +124,17 @@ def test_select_large_T_unstaged_path():
     V = P.vatp()
     T, B, F, R = 70000, 7000, 20, 512
     g = torch.Generator(device="cuda").manual_seed(5)
-    score = torch.rand(1, 2, T, generator=g, device="cuda")
-    score[0, 0, 1000:1100] = 0.5          # a run of ties
-    p = V.make_params(batch=1, heads=2, seq_len=T, head_dim=128, dtype="bf16", budget=B, n_sink=F, n_recent=R)
-    kept = torch.empty(1, 2, B, dtype=torch.int32, device="cuda")
-    V.vatp_select(p, score, kept)
-    torch.cuda.synchronize()
-    from oracle import vatp_oracle as O
-    for h in range(2):
-        want = O.select_keep(score[0, h].cpu().numpy(), B, F, R)
-        assert kept[0, h].cpu().numpy().tolist() == want.tolist()
+    for heads in (80, 2):                  # many units: one CTA each, keys read from global memory; two units: clusters of four
+        score = torch.rand(1, heads, T, generator=g, device="cuda")
+        score[0, 0, 1000:1100] = 0.5          # a run of ties
+        p = V.make_params(batch=1, heads=heads, seq_len=T, head_dim=128, dtype="bf16", budget=B, n_sink=F, n_recent=R)
+        kept = torch.empty(1, heads, B, dtype=torch.int32, device="cuda")
+        V.vatp_select(p, score, kept)
+        torch.cuda.synchronize()
+        from oracle import vatp_oracle as O
+        for h in (0, heads - 1):
+            want = O.select_keep(score[0, h].cpu().numpy(), B, F, R)
+            assert kept[0, h].cpu().numpy().tolist() == want.tolist()
 
 
 def test_strided_inputs():
