@@ -175,11 +175,25 @@ def replica_throughput(units_per_rank: float, ms: float, world: int) -> float:
 
 
 class LayerState:
-    def __init__(self, V, wl, layer, dev, win_rows=False):
+    def __init__(self, V, wl, layer, dev, win_rows=False, kv_heads=0):
         from paper_2406_12335_b200 import synth
-        self.q, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
-        self.p = V.params_for(self.q, budget=wl.budget, n_sink=wl.n_sink, n_recent=wl.n_recent, scale=wl.scale,
-                              indicator=wl.indicator, window=wl.window, norm=wl.norm, decode_overlap=True)
+        if kv_heads:
+            # grouped queries: K and V of kv_heads heads; the queries of a group lean towards their KV head's sinks
+            wl_q, wl = wl, wl.with_(heads=kv_heads)
+            _, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
+            G = wl_q.heads // kv_heads
+            u = synth.sink_direction(wl, layer, dev).repeat_interleave(G, dim=1)
+            gq = torch.Generator(device=dev).manual_seed(977 + layer)
+            shape = (wl_q.batch, wl_q.heads, wl_q.seq_len, wl_q.head_dim)
+            self.q = (torch.randn(shape, generator=gq, device=dev) + synth.sink_alpha(wl) * u).to(self.k.dtype)
+            self.p = V.make_params(batch=wl_q.batch, heads=wl_q.heads, kv_heads=kv_heads, seq_len=wl.seq_len,
+                                   head_dim=wl.head_dim, dtype=wl.dtype, budget=wl.budget, n_sink=wl.n_sink,
+                                   n_recent=wl.n_recent, scale=wl.scale, indicator=wl.indicator, window=wl.window,
+                                   norm=wl.norm, decode_overlap=True)
+        else:
+            self.q, self.k, self.v = synth.prefill_inputs(wl, layer, dev)
+            self.p = V.params_for(self.q, budget=wl.budget, n_sink=wl.n_sink, n_recent=wl.n_recent, scale=wl.scale,
+                                  indicator=wl.indicator, window=wl.window, norm=wl.norm, decode_overlap=True)
         # the same parameters without the opt-in: every decode step then waits for all earlier work in the stream
         self.p_wait = type(self.p).from_buffer_copy(self.p)
         self.p_wait.flags = 0
@@ -188,7 +202,7 @@ class LayerState:
         self.attn_acc = torch.empty(b, h, T, **f32)
         self.vnorm = torch.empty(b, h, T, **f32)
         self.score = torch.empty(b, h, T, **f32)
-        self.lse = torch.empty(b, h, T, **f32)
+        self.lse = torch.empty(b, self.q.shape[1], T, **f32)      # one normaliser row per query head
         # Eq. 3: by default the history of the kept tokens is rebuilt by vatp_compact_window; --win-rows times the
         # variant in which the scoring call writes all w x T probabilities and vatp_compact gathers from them
         self.win_rows = torch.empty(b, h, wl.window, T, **f32) if wl.indicator == "window" and win_rows else None
@@ -196,8 +210,27 @@ class LayerState:
         self.ws = torch.empty(max(V.vatp_workspace_bytes(self.p), 256), dtype=torch.uint8, device=dev)
         self.cache = V.Cache(self.p, device=dev)
         self.dq, self.dk, self.dv = synth.decode_inputs(wl, layer, device=dev)
-        self.out = torch.empty(wl.decode_steps, b, h, wl.head_dim, dtype=self.q.dtype, device=dev)
+        if kv_heads:
+            self.dq = (torch.randn((wl.decode_steps,) + shape[:2] + shape[3:], generator=gq, device=dev)
+                       + synth.sink_alpha(wl) * u.squeeze(2)).to(self.k.dtype)
+        self.out = torch.empty(wl.decode_steps, b, self.q.shape[1], wl.head_dim, dtype=self.q.dtype, device=dev)
         self.evicted = torch.empty(wl.decode_steps, b, h, dtype=torch.int32, device=dev)
+
+
+def prune_launches(wl, args):
+    """Kernels of this library that one layer's scoring + selection + compaction launches (memsets not counted)."""
+    windowed = wl.indicator == "window"
+    tensor_core = wl.dtype == "bf16" and wl.head_dim == 128
+    if tensor_core:
+        # Eq. 2 with the l1 norm: counter reset, pass 1 (value norms on its side warp), pass 2;
+        # otherwise: norm kernel, pass 1 unless the normalisers are given, pass 2
+        scoring = 2 if args.lse_given else 3
+    else:
+        scoring = 1 if args.lse_given else 2       # row statistics, column sums
+    compaction = 2 if windowed else 1              # gather, then the window history (rebuilt or gathered)
+    if args.kv_heads and args.kv_heads < wl.heads:
+        scoring = scoring * (wl.heads // args.kv_heads) + 1    # once per query head of the groups, then the group mean
+    return scoring + 1 + compaction
 
 
 def run_cuda(args, wl):
@@ -215,7 +248,7 @@ def run_cuda(args, wl):
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
     L, steps_dec = args.layers, wl.decode_steps
-    layers = [LayerState(V, wl, l, dev, win_rows=args.win_rows) for l in range(L)]
+    layers = [LayerState(V, wl, l, dev, win_rows=args.win_rows, kv_heads=args.kv_heads) for l in range(L)]
     windowed = wl.indicator == "window"
 
     def compact(ls):
@@ -405,7 +438,8 @@ def run_cuda(args, wl):
 
     if rank != 0:
         return
-    units = wl.batch * wl.heads
+    q_units = wl.batch * wl.heads                              # scoring sweeps run once per query head
+    units = wl.batch * (args.kv_heads or wl.heads)             # kept sets, caches and decode states: one per KV head
     T, d, B = wl.seq_len, wl.head_dim, wl.budget
     tokens = wl.batch * T * L                                  # layer-tokens scored and pruned per step
     value = replica_throughput(tokens, pre_ms, world)
@@ -419,9 +453,9 @@ def run_cuda(args, wl):
     else:
         pairs = T * (T + 1) / 2
     passes = 1 if args.lse_given else 2
-    flops_score = passes * (2.0 * d) * pairs * units           # each pass recomputes the causal part of QK^T
+    flops_score = passes * (2.0 * d) * pairs * q_units         # each pass recomputes the causal part of QK^T
     # fused call: the forward's two contractions over every causal pair, then pass 2's one
-    flops_fused = (2 * (2.0 * d) * (T * (T + 1) / 2) + (2.0 * d) * pairs) * units
+    flops_fused = (2 * (2.0 * d) * (T * (T + 1) / 2) + (2.0 * d) * pairs) * q_units
     bytes_compact = units * (2 * 2 * B * d * 2 + 12 * B)       # K,V rows read + written, 12 B of state per slot
     if wl.indicator == "window":
         # history ring written; with --win-rows the kept columns of the last-w rows are read too
@@ -481,6 +515,9 @@ def run_cuda(args, wl):
         "config": {"workload": f"config{wl.cid} {wl.name}: b{wl.batch} h{wl.heads} d{d} T{T} budget{B} recent{wl.n_recent} "
                                f"sinkF{wl.n_sink} {wl.indicator}, {steps_dec} decode steps, x{L} independently seeded layers",
                    "layers": L,
+                   **({"kv_heads": args.kv_heads, "grouped_queries": f"{wl.heads // args.kv_heads} query heads share each KV "
+                       "head (group-mean indicator): scoring runs per query head, selection / compaction / decode per KV head"}
+                      if args.kv_heads else {}),
                    "l2": f"256 MB flush write between steps; layer rotation over {L} decode states ({L * bytes_decode / 1e6:.0f} MB per visit of all layers)",
                    "replicas": "each GPU runs the whole workload (path does not shard within a call)",
                    "decode_graph": graph is not None},
@@ -490,7 +527,7 @@ def run_cuda(args, wl):
         "e2e": None if host is None else
                {"value": replica_throughput(tokens, e2e_pre_ms, world), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "decode_us_per_layer_step": e2e_dec_ms * 1e3 / (steps_dec * L)},
-        "gpu_launches": args.steps * (L * 4 + steps_dec * L),
+        "gpu_launches": args.steps * L * (prune_launches(wl, args) + steps_dec),
         "clocks": clocks,
     }
     if not args.no_cpu_baseline and world == 1:
@@ -532,6 +569,10 @@ def main():
     ap.add_argument("--lse-given", action="store_true",
                     help="time vatp_prefill_scores_from_lse: the row normalisers come from an earlier attention forward "
                          "(here: from the warm-up's two-pass call), so scoring is one recomputation of QK^T")
+    ap.add_argument("--kv-heads", type=int, default=0,
+                    help="grouped-query attention: the workload's heads become query heads that share this many KV heads "
+                         "(the Limitations section's open case, read as a group-mean indicator); CUDA arm only")
+    ap.add_argument("--batch", type=int, default=None, help="override the workload's batch size")
     ap.add_argument("--norm", default="l1", choices=["l1", "l2", "linf"],
                     help="value norm of Eq. 4: l1 is the method (and the benchmark), l2 / linf the Ablation Study's variants")
     args = ap.parse_args()
@@ -545,6 +586,13 @@ def main():
         pr = presets.appendix_a(method, wl.seq_len, args.budget_ratio)
         wl = wl.with_(budget=pr["budget"], n_sink=pr["n_sink"], n_recent=pr["n_recent"], indicator=pr["indicator"],
                       window=pr["window"], name=f"{wl.name} {method} budget {args.budget_ratio:g}")
+    if args.batch is not None:
+        wl = wl.with_(batch=args.batch, name=f"{wl.name} batch {args.batch}")
+    if args.kv_heads:
+        if wl.heads % args.kv_heads or args.impl == "reference":
+            ap.error("--kv-heads must divide the workload's heads and applies to the CUDA arm only")
+        wl = wl.with_(name=f"{wl.name} {args.kv_heads} kv heads")
+        args.no_cpu_baseline = True          # the sampled oracle baseline is defined for the multi-head workloads
     if args.norm != "l1":
         wl = wl.with_(norm=args.norm, name=f"{wl.name} norm={args.norm}")
     if args.lse_given:
