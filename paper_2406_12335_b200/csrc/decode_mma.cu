@@ -56,6 +56,8 @@ constexpr int ROW_BYTES = HD * 2;
 constexpr int TILE_BYTES = GROUP * 128;    // 16 rows x 64 bf16, 128-byte swizzled
 constexpr int STAGE_BYTES = 4 * TILE_BYTES; // K columns 0-63, K 64-127, V 0-63, V 64-127
 constexpr int MAX_SPLIT = 8;
+constexpr int GQ_HEADS = 8;           // grouped queries: query heads per cache this kernel takes (rows 0-7 of the MMA tiles)
+constexpr int GQ_MAX_SPLIT = 4;       // ... and the CTAs a unit is split over at most
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr unsigned long long NO_KEY = ~0ull;
 
@@ -155,9 +157,14 @@ __device__ __forceinline__ unsigned long long warp_min_key(unsigned long long ke
   return ((unsigned long long)mh << 32) | ml;
 }
 
-template <bool WINDOWED, int MW>
+// GT = 1: one query head per cache (multi-head attention).  GT = GQ_HEADS: grouped queries - up to GQ_HEADS query
+// heads (G of them, a run-time argument) share the cache of unit u: row g of the MMA tiles carries head g, so the
+// streaming loop is the same instructions, and every K and V row is read once for the whole group; the maxima,
+// sums and partial outputs exist per head, and the indicator advances by the MEAN of the heads' probabilities.
+// Only the eight-warp kernel is built for it (the per-head partials take the room a second CTA would need).
+template <bool WINDOWED, int MW, int GT>
 __global__ void __launch_bounds__(MW * 32 + 32, MW == MW_BESIDE ? 2 : 1)
-decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int independent,
+decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v, int independent, int G,
                   int state_in_smem, int split, int chunk, int nstage, int B, int cap, int F, int R, int w, int norm, float scale_log2,
                   vatp_cache c,
                   const __nv_bfloat16* __restrict__ q_new, const __nv_bfloat16* __restrict__ k_new,
@@ -165,6 +172,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
                   int32_t* __restrict__ evicted, int32_t* __restrict__ dev_status) {
   constexpr int WT = MW * 32;           // streaming threads (at least HD: one per output channel where outputs are formed)
   static_assert(WT >= HD, "one streaming thread per output channel");
+  static_assert(GT == 1 || (GT == GQ_HEADS && MW == MW_ALONE), "grouped queries: the eight-warp kernel only");
   extern __shared__ unsigned char dyn_raw[];
   unsigned char* dyn = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(dyn_raw) + 1023) & ~uintptr_t(1023));
   // [MW][nstage] stages | logits[chunk] | acc[chunk] | vnorm[chunk] | pos[chunk]: the per-slot arrays of
@@ -174,9 +182,13 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   // global memory in the tail (state_in_smem == 0).
   unsigned char* stage_base = dyn;
   float* logit_s = reinterpret_cast<float*>(dyn + (size_t)MW * nstage * STAGE_BYTES);
-  float* acc_s = state_in_smem == 2 ? reinterpret_cast<float*>(stage_base) : logit_s + chunk;
+  // (grouped queries: logits[G][chunk], state always here (state_in_smem == 1), then the per-head partial outputs
+  // of the eight streams [NSTREAM][G][HD] and, in rank 0, those of every CTA of the unit [split][G][HD])
+  float* acc_s = state_in_smem == 2 ? reinterpret_cast<float*>(stage_base) : logit_s + (GT > 1 ? G : 1) * chunk;
   float* vn_s = acc_s + chunk;
   int* pos_s = reinterpret_cast<int*>(vn_s + chunk);
+  float* gq_part = reinterpret_cast<float*>(pos_s + chunk);
+  float* gq_xo = gq_part + NSTREAM * (GT > 1 ? G : 0) * HD;
 
   __shared__ __align__(8) uint64_t bars[MW * 4 + 1];
   __shared__ __align__(16) Exch ex;
@@ -184,6 +196,10 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   static_assert(SPW == 1 || SPW == 2, "a warp folds one or two streams");
   __shared__ __align__(16) float part_o[NSTREAM][HD];
   __shared__ float part_m[NSTREAM], part_l[NSTREAM];
+  // grouped queries: per stream and head; per rank and head (pushed by every CTA of the unit); the unit's normalisers
+  __shared__ float gq_pm[GT > 1 ? NSTREAM : 1][GT], gq_pl[GT > 1 ? NSTREAM : 1][GT];
+  __shared__ float gq_m[GT > 1 ? GQ_MAX_SPLIT : 1][GT], gq_l[GT > 1 ? GQ_MAX_SPLIT : 1][GT];
+  __shared__ float gq_fr[GT > 1 ? GQ_MAX_SPLIT : 1][GT], gq_mall[GT], gq_invl[GT];
   __shared__ unsigned long long warp_key[MW];
   __shared__ int ctrl_evicting;
 
@@ -295,7 +311,8 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   const bool owns_last = !independent && ls >= 0 && ls != fs && ls_local >= 0 && ls_local < cnt;
 
   // A operand of q K^T: q replicated over the rows 0-7 of the tile (rows 8-15 zero)
-  const __nv_bfloat16* qn = q_new + (int64_t)u * HD;
+  // (grouped queries: row g of the tile carries head g of the unit's group; rows beyond the group repeat its last head)
+  const __nv_bfloat16* qn = GT > 1 ? q_new + ((int64_t)u * G + min(lane >> 2, G - 1)) * HD : q_new + (int64_t)u * HD;
   uint32_t qa[HD / 16][2];
 #pragma unroll
   for (int ks = 0; ks < HD / 16; ++ks) {
@@ -350,7 +367,16 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     float l = l_run;
     l += __shfl_xor_sync(0xffffffffu, l, 1);
     l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (lane < 4) {
+    if constexpr (GT > 1) {
+      const int hg = lane >> 2;      // this lane's head
+      if (hg < G) {
+        float* po = gq_part + ((size_t)stream * G + hg) * HD;
+#pragma unroll
+        for (int i = 0; i < HD / 8; ++i)
+          *reinterpret_cast<float2*>(&po[i * 8 + 2 * j4]) = make_float2(o_acc[i][0] + o_acc[i][2], o_acc[i][1] + o_acc[i][3]);
+        if (j4 == 0) { gq_pm[stream][hg] = m_run; gq_pl[stream][hg] = l; }
+      }
+    } else if (lane < 4) {
 #pragma unroll
       for (int i = 0; i < HD / 8; ++i)
         *reinterpret_cast<float2*>(&part_o[stream][i * 8 + 2 * j4]) = make_float2(o_acc[i][0] + o_acc[i][2], o_acc[i][1] + o_acc[i][3]);
@@ -405,7 +431,13 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   #pragma unroll
         for (int i = 0; i < 4; ++i)
           if (rows[i] >= cnt) s[i] = -INFINITY;
-        if (lane < 4) {
+        if constexpr (GT > 1) {
+          if ((lane >> 2) < G) {
+  #pragma unroll
+            for (int i = 0; i < 4; ++i)
+              if (rows[i] < cnt) logit_s[(lane >> 2) * chunk + rows[i]] = s[i];
+          }
+        } else if (lane < 4) {
   #pragma unroll
           for (int i = 0; i < 4; ++i)
             if (rows[i] < cnt) logit_s[rows[i]] = s[i];
@@ -413,7 +445,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
         float gmax = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 1));
         gmax = fmaxf(gmax, __shfl_xor_sync(0xffffffffu, gmax, 2));
-        if (gmax > m_run) {          // warp-uniform (r0 < cnt guarantees a live row, so gmax is finite)
+        if (gmax > m_run) {          // uniform over a tile row's four lanes - over the warp with one head (r0 < cnt guarantees a live row, so gmax is finite)
           const float f = ex2(m_run - gmax);   // 0 on the first group
           l_run *= f;
   #pragma unroll
@@ -482,7 +514,34 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   }
 
   // ---- CTA partial: max and sum to every CTA of the unit, partial output to rank 0 ----
-  {
+  if constexpr (GT > 1) {
+    // per head of the group; thread tid < HD merges channel tid of the eight streams, threads HD .. HD + split - 1
+    // push the head's maximum and sum to the unit's CTAs
+    float* xo0 = split > 1 ? cluster.map_shared_rank(gq_xo, 0) : gq_xo;
+    for (int h = 0; h < G; ++h) {
+      float m_c = -INFINITY;
+#pragma unroll
+      for (int i = 0; i < NSTREAM; ++i) m_c = fmaxf(m_c, gq_pm[i][h]);
+      float fw[NSTREAM], l_c = 0.f;
+#pragma unroll
+      for (int i = 0; i < NSTREAM; ++i) {
+        fw[i] = gq_pm[i][h] > -INFINITY ? ex2(gq_pm[i][h] - m_c) : 0.f;
+        l_c += gq_pl[i][h] * fw[i];
+      }
+      if (tid < HD) {
+        float a = 0.f;
+#pragma unroll
+        for (int i = 0; i < NSTREAM; ++i) a = fmaf(gq_part[((size_t)i * G + h) * HD + tid], fw[i], a);
+        xo0[((size_t)rank * G + h) * HD + tid] = a;
+      } else if (tid < HD + split) {
+        const int r = tid - HD;
+        float* rm = split > 1 ? cluster.map_shared_rank(&gq_m[0][0], r) : &gq_m[0][0];
+        float* rl = split > 1 ? cluster.map_shared_rank(&gq_l[0][0], r) : &gq_l[0][0];
+        rm[rank * GT + h] = m_c;
+        rl[rank * GT + h] = l_c;
+      }
+    }
+  } else {
     float m_c = -INFINITY;
 #pragma unroll
     for (int i = 0; i < NSTREAM; ++i) m_c = fmaxf(m_c, part_m[i]);
@@ -508,6 +567,27 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
   if (split > 1) { cluster_arrive_release(); cluster_wait_acquire(); } else workers_sync<WT>();
 
   // ---- every CTA: the unit's softmax normaliser (all data is local now) ----
+  if constexpr (GT > 1) {
+    if (tid < G) {         // one thread per head
+      float m_h = -INFINITY, L_h = 0.f;
+      for (int r = 0; r < split; ++r) m_h = fmaxf(m_h, gq_m[r][tid]);
+      for (int r = 0; r < split; ++r) {
+        const float f = gq_m[r][tid] > -INFINITY ? ex2(gq_m[r][tid] - m_h) : 0.f;
+        gq_fr[r][tid] = f;
+        L_h += gq_l[r][tid] * f;
+      }
+      gq_mall[tid] = m_h;
+      gq_invl[tid] = 1.f / L_h;
+    }
+    workers_sync<WT>();
+    if (rank == 0 && tid < HD) {
+      for (int h = 0; h < G; ++h) {
+        float a = 0.f;
+        for (int r = 0; r < split; ++r) a = fmaf(gq_xo[((size_t)r * G + h) * HD + tid], gq_fr[r][h], a);
+        out[((int64_t)u * G + h) * HD + tid] = __float2bfloat16(a * gq_invl[h]);
+      }
+    }
+  }
   float m_all = -INFINITY, L = 0.f;
   float fr[MAX_SPLIT];
 #pragma unroll
@@ -519,7 +599,7 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
     if (r < split) L += ex.l[r] * fr[r];
   }
   const float invL = 1.f / L;
-  if (rank == 0 && tid < HD) {
+  if (GT == 1 && rank == 0 && tid < HD) {
     float a = 0.f;
 #pragma unroll
     for (int r = 0; r < MAX_SPLIT; ++r)
@@ -542,7 +622,14 @@ decode_mma_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constan
 #pragma unroll 4
     for (int i = tid; i < cnt; i += WT) {
       const int slot = s0 + i;
-      const float p = ex2(lg[i] - m_all) * invL;
+      float p;
+      if constexpr (GT > 1) {      // the mean of the heads' probabilities
+        float a = 0.f;
+        for (int h = 0; h < G; ++h) a = fmaf(ex2(lg[h * chunk + i] - gq_mall[h]), gq_invl[h], a);
+        p = a / (float)G;
+      } else {
+        p = ex2(lg[i] - m_all) * invL;
+      }
       const bool is_new = slot == fs;
       float S;
       if (WINDOWED) {
@@ -730,13 +817,14 @@ void decode_history_forget(cudaStream_t st, bool probe_only) {
 // then takes the general kernel).
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
                               const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
-                              bool may_overlap) {
+                              bool may_overlap, int G) {
   const int cap = cache_capacity(B);
-  if (!vatp_tc_available()) return cudaErrorNotSupported;
+  if (!vatp_tc_available() || G < 1 || G > GQ_HEADS) return cudaErrorNotSupported;
+  const bool grouped = G > 1;           // s.units counts caches (KV heads); q and out hold G rows per unit
   const int sms = device_sm_count();
   // split a unit over a cluster while the grid still fits on the SMs once (a second launch can then be resident too)
   int split = 1;
-  while (split < MAX_SPLIT && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
+  while (split < (grouped ? GQ_MAX_SPLIT : MAX_SPLIT) && s.units * split * 2 <= sms && cap / (split * 2) >= 4 * GROUP) split *= 2;
   int chunk = (cap + split - 1) / split;
   chunk = (chunk + GROUP - 1) / GROUP * GROUP;
   // Shared-memory plan.  A launch that may run beside its neighbours stays within half an SM (two CTAs
@@ -756,6 +844,8 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     const int MW = alone ? MW_ALONE : MW_BESIDE;
     const size_t stage_set = (size_t)MW * STAGE_BYTES;
     size_t state_bytes = 4 * sizeof(float) * tot;
+    if (grouped)    // logits per head, the state, the streams' partial outputs per head, rank 0's copy of every CTA's
+      state_bytes = (size_t)(G + 3) * sizeof(float) * tot + (size_t)(NSTREAM + split) * G * HD * sizeof(float);
     p.state_in_smem = 1;
     const bool fits_half = !alone && state_bytes + 1024 + 2 * stage_set <= half_sm;
     if (!alone && !fits_half && sizeof(float) * tot + 1024 + 2 * stage_set <= half_sm) {
@@ -773,7 +863,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
     p.dyn = (size_t)MW * p.nstage * STAGE_BYTES + state_bytes + 1024;
     return p;
   };
-  const Plan beside = make_plan(false), lone = make_plan(true);
+  const Plan lone = make_plan(true), beside = grouped ? lone : make_plan(false);      // grouped queries: always a whole SM
   if (!beside.ok || !lone.ok) return cudaErrorNotSupported;
   CUtensorMap tm_k, tm_v;
   if (!make_rows_map_bf16(&tm_k, c.k_cache, (uint64_t)s.units * cap, GROUP) ||
@@ -785,12 +875,13 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
                        {(const char*)c.acc, slots * 4}, {(const char*)c.vnorm, slots * 4}, {(const char*)c.pos, slots * 4},
                        {(const char*)c.len, units * 4}, {(const char*)c.free_slot, units * 4},
                        {(const char*)c.next_pos, units * 4}, {(const char*)c.last_slot, units * 4},
-                       {(const char*)out, units * ROW_BYTES}, {(const char*)evicted, evicted ? units * 4 : 0},
+                       {(const char*)out, units * G * ROW_BYTES}, {(const char*)evicted, evicted ? units * 4 : 0},
                        {win ? (const char*)c.ring : nullptr, win ? slots * s.window * 4 : 0},
                        {win ? (const char*)c.acc_fixed : nullptr, win ? slots * 8 : 0},
-                       {(const char*)q, units * ROW_BYTES}, {(const char*)k, units * ROW_BYTES}, {(const char*)v, units * ROW_BYTES}};
-  auto kern_beside = win ? decode_mma_kernel<true, MW_BESIDE> : decode_mma_kernel<false, MW_BESIDE>;
-  auto kern_alone = win ? decode_mma_kernel<true, MW_ALONE> : decode_mma_kernel<false, MW_ALONE>;
+                       {(const char*)q, units * G * ROW_BYTES}, {(const char*)k, units * ROW_BYTES}, {(const char*)v, units * ROW_BYTES}};
+  auto kern_alone = grouped ? (win ? decode_mma_kernel<true, MW_ALONE, GQ_HEADS> : decode_mma_kernel<false, MW_ALONE, GQ_HEADS>)
+                            : (win ? decode_mma_kernel<true, MW_ALONE, 1> : decode_mma_kernel<false, MW_ALONE, 1>);
+  auto kern_beside = grouped ? kern_alone : (win ? decode_mma_kernel<true, MW_BESIDE, 1> : decode_mma_kernel<false, MW_BESIDE, 1>);
   cudaError_t e = cudaFuncSetAttribute(kern_beside, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(kern_alone, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)whole_sm);
   if (e != cudaSuccess) return e;
@@ -798,7 +889,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   auto share_of = [&](const Plan& p, bool alone) {
     int occ = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, alone ? kern_alone : kern_beside,
-                                                      (alone ? MW_ALONE : MW_BESIDE) * 32 + 32, p.dyn) != cudaSuccess || occ < 1)
+                                                      (alone || grouped ? MW_ALONE : MW_BESIDE) * 32 + 32, p.dyn) != cudaSuccess || occ < 1)
       occ = 1;
     return (double)(s.units * split) / ((double)occ * sms);
   };
@@ -810,7 +901,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   const size_t dyn = pl.dyn;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(s.units * split);
-  cfg.blockDim = dim3((independent ? MW_BESIDE : MW_ALONE) * 32 + 32);
+  cfg.blockDim = dim3((independent && !grouped ? MW_BESIDE : MW_ALONE) * 32 + 32);
   cfg.dynamicSmemBytes = dyn;
   cfg.stream = st;
   cudaLaunchAttribute attr[2];
@@ -822,7 +913,7 @@ cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_ca
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, state_in_smem, split, chunk, nstage, B, cap, F, R, s.window, s.norm, s.scale * LOG2E, c,
+  return cudaLaunchKernelEx(&cfg, kern, tm_k, tm_v, independent, G, state_in_smem, split, chunk, nstage, B, cap, F, R, s.window, s.norm, s.scale * LOG2E, c,
                             (const __nv_bfloat16*)q, (const __nv_bfloat16*)k, (const __nv_bfloat16*)v,
                             (__nv_bfloat16*)out, evicted, dev_status);
 }

@@ -266,6 +266,20 @@ vatp_status vatp_decode_step(const vatp_params* p, const vatp_cache* cache, cons
   if (!aligned16(q_new) || !aligned16(k_new) || !aligned16(v_new) || !aligned16(out)) return VATP_ERR_INVALID_ARG;
   if (group_of(p) > 1) {
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    if (p->dtype == VATP_BF16 && p->head_dim == 128 && group_of(p) <= 8) {
+      // tensor-core step: the group's heads ride in the rows of the MMA tiles, every K and V row is read once
+      Shape sh;
+      std::memset(&sh, 0, sizeof(sh));
+      sh.units = p->batch * kv_heads_of(p);
+      sh.heads = kv_heads_of(p);
+      sh.d = p->head_dim;
+      sh.scale = p->scale;
+      sh.window = windowed ? p->window_w : 0;
+      sh.norm = p->norm_kind;
+      const cudaError_t e = launch_decode_mma(sh, p->budget, p->n_sink, p->n_recent, *cache, q_new, k_new, v_new, out, evicted_pos,
+                                              dev_status, st, (p->flags & VATP_FLAG_DECODE_OVERLAP) != 0, group_of(p));
+      if (e != cudaErrorNotSupported) return e == cudaSuccess ? VATP_OK : VATP_ERR_CUDA;
+    }
     decode_history_forget(st);
     const cudaError_t e = launch_decode_gqa(p->batch * kv_heads_of(p), group_of(p), p->head_dim, p->dtype, p->budget, p->n_sink,
                                             p->n_recent, windowed ? p->window_w : 0, p->norm_kind, p->scale, *cache, q_new, k_new,

@@ -136,9 +136,10 @@ cudaError_t launch_decode(const Shape& s, int dtype, int B, int F, int R, const 
 // bf16, head_dim 128 only; cudaErrorNotSupported when the shape does not fit (take launch_decode's general kernel)
 // may_overlap: the caller opted in to launches that run beside earlier decode launches on the stream when they share
 // no buffer with them (VATP_FLAG_DECODE_OVERLAP)
+// G: query heads per cache (grouped-query attention, 1 .. 8): s.units counts caches, q and out hold G rows per unit
 cudaError_t launch_decode_mma(const Shape& s, int B, int F, int R, const vatp_cache& c, const void* q, const void* k,
                               const void* v, void* out, int32_t* evicted, int32_t* dev_status, cudaStream_t st,
-                              bool may_overlap);
+                              bool may_overlap, int G = 1);
 // other work of this library was enqueued on the stream: the next decode launch waits for all of it
 // (probe_only: `st` is only a key of the host-side self-test, not a stream the runtime may be asked about)
 void decode_history_forget(cudaStream_t st, bool probe_only = false);

@@ -656,6 +656,8 @@ def test_bounds_checking_build_reports_no_violation():
     ("f32", 64, 4, 2, 333, 100, 3, 17),        # general kernels
     ("bf16", 64, 8, 1, 257, 128, 2, 16),       # multi-query attention: one KV head
     ("f32", 128, 16, 1, 200, 80, 1, 8),        # sixteen heads per group, 32 pieces per row
+    ("bf16", 128, 16, 2, 900, 300, 2, 20),     # eight heads per group: every row of the decode step's MMA tiles is a head
+    ("bf16", 128, 32, 2, 300, 120, 1, 8),      # sixteen heads per group: beyond the tensor-core step, general decode kernel
 ])
 @pytest.mark.parametrize("fused", [False, True])
 def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R, fused):
@@ -828,3 +830,59 @@ def test_grouped_query_attention_with_history_window(dtype, d, heads, kv_heads, 
         order = np.argsort(pos[live])
         assert pos[live][order].tolist() == st.pos and int(cache.len[bi, g]) == len(st.pos)
         assert P.rel_err(P.to_np64(cache.acc[bi, g])[live][order], st.indicator()) <= 2 * tol
+
+
+@pytest.mark.parametrize("overlap", [True, False])
+@pytest.mark.parametrize("b,heads,kv_heads", [(1, 8, 2), (6, 32, 8)])
+def test_grouped_query_caches_interleaved_match_separate_runs(b, heads, kv_heads, overlap):
+    """The tensor-core decode step with grouped queries (bf16, head_dim 128): steps of three independent caches issued
+    round robin on one stream - with the opt-in flag they may run side by side - give bit for bit what each cache
+    gives when stepped alone with a synchronisation after every step.  (Each step against the oracle:
+    test_grouped_query_attention.)"""
+    V = P.vatp()
+    d, T, B, F, R, steps = 128, 600, 260, 2, 16, 10
+    G = heads // kv_heads
+
+    def prefilled(i, decode_overlap):
+        wl_kv = _small("bf16", d, T, B, F, R, b=b, h=kv_heads, steps=steps, cid=80 + i)
+        _, k, v = synth.prefill_inputs(wl_kv, 0, "cuda")
+        gq = torch.Generator(device="cuda").manual_seed(5000 + i)
+        q = torch.randn(b, heads, T, d, generator=gq, device="cuda").to(k.dtype)
+        dq = torch.randn(steps, b, heads, d, generator=gq, device="cuda").to(k.dtype)
+        _, dk, dv = synth.decode_inputs(wl_kv, 0, device="cuda")
+        p = V.make_params(batch=b, heads=heads, kv_heads=kv_heads, seq_len=T, head_dim=d, dtype="bf16", budget=B, n_sink=F,
+                          n_recent=R, scale=wl_kv.scale, decode_overlap=decode_overlap)
+        f32 = dict(dtype=torch.float32, device="cuda")
+        attn_acc, vnorm, score = (torch.empty(b, kv_heads, T, **f32) for _ in range(3))
+        ws = torch.empty(V.vatp_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        kept = torch.empty(b, kv_heads, B, dtype=torch.int32, device="cuda")
+        cache = V.Cache(p)
+        V.vatp_prefill_scores(p, q, k, v, attn_acc=attn_acc, vnorm=vnorm, score=score, workspace=ws, dev_status=status)
+        V.vatp_select(p, score, kept, dev_status=status)
+        V.vatp_compact(p, k, v, attn_acc, vnorm, kept, cache, dev_status=status)
+        torch.cuda.synchronize()
+        return dict(p=p, cache=cache, status=status, dq=dq, dk=dk, dv=dv,
+                    out=torch.empty(steps, b, heads, d, dtype=k.dtype, device="cuda"),
+                    ev=torch.empty(steps, b, kv_heads, dtype=torch.int32, device="cuda"))
+
+    def step(c, s):
+        V.vatp_decode_step(c["p"], c["cache"], c["dq"][s], c["dk"][s], c["dv"][s], c["out"][s], evicted_pos=c["ev"][s],
+                           dev_status=c["status"])
+
+    alone = [prefilled(i, False) for i in range(3)]
+    for c in alone:
+        for s in range(steps):
+            step(c, s)
+            torch.cuda.synchronize()
+    inter = [prefilled(i, overlap) for i in range(3)]
+    for s in range(steps):
+        for c in inter:
+            step(c, s)
+    torch.cuda.synchronize()
+    for ca, cb in zip(alone, inter):
+        assert int(ca["status"].item()) == 0 and int(cb["status"].item()) == 0
+        assert torch.all(ca["ev"][-1] >= 0), "the last step evicts in every unit"
+        assert torch.equal(ca["out"], cb["out"]) and torch.equal(ca["ev"], cb["ev"])
+        for name in ("k_cache", "v_cache", "acc", "vnorm", "pos", "len", "free_slot", "next_pos"):
+            assert torch.equal(getattr(ca["cache"], name), getattr(cb["cache"], name)), name
