@@ -5,6 +5,7 @@
 // and the exact fixed-point window sum moves by it), Eq. 4 multiplies by the norm of the shared value row, and
 // the lowest importance is released as in the multi-head step.
 //
+// (bf16 with head_dim 128 and up to eight heads per group takes the tensor-core step of decode_mma.cu instead.)
 // A general kernel (any dtype and head_dim; CTAs of 512 threads, the probabilities of all heads in shared memory), laid
 // out so that every K and V row is read ONCE for all heads of the group.  A unit's slots are split over a cluster of
 // four or two CTAs while the grid still fits the SMs at once: every CTA forms the maxima, sums and partial outputs of

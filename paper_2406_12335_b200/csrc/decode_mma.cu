@@ -26,7 +26,10 @@
 //     the next launch at once and only holds the CTA until the previous launch has completed, so
 //     launches still complete in order and the number in flight is bounded by what fits on the
 //     machine (two CTAs fit on an SM).  A launch that does wait has its SMs to itself and runs the
-//     eight-warp variant of the kernel (same arithmetic, see MW below).
+//     eight-warp variant of the kernel (same arithmetic, see MW below);
+//   * grouped-query attention (several query heads share one cache; the paper leaves the case open and points at
+//     a group-wise score, read here as the MEAN of the heads' probabilities): up to eight heads of a group ride
+//     in the rows of the MMA tiles (template parameter GT), so a K or V row is still read once per step.
 #include <cooperative_groups.h>
 
 #include <mutex>
