@@ -640,7 +640,8 @@ def test_bounds_checking_build_reports_no_violation():
     env = dict(os.environ, VATP_LIBRARY=lib)
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     sel = ("ragged or degenerate or windowed_indicator_shapes or general_kernels or large_cache or few_units "
-           "or exact_ties or unstaged or strided or static_scratch_matches or rebuilt or (fused_attention and not config1)")
+           "or exact_ties or unstaged or strided or static_scratch_matches or rebuilt or (fused_attention and not config1) "
+           "or grouped_query_caches")
     r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_gpu_parity.py", "tests/test_zz_no_alloc.py", "-x", "-q",
                         "-m", "gpu", "-k", sel, "-p", "no:cacheprovider"], cwd=root, env=env, capture_output=True, text=True)
     tail = (r.stdout + r.stderr)[-2000:]
