@@ -659,6 +659,7 @@ def test_bounds_checking_build_reports_no_violation():
     ("f32", 128, 16, 1, 200, 80, 1, 8),        # sixteen heads per group, 32 pieces per row
     ("bf16", 128, 16, 2, 900, 300, 2, 20),     # eight heads per group: every row of the decode step's MMA tiles is a head
     ("bf16", 128, 32, 2, 300, 120, 1, 8),      # sixteen heads per group: beyond the tensor-core step, general decode kernel
+    ("bf16", 128, 10, 2, 500, 200, 1, 12),     # five heads per group: three rows of the MMA tiles repeat the last head
 ])
 @pytest.mark.parametrize("fused", [False, True])
 def test_grouped_query_attention(dtype, d, heads, kv_heads, T, B, F, R, fused):
