@@ -60,7 +60,7 @@ constexpr int TILE_BYTES = GROUP * 128;    // 16 rows x 64 bf16, 128-byte swizzl
 constexpr int STAGE_BYTES = 4 * TILE_BYTES; // K columns 0-63, K 64-127, V 0-63, V 64-127
 constexpr int MAX_SPLIT = 8;
 constexpr int GQ_HEADS = 8;           // grouped queries: query heads per cache this kernel takes (rows 0-7 of the MMA tiles)
-constexpr int GQ_MAX_SPLIT = 4;       // ... and the CTAs a unit is split over at most
+constexpr int GQ_MAX_SPLIT = MAX_SPLIT;   // ... and the CTAs a unit is split over at most
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr unsigned long long NO_KEY = ~0ull;
 
