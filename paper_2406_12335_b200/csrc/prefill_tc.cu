@@ -373,6 +373,10 @@ __device__ __forceinline__ void consume32(float (&x)[32], int c0, int row, float
 
 struct TcArgs {
   int units, heads, T, nt, nch, Tpad;  // nt tiles of 128 tokens, nch = ceil(nt / 2) chunks, Tpad = 256 nch
+  // Grouped queries in one launch (G > 1): the units are the query heads, unit (b, h) reads K and V of KV head h / G;
+  // value norms exist per KV unit, and pass 2 writes query head h's indicator to slice h % G of attn_acc
+  // ([G][kv_units][T]: the group mean is taken afterwards) and no score.  G = 1: kv_units = units, kv_heads = heads.
+  int G, kv_units, kv_heads;
   float scale_log2;
   const __nv_bfloat16* v;
   int64_t sb, sh, st;       // element strides of v
@@ -413,6 +417,12 @@ struct Item {
   int u, tile, c_first, c_count;
   int lo;   // pass 2: first query tile that counts for this key tile
 };
+// the KV unit whose keys and values unit u attends over
+__device__ __forceinline__ int kv_unit_of(const TcArgs& a, int u) {
+  if (a.G == 1) return u;
+  const int b = u / a.heads, h = u - b * a.heads;
+  return b * a.kv_heads + h / a.G;
+}
 template <int PASS>
 __device__ __forceinline__ Item item_of(int id, const TcArgs& a) {
   Item it;
@@ -437,11 +447,11 @@ __device__ __forceinline__ bool tile_needed(const Item& it, int st, int nt) {
 // Value norms of all (unit, token tile) pairs, shared out over the CTAs: the work of pass 1's side warp.
 template <int KIND>
 __device__ __forceinline__ void side_value_norms(const TcArgs& a, int lane) {
-  for (int id = blockIdx.x; id < a.units * a.nt; id += gridDim.x) {
+  for (int id = blockIdx.x; id < a.kv_units * a.nt; id += gridDim.x) {
     Item it;
-    it.tile = id / a.units;
-    it.u = id - it.tile * a.units;
-    const int b = it.u / a.heads, h = it.u - b * a.heads;
+    it.tile = id / a.kv_units;
+    it.u = id - it.tile * a.kv_units;      // a KV unit
+    const int b = it.u / a.kv_heads, h = it.u - b * a.kv_heads;
     const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
     // 16 lanes per row, two rows per load instruction, 16 rows in flight per lane group
     const int sub = lane >> 4, part = lane & 15;
@@ -463,7 +473,7 @@ __device__ __forceinline__ void side_value_norms(const TcArgs& a, int lane) {
 #pragma unroll
         for (int o = 8; o; o >>= 1) acc = norm_merge(KIND, acc, __shfl_xor_sync(0xffffffffu, acc, o));
         const int tok = it.tile * TILE + r0 + 2 * j + sub;
-        if (part == 0 && tok < a.T && VATP_INB((int64_t)it.u * a.T + tok, (int64_t)a.units * a.T, a.dev_status))
+        if (part == 0 && tok < a.T && VATP_INB((int64_t)it.u * a.T + tok, (int64_t)a.kv_units * a.T, a.dev_status))
           a.vnorm[(int64_t)it.u * a.T + tok] = norm_finish(KIND, acc);
       }
     }
@@ -553,11 +563,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         next = (int)atomicAdd(&a.counters[PASS - 1], 1u);     // in flight while this item's tiles are requested
         const int b = it.u / a.heads, h = it.u - b * a.heads;
         const int fb = itl & 1;
+        // head coordinate of the fixed and of the streamed operand (K is the streamed one in pass 1, the fixed one in pass 2)
+        const int hk = a.G > 1 ? h / a.G : h;
+        const int h_fix = PASS == 1 ? h : hk, h_str = PASS == 1 ? hk : h;
         ok = mbar_wait<20>(&sm.fixed_empty[fb], ((itl >> 1) & 1) ^ 1, abort_flag, a.dev_status);
         if (!ok) break;
         mbar_expect_tx(&sm.fixed_full[fb], TILE_BYTES);
-        tma_load_4d(sm.fixed[fb], tm_fixed, &sm.fixed_full[fb], 0, it.tile * TILE, h, b);
-        tma_load_4d(sm.fixed[fb] + SLAB_BYTES, tm_fixed, &sm.fixed_full[fb], 64, it.tile * TILE, h, b);
+        tma_load_4d(sm.fixed[fb], tm_fixed, &sm.fixed_full[fb], 0, it.tile * TILE, h_fix, b);
+        tma_load_4d(sm.fixed[fb] + SLAB_BYTES, tm_fixed, &sm.fixed_full[fb], 64, it.tile * TILE, h_fix, b);
         for (int c = 0; c < it.c_count; ++c, ++n) {
           const int stg = n % NS;
           ok = mbar_wait<20>(&sm.empty[stg], ((n / NS) & 1) ^ 1, abort_flag, a.dev_status);
@@ -570,7 +583,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 #pragma unroll
             for (int hh = 0; hh < 2; ++hh)
               tma_load_4d(sm.stream[stg] + kh * (2 * SLAB_BYTES) + hh * SLAB_BYTES, tm_stream, &sm.full[stg], 64 * kh,
-                          tok0 + hh * TILE, h, b);
+                          tok0 + hh * TILE, h_str, b);
           if (PASS == 2) {
             // The chunk's 256 normalisers travel with its tiles and are complete when its MMAs are.  Ring slot
             // n % NLSE: the MMAs of chunk n - 2 have completed (that freed this stage), so every softmax warp
@@ -639,7 +652,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
       const int tok = it.tile * TILE + row;       // query (pass 1) or key (pass 2) index of this thread
       // pass 2: this key's value norm, written by pass 1; fetched now, used in the item's epilogue
       float n1 = 0.f;
-      if (PASS == 2 && g == 0 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)u * a.T + tok);
+      if (PASS == 2 && g == 0 && tok < a.T) n1 = __ldg(a.vnorm + (int64_t)kv_unit_of(a, u) * a.T + tok);
       float m_run = -INFINITY, l_run = 0.f;       // pass 1
       f32x2 cs[2] = {pk2(0.f, 0.f), pk2(0.f, 0.f)};   // pass 2: four running sums, packed
       const uint32_t n0 = n;
@@ -743,9 +756,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
           const float tot = hsum2(add2(cs[0], cs[1])) + (sm.part_a[pi][0][row] + sm.part_a[pi][1][row]) + sm.part_a[pi][2][row];
           mbar_arrive(&sm.comb_empty[pi]);
           if (tok < a.T && VATP_INB((int64_t)u * a.T + tok, (int64_t)a.units * a.T, a.dev_status)) {
-            const int64_t o = (int64_t)u * a.T + tok;
-            a.attn_acc[o] = tot;
-            a.score[o] = tot * n1;
+            if (a.G == 1) {
+              const int64_t o = (int64_t)u * a.T + tok;
+              a.attn_acc[o] = tot;
+              a.score[o] = tot * n1;
+            } else {      // query head h's indicator: slice h % G of the partial indicators, row of its KV unit
+              const int h = u % a.heads;
+              a.attn_acc[((int64_t)(h % a.G) * a.kv_units + kv_unit_of(a, u)) * a.T + tok] = tot;
+            }
           }
         }
       }
@@ -979,13 +997,14 @@ attention_fwd_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_c
           ok = mbar_wait<20>(&sm.k_empty[stg], par, abort_flag, a.dev_status);
           if (!ok) break;
           mbar_expect_tx(&sm.k_full[stg], TILE_BYTES);     // tokens beyond T arrive as zeros
-          tma_load_4d(sm.k[stg], &tm_k, &sm.k_full[stg], 0, c * TILE, h, b);
-          tma_load_4d(sm.k[stg] + SLAB_BYTES, &tm_k, &sm.k_full[stg], 64, c * TILE, h, b);
+          const int hk = a.G > 1 ? h / a.G : h;      // grouped queries: the KV head of this query head
+          tma_load_4d(sm.k[stg], &tm_k, &sm.k_full[stg], 0, c * TILE, hk, b);
+          tma_load_4d(sm.k[stg] + SLAB_BYTES, &tm_k, &sm.k_full[stg], 64, c * TILE, hk, b);
           ok = mbar_wait<20>(&sm.v_empty[stg], par, abort_flag, a.dev_status);
           if (!ok) break;
           mbar_expect_tx(&sm.v_full[stg], TILE_BYTES);
-          tma_load_4d(sm.v[stg], &tm_v, &sm.v_full[stg], 0, c * TILE, h, b);
-          tma_load_4d(sm.v[stg] + SLAB_BYTES, &tm_v, &sm.v_full[stg], 64, c * TILE, h, b);
+          tma_load_4d(sm.v[stg], &tm_v, &sm.v_full[stg], 0, c * TILE, hk, b);
+          tma_load_4d(sm.v[stg] + SLAB_BYTES, &tm_v, &sm.v_full[stg], 64, c * TILE, hk, b);
         }
       }
     }
@@ -1265,7 +1284,7 @@ __global__ void __launch_bounds__(256) vnorm_kernel(TcArgs a, const float* __res
       a.lse2[(int64_t)u * a.Tpad + i] = x;
     }
   }
-  const int b = u / a.heads, h = u - b * a.heads;
+  const int b = u / a.kv_heads, h = u - b * a.kv_heads;      // (one CTA column per KV unit)
   const __nv_bfloat16* vu = a.v + (int64_t)b * a.sb + (int64_t)h * a.sh;
   const int sub = threadIdx.x >> 4, part = threadIdx.x & 15;       // 16 rows per pass of the CTA
   const int row0 = blockIdx.y * 128 + sub;
@@ -1464,7 +1483,8 @@ EncodeTiledFn encode_fn() {
 
 // [batch, heads, T, 128] bf16 with element strides (sb, sh, st, 1); box = 64 x 128 rows, 128-byte swizzle
 bool make_map(CUtensorMap* m, const void* base, const Shape& s, bool of_q = false) {
-  const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)s.T, (cuuint64_t)s.heads, (cuuint64_t)(s.units / s.heads)};
+  const int heads = (!of_q && s.kv_heads > 0) ? s.kv_heads : s.heads;      // k and v of grouped queries: the KV heads
+  const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)s.T, (cuuint64_t)heads, (cuuint64_t)(s.units / s.heads)};
   const cuuint64_t strides[3] = {(cuuint64_t)s.st * 2, (cuuint64_t)(of_q ? s.qsh : s.sh) * 2, (cuuint64_t)(of_q ? s.qsb : s.sb) * 2};
   const cuuint32_t box[4] = {64, TILE, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -1538,6 +1558,10 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
   if (attn_out && (lse_in || !make_map(&tm_v, v, s))) return cudaErrorInvalidValue;
   TcArgs a;
   a.units = s.units; a.heads = s.heads; a.T = s.T;
+  a.kv_heads = s.kv_heads > 0 ? s.kv_heads : s.heads;
+  a.G = s.heads / a.kv_heads;
+  a.kv_units = s.units / a.G;
+  if (a.G > 1 && (lse_in || win_rows)) return cudaErrorInvalidValue;
   a.nt = (s.T + TILE - 1) / TILE;
   a.nch = (a.nt + 1) / 2;
   a.Tpad = a.nch * CHUNK;
@@ -1585,7 +1609,7 @@ cudaError_t launch_prefill_tc(const Shape& s, const void* q, const void* k, cons
     return e;
   }
   if (!a.side_norm) {
-    const dim3 grid(a.units, (s.T + 127) / 128);
+    const dim3 grid(a.kv_units, (s.T + 127) / 128);
     if (a.norm == VATP_NORM_L1) vnorm_kernel<VATP_NORM_L1><<<grid, 256, 0, st>>>(a, lse_in);
     else if (a.norm == VATP_NORM_L2) vnorm_kernel<VATP_NORM_L2><<<grid, 256, 0, st>>>(a, lse_in);
     else vnorm_kernel<VATP_NORM_LINF><<<grid, 256, 0, st>>>(a, lse_in);

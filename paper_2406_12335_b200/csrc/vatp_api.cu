@@ -39,6 +39,7 @@ vatp_status make_shape(const vatp_params* p, Shape* s) {
   const int kvh = kv_heads_of(p), G = group_of(p);
   s->units = p->batch * kvh;
   s->heads = kvh;
+  s->kv_heads = 0;
   s->T = p->seq_len;
   s->d = p->head_dim;
   s->st = p->stride_t ? p->stride_t : p->head_dim;
@@ -62,7 +63,7 @@ vatp_status make_shape(const vatp_params* p, Shape* s) {
 // row normalisers of pass 1, padded to whole 128-row tiles per unit; with grouped queries, then the G partial
 // indicators [G][units][T] that the group mean is taken of
 inline size_t lse_bytes(const vatp_params* p) {
-  size_t n = prefill_tc_workspace_bytes(p->batch * kv_heads_of(p), p->seq_len);
+  size_t n = prefill_tc_workspace_bytes(p->batch * p->heads, p->seq_len);      // (one row per query head)
   return (n + 255) / 256 * 256;
 }
 inline size_t workspace_need(const vatp_params* p) {
@@ -113,7 +114,22 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
     // the general kernel keeps its (natural-log) normalisers in the caller's layout: lse_out, or a scratch copy of
     // that layout at the head of the workspace when the caller wants none (it fits: G * units * T floats <= `part`)
     e = cudaSuccess;
-    for (int g = 0; g < G && e == cudaSuccess; ++g) {
+    if (tc) {
+      // tensor cores: ONE launch over all query heads; unit (b, h) reads KV head h / G, and pass 2 files its indicator
+      // under slice h % G of the partial indicators
+      Shape sq = sh;
+      sq.units = p->batch * p->heads;
+      sq.heads = p->heads;
+      sq.kv_heads = kv_heads_of(p);
+      sq.qsh = sh.sh;
+      sq.qsb = (int64_t)p->heads * sh.sh;
+      sq.lse_sh = sh.T;
+      sq.lse_sb = (int64_t)p->heads * sh.T;
+      sq.osh = (int64_t)sh.T * sh.d;
+      sq.osb = (int64_t)p->heads * sh.T * sh.d;
+      e = launch_prefill_tc(sq, q, k, v, ws, lse_out, part, vnorm, score, nullptr, dev_status, st, nullptr, attn_out);
+    }
+    for (int g = 0; g < G && e == cudaSuccess && !tc; ++g) {
       const char* qg = static_cast<const char*>(q) + (size_t)g * sh.sh * eb;
       float* lse_g = lse_out ? lse_out + (size_t)g * sh.T : nullptr;
       // the fused call: this round's query heads' rows of the attention output (head kvh * G + g of every KV group)

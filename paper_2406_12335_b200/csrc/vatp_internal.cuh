@@ -13,6 +13,8 @@ namespace vatp {
 struct Shape {
   int units;           // batch * heads
   int heads;
+  int kv_heads;        // 0: k and v have `heads` heads; else grouped queries in ONE launch: the units are the query heads,
+                       // k and v have kv_heads heads and unit (b, h) reads KV head h / (heads / kv_heads) of batch b
   int T, d;
   int64_t sb, sh, st;  // element strides of k and v (and of q, unless qsb / qsh say otherwise)
   int64_t qsb, qsh;    // batch and head strides of q (grouped-query attention runs one query head of every KV

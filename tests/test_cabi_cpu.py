@@ -86,7 +86,8 @@ def test_host_side_validation(V):
     # grouped-query attention: kv_heads divides heads, contiguous layouts only; the workspace also holds the G partial indicators
     gq = dict(ok, heads=4)
     assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=4)) == V.vatp_workspace_bytes(V.make_params(**gq))
-    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=2)) == (2 * 256 * 4 + 256) + 2 * 2 * 64 * 4
+    # (normalisers of the 4 query heads, padded to 256 tokens, the counters, then 2 partial indicators of 2 KV units)
+    assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=2)) == (4 * 256 * 4 + 256) + 2 * 2 * 64 * 4
     assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=3)) == 0
     assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=8)) == 0
     assert V.vatp_workspace_bytes(V.make_params(**gq, kv_heads=2, strides=(0, 0, 128))) == 0
