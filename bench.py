@@ -229,7 +229,8 @@ def prune_launches(wl, args):
         scoring = 1 if args.lse_given else 2       # row statistics, column sums
     compaction = 2 if windowed else 1              # gather, then the window history (rebuilt or gathered)
     if args.kv_heads and args.kv_heads < wl.heads:
-        scoring = scoring * (wl.heads // args.kv_heads) + 1    # once per query head of the groups, then the group mean
+        # tensor cores: one launch over all query heads; general kernels: once per query head of the groups; then the group mean
+        scoring = (scoring if tensor_core else scoring * (wl.heads // args.kv_heads)) + 1
     return scoring + 1 + compaction
 
 

@@ -34,8 +34,8 @@
  *     vatp_compact_window, which then needs lse for all `heads` query heads).  Layouts must be
  *     contiguous (stride fields 0); vatp_prefill_scores_from_lse and win_rows (hence vatp_compact
  *     with a history window) are not available with it (VATP_ERR_UNSUPPORTED), and the workspace
- *     grows by G partial indicators.  The decode step takes the tensor-core kernel for bf16,
- *     head_dim 128 and G <= 8 (VATP_FLAG_DECODE_OVERLAP applies as in the multi-head case) and a
+ *     holds a normaliser row per query head and G partial indicators.  The decode step takes
+ *     the tensor-core kernel for bf16, head_dim 128 and G <= 8 (VATP_FLAG_DECODE_OVERLAP applies as in the multi-head case) and a
  *     general kernel otherwise; the history rebuild runs a general kernel.
  *   - Inputs are assumed finite.
  *   - A second build of the library (compiled with -DVATP_DEBUG_BOUNDS) range-checks every row, slot,

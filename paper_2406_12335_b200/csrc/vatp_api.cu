@@ -33,8 +33,9 @@ inline int group_of(const vatp_params* p) { return p->kv_heads > 0 ? p->heads / 
 inline int kv_heads_of(const vatp_params* p) { return p->kv_heads > 0 ? p->kv_heads : p->heads; }
 
 // The units are the (batch, KV head) pairs.  With grouped queries (contiguous layouts only) q has G times as many
-// heads: a launch takes one query head of every group, i.e. q as a view with head stride G * T * d (the caller
-// offsets the q pointer by g * T * d and the row-normaliser pointer by g * T).
+// heads.  The general kernels take one query head of every group per launch, i.e. q as a view with head stride
+// G * T * d (the caller offsets the q pointer by g * T * d and the row-normaliser pointer by g * T); the tensor-core
+// kernels take all query heads in one launch (Shape::kv_heads).
 vatp_status make_shape(const vatp_params* p, Shape* s) {
   const int kvh = kv_heads_of(p), G = group_of(p);
   s->units = p->batch * kvh;
@@ -105,8 +106,9 @@ vatp_status prefill_impl(const vatp_params* p, const void* q, const void* k, con
   decode_history_forget(st);
   cudaError_t e;
   if (G > 1) {
-    // One query head of every KV group per round: the multi-head kernels on strided views of q, each round's
-    // indicator into its own slice of the workspace, then the mean over the rounds (fixed order) and Eq. 4.
+    // Every query head's indicator goes to a slice of the workspace - head g of its group to slice g - then the mean
+    // over the slices (fixed order) and Eq. 4.  General kernels: one query head of every KV group per round, the
+    // multi-head kernels on strided views of q.
     const size_t n = (size_t)sh.units * sh.T;
     float* part = reinterpret_cast<float*>(static_cast<char*>(workspace) + lse_bytes(p));
     const int eb = p->dtype == VATP_F32 ? 4 : 2;
