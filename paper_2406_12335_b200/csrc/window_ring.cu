@@ -52,95 +52,131 @@ window_ring_general_kernel(int heads, int T_len, int d, int w, int B, int cap, f
 }
 
 // Grouped-query attention: the history holds the MEAN over the KV group's G query heads of their probabilities
-// (the group-mean indicator's rows).  One thread per slot, 128 slots per CTA.  The CTA's 128 key rows are staged in
-// shared memory once, as fp32 and transposed ([d][129]: a thread walks its own column without bank conflicts); two
-// window queries of all G heads are staged per step ([2][d][G padded to fours]), so that one key element from shared
-// memory meets eight query values (two queries x four heads) in registers.  Per (slot, query) the heads are summed in
-// ascending order and the dot products in ascending channel order.
-constexpr int WR_SLOTS = 128, WR_KPAD = WR_SLOTS + 1, WR_Q = 2;
+// (the group-mean indicator's rows).  A CTA of four warps takes 128 slots: their key rows are staged in shared memory
+// once, as fp32 and transposed ([d][132]), and eight window queries of all G heads per step ([8][d][G padded to fours]).
+// A thread owns four neighbouring slots, a warp two of the step's queries: per channel one 16-byte load of four key
+// elements and two of four heads' query elements feed 32 FMAs.  Per (slot, query) the heads are summed in ascending order
+// and the dot products in ascending channel order; the fixed-point window sums of the four warps are integers and are
+// added at the end.
+constexpr int WR_SLOTS = 128, WR_KPAD = WR_SLOTS + 4, WR_Q = 2, WR_WARPS = 4, WR_STEP = WR_Q * WR_WARPS;
 template <typename T>
-__global__ void __launch_bounds__(WR_SLOTS)
+__global__ void __launch_bounds__(WR_WARPS * 32)
 window_ring_grouped_kernel(int G, int kv_heads, int T_len, int d, int w, int B, int cap, float scale, const T* __restrict__ q,
                            int64_t qsb, int64_t qsh, int64_t q_head, int64_t st, const float* __restrict__ lse, int64_t lse_sb,
                            int64_t lse_sh, vatp_cache c) {
   extern __shared__ __align__(16) float wr_smem[];
   const int GP = (G + 3) & ~3;
   float* k_s = wr_smem;                          // [d][WR_KPAD]
-  float* q_s = wr_smem + (size_t)d * WR_KPAD;    // [WR_Q][d][GP]  (d is a multiple of four: 16-byte aligned)
-  const int u = blockIdx.y, tid = threadIdx.x;
-  const int slot0 = blockIdx.x * WR_SLOTS, slot = slot0 + tid;
+  float* q_s = wr_smem + (size_t)d * WR_KPAD;    // [WR_STEP][d][GP]  (16-byte aligned: WR_KPAD is a multiple of four)
+  const int u = blockIdx.y, tid = threadIdx.x, lane = tid & 31, wq = tid >> 5;
+  const int slot0 = blockIdx.x * WR_SLOTS;
+  const int sl4 = lane * 4;                      // this thread's slots: slot0 + sl4 .. + 3
   const int len = min(T_len, B);
   const int b = u / kv_heads, h = u - b * kv_heads;
   const T* qu = q + (int64_t)b * qsb + (int64_t)h * qsh;
   const float* lu = lse + (int64_t)b * lse_sb + (int64_t)h * lse_sh;
   const T* kbase = static_cast<const T*>(c.k_cache) + (int64_t)u * cap * d;
-  const int ps = slot < len ? c.pos[(int64_t)u * cap + slot] : -1;
+  int ps[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) ps[k] = slot0 + sl4 + k < len ? c.pos[(int64_t)u * cap + slot0 + sl4 + k] : -1;
   const float invG = 1.f / (float)G;
-  for (int idx = tid; idx < WR_SLOTS * d; idx += WR_SLOTS) {       // consecutive threads: consecutive elements of a row
+  for (int idx = tid; idx < WR_SLOTS * d; idx += WR_WARPS * 32) {       // consecutive threads: consecutive elements of a row
     const int sl = idx / d, i = idx - sl * d;
     k_s[i * WR_KPAD + sl] = slot0 + sl < cap ? to_f32(kbase[(int64_t)(slot0 + sl) * d + i]) : 0.f;
   }
-  for (int idx = tid; idx < WR_Q * d * GP; idx += WR_SLOTS) q_s[idx] = 0.f;      // the padding heads stay zero
-  long long fx = 0;
-  for (int r0 = 0; r0 < w; r0 += WR_Q) {
+  for (int idx = tid; idx < WR_STEP * d * GP; idx += WR_WARPS * 32) q_s[idx] = 0.f;      // the padding heads stay zero
+  long long fx[4] = {0, 0, 0, 0};
+  for (int r0 = 0; r0 < w; r0 += WR_STEP) {
     __syncthreads();
-    for (int idx = tid; idx < WR_Q * G * d; idx += WR_SLOTS) {
+    for (int idx = tid; idx < WR_STEP * G * d; idx += WR_WARPS * 32) {
       const int jj = idx / (G * d), rem = idx - jj * (G * d);
       const int g = rem / d, i = rem - g * d;
       const int j = T_len - w + r0 + jj;
       q_s[(jj * d + i) * GP + g] = (r0 + jj < w && j >= 0) ? to_f32(qu[(int64_t)g * q_head + (int64_t)j * st + i]) : 0.f;
     }
     __syncthreads();
-    float p[WR_Q];
-    bool live[WR_Q];
+    const int rq = r0 + wq * WR_Q;               // this warp's window rows: rq, rq + 1
+    float p[WR_Q][4];
+    bool live[WR_Q][4], any = false;
 #pragma unroll
     for (int jj = 0; jj < WR_Q; ++jj) {
-      const int j = T_len - w + r0 + jj;
-      p[jj] = 0.f;
-      live[jj] = slot < cap && r0 + jj < w && j >= 0 && ps >= 0 && ps <= j;      // causal: the token precedes the query
-    }
-    if (live[0] || live[1]) {
-      for (int g0 = 0; g0 < G; g0 += 4) {
-        float a[WR_Q][4];
+      const int j = T_len - w + rq + jj;
 #pragma unroll
-        for (int jj = 0; jj < WR_Q; ++jj) a[jj][0] = a[jj][1] = a[jj][2] = a[jj][3] = 0.f;
-#pragma unroll 4
+      for (int k = 0; k < 4; ++k) {
+        p[jj][k] = 0.f;
+        // causal: the token precedes the query
+        live[jj][k] = slot0 + sl4 + k < cap && rq + jj < w && j >= 0 && ps[k] >= 0 && ps[k] <= j;
+        any = any || live[jj][k];
+      }
+    }
+    if (any) {
+      for (int g0 = 0; g0 < G; g0 += 4) {
+        float a[WR_Q][4][4];                     // [query][head][slot]
+#pragma unroll
+        for (int jj = 0; jj < WR_Q; ++jj)
+#pragma unroll
+          for (int hh = 0; hh < 4; ++hh) a[jj][hh][0] = a[jj][hh][1] = a[jj][hh][2] = a[jj][hh][3] = 0.f;
+        const float* qw = q_s + (size_t)(wq * WR_Q) * d * GP + g0;
+#pragma unroll 2
         for (int i = 0; i < d; ++i) {
-          const float kv = k_s[i * WR_KPAD + tid];
+          const float4 kv = *reinterpret_cast<const float4*>(&k_s[i * WR_KPAD + sl4]);
 #pragma unroll
           for (int jj = 0; jj < WR_Q; ++jj) {
-            const float4 qv = *reinterpret_cast<const float4*>(&q_s[(jj * d + i) * GP + g0]);
-            a[jj][0] = fmaf(qv.x, kv, a[jj][0]);
-            a[jj][1] = fmaf(qv.y, kv, a[jj][1]);
-            a[jj][2] = fmaf(qv.z, kv, a[jj][2]);
-            a[jj][3] = fmaf(qv.w, kv, a[jj][3]);
+            const float4 qv = *reinterpret_cast<const float4*>(&qw[((size_t)jj * d + i) * GP]);
+            const float qh[4] = {qv.x, qv.y, qv.z, qv.w};
+#pragma unroll
+            for (int hh = 0; hh < 4; ++hh) {
+              a[jj][hh][0] = fmaf(qh[hh], kv.x, a[jj][hh][0]);
+              a[jj][hh][1] = fmaf(qh[hh], kv.y, a[jj][hh][1]);
+              a[jj][hh][2] = fmaf(qh[hh], kv.z, a[jj][hh][2]);
+              a[jj][hh][3] = fmaf(qh[hh], kv.w, a[jj][hh][3]);
+            }
           }
         }
 #pragma unroll
         for (int jj = 0; jj < WR_Q; ++jj) {
-          const int j = T_len - w + r0 + jj;
-          if (live[jj]) {
+          const int j = T_len - w + rq + jj;
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-              if (g0 + k < G) p[jj] += __expf(a[jj][k] * scale - __ldg(lu + (int64_t)(g0 + k) * T_len + j));
+          for (int hh = 0; hh < 4; ++hh) {
+            if (g0 + hh < G && rq + jj < w && j >= 0) {
+              const float l = __ldg(lu + (int64_t)(g0 + hh) * T_len + j);
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                if (live[jj][k]) p[jj][k] += __expf(a[jj][hh][k] * scale - l);
+            }
           }
         }
       }
     }
 #pragma unroll
     for (int jj = 0; jj < WR_Q; ++jj) {
-      const int j = T_len - w + r0 + jj;
-      if (r0 + jj < w && slot < cap) {
-        const float pj = live[jj] ? p[jj] * invG : 0.f;
+      const int j = T_len - w + rq + jj;
+      if (rq + jj < w) {
         const int rr = ((j % w) + w) % w;
-        c.ring[((int64_t)u * w + rr) * cap + slot] = pj;
-        fx += prob_to_fixed(pj);
+        float* row = c.ring + ((int64_t)u * w + rr) * cap + slot0 + sl4;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          if (slot0 + sl4 + k < cap) {
+            const float pj = live[jj][k] ? p[jj][k] * invG : 0.f;
+            row[k] = pj;
+            fx[k] += prob_to_fixed(pj);
+          }
+        }
       }
     }
   }
+  __syncthreads();                               // every warp is past its last read of q_s
+  long long* fx_s = reinterpret_cast<long long*>(q_s);      // [WR_WARPS][WR_SLOTS]
+#pragma unroll
+  for (int k = 0; k < 4; ++k) fx_s[wq * WR_SLOTS + sl4 + k] = fx[k];
+  __syncthreads();
+  const int slot = slot0 + tid;
   if (slot < cap) {
-    c.acc_fixed[(int64_t)u * cap + slot] = fx;
-    c.acc[(int64_t)u * cap + slot] = fixed_to_prob(fx);
+    long long tot = 0;
+#pragma unroll
+    for (int ww = 0; ww < WR_WARPS; ++ww) tot += fx_s[ww * WR_SLOTS + tid];
+    c.acc_fixed[(int64_t)u * cap + slot] = tot;
+    c.acc[(int64_t)u * cap + slot] = fixed_to_prob(tot);
   }
 }
 
@@ -150,7 +186,9 @@ window_ring_grouped_kernel(int G, int kv_heads, int T_len, int d, int w, int B, 
 cudaError_t launch_window_ring_grouped(const Shape& s, int G, int dtype, int B, const void* q, const float* lse, const vatp_cache& c,
                                        cudaStream_t st) {
   const int cap = cache_capacity(B);
-  const size_t smem = ((size_t)s.d * WR_KPAD + (size_t)WR_Q * s.d * ((G + 3) & ~3)) * sizeof(float);
+  size_t q_bytes = (size_t)WR_STEP * s.d * ((G + 3) & ~3) * sizeof(float);
+  if (q_bytes < (size_t)WR_WARPS * WR_SLOTS * sizeof(long long)) q_bytes = (size_t)WR_WARPS * WR_SLOTS * sizeof(long long);   // the warps' window sums land there at the end
+  const size_t smem = (size_t)s.d * WR_KPAD * sizeof(float) + q_bytes;
   if (smem > 200 * 1024 || (s.d & 3)) return cudaErrorNotSupported;
   cudaError_t e = cudaFuncSetAttribute(window_ring_grouped_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e == cudaSuccess)
